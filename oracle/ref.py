@@ -1,0 +1,181 @@
+"""ctypes loader for libmtmcref, the fp64 CPU oracle (TEST INFRASTRUCTURE ONLY).
+
+Only tests, the smoke check and the benchmark's CPU legs may import this module.
+It never imports the CUDA package and shares nothing with it.  Arrays are numpy:
+bf16 operands travel as uint16 bit patterns, bias as float32, results as float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "mtmc_ref.cpp")
+_LIB = os.path.join(_HERE, "libmtmcref.so")
+
+ACT_NONE, ACT_RELU, ACT_GELU_TANH, ACT_SILU = 0, 1, 2, 3
+
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle/mtmc_ref.cpp -> oracle/libmtmcref.so with g++ (no CUDA involved)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(
+            ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-pthread", "-o", tmp, _SRC]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        i64, vp, dbl, ci = ctypes.c_int64, ctypes.c_void_p, ctypes.c_double, ctypes.c_int
+        L.mtmc_ref_set_threads.argtypes = [ci]
+        L.mtmc_ref_get_threads.restype = ci
+        L.mtmc_ref_act.argtypes = [ci, dbl]
+        L.mtmc_ref_act.restype = dbl
+        L.mtmc_ref_fused_linear.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp]
+        L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
+        L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+        L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
+        L.mtmc_ref_linear_lse.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
+        L.mtmc_ref_linear_lse_rows.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
+        L.mtmc_ref_lse_vector.argtypes = [vp, i64]
+        L.mtmc_ref_lse_vector.restype = dbl
+        L.mtmc_ref_compare.argtypes = [vp, vp, i64, dbl, dbl, vp]
+        L.mtmc_ref_compare.restype = i64
+        _lib = L
+    return _lib
+
+
+def _bf16(a, shape) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint16 or tuple(a.shape) != tuple(shape):
+        raise TypeError("bf16 operand must be a uint16 bit-pattern array of shape %r" % (shape,))
+    return a
+
+
+def _bias(b, N):
+    if b is None:
+        return None, None
+    b = np.ascontiguousarray(b)
+    if b.dtype != np.float32 or b.shape != (N,):
+        raise TypeError("bias must be float32 [N]")
+    return b, b.ctypes.data
+
+
+def _idx(v) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(v, dtype=np.int64))
+
+
+def _check(rc: int, name: str) -> None:
+    if rc != 0:
+        raise ValueError("%s rejected its arguments (status %d)" % (name, rc))
+
+
+def set_threads(n: int) -> None:
+    lib().mtmc_ref_set_threads(int(n))
+
+
+def get_threads() -> int:
+    return int(lib().mtmc_ref_get_threads())
+
+
+def act(kind: int, z: float) -> float:
+    return float(lib().mtmc_ref_act(int(kind), float(z)))
+
+
+def fused_linear(X, W, b, act_kind: int) -> np.ndarray:
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear(X.ctypes.data, W.ctypes.data, bp, M, N, K, int(act_kind), out.ctypes.data),
+           "mtmc_ref_fused_linear")
+    return out
+
+
+def fused_linear_points(X, W, b, act_kind: int, rows, cols) -> np.ndarray:
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    rows, cols = _idx(rows), _idx(cols)
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear_points(X.ctypes.data, W.ctypes.data, bp, M, N, K, int(act_kind),
+                                              rows.ctypes.data, cols.ctypes.data, rows.shape[0], out.ctypes.data),
+           "mtmc_ref_fused_linear_points")
+    return out
+
+
+def swiglu(X, Wg, Wu) -> np.ndarray:
+    M, K = X.shape
+    N = Wg.shape[0]
+    X, Wg, Wu = _bf16(X, (M, K)), _bf16(Wg, (N, K)), _bf16(Wu, (N, K))
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_swiglu(X.ctypes.data, Wg.ctypes.data, Wu.ctypes.data, M, N, K, out.ctypes.data),
+           "mtmc_ref_swiglu")
+    return out
+
+
+def swiglu_points(X, Wg, Wu, rows, cols) -> np.ndarray:
+    M, K = X.shape
+    N = Wg.shape[0]
+    X, Wg, Wu = _bf16(X, (M, K)), _bf16(Wg, (N, K)), _bf16(Wu, (N, K))
+    rows, cols = _idx(rows), _idx(cols)
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _check(lib().mtmc_ref_swiglu_points(X.ctypes.data, Wg.ctypes.data, Wu.ctypes.data, M, N, K,
+                                        rows.ctypes.data, cols.ctypes.data, rows.shape[0], out.ctypes.data),
+           "mtmc_ref_swiglu_points")
+    return out
+
+
+def linear_lse(X, W, b, want_logits: bool = False):
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    lse = np.empty(M, dtype=np.float64)
+    logits = np.empty((M, N), dtype=np.float64) if want_logits else None
+    _check(lib().mtmc_ref_linear_lse(X.ctypes.data, W.ctypes.data, bp, M, N, K, lse.ctypes.data,
+                                     logits.ctypes.data if want_logits else None), "mtmc_ref_linear_lse")
+    return (lse, logits) if want_logits else lse
+
+
+def linear_lse_rows(X, W, b, rows) -> np.ndarray:
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    rows = _idx(rows)
+    lse = np.empty(rows.shape[0], dtype=np.float64)
+    _check(lib().mtmc_ref_linear_lse_rows(X.ctypes.data, W.ctypes.data, bp, M, N, K,
+                                          rows.ctypes.data, rows.shape[0], lse.ctypes.data),
+           "mtmc_ref_linear_lse_rows")
+    return lse
+
+
+def lse_vector(z) -> float:
+    z = np.ascontiguousarray(np.asarray(z, dtype=np.float64))
+    return float(lib().mtmc_ref_lse_vector(z.ctypes.data, z.shape[0]))
+
+
+def compare(got, ref, atol: float, rtol: float) -> dict:
+    """|got-ref| <= atol + rtol*|ref| element-wise; NaN/Inf on either side fails."""
+    got = np.ascontiguousarray(np.asarray(got, dtype=np.float64)).ravel()
+    ref = np.ascontiguousarray(np.asarray(ref, dtype=np.float64)).ravel()
+    if got.shape != ref.shape:
+        raise ValueError("shape mismatch: %r vs %r" % (got.shape, ref.shape))
+    stats = np.zeros(4, dtype=np.float64)
+    bad = lib().mtmc_ref_compare(got.ctypes.data, ref.ctypes.data, got.shape[0], float(atol), float(rtol),
+                                 stats.ctypes.data)
+    return {"violations": int(bad), "max_abs_err": float(stats[0]), "max_ratio": float(stats[1]),
+            "worst_index": int(stats[2]), "count": int(got.shape[0]), "ok": bad == 0}

@@ -1,0 +1,102 @@
+"""Seeded synthetic inputs shared by the CUDA tests, the oracle tests and the benchmark.
+
+This module holds none of the method's arithmetic: it only draws random tensors
+with the stated distributions and rounds them to bf16.  Both the CUDA path and
+the CPU oracle receive the very same arrays, so parity never depends on the
+generator.
+
+Recipe ("seed s"): a torch CPU generator seeded with s; fp32 draws in the fixed
+order X, W (or Wg then Wu), b:
+    X  = randn(M, K)                 -> bf16 (round to nearest even)
+    W  = randn(N, K) * K**-0.5       -> bf16   (variance 1/K, so X.W^T ~ N(0,1))
+    b  = rand(N) * 0.2 - 0.1         (fp32, U(-0.1, 0.1), not rounded)
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+# The five benchmark configurations (shape, call, seed).
+CONFIGS = {
+    "C1": dict(op="fused_linear", M=256, N=256, K=256, act="relu", out_dtype="fp32", seed=0),
+    "C2": dict(op="fused_linear", M=4096, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=1),
+    "C3": dict(op="swiglu", M=8192, N=11008, K=4096, seed=2),
+    "C4": dict(op="linear_lse", M=4096, N=32000, K=4096, seed=3),
+    "C5": dict(op="fused_linear", M=16, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=4),
+}
+
+
+@dataclass
+class LinearInputs:
+    X: torch.Tensor            # [M, K] bf16, CPU
+    W: torch.Tensor            # [N, K] bf16, CPU
+    b: torch.Tensor | None     # [N] fp32, CPU
+
+
+@dataclass
+class SwigluInputs:
+    X: torch.Tensor            # [M, K] bf16
+    Wg: torch.Tensor           # [N, K] bf16
+    Wu: torch.Tensor           # [N, K] bf16
+
+
+def _gen(seed: int) -> torch.Generator:
+    g = torch.Generator(device="cpu")
+    g.manual_seed(int(seed))
+    return g
+
+
+def linear_inputs(M: int, N: int, K: int, seed: int, bias: bool = True) -> LinearInputs:
+    g = _gen(seed)
+    X = torch.randn(M, K, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    W = (torch.randn(N, K, generator=g, dtype=torch.float32) * (float(K) ** -0.5)).to(torch.bfloat16)
+    b = (torch.rand(N, generator=g, dtype=torch.float32) * 0.2 - 0.1) if bias else None
+    return LinearInputs(X, W, b)
+
+
+def swiglu_inputs(M: int, N: int, K: int, seed: int) -> SwigluInputs:
+    g = _gen(seed)
+    X = torch.randn(M, K, generator=g, dtype=torch.float32).to(torch.bfloat16)
+    Wg = (torch.randn(N, K, generator=g, dtype=torch.float32) * (float(K) ** -0.5)).to(torch.bfloat16)
+    Wu = (torch.randn(N, K, generator=g, dtype=torch.float32) * (float(K) ** -0.5)).to(torch.bfloat16)
+    return SwigluInputs(X, Wg, Wu)
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 tensor (CPU) -> uint16 numpy array of the same shape holding the raw bit patterns."""
+    assert t.dtype == torch.bfloat16
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def bits_to_bf16(a: np.ndarray) -> torch.Tensor:
+    """uint16 bit patterns -> bf16 torch tensor (CPU) of the same shape."""
+    assert a.dtype == np.uint16
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16)
+
+
+def f32(t: torch.Tensor | None) -> np.ndarray | None:
+    return None if t is None else t.detach().cpu().contiguous().numpy()
+
+
+def to_f64(t: torch.Tensor) -> np.ndarray:
+    """Exact widening of a result tensor (fp32 or bf16, any device) to float64 numpy."""
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
+def sample_points(M: int, N: int, count: int, seed: int, tile_m: int = 128, tile_n: int = 128):
+    """(rows, cols) for sampled parity: the four corners of the output, first/last
+    element of tile-edge rows and columns, plus `count` seeded uniform positions."""
+    rng = np.random.default_rng(seed)
+    rows = list(rng.integers(0, M, size=count))
+    cols = list(rng.integers(0, N, size=count))
+    edge_r = sorted({0, M - 1, min(tile_m - 1, M - 1), min(tile_m, M - 1), (M // tile_m) * tile_m - 1 if M >= tile_m else 0,
+                     min((M // tile_m) * tile_m, M - 1)})
+    edge_c = sorted({0, N - 1, min(tile_n - 1, N - 1), min(tile_n, N - 1), (N // tile_n) * tile_n - 1 if N >= tile_n else 0,
+                     min((N // tile_n) * tile_n, N - 1)})
+    for r in edge_r:
+        for c in edge_c:
+            rows.append(r)
+            cols.append(c)
+    return np.asarray(rows, dtype=np.int64), np.asarray(cols, dtype=np.int64)

@@ -1,0 +1,300 @@
+"""Pins for the fp64 CPU oracle: every check here is against something OTHER than the
+oracle itself -- exact rational brute force, hand-worked values, 40-digit closed
+forms, algebraic laws of the operators, and torch's fp64 library routines.  A
+dropped term, a wrong sign or index, or a transposed operand fails at least one.
+CPU only."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2511_20100_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+ACTS = [ref.ACT_NONE, ref.ACT_RELU, ref.ACT_GELU_TANH, ref.ACT_SILU]
+
+
+def bits(a) -> np.ndarray:
+    """float array (values exactly representable in bf16, or to be RNE-rounded) -> uint16 bit patterns."""
+    return inputs.bf16_bits(torch.as_tensor(np.asarray(a, dtype=np.float32)).to(torch.bfloat16))
+
+
+def widen(b16: np.ndarray) -> np.ndarray:
+    return inputs.bits_to_bf16(b16).to(torch.float64).numpy()
+
+
+def py_act(kind, z):
+    """Independent scalar restatement used only where the GEMM part is under test."""
+    if kind == ref.ACT_NONE:
+        return z
+    if kind == ref.ACT_RELU:
+        return max(z, 0.0)
+    if kind == ref.ACT_GELU_TANH:
+        return float(torch.nn.functional.gelu(torch.tensor(z, dtype=torch.float64), approximate="tanh"))
+    return float(torch.nn.functional.silu(torch.tensor(z, dtype=torch.float64)))
+
+
+# ---------------------------------------------------------------- bf16 decode
+def test_bf16_decode_known_patterns():
+    # 0x3F80 = 1, 0xC000 = -2, 0x3FC0 = 1.5, 0x0001 = 2^-133 (denormal), 0x8000 = -0
+    pats = np.array([[0x3F80, 0xC000, 0x3FC0, 0x0001, 0x8000]], dtype=np.uint16).T.copy()  # X [5,1]
+    one = np.array([[0x3F80]], dtype=np.uint16)                                                # W [1,1] = 1
+    z = ref.fused_linear(pats, one, None, ref.ACT_NONE)[:, 0]
+    assert z.tolist() == [1.0, -2.0, 1.5, 2.0 ** -133, 0.0]
+
+
+# ---------------------------------------------------------------- GEMM core
+def test_hand_worked_example():
+    blocks, cur = {}, None
+    for line in open(os.path.join(GOLDEN, "gemm_2x3x4.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        tok = line.split()
+        if tok[0] in ("X", "W", "b", "Z"):
+            cur = tok[0]
+            blocks[cur] = []
+        else:
+            blocks[cur].append([float(t) for t in tok])
+    X, W, b, Z = (np.array(blocks[k]) for k in ("X", "W", "b", "Z"))
+    got = ref.fused_linear(bits(X), bits(W), b[0].astype(np.float32), ref.ACT_NONE)
+    assert got.shape == (2, 3)
+    assert np.array_equal(got, Z)
+    # and through the sampled entry point
+    rows, cols = np.array([0, 1, 1]), np.array([2, 0, 2])
+    pts = ref.fused_linear_points(bits(X), bits(W), b[0].astype(np.float32), ref.ACT_NONE, rows, cols)
+    assert pts.tolist() == [Z[0, 2], Z[1, 0], Z[1, 2]]
+
+
+@pytest.mark.parametrize("M,N,K", [(4, 4, 4), (3, 5, 7), (1, 1, 1), (2, 6, 3)])
+def test_exact_rational_brute_force(M, N, K):
+    vals = [0.0, 0.5, -0.5, 1.0, -1.0, 1.5, -1.5, 2.0, -2.0, 3.0, -3.0]
+    rng = np.random.default_rng(100 + M * 49 + N * 7 + K)
+    X = rng.choice(vals, size=(M, K))
+    W = rng.choice(vals, size=(N, K))
+    b = rng.choice([0.0, 0.25, -0.75, 1.0], size=N).astype(np.float32)
+    got = ref.fused_linear(bits(X), bits(W), b, ref.ACT_NONE)
+    for m in range(M):
+        for n in range(N):
+            exact = sum((Fraction(X[m, k]) * Fraction(W[n, k]) for k in range(K)), Fraction(float(b[n])))
+            assert Fraction(got[m, n]) == exact, (m, n)
+
+
+def test_identity_weight_gives_act_of_x_plus_b():
+    li = inputs.linear_inputs(9, 16, 16, seed=11)
+    eye = bits(np.eye(16))
+    Xd, b = widen(inputs.bf16_bits(li.X)), inputs.f32(li.b)
+    for kind in ACTS:
+        got = ref.fused_linear(inputs.bf16_bits(li.X), eye, b, kind)
+        want = np.array([[py_act(kind, Xd[m, n] + float(b[n])) for n in range(16)] for m in range(9)])
+        np.testing.assert_allclose(got, want, rtol=1e-14, atol=1e-15)
+
+
+def test_zero_input_gives_act_of_bias():
+    li = inputs.linear_inputs(5, 12, 24, seed=12)
+    X0 = np.zeros((5, 24), dtype=np.uint16)
+    b = inputs.f32(li.b)
+    for kind in ACTS:
+        got = ref.fused_linear(X0, inputs.bf16_bits(li.W), b, kind)
+        want = np.array([py_act(kind, float(v)) for v in b])
+        for m in range(5):
+            np.testing.assert_allclose(got[m], want, rtol=1e-14, atol=1e-16)
+
+
+def test_k_split_additivity_permutation_and_scaling():
+    li = inputs.linear_inputs(6, 10, 40, seed=13)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    z = ref.fused_linear(X, W, None, ref.ACT_NONE)
+    z1 = ref.fused_linear(X[:, :24].copy(), W[:, :24].copy(), None, ref.ACT_NONE)
+    z2 = ref.fused_linear(X[:, 24:].copy(), W[:, 24:].copy(), None, ref.ACT_NONE)
+    np.testing.assert_allclose(z, z1 + z2, rtol=0, atol=1e-13)
+    perm = np.random.default_rng(5).permutation(40)
+    zp = ref.fused_linear(X[:, perm].copy(), W[:, perm].copy(), None, ref.ACT_NONE)
+    np.testing.assert_allclose(z, zp, rtol=0, atol=1e-13)
+    nperm = np.random.default_rng(6).permutation(10)
+    zb = ref.fused_linear(X, W, b, ref.ACT_NONE)
+    zn = ref.fused_linear(X, W[nperm].copy(), b[nperm].copy(), ref.ACT_NONE)
+    assert np.array_equal(zn, zb[:, nperm])
+    W2 = bits(2.0 * widen(W))                      # doubling is exact in bf16
+    assert np.array_equal(ref.fused_linear(X, W2, None, ref.ACT_NONE), 2.0 * z)
+    # bias enters once, after the sum
+    np.testing.assert_allclose(zb - z, np.broadcast_to(b.astype(np.float64), z.shape), rtol=0, atol=1e-14)
+
+
+@pytest.mark.parametrize("M,N,K,seed", [(7, 13, 64, 21), (33, 5, 129, 22)])
+def test_against_torch_fp64_matmul(M, N, K, seed):
+    li = inputs.linear_inputs(M, N, K, seed=seed)
+    want = li.X.double() @ li.W.double().T + li.b.double()
+    got = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_NONE)
+    np.testing.assert_allclose(got, want.numpy(), rtol=0, atol=1e-12)
+    for kind, fn in [(ref.ACT_RELU, torch.relu),
+                     (ref.ACT_GELU_TANH, lambda t: torch.nn.functional.gelu(t, approximate="tanh")),
+                     (ref.ACT_SILU, torch.nn.functional.silu)]:
+        got = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), kind)
+        np.testing.assert_allclose(got, fn(want).numpy(), rtol=1e-12, atol=1e-13)
+
+
+# ---------------------------------------------------------------- activations
+def _closed_forms():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "closed_forms.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        kind, arg, val = line.split()
+        rows.append((kind, arg, float(val)))
+    return rows
+
+
+def test_activation_closed_forms():
+    ids = {"relu": ref.ACT_RELU, "gelu_tanh": ref.ACT_GELU_TANH, "silu": ref.ACT_SILU}
+    seen = 0
+    for kind, arg, val in _closed_forms():
+        if kind in ids:
+            got = ref.act(ids[kind], float(arg))
+            # 1 + tanh(.) cancels for very negative z: the formula in double carries ~1e-16 absolute error there
+            assert got == pytest.approx(val, rel=4e-15, abs=1e-15), (kind, arg)
+            seen += 1
+    assert seen == 39
+
+
+def test_activation_identities():
+    zs = np.linspace(-9.0, 9.0, 181)
+    for kind in (ref.ACT_RELU, ref.ACT_GELU_TANH, ref.ACT_SILU):
+        for z in zs:
+            # act(z) - act(-z) = z for ReLU, GELU-tanh (tanh odd) and SiLU (sigma(z)+sigma(-z)=1)
+            assert ref.act(kind, z) - ref.act(kind, -z) == pytest.approx(z, abs=1e-14)
+        assert ref.act(kind, 0.0) == 0.0
+        assert ref.act(kind, 40.0) == pytest.approx(40.0, rel=1e-15)
+        assert abs(ref.act(kind, -40.0)) < 1e-15
+    h = 1e-6   # slope one half at the origin for the two smooth activations
+    for kind in (ref.ACT_GELU_TANH, ref.ACT_SILU):
+        assert (ref.act(kind, h) - ref.act(kind, -h)) / (2 * h) == pytest.approx(0.5, abs=1e-9)
+    assert ref.act(ref.ACT_RELU, 2 * 1.7) == 2 * ref.act(ref.ACT_RELU, 1.7)
+    assert ref.act(ref.ACT_NONE, -3.25) == -3.25
+
+
+# ---------------------------------------------------------------- SwiGLU
+def test_swiglu_laws():
+    si = inputs.swiglu_inputs(6, 9, 32, seed=31)
+    X, Wg, Wu = (inputs.bf16_bits(t) for t in (si.X, si.Wg, si.Wu))
+    out = ref.swiglu(X, Wg, Wu)
+    # equal weights: silu(z) * z
+    z = ref.fused_linear(X, Wg, None, ref.ACT_NONE)
+    same = ref.swiglu(X, Wg, Wg)
+    want = torch.nn.functional.silu(torch.from_numpy(z)) * torch.from_numpy(z)
+    np.testing.assert_allclose(same, want.numpy(), rtol=1e-13, atol=1e-15)
+    zero = np.zeros_like(Wu)
+    assert np.all(ref.swiglu(X, Wg, zero) == 0.0)        # up = 0
+    assert np.all(ref.swiglu(X, zero, Wu) == 0.0)        # silu(0) = 0
+    Wu2 = bits(2.0 * widen(Wu))
+    assert np.array_equal(ref.swiglu(X, Wg, Wu2), 2.0 * out)
+    gate = ref.fused_linear(X, Wg, None, ref.ACT_SILU)
+    up = ref.fused_linear(X, Wu, None, ref.ACT_NONE)
+    assert np.array_equal(out, gate * up)
+    tw = torch.nn.functional.silu(si.X.double() @ si.Wg.double().T) * (si.X.double() @ si.Wu.double().T)
+    np.testing.assert_allclose(out, tw.numpy(), rtol=1e-12, atol=1e-13)
+    # gate and up are not interchangeable
+    assert not np.allclose(out, ref.swiglu(X, Wu, Wg))
+    rows, cols = np.array([0, 5, 3]), np.array([8, 0, 4])
+    assert np.array_equal(ref.swiglu_points(X, Wg, Wu, rows, cols), out[rows, cols])
+
+
+# ---------------------------------------------------------------- logsumexp
+def test_lse_closed_forms():
+    seen = 0
+    for kind, arg, val in _closed_forms():
+        if kind == "lse":
+            v = [float(t) for t in arg.split(",")]
+            assert ref.lse_vector(v) == pytest.approx(val, rel=4e-15), arg
+            seen += 1
+    assert seen == 6
+    assert ref.lse_vector([0, 0, 0, 0]) == pytest.approx(math.log(4.0), rel=1e-15)
+
+
+def test_lse_laws_on_vectors():
+    rng = np.random.default_rng(41)
+    z = rng.normal(size=200)
+    base = ref.lse_vector(z)
+    for c in (-700.0, -3.5, 12.25, 900.0):
+        assert ref.lse_vector(z + c) == pytest.approx(base + c, abs=1e-12 * max(1.0, abs(c)))   # shift law
+    assert np.sum(np.exp(z - base)) == pytest.approx(1.0, abs=1e-13)                           # softmax sums to 1
+    assert z.max() <= base <= z.max() + math.log(z.size)
+    assert ref.lse_vector(np.full(37, -2.5)) == pytest.approx(-2.5 + math.log(37), rel=1e-15)
+    assert ref.lse_vector([4.75]) == 4.75
+    assert ref.lse_vector(z[rng.permutation(200)]) == pytest.approx(base, abs=1e-13)
+    a, b = ref.lse_vector(z[:77]), ref.lse_vector(z[77:])                                     # merge law
+    assert math.log(math.exp(a) + math.exp(b)) == pytest.approx(base, abs=1e-13)
+    assert base == pytest.approx(float(torch.logsumexp(torch.from_numpy(z), 0)), abs=1e-13)
+
+
+def test_linear_lse_end_to_end():
+    li = inputs.linear_inputs(5, 300, 48, seed=42)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    lse, logits = ref.linear_lse(X, W, b, want_logits=True)
+    z = (li.X.double() @ li.W.double().T + li.b.double())
+    np.testing.assert_allclose(logits, z.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(lse, torch.logsumexp(z, -1).numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(np.exp(logits - lse[:, None]).sum(axis=1), np.ones(5), rtol=0, atol=1e-12)
+    # adding c to every bias shifts every lse by c (c exactly representable)
+    b_shift = (li.b.double() + 2.0).float().numpy()
+    exact_shift = b_shift.astype(np.float64) - b.astype(np.float64)   # what fp32 rounding really added per column
+    lse_s = ref.linear_lse(X, W, b_shift, False)
+    assert np.all(np.abs(lse_s - lse - 2.0) <= np.abs(exact_shift - 2.0).max() + 1e-12)
+    # zero weights: lse = lse(b); no bias and zero weights: ln N
+    W0 = np.zeros_like(W)
+    assert ref.linear_lse(X, W0, b, False)[0] == pytest.approx(ref.lse_vector(b.astype(np.float64)), abs=1e-13)
+    assert ref.linear_lse(X, W0, None, False)[3] == pytest.approx(math.log(300), rel=1e-15)
+    # N = 1: lse = z
+    l1 = ref.linear_lse(X, W[:1].copy(), b[:1].copy(), False)
+    np.testing.assert_allclose(l1, z.numpy()[:, 0], rtol=0, atol=1e-12)
+    rows = np.array([4, 0, 2])
+    np.testing.assert_array_equal(ref.linear_lse_rows(X, W, b, rows), lse[rows])
+
+
+def test_lse_expected_level_for_unit_variance_logits():
+    # logits ~ N(0,1) + small bias over N columns: lse ~ ln N + 1/2 (lognormal mean)
+    li = inputs.linear_inputs(4, 4000, 256, seed=43)
+    lse = ref.linear_lse(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b))
+    assert np.all(np.abs(lse - (math.log(4000) + 0.5)) < 0.15)
+
+
+# ---------------------------------------------------------------- sampled variants, threads, comparator
+def test_points_match_full_and_threads_do_not_matter():
+    li = inputs.linear_inputs(20, 31, 72, seed=51)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    rows, cols = inputs.sample_points(20, 31, 25, seed=3, tile_m=8, tile_n=8)
+    full = ref.fused_linear(X, W, b, ref.ACT_GELU_TANH)
+    assert np.array_equal(ref.fused_linear_points(X, W, b, ref.ACT_GELU_TANH, rows, cols), full[rows, cols])
+    ref.set_threads(1)
+    try:
+        assert np.array_equal(ref.fused_linear(X, W, b, ref.ACT_GELU_TANH), full)
+    finally:
+        ref.set_threads(0)
+    assert ref.get_threads() >= 1
+
+
+def test_bad_arguments_are_rejected():
+    X = np.zeros((2, 4), dtype=np.uint16)
+    W = np.zeros((3, 4), dtype=np.uint16)
+    with pytest.raises(ValueError):
+        ref.fused_linear(X, W, None, 7)
+    with pytest.raises(ValueError):
+        ref.fused_linear_points(X, W, None, 0, [2], [0])
+    with pytest.raises(TypeError):
+        ref.fused_linear(X.astype(np.float32), W, None, 0)
+
+
+def test_comparator():
+    refv = np.array([1.0, -2.0, 0.0, 100.0])
+    ok = ref.compare(refv + np.array([0.019, -0.029, 0.0099, 1.0]), refv, 1e-2, 1e-2)
+    assert ok["ok"] and ok["violations"] == 0 and ok["max_abs_err"] == pytest.approx(1.0)
+    bad = ref.compare(refv + np.array([0.021, 0.0, 0.0, 0.0]), refv, 1e-2, 1e-2)
+    assert not bad["ok"] and bad["violations"] == 1 and bad["worst_index"] == 0
+    nan = ref.compare(np.array([np.nan, 1.0]), np.array([0.0, 1.0]), 1.0, 1.0)
+    assert nan["violations"] == 1
+    inf = ref.compare(np.array([np.inf]), np.array([np.inf]), 1.0, 1.0)
+    assert inf["violations"] == 1
