@@ -1,0 +1,149 @@
+/* libmtmcfused -- B200 (sm_100a) fused linear layers:  Y = epilogue(X . W^T + b).
+ *
+ * The operator family is the "GEMM followed by an epilogue" class the paper's
+ * Level-2 fused-operator tasks stand for (Table "Details of KernelBench and
+ * TritonBench"; the Fusion, Tiling, Pipeline and Reordering principles of section
+ * "Optimization Principles"); correctness is the paper's Eq. 1 constraint: the
+ * result equals the high-level reference semantics of the operator sequence.
+ *
+ * Conventions shared by every entry point
+ *   - extern "C"; every function returns an int status (MTMC_OK = 0).
+ *   - X [M,K], W / Wg / Wu [N,K], out [M,N]: dense row-major.  "bf16" is the upper
+ *     16 bits of an IEEE-754 binary32.  b is binary32 [N]; b == NULL means no bias.
+ *   - Unless a function name ends in _host, every pointer is a DEVICE pointer on
+ *     the current CUDA device, 16-byte aligned, owned by the caller, and must stay
+ *     valid until the enqueued work has run.  Outputs must not alias inputs.
+ *   - Work is enqueued on the stream set by mtmc_set_stream() (default: the
+ *     legacy default stream) and the call returns without synchronising.
+ *     Argument errors are reported synchronously and enqueue nothing.  A device
+ *     side bounded wait that expires sets a sticky status that
+ *     mtmc_check_status() returns after synchronising the stream.
+ *   - Shapes: M, N, K >= 1 and K % 8 == 0 (a row of X or W must be a multiple of
+ *     16 bytes for the TMA descriptors).  Tails in M, N and K (K % 64 != 0) are
+ *     handled by TMA zero fill and predicated stores.  M, N, K < 2^31.
+ *   - Only compute capability 10.x is accepted; there is no fallback of any kind.
+ *   - Results are bit-reproducible run to run for a fixed shape and device.
+ *   - Scratch: split-K partial sums and logsumexp partials live in a workspace.
+ *     By default the library owns one per device (cudaMalloc, grow-only; so the
+ *     first call of a larger shape allocates and must not run under stream
+ *     capture); mtmc_set_workspace() substitutes caller-owned memory.
+ */
+#ifndef MTMC_FUSED_H_
+#define MTMC_FUSED_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define MTMC_OK 0
+#define MTMC_ERR_INVALID_ARG 1        /* null / misaligned pointer, M/N/K <= 0, unknown enum */
+#define MTMC_ERR_UNSUPPORTED_SHAPE 2  /* K % 8 != 0, or a dimension >= 2^31 */
+#define MTMC_ERR_UNSUPPORTED_DEVICE 3 /* not compute capability 10.x */
+#define MTMC_ERR_CUDA 4               /* CUDA runtime / driver error; text in mtmc_last_error() */
+#define MTMC_ERR_DEVICE_TIMEOUT 5     /* a bounded device-side wait expired */
+#define MTMC_ERR_WORKSPACE 6          /* caller-provided workspace too small */
+
+/* activation ids for mtmc_fused_linear */
+#define MTMC_ACT_NONE 0
+#define MTMC_ACT_RELU 1
+#define MTMC_ACT_GELU_TANH 2 /* 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))) */
+#define MTMC_ACT_SILU 3      /* z / (1 + exp(-z)) */
+
+/* output element types for mtmc_fused_linear */
+#define MTMC_OUT_FP32 0
+#define MTMC_OUT_BF16 1 /* round to nearest even, once, at the final store */
+
+/* operation ids for mtmc_workspace_bytes */
+#define MTMC_OP_FUSED_LINEAR 0
+#define MTMC_OP_SWIGLU 1
+#define MTMC_OP_LINEAR_LSE 2
+
+/* out[m][n] = act( sum_k X[m][k] W[n][k] + b[n] ).
+ * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
+ * the bias add and activation happen in fp32 on the fp32 accumulator, with no
+ * intermediate rounding.)  X, W bf16; b fp32 or NULL; out fp32 or bf16 [M,N]
+ * according to out_dtype.  Shapes with M <= 16 and a long K take the split-K
+ * weight-streaming path (HBM-bound decode shape); all others the tiled
+ * tensor-core path.  Needs workspace only on the split-K path. */
+int mtmc_fused_linear(const void* X, const void* W, const float* b,
+                      int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+
+/* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
+ * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate
+ * product fused in one kernel; neither GEMM result is written to memory.) */
+int mtmc_swiglu(const void* X, const void* Wg, const void* Wu,
+                int64_t M, int64_t N, int64_t K, void* out);
+
+/* lse_out[m] = log sum_n exp( sum_k X[m][k] W[n][k] + b[n] ),  fp32 [M].
+ * (A row reduction fused into a linear layer -- the paper's own example of a
+ * semantic action is fusing a linear with a row maximum, section "Training
+ * Process".  The M x N logits are never written to memory: each tile keeps an
+ * online (max, sum-exp) per row, partials go to the workspace and are merged.)
+ * Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_LSE, M, N, K) bytes of workspace. */
+int mtmc_linear_lse(const void* X, const void* W, const float* b,
+                    int64_t M, int64_t N, int64_t K, float* lse_out);
+
+/* Same three operations with every pointer a HOST pointer (pageable or pinned).
+ * The library copies the operands to device buffers it owns (cudaMalloc,
+ * grow-only, per device), runs the device entry point on the current stream,
+ * copies the result back and synchronises the stream before returning.  These
+ * allocate and synchronise; they are a convenience for callers without device
+ * memory management and the end-to-end leg of the benchmark.  (No counterpart in
+ * the paper: its measurements are device-resident.) */
+int mtmc_fused_linear_host(const void* X, const void* W, const float* b,
+                           int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+int mtmc_swiglu_host(const void* X, const void* Wg, const void* Wu,
+                     int64_t M, int64_t N, int64_t K, void* out);
+int mtmc_linear_lse_host(const void* X, const void* W, const float* b,
+                         int64_t M, int64_t N, int64_t K, float* lse_out);
+
+/* Stream on which later calls from this host thread enqueue (a cudaStream_t;
+ * NULL = legacy default stream).  Thread-local. */
+int mtmc_set_stream(void* cuda_stream);
+
+/* Use caller-owned device scratch instead of the library's own.  dptr must be
+ * 256-byte aligned and stay valid while calls are in flight; (NULL, 0) returns to
+ * library-owned scratch.  A call whose requirement exceeds `bytes` fails with
+ * MTMC_ERR_WORKSPACE.  Calls in flight on different streams must not share one
+ * workspace.  Thread-local. */
+int mtmc_set_workspace(void* dptr, size_t bytes);
+
+/* Scratch bytes the given operation needs for this shape on the current device
+ * (0 if none; (size_t)-1 on invalid arguments). */
+size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
+
+/* Synchronises the current stream, then returns and clears the sticky device
+ * status (MTMC_OK, MTMC_ERR_DEVICE_TIMEOUT or MTMC_ERR_CUDA). */
+int mtmc_check_status(void);
+
+/* Text for the last non-OK status returned on this host thread ("" if none). */
+const char* mtmc_last_error(void);
+
+/* Number of kernels this library has launched from this process so far. */
+int64_t mtmc_launch_count(void);
+
+/* Device time, in milliseconds, of the most recent mtmc_* device entry point on
+ * this host thread's current device, measured with CUDA events recorded on the
+ * launching stream around the library's kernels.  Synchronises on the end event.
+ * Timing is recorded only while enabled with mtmc_set_timing(1).
+ * Returns a negative value if no timed call has been made. */
+int mtmc_set_timing(int enabled);
+float mtmc_last_kernel_ms(void);
+
+/* Tuning hooks (0 / negative = automatic).  They select among kernels of this
+ * library only; results stay within tolerance of each other.
+ *   split_k : number of K splits requested on the skinny path
+ *   tile_n  : 128 or 256, accumulator tile width of the tiled path          */
+int mtmc_set_tuning(int split_k, int tile_n);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int mtmc_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MTMC_FUSED_H_ */

@@ -1,0 +1,202 @@
+"""Thin ctypes binding to libmtmcfused.so: argument marshalling only.
+
+Same names as the C ABI (include/mtmc_fused.h).  torch supplies device memory and
+the stream; every step of the computation runs inside the library's kernels.
+There is no fallback: a missing library, a missing GPU or a non-Blackwell GPU is
+an error.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmtmcfused.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_WORKSPACE = 1, 2, 3, 4, 5, 6
+ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}
+OUT_DTYPE = {"fp32": 0, "bf16": 1}
+OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2}
+
+EXPORTS = [
+    "mtmc_fused_linear", "mtmc_swiglu", "mtmc_linear_lse",
+    "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
+    "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
+    "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
+    "mtmc_set_tuning", "mtmc_version",
+]
+
+_lib = None
+
+
+class MtmcError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("libmtmcfused status %d: %s" % (status, message))
+        self.status = status
+
+
+def load() -> ctypes.CDLL:
+    """Loads the library (built in-tree by paper_2511_20100_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libmtmcfused.so is missing at %s: build it with "
+                           "`python -m paper_2511_20100_b200.build` (there is no fallback path)" % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+    for name in ("mtmc_fused_linear", "mtmc_fused_linear_host"):
+        getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host"):
+        getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    L.mtmc_set_stream.argtypes = [vp]
+    L.mtmc_set_workspace.argtypes = [vp, sz]
+    L.mtmc_workspace_bytes.argtypes = [ci, i64, i64, i64]
+    L.mtmc_workspace_bytes.restype = sz
+    L.mtmc_last_error.restype = ctypes.c_char_p
+    L.mtmc_launch_count.restype = i64
+    L.mtmc_set_timing.argtypes = [ci]
+    L.mtmc_last_kernel_ms.restype = ctypes.c_float
+    L.mtmc_set_tuning.argtypes = [ci, ci]
+    _lib = L
+    return L
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise MtmcError(rc, load().mtmc_last_error().decode())
+
+
+def _dev(t: torch.Tensor, dtype, shape, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise TypeError("%s must be contiguous %s of shape %r (got %s %r)" % (name, dtype, tuple(shape), t.dtype, tuple(t.shape)))
+    return t.data_ptr()
+
+
+def _use_current_stream(device) -> None:
+    torch.cuda.set_device(device)
+    load().mtmc_set_stream(ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream))
+
+
+def mtmc_fused_linear(X, W, b, act="none", out_dtype="bf16", out=None):
+    """out = act(X @ W.T + b) on the current CUDA stream; X [M,K], W [N,K] bf16, b [N] fp32 or None."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_fused_linear(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                    None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                    M, N, K, ACT[act], OUT_DTYPE[out_dtype], _dev(out, odt, (M, N), "out")))
+    return out
+
+
+def mtmc_swiglu(X, Wg, Wu, out=None):
+    """out = silu(X @ Wg.T) * (X @ Wu.T), bf16 [M,N]."""
+    M, K = X.shape
+    N = Wg.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_swiglu(_dev(X, torch.bfloat16, (M, K), "X"), _dev(Wg, torch.bfloat16, (N, K), "Wg"),
+                              _dev(Wu, torch.bfloat16, (N, K), "Wu"), M, N, K, _dev(out, torch.bfloat16, (M, N), "out")))
+    return out
+
+
+def mtmc_linear_lse(X, W, b, lse_out=None):
+    """lse_out[m] = logsumexp_n(X @ W.T + b), fp32 [M]; the logits are never materialised."""
+    M, K = X.shape
+    N = W.shape[0]
+    if lse_out is None:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_linear_lse(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                  None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                  M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
+
+
+def _host(t: torch.Tensor, dtype, shape, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or t.is_cuda:
+        raise TypeError("%s must be a CPU tensor" % name)
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or not t.is_contiguous():
+        raise TypeError("%s must be contiguous %s of shape %r" % (name, dtype, tuple(shape)))
+    return t.data_ptr()
+
+
+def mtmc_fused_linear_host(X, W, b, act="none", out_dtype="bf16", out=None, device=0):
+    """Host-pointer variant: CPU tensors in, CPU tensor out; copies and synchronises inside the library."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt)
+    _use_current_stream(torch.device("cuda", device))
+    _check(load().mtmc_fused_linear_host(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
+                                         None if b is None else _host(b, torch.float32, (N,), "b"),
+                                         M, N, K, ACT[act], OUT_DTYPE[out_dtype], _host(out, odt, (M, N), "out")))
+    return out
+
+
+def mtmc_swiglu_host(X, Wg, Wu, out=None, device=0):
+    M, K = X.shape
+    N = Wg.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16)
+    _use_current_stream(torch.device("cuda", device))
+    _check(load().mtmc_swiglu_host(_host(X, torch.bfloat16, (M, K), "X"), _host(Wg, torch.bfloat16, (N, K), "Wg"),
+                                   _host(Wu, torch.bfloat16, (N, K), "Wu"), M, N, K, _host(out, torch.bfloat16, (M, N), "out")))
+    return out
+
+
+def mtmc_linear_lse_host(X, W, b, lse_out=None, device=0):
+    M, K = X.shape
+    N = W.shape[0]
+    if lse_out is None:
+        lse_out = torch.empty((M,), dtype=torch.float32)
+    _use_current_stream(torch.device("cuda", device))
+    _check(load().mtmc_linear_lse_host(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
+                                       None if b is None else _host(b, torch.float32, (N,), "b"),
+                                       M, N, K, _host(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
+
+
+def mtmc_set_workspace(t: torch.Tensor | None) -> None:
+    if t is None:
+        _check(load().mtmc_set_workspace(None, 0))
+    else:
+        _check(load().mtmc_set_workspace(ctypes.c_void_p(t.data_ptr()), t.numel() * t.element_size()))
+
+
+def mtmc_workspace_bytes(op: str, M: int, N: int, K: int) -> int:
+    return int(load().mtmc_workspace_bytes(OP[op], M, N, K))
+
+
+def mtmc_check_status() -> None:
+    _check(load().mtmc_check_status())
+
+
+def mtmc_launch_count() -> int:
+    return int(load().mtmc_launch_count())
+
+
+def mtmc_set_timing(enabled: bool) -> None:
+    load().mtmc_set_timing(1 if enabled else 0)
+
+
+def mtmc_last_kernel_ms() -> float:
+    return float(load().mtmc_last_kernel_ms())
+
+
+def mtmc_set_tuning(split_k: int = 0, tile_n: int = 0) -> None:
+    _check(load().mtmc_set_tuning(int(split_k), int(tile_n)))
+
+
+def mtmc_version() -> int:
+    return int(load().mtmc_version())

@@ -1,0 +1,508 @@
+// libmtmcfused: the C-ABI boundary (see include/mtmc_fused.h).  Host side only:
+// argument validation, per-device state, TMA descriptor encoding, kernel selection
+// by shape and launches.  All arithmetic is in the kernels.
+#include "../../include/mtmc_fused.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include "skinny.cuh"
+
+namespace {
+
+using namespace mtmc;
+
+constexpr int MAX_DEVICES = 64;
+constexpr size_t TICKET_BYTES = 64 * 1024;   // library-owned split-K tickets: 16384 tiles
+constexpr int SKINNY_MAX_M = 16;
+
+struct DeviceState {
+    bool ready = false;
+    int sm_count = 0;
+    uint32_t* status = nullptr;      // device status word (256 bytes reserved)
+    uint32_t* tickets = nullptr;     // library-owned split-K tickets, zero between launches
+    bool tickets_dirty = false;
+    void* ws = nullptr;              // library-owned workspace (grow-only)
+    size_t ws_bytes = 0;
+    void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // device copies for the *_host calls
+    size_t stage_bytes[5] = {0, 0, 0, 0, 0};
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    bool timed = false;
+};
+
+std::mutex g_mutex;
+DeviceState g_dev[MAX_DEVICES];
+std::atomic<long long> g_launches{0};
+
+thread_local cudaStream_t t_stream = nullptr;
+thread_local void* t_user_ws = nullptr;
+thread_local size_t t_user_ws_bytes = 0;
+thread_local int t_split_k = 0;
+thread_local int t_tile_n = 0;
+thread_local int t_timing = 0;
+thread_local char t_error[512] = "";
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int fail(int code, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(t_error, sizeof t_error, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CUDA_TRY(expr)                                                                      \
+    do {                                                                                    \
+        cudaError_t e_ = (expr);                                                            \
+        if (e_ != cudaSuccess) return fail(MTMC_ERR_CUDA, "%s: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+int get_device(DeviceState** out, int* dev_out = nullptr) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return fail(MTMC_ERR_UNSUPPORTED_DEVICE, "device index %d out of range", dev);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& d = g_dev[dev];
+    if (!d.ready) {
+        int major = 0, minor = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+        if (major != 10)
+            return fail(MTMC_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d: this library only runs on 10.x (B200)", major, minor);
+        CUDA_TRY(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+            if (!fn || qres != cudaDriverEntryPointSuccess)
+                return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        CUDA_TRY(cudaMalloc(&d.status, 256));
+        CUDA_TRY(cudaMemset(d.status, 0, 256));
+        CUDA_TRY(cudaMalloc(&d.tickets, TICKET_BYTES));
+        CUDA_TRY(cudaMemset(d.tickets, 0, TICKET_BYTES));
+        CUDA_TRY(cudaEventCreate(&d.ev0));
+        CUDA_TRY(cudaEventCreate(&d.ev1));
+        d.ready = true;
+    }
+    *out = &d;
+    if (dev_out) *dev_out = dev;
+    return MTMC_OK;
+}
+
+// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
+int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+    cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+    return MTMC_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_common(const void* X, const void* W, const void* out, int64_t M, int64_t N, int64_t K) {
+    if (!X || !W || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive (got %lld, %lld, %lld)",
+                                                 (long long)M, (long long)N, (long long)K);
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31))
+        return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "dimensions must be below 2^31");
+    if (K % 8 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 8 (16-byte rows for TMA)", (long long)K);
+    if (!aligned16(X) || !aligned16(W) || !aligned16(out)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    return MTMC_OK;
+}
+
+// Scratch for this call: the caller's if set, else the library's (grown on demand).
+int get_workspace(DeviceState* d, size_t need, void** out) {
+    if (need == 0) { *out = nullptr; return MTMC_OK; }
+    if (t_user_ws) {
+        if (t_user_ws_bytes < need)
+            return fail(MTMC_ERR_WORKSPACE, "workspace of %zu bytes given, %zu needed", t_user_ws_bytes, need);
+        *out = t_user_ws;
+        return MTMC_OK;
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (d->ws_bytes < need) {
+        if (d->ws) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(d->ws)); d->ws = nullptr; d->ws_bytes = 0; }
+        size_t bytes = (need + (1u << 20) - 1) & ~static_cast<size_t>((1u << 20) - 1);
+        CUDA_TRY(cudaMalloc(&d->ws, bytes));
+        d->ws_bytes = bytes;
+    }
+    *out = d->ws;
+    return MTMC_OK;
+}
+
+size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+
+int pick_tile_n(int64_t N) {
+    if (t_tile_n == 128 || t_tile_n == 256) return t_tile_n;
+    return N > 128 ? 256 : 128;
+}
+
+int pick_group_m(int m_tiles) { return m_tiles < 16 ? m_tiles : 16; }
+
+struct TimedRegion {
+    DeviceState* d;
+    bool on;
+    TimedRegion(DeviceState* dev) : d(dev), on(t_timing != 0) {
+        if (on) cudaEventRecord(d->ev0, t_stream);
+    }
+    void stop() {
+        if (on) { cudaEventRecord(d->ev1, t_stream); d->timed = true; }
+    }
+};
+
+template <int EPI, int BN, bool OUT_BF16>
+int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, GemmParams p) {
+    using Cfg = TileCfg<EPI, BN>;
+    auto kern = gemm_tiled_kernel<EPI, BN, OUT_BF16>;
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB2, p);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
+void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n) {
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.m_tiles = static_cast<int>((M + 127) / 128);
+    p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
+    p.num_tiles = p.m_tiles * p.n_tiles;
+    p.k_blocks = static_cast<int>((K + 63) / 64);
+    p.group_m = pick_group_m(p.m_tiles);
+}
+
+int skinny_cta_of_unit_host(long long u, long long total, int grid) {
+    return static_cast<int>(((u + 1) * grid - 1) / total);
+}
+
+struct SkinnyPlan {
+    int n_tiles, k_blocks, grid, max_slots;
+    long long total;
+    size_t ticket_bytes, partial_bytes;
+};
+
+SkinnyPlan plan_skinny(int sm_count, int64_t N, int64_t K) {
+    SkinnyPlan s;
+    s.n_tiles = static_cast<int>((N + 127) / 128);
+    s.k_blocks = static_cast<int>((K + 63) / 64);
+    s.total = static_cast<long long>(s.n_tiles) * s.k_blocks;
+    long long g = t_split_k > 0 ? static_cast<long long>(s.n_tiles) * t_split_k : sm_count;
+    if (g > s.total) g = s.total;
+    if (g > 65535 * 16) g = 65535 * 16;
+    s.grid = static_cast<int>(g);
+    int mx = 1;
+    for (int t = 0; t < s.n_tiles; ++t) {
+        long long first = static_cast<long long>(t) * s.k_blocks;
+        int nc = skinny_cta_of_unit_host(first + s.k_blocks - 1, s.total, s.grid) - skinny_cta_of_unit_host(first, s.total, s.grid) + 1;
+        if (nc > mx) mx = nc;
+    }
+    s.max_slots = mx;
+    s.ticket_bytes = round256(static_cast<size_t>(s.n_tiles) * 4);
+    s.partial_bytes = static_cast<size_t>(s.n_tiles) * s.max_slots * 16 * 128 * 4;
+    return s;
+}
+
+bool use_skinny(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 127) / 128 <= static_cast<int64_t>(TICKET_BYTES / 4); }
+
+int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
+               int out_dtype, void* out) {
+    SkinnyPlan s = plan_skinny(d->sm_count, N, K);
+    SkinnyParams p;
+    p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
+    p.act = act; p.bias = b; p.out = out; p.status = d->status;
+    void* ws = nullptr;
+    if (t_user_ws) {
+        int rc = get_workspace(d, s.ticket_bytes + s.partial_bytes, &ws);
+        if (rc) return rc;
+        p.tickets = static_cast<uint32_t*>(ws);
+        p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + s.ticket_bytes);
+        CUDA_TRY(cudaMemsetAsync(p.tickets, 0, s.ticket_bytes, t_stream));
+    } else {
+        int rc = get_workspace(d, s.partial_bytes, &ws);
+        if (rc) return rc;
+        p.tickets = d->tickets;
+        p.partial = static_cast<float*>(ws);
+        if (d->tickets_dirty) {
+            CUDA_TRY(cudaMemsetAsync(d->tickets, 0, TICKET_BYTES, t_stream));
+            d->tickets_dirty = false;
+        }
+    }
+    CUtensorMap tmW, tmX;
+    int rc = encode_bf16_2d(&tmW, W, N, K, SkinnyCfg::BNW);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmX, X, M, K, SkinnyCfg::MX);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    if (out_dtype == MTMC_OUT_BF16) {
+        auto kern = skinny_splitk_kernel<true>;
+        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
+        kern<<<s.grid, 192, SkinnyCfg::SMEM_BYTES, t_stream>>>(tmW, tmX, p);
+    } else {
+        auto kern = skinny_splitk_kernel<false>;
+        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
+        kern<<<s.grid, 192, SkinnyCfg::SMEM_BYTES, t_stream>>>(tmW, tmX, p);
+    }
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    tr.stop();
+    return MTMC_OK;
+}
+
+// Device buffer i of the *_host entry points, at least `bytes` large.
+int stage_buffer(DeviceState* d, int i, size_t bytes, void** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (d->stage_bytes[i] < bytes) {
+        if (d->stage[i]) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(d->stage[i])); d->stage[i] = nullptr; d->stage_bytes[i] = 0; }
+        CUDA_TRY(cudaMalloc(&d->stage[i], bytes));
+        d->stage_bytes[i] = bytes;
+    }
+    *out = d->stage[i];
+    return MTMC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mtmc_version(void) { return 100; }
+
+int mtmc_set_stream(void* cuda_stream) {
+    t_stream = static_cast<cudaStream_t>(cuda_stream);
+    return MTMC_OK;
+}
+
+int mtmc_set_workspace(void* dptr, size_t bytes) {
+    if (dptr == nullptr) { t_user_ws = nullptr; t_user_ws_bytes = 0; return MTMC_OK; }
+    if ((reinterpret_cast<uintptr_t>(dptr) & 255u) != 0) return fail(MTMC_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    t_user_ws = dptr;
+    t_user_ws_bytes = bytes;
+    return MTMC_OK;
+}
+
+int mtmc_set_tuning(int split_k, int tile_n) {
+    if (tile_n > 0 && tile_n != 128 && tile_n != 256) return fail(MTMC_ERR_INVALID_ARG, "tile_n must be 128 or 256");
+    t_split_k = split_k > 0 ? split_k : 0;
+    t_tile_n = tile_n > 0 ? tile_n : 0;
+    return MTMC_OK;
+}
+
+int mtmc_set_timing(int enabled) { t_timing = enabled ? 1 : 0; return MTMC_OK; }
+
+float mtmc_last_kernel_ms(void) {
+    DeviceState* d = nullptr;
+    if (get_device(&d) != MTMC_OK || !d->timed) return -1.0f;
+    if (cudaEventSynchronize(d->ev1) != cudaSuccess) return -1.0f;
+    float ms = -1.0f;
+    if (cudaEventElapsedTime(&ms, d->ev0, d->ev1) != cudaSuccess) return -1.0f;
+    return ms;
+}
+
+int64_t mtmc_launch_count(void) { return g_launches.load(); }
+
+const char* mtmc_last_error(void) { return t_error; }
+
+size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
+    if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
+    switch (op) {
+        case MTMC_OP_FUSED_LINEAR: {
+            if (!use_skinny(M, N)) return 0;
+            DeviceState* d = nullptr;
+            if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
+            SkinnyPlan s = plan_skinny(d->sm_count, N, K);
+            return s.ticket_bytes + s.partial_bytes;
+        }
+        case MTMC_OP_SWIGLU: return 0;
+        case MTMC_OP_LINEAR_LSE: return round256(static_cast<size_t>((N + 127) / 128) * static_cast<size_t>(M) * sizeof(float2));
+        default: return static_cast<size_t>(-1);
+    }
+}
+
+int mtmc_check_status(void) {
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    uint32_t st = 0;
+    CUDA_TRY(cudaMemcpy(&st, d->status, sizeof st, cudaMemcpyDeviceToHost));
+    if (st != 0) {
+        CUDA_TRY(cudaMemset(d->status, 0, sizeof st));
+        d->tickets_dirty = true;
+        return fail(MTMC_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (status word 0x%x)", st);
+    }
+    return MTMC_OK;
+}
+
+int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
+                      int out_dtype, void* out) {
+    int rc = check_common(X, W, out, M, N, K);
+    if (rc) return rc;
+    if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    rc = get_device(&d);
+    if (rc) return rc;
+    if (use_skinny(M, N)) return run_skinny(d, X, W, b, M, N, K, act, out_dtype, out);
+
+    const int bn = pick_tile_n(N);
+    GemmParams p{};
+    fill_tiling(p, M, N, K, bn);
+    p.act = act; p.bias = b; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    CUtensorMap tmA, tmB;
+    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmB, W, N, K, bn);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    if (bn == 256) {
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, p)
+                                        : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, p);
+    } else {
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, p)
+                                        : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, p);
+    }
+    tr.stop();
+    return rc;
+}
+
+int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
+    int rc = check_common(X, Wg, out, M, N, K);
+    if (rc) return rc;
+    if (!Wu) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(Wu)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    rc = get_device(&d);
+    if (rc) return rc;
+    GemmParams p{};
+    fill_tiling(p, M, N, K, 128);               // 128 output columns = 128 gate + 128 up accumulator columns
+    p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    CUtensorMap tmA, tmG, tmU;
+    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmG, Wg, N, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmU, Wu, N, K, 128);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, p);
+    tr.stop();
+    return rc;
+}
+
+int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
+    int rc = check_common(X, W, lse_out, M, N, K);
+    if (rc) return rc;
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    rc = get_device(&d);
+    if (rc) return rc;
+    const int bn = pick_tile_n(N);
+    GemmParams p{};
+    fill_tiling(p, M, N, K, bn);
+    void* ws = nullptr;
+    rc = get_workspace(d, round256(static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M) * sizeof(float2)), &ws);
+    if (rc) return rc;
+    p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
+    CUtensorMap tmA, tmB;
+    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmB, W, N, K, bn);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    rc = bn == 256 ? launch_tiled<EPI_LSE, 256, false>(d, tmA, tmB, tmB, p) : launch_tiled<EPI_LSE, 128, false>(d, tmA, tmB, tmB, p);
+    tr.stop();
+    if (rc) return rc;
+    const int rows_per_block = 8;
+    lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
+        p.lse_partial, p.M, p.n_tiles, lse_out);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
+// ---------------------------------------------------------------------------- host-pointer variants
+int mtmc_fused_linear_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
+                           int out_dtype, void* out) {
+    if (!X || !W || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
+    const size_t ob = static_cast<size_t>(M) * N * (out_dtype == MTMC_OUT_BF16 ? 2 : 4);
+    void *dX, *dW, *dB = nullptr, *dO;
+    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dW)) || (rc = stage_buffer(d, 4, ob, &dO))) return rc;
+    if (b && (rc = stage_buffer(d, 3, bb, &dB))) return rc;
+    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
+    CUDA_TRY(cudaMemcpyAsync(dW, W, wb, cudaMemcpyHostToDevice, t_stream));
+    if (b) CUDA_TRY(cudaMemcpyAsync(dB, b, bb, cudaMemcpyHostToDevice, t_stream));
+    rc = mtmc_fused_linear(dX, dW, static_cast<const float*>(dB), M, N, K, act, out_dtype, dO);
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
+    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    return MTMC_OK;
+}
+
+int mtmc_swiglu_host(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
+    if (!X || !Wg || !Wu || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, ob = static_cast<size_t>(M) * N * 2;
+    void *dX, *dG, *dU, *dO;
+    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dG)) || (rc = stage_buffer(d, 2, wb, &dU)) ||
+        (rc = stage_buffer(d, 4, ob, &dO)))
+        return rc;
+    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
+    CUDA_TRY(cudaMemcpyAsync(dG, Wg, wb, cudaMemcpyHostToDevice, t_stream));
+    CUDA_TRY(cudaMemcpyAsync(dU, Wu, wb, cudaMemcpyHostToDevice, t_stream));
+    rc = mtmc_swiglu(dX, dG, dU, M, N, K, dO);
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
+    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    return MTMC_OK;
+}
+
+int mtmc_linear_lse_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
+    if (!X || !W || !lse_out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
+    const size_t ob = static_cast<size_t>(M) * 4;
+    void *dX, *dW, *dB = nullptr, *dO;
+    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dW)) || (rc = stage_buffer(d, 4, ob, &dO))) return rc;
+    if (b && (rc = stage_buffer(d, 3, bb, &dB))) return rc;
+    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
+    CUDA_TRY(cudaMemcpyAsync(dW, W, wb, cudaMemcpyHostToDevice, t_stream));
+    if (b) CUDA_TRY(cudaMemcpyAsync(dB, b, bb, cudaMemcpyHostToDevice, t_stream));
+    rc = mtmc_linear_lse(dX, dW, static_cast<const float*>(dB), M, N, K, static_cast<float*>(dO));
+    if (rc) return rc;
+    CUDA_TRY(cudaMemcpyAsync(lse_out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
+    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    return MTMC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,373 @@
+// The tiled tensor-core path: persistent, warp-specialised CTAs, one per SM.
+//
+//   warp 0 (one lane)  TMA producer: X and W tiles, HBM/L2 -> 128B-swizzled shared
+//                      memory ring, mbarrier full/empty per stage  (Pipeline principle)
+//   warp 1 (one lane)  tcgen05.mma issuer: 128 x BN x 16 bf16 MMAs accumulating fp32
+//                      in tensor memory; two accumulator buffers so the next tile's
+//                      mainloop overlaps this tile's epilogue     (Tiling principle)
+//   warps 2-5          epilogue: tcgen05.ld -> registers -> bias / activation / gate
+//                      product / row (max, sum-exp) -> global     (Fusion principle)
+//
+// Tile order walks M fastest inside groups of group_m row blocks so that the CTAs
+// running at the same time share W tiles through L2 (Reordering principle).
+#pragma once
+#include "ptx.cuh"
+
+namespace mtmc {
+
+enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2 };
+enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
+
+struct GemmParams {
+    int M, N, K;
+    int m_tiles, n_tiles, num_tiles, k_blocks;
+    int group_m;
+    int act;
+    const float* bias;    // [N] or null
+    void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
+    float2* lse_partial;  // [n_tiles][M] (max, sum-exp) per row and column tile (EPI_LSE)
+    uint32_t* status;     // device status word
+};
+
+template <int EPI, int BN>
+struct TileCfg {
+    static constexpr int BM = 128;                       // accumulator rows = TMEM lanes
+    static constexpr int BK = 64;                        // one 128-byte swizzle row of bf16
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : 6;
+    static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
+    static constexpr int TMEM_COLS = 2 * BN;             // two accumulator buffers
+    static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;  // + alignment slack
+    static constexpr int THREADS = 192;
+};
+
+__device__ __forceinline__ void tile_coords(const GemmParams& p, int idx, int& mb, int& nb) {
+    const int per_group = p.group_m * p.n_tiles;
+    const int g = idx / per_group;
+    const int r = idx - g * per_group;
+    const int m_first = g * p.group_m;
+    const int gm = min(p.group_m, p.m_tiles - m_first);
+    nb = r / gm;
+    mb = m_first + (r - nb * gm);
+}
+
+// z / (1 + exp(-z))
+__device__ __forceinline__ float silu_f(float z) {
+    return z * rcp_approx(1.0f + ex2_approx(-1.4426950408889634f * z));
+}
+// 0.5 z (1 + tanh(u)) = z * sigmoid(2u),  u = sqrt(2/pi) (z + 0.044715 z^3)
+__device__ __forceinline__ float gelu_tanh_f(float z) {
+    const float u2 = 1.5957691216057308f * z * fmaf(0.044715f * z, z, 1.0f);   // 2u
+    return z * rcp_approx(1.0f + ex2_approx(-1.4426950408889634f * u2));
+}
+__device__ __forceinline__ float apply_act(int act, float z) {
+    switch (act) {
+        case ACT_RELU: return fmaxf(z, 0.0f);
+        case ACT_GELU_TANH: return gelu_tanh_f(z);
+        case ACT_SILU: return silu_f(z);
+        default: return z;
+    }
+}
+
+__device__ __forceinline__ void apply_act_chunk(int act, float (&y)[32]) {
+    if (act == ACT_RELU) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) y[j] = fmaxf(y[j], 0.0f);
+    } else if (act == ACT_GELU_TANH) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) y[j] = gelu_tanh_f(y[j]);
+    } else if (act == ACT_SILU) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) y[j] = silu_f(y[j]);
+    }
+}
+
+// Stores 32 consecutive columns [n0, n0+32) of one output row; 128-bit stores when
+// the row segment is whole and 16-byte aligned, predicated scalar stores otherwise.
+template <bool OUT_BF16>
+__device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int N, const float (&y)[32], bool vec_ok) {
+    if (OUT_BF16) {
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N + n0;
+        if (vec_ok && n0 + 32 <= N) {
+            uint4* o4 = reinterpret_cast<uint4*>(o);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                uint4 q;
+                q.x = pack_bf16x2(y[8 * v + 0], y[8 * v + 1]);
+                q.y = pack_bf16x2(y[8 * v + 2], y[8 * v + 3]);
+                q.z = pack_bf16x2(y[8 * v + 4], y[8 * v + 5]);
+                q.w = pack_bf16x2(y[8 * v + 6], y[8 * v + 7]);
+                o4[v] = q;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (n0 + j < N) o[j] = __float2bfloat16_rn(y[j]);
+        }
+    } else {
+        float* o = reinterpret_cast<float*>(out) + static_cast<size_t>(row) * N + n0;
+        if (vec_ok && n0 + 32 <= N) {
+            float4* o4 = reinterpret_cast<float4*>(o);
+#pragma unroll
+            for (int v = 0; v < 8; ++v) o4[v] = make_float4(y[4 * v], y[4 * v + 1], y[4 * v + 2], y[4 * v + 3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (n0 + j < N) o[j] = y[j];
+        }
+    }
+}
+
+// Loads bias[n0 .. n0+32) into registers (zeros past N or without bias).
+__device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N, float (&b)[32]) {
+    if (bias == nullptr) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) b[j] = 0.0f;
+    } else if (n0 + 32 <= N) {
+        const float4* b4 = reinterpret_cast<const float4*>(bias + n0);
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+            const float4 t = __ldg(b4 + v);
+            b[4 * v] = t.x; b[4 * v + 1] = t.y; b[4 * v + 2] = t.z; b[4 * v + 3] = t.w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) b[j] = (n0 + j < N) ? __ldg(bias + n0 + j) : 0.0f;
+    }
+}
+
+template <int EPI, int BN, bool OUT_BF16>
+__global__ void __launch_bounds__(192, 1)
+gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                  const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
+    using Cfg = TileCfg<EPI, BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
+    const uint32_t bar_base = base + STAGES * Cfg::STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
+    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+        *abort_flag = 0u;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+        if (EPI == EPI_SWIGLU) tma_prefetch_desc(&tmB2);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
+                int mb, nb;
+                tile_coords(p, t, mb, nb);
+                const int m0 = mb * Cfg::BM;
+                const int n0 = nb * Cfg::OUT_TILE_N;
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 1u)) { ok = false; break; }
+                    const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
+                    const uint32_t b_dst = a_dst + Cfg::A_BYTES;
+                    mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    tma_load_2d(a_dst, &tmA, full_bar(s), kb * Cfg::BK, m0);
+                    if (EPI == EPI_SWIGLU) {
+                        tma_load_2d(b_dst, &tmB, full_bar(s), kb * Cfg::BK, n0);
+                        tma_load_2d(b_dst + Cfg::B_BYTES / 2, &tmB2, full_bar(s), kb * Cfg::BK, n0);
+                    } else {
+                        tma_load_2d(b_dst, &tmB, full_bar(s), kb * Cfg::BK, n0);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(Cfg::BM, BN);
+            int s = 0;
+            uint32_t ph = 0;
+            uint32_t acc_ph[2] = {0u, 0u};
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++it) {
+                const int buf = it & 1;
+                if (!mbar_wait(acce_bar(buf), acc_ph[buf] ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 1u)) { ok = false; break; }
+                acc_ph[buf] ^= 1u;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * BN);
+                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 2u)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
+                    const uint64_t a_desc = umma_smem_desc_sw128(a_src);
+                    const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < Cfg::BK / 16; ++k)
+                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty_bar(s));      // frees the stage once these MMAs have read it
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma_commit(accf_bar(buf));  // accumulator complete
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
+        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        uint32_t acc_ph[2] = {0u, 0u};
+        int it = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++it) {
+            const int buf = it & 1;
+            int mb, nb;
+            tile_coords(p, t, mb, nb);
+            const int row = mb * Cfg::BM + q * 32 + lane;
+            const int n_tile0 = nb * Cfg::OUT_TILE_N;
+            if (!mbar_wait(accf_bar(buf), acc_ph[buf], abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 1u)) { ok = false; break; }
+            acc_ph[buf] ^= 1u;
+            tc_fence_after();
+            const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * BN);
+
+            if (EPI == EPI_ACT) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    const int n0 = n_tile0 + c * 32;
+                    if (n0 >= p.N) break;            // warp-uniform
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(t_addr + c * 32, r);
+                    float bv[32], y[32];
+                    load_bias_chunk(p.bias, n0, p.N, bv);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
+                    apply_act_chunk(p.act, y);
+                    if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, vec_ok);
+                }
+            } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+                for (int c = 0; c < BN / 64; ++c) {
+                    const int n0 = n_tile0 + c * 32;
+                    if (n0 >= p.N) break;
+                    uint32_t g[32], u[32];
+                    tmem_ld_32x32b_x32(t_addr + c * 32, g);                 // gate columns
+                    tmem_ld_32x32b_x32(t_addr + BN / 2 + c * 32, u);        // up columns
+                    tmem_ld_wait();
+                    float y[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+                    if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, vec_ok);
+                }
+            } else {
+                // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
+                constexpr float LOG2E = 1.4426950408889634f;
+                float mx = -INFINITY, sum = 0.0f;
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    const int n0 = n_tile0 + c * 32;
+                    if (n0 >= p.N) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(t_addr + c * 32, r);
+                    float bv[32], tv[32];
+                    load_bias_chunk(p.bias, n0, p.N, bv);
+                    tmem_ld_wait();
+                    float cm = -INFINITY;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        // columns past N are zero-filled weight rows: mask them out of the reduction
+                        tv[j] = (n0 + j < p.N) ? (__uint_as_float(r[j]) + bv[j]) * LOG2E : -INFINITY;
+                        cm = fmaxf(cm, tv[j]);
+                    }
+                    const float nm = fmaxf(mx, cm);
+                    float cs = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) cs += ex2_approx(tv[j] - nm);
+                    sum = sum * ex2_approx(mx - nm) + cs;
+                    mx = nm;
+                }
+                if (row < p.M)
+                    p.lse_partial[static_cast<size_t>(nb) * p.M + row] = make_float2(mx * 0.6931471805599453f, sum);
+            }
+            // accumulator buffer drained: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(buf));
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag != 0u) {
+        // A wait gave up: let copies / MMAs already in flight land before freeing anything.
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+// (m, s) <- (m, s) (+) (om, os):  max of the maxima, sums rescaled to it.  A side that
+// has seen nothing yet holds (-inf, 0) and stays neutral.
+__device__ __forceinline__ void lse_combine(float& m, float& s, float om, float os) {
+    const float nm = fmaxf(m, om);
+    const float a = (m == -INFINITY) ? 0.0f : __expf(m - nm);
+    const float b = (om == -INFINITY) ? 0.0f : __expf(om - nm);
+    s = s * a + os * b;
+    m = nm;
+}
+
+// Merges the per-column-tile (max, sum-exp) partials of each row, in ascending
+// tile order, into lse[row] = max + ln(sum).  One warp per row; lanes stride over
+// the partials and combine with shuffles.
+__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int n_parts, float* __restrict__ lse) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    float mx = -INFINITY, sum = 0.0f;
+    for (int i = lane; i < n_parts; i += 32) {
+        const float2 v = __ldcg(partial + static_cast<size_t>(i) * M + row);
+        lse_combine(mx, sum, v.x, v.y);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, mx, off);
+        const float os = __shfl_xor_sync(0xffffffffu, sum, off);
+        lse_combine(mx, sum, om, os);
+    }
+    if (lane == 0) lse[row] = mx + __logf(sum);
+}
+
+}  // namespace mtmc

@@ -1,0 +1,282 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 CPU oracle, element by
+element, on the same seeded inputs.  Tolerances are the stated ones:
+    bf16 outputs : |err| <= 1e-2 + 1e-2 |ref|
+    fp32 outputs and lse : |err| <= 1e-3 + 1e-3 |ref|
+Outputs are pre-filled with NaN and surrounded by canaries, so an element the
+kernel never wrote, or a write outside the output, fails the test."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ref
+from paper_2511_20100_b200 import inputs
+from paper_2511_20100_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+TOL = {"bf16": (1e-2, 1e-2), "fp32": (1e-3, 1e-3)}
+PAD = 512   # canary elements before and after every output
+
+
+def _guarded(shape, dtype):
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * PAD,), float("nan"), dtype=dtype, device="cuda")
+    buf[:PAD] = 7.0
+    buf[PAD + n:] = 7.0
+    return buf, buf[PAD:PAD + n].view(*shape)
+
+
+def _canaries_intact(buf, n):
+    return bool((buf[:PAD] == 7.0).all()) and bool((buf[PAD + n:] == 7.0).all())
+
+
+def _assert_close(got, want, tol, what):
+    r = ref.compare(got, want, *tol)
+    assert r["ok"], "%s: %d/%d outside tolerance, max |err| %.3e, worst ratio %.2f at flat index %d" % (
+        what, r["violations"], r["count"], r["max_abs_err"], r["max_ratio"], r["worst_index"])
+    return r
+
+
+def run_linear(M, N, K, act, odt, seed, bias=True):
+    li = inputs.linear_inputs(M, N, K, seed, bias=bias)
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), None if li.b is None else li.b.cuda(), act, odt, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    return li, out
+
+
+# ------------------------------------------------------------------ small shapes, full oracle
+SMALL = [
+    # M, N, K  -- several tiles, ragged tails in every dimension, K not a multiple of 64
+    (1, 8, 8), (17, 8, 64), (100, 72, 136), (128, 128, 64), (129, 257, 72), (136, 384, 256),
+    (256, 100, 1024), (384, 640, 512), (300, 520, 200), (64, 1000, 320),
+]
+
+
+@pytest.mark.parametrize("M,N,K", SMALL)
+@pytest.mark.parametrize("act", ["none", "relu", "gelu_tanh", "silu"])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_fused_linear_small(M, N, K, act, odt):
+    li, out = run_linear(M, N, K, act, odt, seed=1000 + M + N + K)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[act])
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "fused_linear %dx%dx%d %s %s" % (M, N, K, act, odt))
+
+
+@pytest.mark.parametrize("tile_n", [128, 256])
+def test_fused_linear_both_tile_widths(tile_n):
+    B.mtmc_set_tuning(tile_n=tile_n)
+    try:
+        li, out = run_linear(260, 392, 328, "gelu_tanh", "fp32", seed=77)
+    finally:
+        B.mtmc_set_tuning()
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT["gelu_tanh"])
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "tile_n %d" % tile_n)
+
+
+def test_fused_linear_exact_integers_and_no_bias():
+    # integer-valued operands: every product and fp32 partial sum is exact, so the result must be too
+    g = torch.Generator().manual_seed(5)
+    X = torch.randint(-3, 4, (200, 192), generator=g).to(torch.bfloat16)
+    W = torch.randint(-3, 4, (264, 192), generator=g).to(torch.bfloat16)
+    out = B.mtmc_fused_linear(X.cuda(), W.cuda(), None, "none", "fp32")
+    B.mtmc_check_status()
+    want = ref.fused_linear(inputs.bf16_bits(X), inputs.bf16_bits(W), None, ref.ACT_NONE)
+    assert np.array_equal(inputs.to_f64(out), want)
+
+
+def test_identity_weight_and_zero_input():
+    li = inputs.linear_inputs(130, 192, 192, seed=3)
+    eye = torch.eye(192).to(torch.bfloat16)
+    out = B.mtmc_fused_linear(li.X.cuda(), eye.cuda(), li.b.cuda(), "silu", "fp32")
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(eye), inputs.f32(li.b), ref.ACT_SILU)
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "W = I")
+    zero = torch.zeros_like(li.X)
+    out0 = B.mtmc_fused_linear(zero.cuda(), li.W.cuda(), li.b.cuda(), "gelu_tanh", "fp32")
+    B.mtmc_check_status()
+    want0 = np.array([ref.act(ref.ACT_GELU_TANH, float(v)) for v in li.b])
+    _assert_close(inputs.to_f64(out0), np.broadcast_to(want0, (130, 192)), TOL["fp32"], "X = 0")
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (100, 72, 136), (300, 392, 256), (128, 1000, 512), (513, 136, 64)])
+def test_swiglu_small(M, N, K):
+    si = inputs.swiglu_inputs(M, N, K, seed=2000 + M + N)
+    buf, out = _guarded((M, N), torch.bfloat16)
+    B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda(), out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    want = ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu))
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "swiglu %dx%dx%d" % (M, N, K))
+
+
+def test_swiglu_equal_weights_is_silu_z_times_z():
+    si = inputs.swiglu_inputs(140, 256, 192, seed=31)
+    out = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wg.cuda())
+    B.mtmc_check_status()
+    z = ref.fused_linear(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), None, ref.ACT_NONE)
+    want = np.vectorize(lambda v: ref.act(ref.ACT_SILU, v) * v)(z)
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "Wg = Wu")
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 8, 64), (200, 1000, 256), (129, 257, 72), (64, 3000, 128), (260, 512, 320)])
+@pytest.mark.parametrize("bias", [True, False])
+def test_linear_lse_small(M, N, K, bias):
+    li = inputs.linear_inputs(M, N, K, seed=3000 + M + N, bias=bias)
+    buf, out = _guarded((M,), torch.float32)
+    B.mtmc_linear_lse(li.X.cuda(), li.W.cuda(), None if li.b is None else li.b.cuda(), lse_out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M)
+    want = ref.linear_lse(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b))
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "lse %dx%dx%d" % (M, N, K))
+
+
+def test_linear_lse_shift_law():
+    li = inputs.linear_inputs(150, 700, 128, seed=41)
+    a = B.mtmc_linear_lse(li.X.cuda(), li.W.cuda(), li.b.cuda())
+    b = B.mtmc_linear_lse(li.X.cuda(), li.W.cuda(), (li.b + 3.0).cuda())
+    B.mtmc_check_status()
+    assert torch.allclose(b - a, torch.full_like(a, 3.0), atol=2e-3)
+
+
+# ------------------------------------------------------------------ skinny / split-K path
+@pytest.mark.parametrize("M,N,K", [(16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392)])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_skinny_small(M, N, K, odt):
+    li, out = run_linear(M, N, K, "gelu_tanh", odt, seed=4000 + M + N)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "skinny %dx%dx%d %s" % (M, N, K, odt))
+
+
+@pytest.mark.parametrize("split_k", [1, 2, 8, 37])
+def test_skinny_result_independent_of_split(split_k):
+    li = inputs.linear_inputs(16, 640, 4096, seed=44)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
+    B.mtmc_set_tuning(split_k=split_k)
+    try:
+        Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+        first = B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32")
+        again = B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(first), want, TOL["fp32"], "split_k %d" % split_k)
+    assert torch.equal(first, again), "split-K result must be bit-stable run to run"
+
+
+def test_skinny_with_caller_workspace():
+    li = inputs.linear_inputs(16, 512, 2048, seed=45)
+    need = B.mtmc_workspace_bytes("fused_linear", 16, 512, 2048)
+    assert need > 0
+    ws = torch.full((need + 256,), 255, dtype=torch.uint8, device="cuda")   # dirty on purpose
+    off = (-ws.data_ptr()) % 256
+    B.mtmc_set_workspace(ws[off:off + need])
+    try:
+        out = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), "gelu_tanh", "bf16")
+        B.mtmc_check_status()
+        with pytest.raises(B.MtmcError) as e:
+            B.mtmc_set_workspace(ws[off:off + 1024])
+            B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), "gelu_tanh", "bf16")
+        assert e.value.status == B.ERR_WORKSPACE
+    finally:
+        B.mtmc_set_workspace(None)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "caller workspace")
+
+
+# ------------------------------------------------------------------ the five benchmark configurations
+def test_config_c1_full():
+    c = inputs.CONFIGS["C1"]
+    li, out = run_linear(c["M"], c["N"], c["K"], c["act"], c["out_dtype"], c["seed"])
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[c["act"]])
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "C1")
+
+
+def test_config_c2_sampled():
+    c = inputs.CONFIGS["C2"]
+    li, out = run_linear(c["M"], c["N"], c["K"], c["act"], c["out_dtype"], c["seed"])
+    rows, cols = inputs.sample_points(c["M"], c["N"], 6000, seed=1, tile_n=256)
+    want = ref.fused_linear_points(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[c["act"]], rows, cols)
+    got = inputs.to_f64(out[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()])
+    _assert_close(got, want, TOL["bf16"], "C2 sampled")
+    assert bool(torch.isfinite(out.float()).all())       # every element was written with a finite value
+
+
+def test_config_c3_sampled():
+    c = inputs.CONFIGS["C3"]
+    si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
+    buf, out = _guarded((c["M"], c["N"]), torch.bfloat16)
+    B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda(), out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, c["M"] * c["N"])
+    rows, cols = inputs.sample_points(c["M"], c["N"], 6000, seed=2)
+    want = ref.swiglu_points(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu), rows, cols)
+    got = inputs.to_f64(out[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()])
+    _assert_close(got, want, TOL["bf16"], "C3 sampled")
+    assert bool(torch.isfinite(out.float()).all())
+
+
+def test_config_c4_sampled_rows():
+    c = inputs.CONFIGS["C4"]
+    li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+    buf, out = _guarded((c["M"],), torch.float32)
+    B.mtmc_linear_lse(li.X.cuda(), li.W.cuda(), li.b.cuda(), lse_out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, c["M"])
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 127, 128, c["M"] - 1], rng.integers(0, c["M"], size=12)]))
+    want = ref.linear_lse_rows(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), rows)
+    _assert_close(inputs.to_f64(out[torch.from_numpy(rows).cuda()]), want, TOL["fp32"], "C4 sampled rows")
+    # property that holds at any size: logits ~ N(0,1)+b, so every lse sits near ln N + 1/2
+    allv = inputs.to_f64(out)
+    assert np.all(np.isfinite(allv)) and np.all(np.abs(allv - (np.log(c["N"]) + 0.5)) < 0.2)
+
+
+def test_config_c5_full():
+    c = inputs.CONFIGS["C5"]
+    li, out = run_linear(c["M"], c["N"], c["K"], c["act"], c["out_dtype"], c["seed"])
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[c["act"]])
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "C5")
+
+
+# ------------------------------------------------------------------ determinism, errors
+def test_bit_reproducible():
+    li = inputs.linear_inputs(300, 520, 448, seed=9)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    first = B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "bf16")
+    l0 = B.mtmc_linear_lse(Xd, Wd, bd)
+    for _ in range(10):
+        assert torch.equal(first, B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "bf16"))
+        assert torch.equal(l0, B.mtmc_linear_lse(Xd, Wd, bd))
+    B.mtmc_check_status()
+
+
+def test_argument_errors_enqueue_nothing():
+    L = B.load()
+    x = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    o = torch.zeros(64, 64, dtype=torch.float32, device="cuda")
+    before = B.mtmc_launch_count()
+    assert L.mtmc_fused_linear(None, x.data_ptr(), None, 64, 64, 64, 0, 0, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_fused_linear(x.data_ptr(), x.data_ptr(), None, 64, 64, 0, 0, 0, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_fused_linear(x.data_ptr(), x.data_ptr(), None, 64, 64, 64, 9, 0, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_fused_linear(x.data_ptr(), x.data_ptr(), None, 64, 64, 64, 0, 5, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_fused_linear(x.data_ptr(), x.data_ptr(), None, 64, 64, 60, 0, 0, o.data_ptr()) == B.ERR_UNSUPPORTED_SHAPE
+    assert L.mtmc_fused_linear(x.data_ptr() + 2, x.data_ptr(), None, 32, 64, 64, 0, 0, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_swiglu(x.data_ptr(), x.data_ptr(), None, 64, 64, 64, o.data_ptr()) == B.ERR_INVALID_ARG
+    assert L.mtmc_linear_lse(x.data_ptr(), x.data_ptr(), None, 64, 64, 64, None) == B.ERR_INVALID_ARG
+    assert B.mtmc_launch_count() == before
+    assert len(L.mtmc_last_error()) > 0
+    B.mtmc_check_status()
+
+
+def test_host_pointer_entry_points():
+    li = inputs.linear_inputs(150, 264, 128, seed=61)
+    out = B.mtmc_fused_linear_host(li.X, li.W, li.b, "relu", "fp32")
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_RELU)
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "fused_linear_host")
+    lse = B.mtmc_linear_lse_host(li.X, li.W, li.b)
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)),
+                  TOL["fp32"], "linear_lse_host")
+    si = inputs.swiglu_inputs(150, 264, 128, seed=62)
+    sw = B.mtmc_swiglu_host(si.X, si.Wg, si.Wu)
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "swiglu_host")
