@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the fused-linear hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole hot path: the five benchmark configurations, one call
+each, back to back on one stream (tiled fused linear, SwiGLU, linear + logsumexp,
+split-K skinny linear).  The metric is TFLOP/s (algorithmic FLOPs of all calls / device
+time); per-configuration times, TFLOP/s or GB/s and roofline fractions ride along in
+the same JSON line.  Inputs are seeded synthetic tensors resident in HBM; a step touches
+about 1 GB of distinct operands, far more than the 126 MB L2, so every call starts
+L2-cold.  With N > 1 (torchrun) every rank runs an independent replica of the same
+step on its own GPU -- the path does not shard and there is no data-path collective.
+
+`--impl reference` times the fp64 CPU oracle (as it stands, never tuned) on the host
+cores on a bounded row-sample of the same five configurations.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2511_20100_b200 import inputs
+
+ORDER = ["C1", "C2", "C3", "C4", "C5"]
+# rows of X the CPU reference computes per step and per configuration (bounded sample)
+REF_ROWS = {"C1": 256, "C2": 64, "C3": 32, "C4": 32, "C5": 16}
+
+
+def flops(c) -> float:
+    f = 2.0 * c["M"] * c["N"] * c["K"]
+    return 2.0 * f if c["op"] == "swiglu" else f
+
+
+def algorithmic_bytes(c) -> float:
+    """Each operand read once, each output written once."""
+    M, N, K = c["M"], c["N"], c["K"]
+    if c["op"] == "swiglu":
+        return 2.0 * (M * K + 2 * N * K) + 2.0 * M * N
+    if c["op"] == "linear_lse":
+        return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M
+    out_b = 2.0 if c["out_dtype"] == "bf16" else 4.0
+    return 2.0 * (M * K + N * K) + 4.0 * N + out_b * M * N
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            p = json.load(open(path))
+            return {"hbm_gbs": float(p["hbm_gbs"]), "tflops_burst": float(p["bf16_tflops"]),
+                    "tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------- our arm
+def make_device_problem(name, device):
+    c = inputs.CONFIGS[name]
+    if c["op"] == "swiglu":
+        si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
+        host = [si.X, si.Wg, si.Wu]
+    else:
+        li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+        host = [li.X, li.W, li.b]
+    dev = [t.to(device) for t in host]
+    if c["op"] == "linear_lse":
+        out = torch.empty((c["M"],), dtype=torch.float32, device=device)
+    else:
+        odt = torch.bfloat16 if c.get("out_dtype", "bf16") == "bf16" else torch.float32
+        out = torch.empty((c["M"], c["N"]), dtype=odt, device=device)
+    return {"name": name, "cfg": c, "host": host, "dev": dev, "out": out}
+
+
+def call_device(B, pr):
+    c, d = pr["cfg"], pr["dev"]
+    if c["op"] == "swiglu":
+        B.mtmc_swiglu(d[0], d[1], d[2], out=pr["out"])
+    elif c["op"] == "linear_lse":
+        B.mtmc_linear_lse(d[0], d[1], d[2], lse_out=pr["out"])
+    else:
+        B.mtmc_fused_linear(d[0], d[1], d[2], c["act"], c["out_dtype"], out=pr["out"])
+
+
+def call_host(B, pr, pinned, dev_index):
+    c = pr["cfg"]
+    if c["op"] == "swiglu":
+        B.mtmc_swiglu_host(pinned["in"][0], pinned["in"][1], pinned["in"][2], out=pinned["out"], device=dev_index)
+    elif c["op"] == "linear_lse":
+        B.mtmc_linear_lse_host(pinned["in"][0], pinned["in"][1], pinned["in"][2], lse_out=pinned["out"], device=dev_index)
+    else:
+        B.mtmc_fused_linear_host(pinned["in"][0], pinned["in"][1], pinned["in"][2], c["act"], c["out_dtype"],
+                                 out=pinned["out"], device=dev_index)
+
+
+def cpu_baseline_sample():
+    """The oracle timed on a bounded sample: the first REF_ROWS rows of every configuration."""
+    from oracle import ref
+    t_total, fl_total = 0.0, 0.0
+    for name in ORDER:
+        t, fl = reference_step_one(ref, name, prepared_reference_inputs(name))
+        t_total += t
+        fl_total += fl
+    return fl_total / t_total / 1e12, ref.get_threads()
+
+
+_ref_cache = {}
+
+
+def prepared_reference_inputs(name):
+    if name not in _ref_cache:
+        c = inputs.CONFIGS[name]
+        r = min(REF_ROWS[name], c["M"])
+        if c["op"] == "swiglu":
+            si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
+            _ref_cache[name] = (inputs.bf16_bits(si.X[:r].contiguous()), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu))
+        else:
+            li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+            _ref_cache[name] = (inputs.bf16_bits(li.X[:r].contiguous()), inputs.bf16_bits(li.W), inputs.f32(li.b))
+    return _ref_cache[name]
+
+
+def reference_step_one(ref, name, arrs):
+    c = inputs.CONFIGS[name]
+    r = arrs[0].shape[0]
+    t0 = time.perf_counter()
+    if c["op"] == "swiglu":
+        ref.swiglu(arrs[0], arrs[1], arrs[2])
+    elif c["op"] == "linear_lse":
+        ref.linear_lse(arrs[0], arrs[1], arrs[2])
+    else:
+        ref.fused_linear(arrs[0], arrs[1], arrs[2], {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}[c["act"]])
+    dt = time.perf_counter() - t0
+    return dt, flops(c) * r / c["M"]
+
+
+def sample_description():
+    return "first rows of X per configuration: " + ", ".join("%s %d/%d" % (n, min(REF_ROWS[n], inputs.CONFIGS[n]["M"]),
+                                                                               inputs.CONFIGS[n]["M"]) for n in ORDER)
+
+
+def run_ours(args, rank, world, local_rank):
+    from paper_2511_20100_b200 import binding as B   # raises if the CUDA library is missing: no fallback
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU path")
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+    B.load()
+    problems = [make_device_problem(n, device) for n in ORDER]
+    peaks = measured_peaks()
+
+    def step(events=None):
+        for i, pr in enumerate(problems):
+            call_device(B, pr)
+            if events is not None:
+                events[i + 1].record()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    B.mtmc_check_status()
+    torch.cuda.synchronize()
+
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(ORDER) + 1)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = B.mtmc_launch_count()
+    for k in range(args.steps):
+        ev[k][0].record()
+        step(ev[k])
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    launches = B.mtmc_launch_count() - launches0
+    clocks = sampler.stop()
+    B.mtmc_check_status()
+
+    total_ms = sum(ev[k][0].elapsed_time(ev[k][-1]) for k in range(args.steps))
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    per_cfg_ms = {n: statistics.mean(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps))
+                  for i, n in enumerate(ORDER)}
+    per_cfg_best = {n: min(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)) for i, n in enumerate(ORDER)}
+    step_flops = sum(flops(inputs.CONFIGS[n]) for n in ORDER)
+    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+
+    per_config = {}
+    for n in ORDER:
+        c = inputs.CONFIGS[n]
+        ms = per_cfg_ms[n]
+        entry = {"call": c["op"], "M": c["M"], "N": c["N"], "K": c["K"], "ms": round(ms, 5), "ms_best": round(per_cfg_best[n], 5),
+                 "tflops": round(flops(c) / (ms * 1e-3) / 1e12, 3), "gbs": round(algorithmic_bytes(c) / (ms * 1e-3) / 1e9, 2)}
+        if n == "C5":
+            entry["roofline"] = {"bound": "hbm", "achieved": entry["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                 "frac": round(entry["gbs"] / peaks["hbm_gbs"], 4), "of": peaks["source"],
+                                 "frac_of_nominal_8000": round(entry["gbs"] / 8000.0, 4)}
+        elif n != "C1":
+            entry["roofline"] = {"bound": "tensor", "achieved": entry["tflops"], "peak": peaks["tflops_sustained"],
+                                 "unit": "TFLOP/s", "frac": round(entry["tflops"] / peaks["tflops_sustained"], 4),
+                                 "of": peaks["source"] + " (sustained cuBLAS bf16)",
+                                 "frac_of_burst": round(entry["tflops"] / peaks["tflops_burst"], 4),
+                                 "frac_of_nominal_2250": round(entry["tflops"] / 2250.0, 4)}
+        else:
+            entry["note"] = "launch-latency bound parity configuration"
+        per_config[n] = entry
+
+    # dominant kernel of the step: the tiled tcgen05 kernel, on its longest launch (C3, SwiGLU)
+    dom = per_config["C3"]
+    roofline = {"bound": "tensor", "kernel": "gemm_tiled_kernel<SWIGLU,256,bf16> on C3",
+                "achieved": dom["tflops"], "peak": peaks["tflops_sustained"], "unit": "TFLOP/s",
+                "frac": round(dom["tflops"] / peaks["tflops_sustained"], 4), "peak_source": peaks["source"] + ", sustained cuBLAS bf16",
+                "traffic": None}
+    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(prof):
+        try:
+            roofline["traffic"] = json.load(open(prof)).get("C3_dram_bytes_per_launch")
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ end to end through the host-pointer C ABI
+    e2e = None
+    if rank == 0 or world > 1:
+        pinned = []
+        h2d = d2h = 0
+        for pr in problems:
+            ins = [None if t is None else t.pin_memory() for t in pr["host"]]
+            out = torch.empty(pr["out"].shape, dtype=pr["out"].dtype).pin_memory()
+            pinned.append({"in": ins, "out": out})
+            h2d += sum(t.numel() * t.element_size() for t in ins if t is not None)
+            d2h += out.numel() * out.element_size()
+        for pr, pn in zip(problems, pinned):       # warm-up: sizes the library's staging buffers
+            call_host(B, pr, pn, local_rank)
+        e2e_steps = max(2, min(args.steps, 5))
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            for pr, pn in zip(problems, pinned):
+                call_host(B, pr, pn, local_rank)
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([e2e_s], dtype=torch.float64, device=device)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = float(t.item())
+        e2e = {"value": round(world * step_flops * e2e_steps / e2e_s / 1e12, 3), "unit": "TFLOP/s",
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
+               "ms_per_step": round(e2e_s / e2e_steps * 1e3, 3),
+               "api": "mtmc_*_host: pinned host buffers in, host result out, copies inside the timed region"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores = cpu_baseline_sample()
+        cpu = {"value": round(v, 6), "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample_description()}
+
+    if rank == 0:
+        line = {
+            "metric": "TFLOP/s over one pass of the fused-linear hot path (per-config TFLOP/s, GB/s and roofline fractions in per_config)",
+            "value": round(value, 3), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "C1+C2+C3+C4+C5 (all five configurations, one call each per step)",
+                       "l2": "inputs larger than L2: a step reads ~1.0 GB of distinct operands (L2 126 MB), every call starts cold",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "per_config": per_config, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------- reference arm
+def run_reference(args, rank, world):
+    if rank != 0:
+        return
+    from oracle import ref
+    arrs = {n: prepared_reference_inputs(n) for n in ORDER}
+    steps, warm = args.steps, max(args.warmup, 1)
+    for _ in range(warm):
+        for n in ORDER:
+            reference_step_one(ref, n, arrs[n])
+    t_total, fl_total = 0.0, 0.0
+    for _ in range(steps):
+        for n in ORDER:
+            t, fl = reference_step_one(ref, n, arrs[n])
+            t_total += t
+            fl_total += fl
+    value = fl_total / t_total / 1e12
+    line = {
+        "impl": "reference",
+        "metric": "TFLOP/s over one pass of the fused-linear hot path (per-config TFLOP/s, GB/s and roofline fractions in per_config)",
+        "value": round(value, 6), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warm,
+        "ms_per_step": round(t_total / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "C1+C2+C3+C4+C5 (all five configurations, one call each per step)",
+                   "sample": sample_description()},
+        "cpu_baseline": {"value": round(value, 6), "unit": "TFLOP/s", "cores": ref.get_threads(), "kind": "oracle",
+                         "sample": sample_description()},
+        "e2e": {"value": round(value, 6), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
