@@ -87,6 +87,40 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu,
 int mtmc_linear_lse(const void* X, const void* W, const float* b,
                     int64_t M, int64_t N, int64_t K, float* lse_out);
 
+/* Allocation-free variant of mtmc_linear_lse: same arguments, same result (same
+ * kernels), but the (max, sum-exp) partials live in an 8 MiB array that is part of
+ * the library image instead of a workspace from cudaMalloc.  (The paper has no
+ * counterpart; this exists for callers that must not allocate.)
+ *
+ * Who needs it: code that runs where device memory is not theirs to ask for -- an
+ * operator called from inside an inference server's request loop, where a
+ * cudaMalloc would stall every stream of the device; a plug-in whose host
+ * framework has already claimed the whole GPU for its own pool, so a raw
+ * allocation fails or fragments it; a job with a fixed memory budget audited at
+ * start-up.  This call makes no cudaMalloc / cudaFree and calls no allocating
+ * library routine, on any call including the first.
+ *
+ * Limits and rules:
+ *   - ceil(N / 256) * M  (ceil(N / 128) * M when N <= 128 or tile_n = 128 is
+ *     forced) must not exceed 1,048,576 partials; larger shapes are rejected with
+ *     MTMC_ERR_UNSUPPORTED_SHAPE and the message names mtmc_linear_lse instead.
+ *     The benchmark's LM-head shape (M=4096, N=32000) needs 512,000.
+ *   - Every GPU that loads the library holds the 8 MiB until the process exits.
+ *   - The first call on each device performs a one-time set-up (device attribute
+ *     queries, driver entry point lookup, cudaGetSymbolAddress of the scratch,
+ *     one 4-byte synchronous copy).  Make that first call before starting any
+ *     stream capture.
+ *   - All calls on a device share the one array, which keeps whatever the last
+ *     call left in it.  Nothing in it needs clearing: every slot a call reads
+ *     has been written by that same call first.  Two calls that overlap on the
+ *     GPU (different streams, or different host threads) race on it and give
+ *     wrong results; serialise them on one stream.
+ *   - Device-side timeouts of this path go to a status word of their own:
+ *     a later call to this function returns MTMC_ERR_DEVICE_TIMEOUT if it finds
+ *     the stream idle and the word set; mtmc_check_status() does not see it. */
+int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b,
+                            int64_t M, int64_t N, int64_t K, float* lse_out);
+
 /* Same three operations with every pointer a HOST pointer (pageable or pinned).
  * The library copies the operands to device buffers it owns (cudaMalloc,
  * grow-only, per device), runs the device entry point on the current stream,

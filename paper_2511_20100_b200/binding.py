@@ -23,6 +23,7 @@ OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2}
 
 EXPORTS = [
     "mtmc_fused_linear", "mtmc_swiglu", "mtmc_linear_lse",
+    "mtmc_linear_lse_noalloc",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
@@ -50,7 +51,7 @@ def load() -> ctypes.CDLL:
     vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
     for name in ("mtmc_fused_linear", "mtmc_fused_linear_host"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
-    for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host"):
+    for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_set_stream.argtypes = [vp]
     L.mtmc_set_workspace.argtypes = [vp, sz]
@@ -119,6 +120,23 @@ def mtmc_linear_lse(X, W, b, lse_out=None):
     _check(load().mtmc_linear_lse(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
                                   None if b is None else _dev(b, torch.float32, (N,), "b"),
                                   M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
+
+
+def mtmc_linear_lse_noalloc(X, W, b, lse_out):
+    """mtmc_linear_lse without any allocation inside the library: the partials go to an
+    8 MiB array built into the library image (ceil(N/256) * M <= 1,048,576).  For
+    callers that may not allocate device memory -- a request loop that cannot afford
+    cudaMalloc's device-wide stall, a plug-in inside a framework that owns the whole
+    GPU.  The caller passes every buffer, lse_out included, so this wrapper allocates
+    nothing either.  Calls sharing a GPU must not overlap; make the first call on a
+    device before any stream capture."""
+    M, K = X.shape
+    N = W.shape[0]
+    _use_current_stream(X.device)
+    _check(load().mtmc_linear_lse_noalloc(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                          None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                          M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
     return lse_out
 
 

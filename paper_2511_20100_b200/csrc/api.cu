@@ -439,6 +439,122 @@ int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int
     return MTMC_OK;
 }
 
+}  // extern "C"
+
+// ---------------------------------------------------------------------------- allocation-free variant
+// Scratch for mtmc_linear_lse_noalloc: the per-(column tile, row) (max, sum-exp)
+// partials and a status word live in the library image itself.  Every GPU that loads
+// the library carries these 8 MiB until the process exits.  In host code the names
+// below are host-side stand-ins, not device addresses; the device addresses are
+// fetched once per device with cudaGetSymbolAddress and cached.
+constexpr size_t NOALLOC_MAX_PARTIALS = 1u << 20;           // float2 entries = 8 MiB
+static __device__ __align__(256) float2 g_noalloc_partials[NOALLOC_MAX_PARTIALS];
+static __device__ __align__(256) uint32_t g_noalloc_status[64];
+
+namespace {
+struct NoAllocDevice {
+    bool ready = false;
+    int sm_count = 0;
+    float2* partials = nullptr;   // device address of g_noalloc_partials on this device
+    uint32_t* status = nullptr;   // device address of g_noalloc_status on this device
+};
+NoAllocDevice g_noalloc_dev[MAX_DEVICES];
+
+// One-time set-up for the current device.  Queries attributes and symbol addresses only.
+int noalloc_device(NoAllocDevice** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return fail(MTMC_ERR_UNSUPPORTED_DEVICE, "device index %d out of range", dev);
+    std::lock_guard<std::mutex> lock(g_mutex);
+    NoAllocDevice& d = g_noalloc_dev[dev];
+    if (!d.ready) {
+        int major = 0, minor = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        CUDA_TRY(cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev));
+        if (major != 10)
+            return fail(MTMC_ERR_UNSUPPORTED_DEVICE, "compute capability %d.%d: this library only runs on 10.x (B200)", major, minor);
+        CUDA_TRY(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        if (!g_encode) {
+            void* fn = nullptr;
+            cudaDriverEntryPointQueryResult qres;
+            CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+            if (!fn || qres != cudaDriverEntryPointSuccess)
+                return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
+            g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        void* ptr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_partials));
+        d.partials = static_cast<float2*>(ptr);
+        CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_status));
+        d.status = static_cast<uint32_t*>(ptr);
+        uint32_t zero = 0;
+        CUDA_TRY(cudaMemcpy(d.status, &zero, sizeof zero, cudaMemcpyHostToDevice));
+        d.ready = true;
+    }
+    *out = &d;
+    return MTMC_OK;
+}
+
+template <int BN>
+int launch_lse_noalloc(NoAllocDevice* d, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams p) {
+    using Cfg = TileCfg<EPI_LSE, BN>;
+    auto kern = gemm_tiled_kernel<EPI_LSE, BN, false>;
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB, p);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+}  // namespace
+
+extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K,
+                                       float* lse_out) {
+    int rc = check_common(X, W, lse_out, M, N, K);
+    if (rc) return rc;
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    NoAllocDevice* d = nullptr;
+    rc = noalloc_device(&d);
+    if (rc) return rc;
+    const int bn = pick_tile_n(N);
+    GemmParams p{};
+    fill_tiling(p, M, N, K, bn);
+    const size_t need = static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M);
+    if (need > NOALLOC_MAX_PARTIALS)
+        return fail(MTMC_ERR_UNSUPPORTED_SHAPE,
+                    "mtmc_linear_lse_noalloc: ceil(N/%d) * M = %zu partials exceed the built-in scratch of %zu "
+                    "(8 MiB); use mtmc_linear_lse for this shape", bn, need, NOALLOC_MAX_PARTIALS);
+    // A timeout recorded by an earlier call is reported once the stream has gone idle
+    // (never by waiting for it).
+    if (cudaStreamQuery(t_stream) == cudaSuccess) {
+        uint32_t st = 0;
+        CUDA_TRY(cudaMemcpy(&st, d->status, sizeof st, cudaMemcpyDeviceToHost));
+        if (st != 0) {
+            uint32_t zero = 0;
+            CUDA_TRY(cudaMemcpy(d->status, &zero, sizeof zero, cudaMemcpyHostToDevice));
+            return fail(MTMC_ERR_DEVICE_TIMEOUT, "an earlier mtmc_linear_lse_noalloc call timed out on the device (status word 0x%x)", st);
+        }
+    } else {
+        (void)cudaGetLastError();   // cudaErrorNotReady is not an error here
+    }
+    p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = d->partials; p.status = d->status;
+    CUtensorMap tmA, tmB;
+    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmB, W, N, K, bn);
+    if (rc) return rc;
+    rc = bn == 256 ? launch_lse_noalloc<256>(d, tmA, tmB, p) : launch_lse_noalloc<128>(d, tmA, tmB, p);
+    if (rc) return rc;
+    const int rows_per_block = 8;
+    lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
+        p.lse_partial, p.M, p.n_tiles, lse_out);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
+extern "C" {
+
 // ---------------------------------------------------------------------------- host-pointer variants
 int mtmc_fused_linear_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
                            int out_dtype, void* out) {
