@@ -36,6 +36,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("MTMC_NVCC_FLAGS", "").split()
     cmd += [os.path.join(CSRC, f) for f in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -10,6 +10,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -35,6 +36,7 @@ struct DeviceState {
     size_t stage_bytes[5] = {0, 0, 0, 0, 0};
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     bool timed = false;
+    int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
 };
 
 std::mutex g_mutex;
@@ -194,40 +196,121 @@ int skinny_cta_of_unit_host(long long u, long long total, int grid) {
 }
 
 struct SkinnyPlan {
-    int n_tiles, k_blocks, grid, max_slots;
+    int n_tiles, k_blocks, grid, max_slots, tile_rows, stages, pair;
     long long total;
     size_t ticket_bytes, partial_bytes;
 };
 
-SkinnyPlan plan_skinny(int sm_count, int64_t N, int64_t K) {
+// Bands of W rows and the grid.
+//  * pair plan (default when W has at least 32 rows per CTA pair): one band per cluster of two
+//    CTAs, bands sized so that the clusters cover the SMs; each CTA takes half of K and the
+//    pair reduces through distributed shared memory.
+//  * ticket plan (few rows, or a forced split): 128-row bands, the (band, k-block) list cut
+//    evenly over the SMs or over n_tiles * split_k CTAs; partials and tickets in the workspace.
+SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
     SkinnyPlan s;
-    s.n_tiles = static_cast<int>((N + 127) / 128);
     s.k_blocks = static_cast<int>((K + 63) / 64);
-    s.total = static_cast<long long>(s.n_tiles) * s.k_blocks;
+    s.tile_rows = 128;
+    s.n_tiles = static_cast<int>((N + 127) / 128);
+    s.pair = 0;
     long long g = t_split_k > 0 ? static_cast<long long>(s.n_tiles) * t_split_k : sm_count;
-    if (g > s.total) g = s.total;
-    if (g > 65535 * 16) g = 65535 * 16;
+    if (t_split_k == 0 && pairs > 0 && s.k_blocks >= 2) {
+        int64_t rows = (N + pairs - 1) / pairs;               // rows per band if every pair gets one band
+        rows = (rows + 7) / 8 * 8;
+        if (rows >= 32 && rows <= 128) {
+            s.pair = 1;
+            s.tile_rows = static_cast<int>(rows);
+            s.n_tiles = static_cast<int>((N + rows - 1) / rows);
+            g = 2ll * s.n_tiles;
+        }
+    }
+    if (const char* e = getenv("MTMC_SKINNY")) {   // development knob: "rows,split" (ticket plan)
+        int r = 0, sp = 0;
+        if (sscanf(e, "%d,%d", &r, &sp) == 2 && r >= 8 && r <= 128 && r % 8 == 0) {
+            s.pair = 0;
+            s.tile_rows = r;
+            s.n_tiles = static_cast<int>((N + r - 1) / r);
+            g = sp > 0 ? static_cast<long long>(s.n_tiles) * sp : sm_count;
+        }
+    }
+    s.total = static_cast<long long>(s.n_tiles) * s.k_blocks;
+    if (!s.pair) {
+        if (g > s.total) g = s.total;
+        if (g > 65535 * 16) g = 65535 * 16;
+    }
     s.grid = static_cast<int>(g);
+    s.stages = SkinnyCfg::stages_for(s.tile_rows);
     int mx = 1;
-    for (int t = 0; t < s.n_tiles; ++t) {
-        long long first = static_cast<long long>(t) * s.k_blocks;
-        int nc = skinny_cta_of_unit_host(first + s.k_blocks - 1, s.total, s.grid) - skinny_cta_of_unit_host(first, s.total, s.grid) + 1;
-        if (nc > mx) mx = nc;
+    if (!s.pair) {
+        for (int t = 0; t < s.n_tiles; ++t) {
+            long long first = static_cast<long long>(t) * s.k_blocks;
+            int nc = skinny_cta_of_unit_host(first + s.k_blocks - 1, s.total, s.grid) - skinny_cta_of_unit_host(first, s.total, s.grid) + 1;
+            if (nc > mx) mx = nc;
+        }
     }
     s.max_slots = mx;
-    s.ticket_bytes = round256(static_cast<size_t>(s.n_tiles) * 4);
-    s.partial_bytes = static_cast<size_t>(s.n_tiles) * s.max_slots * 16 * 128 * 4;
+    s.ticket_bytes = s.pair ? 0 : round256(static_cast<size_t>(s.n_tiles) * 4);
+    s.partial_bytes = mx > 1 ? static_cast<size_t>(s.n_tiles) * s.max_slots * 16 * 128 * 4 : 0;
     return s;
 }
 
-bool use_skinny(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 127) / 128 <= static_cast<int64_t>(TICKET_BYTES / 4); }
+bool use_skinny(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 31) / 32 <= static_cast<int64_t>(TICKET_BYTES / 4); }
+
+template <bool OUT_BF16, bool PAIR>
+int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap& tmX, const SkinnyParams& p) {
+    auto kern = skinny_splitk_kernel<OUT_BF16, PAIR>;
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(s.grid), 1, 1);
+    cfg.blockDim = dim3(192, 1, 1);
+    cfg.dynamicSmemBytes = SkinnyCfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmW, tmX, p));
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
+// How many 2-CTA clusters of the skinny kernel the device can hold at once (0 if clusters
+// cannot be scheduled): the pair plan sizes its bands to this.
+int skinny_pairs(DeviceState* d) {
+    if (d->max_pairs < 0) {
+        auto kern = skinny_splitk_kernel<true, true>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2u * static_cast<unsigned>(d->sm_count), 1, 1);
+        cfg.blockDim = dim3(192, 1, 1);
+        cfg.dynamicSmemBytes = SkinnyCfg::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        d->max_pairs = n;
+    }
+    return d->max_pairs;
+}
 
 int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
                int out_dtype, void* out) {
-    SkinnyPlan s = plan_skinny(d->sm_count, N, K);
+    SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), N, K);
     SkinnyParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
+    p.tile_rows = s.tile_rows; p.num_stages = s.stages;
     p.act = act; p.bias = b; p.out = out; p.status = d->status;
     void* ws = nullptr;
     if (t_user_ws) {
@@ -235,7 +318,7 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, int
         if (rc) return rc;
         p.tickets = static_cast<uint32_t*>(ws);
         p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + s.ticket_bytes);
-        CUDA_TRY(cudaMemsetAsync(p.tickets, 0, s.ticket_bytes, t_stream));
+        if (s.ticket_bytes) CUDA_TRY(cudaMemsetAsync(p.tickets, 0, s.ticket_bytes, t_stream));
     } else {
         int rc = get_workspace(d, s.partial_bytes, &ws);
         if (rc) return rc;
@@ -247,24 +330,15 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, int
         }
     }
     CUtensorMap tmW, tmX;
-    int rc = encode_bf16_2d(&tmW, W, N, K, SkinnyCfg::BNW);
+    int rc = encode_bf16_2d(&tmW, W, N, K, s.tile_rows);
     if (rc) return rc;
     rc = encode_bf16_2d(&tmX, X, M, K, SkinnyCfg::MX);
     if (rc) return rc;
     TimedRegion tr(d);
-    if (out_dtype == MTMC_OUT_BF16) {
-        auto kern = skinny_splitk_kernel<true>;
-        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
-        kern<<<s.grid, 192, SkinnyCfg::SMEM_BYTES, t_stream>>>(tmW, tmX, p);
-    } else {
-        auto kern = skinny_splitk_kernel<false>;
-        CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
-        kern<<<s.grid, 192, SkinnyCfg::SMEM_BYTES, t_stream>>>(tmW, tmX, p);
-    }
-    CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1);
+    rc = out_dtype == MTMC_OUT_BF16 ? (s.pair ? launch_skinny<true, true>(s, tmW, tmX, p) : launch_skinny<true, false>(s, tmW, tmX, p))
+                                    : (s.pair ? launch_skinny<false, true>(s, tmW, tmX, p) : launch_skinny<false, false>(s, tmW, tmX, p));
     tr.stop();
-    return MTMC_OK;
+    return rc;
 }
 
 // Device buffer i of the *_host entry points, at least `bytes` large.
@@ -327,7 +401,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
             if (!use_skinny(M, N)) return 0;
             DeviceState* d = nullptr;
             if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
-            SkinnyPlan s = plan_skinny(d->sm_count, N, K);
+            SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), N, K);
             return s.ticket_bytes + s.partial_bytes;
         }
         case MTMC_OP_SWIGLU: return 0;
@@ -507,6 +581,25 @@ int launch_lse_noalloc(NoAllocDevice* d, const CUtensorMap& tmA, const CUtensorM
     return MTMC_OK;
 }
 }  // namespace
+
+#ifdef MTMC_TRACE
+__global__ void __launch_bounds__(192, 1) null_kernel(const __grid_constant__ CUtensorMap a, const __grid_constant__ CUtensorMap b, int x) {
+    extern __shared__ uint8_t sm[];
+    if (x == 12345) sm[threadIdx.x] = reinterpret_cast<const uint8_t*>(&a)[threadIdx.x & 63] + reinterpret_cast<const uint8_t*>(&b)[0];
+}
+extern "C" int mtmc_debug_null(int grid, int smem) {
+    CUtensorMap m; memset(&m, 0, sizeof m);
+    cudaFuncSetAttribute(null_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    null_kernel<<<grid, 192, smem, t_stream>>>(m, m, 0);
+    return cudaGetLastError() == cudaSuccess ? 0 : 4;
+}
+extern "C" int mtmc_debug_span(unsigned long long* out) {
+    return cudaMemcpyFromSymbol(out, mtmc::g_span, sizeof(unsigned long long) * 2048) == cudaSuccess ? 0 : 4;
+}
+extern "C" int mtmc_debug_trace(long long* out) {
+    return cudaMemcpyFromSymbol(out, mtmc::g_trace, sizeof(long long) * 8 * 16) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K,
                                        float* lse_out) {

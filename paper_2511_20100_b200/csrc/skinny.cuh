@@ -1,14 +1,31 @@
 // The skinny (decode-shaped, M <= 16) path: HBM-bound weight streaming with split-K.
 //
-// The roles are swapped relative to the tiled path ("swap-AB"): the 128 TMEM lanes
-// carry 128 rows of W (output columns n), the MMA's N side carries the M <= 16
-// rows of X.  Work is the flat list of (n-tile, k-block) units, cut into one
-// contiguous, equal share per CTA (stream-K), so every SM streams the same number
-// of weight bytes through a deep TMA ring.  A CTA whose share covers only part of
-// a tile's K range writes its fp32 partial [16 x 128] to the workspace and takes a
-// ticket; the CTA that takes the last ticket of a tile adds the partials in slot
-// order (so the result does not depend on arrival order), applies bias and
-// activation and stores.  No CTA ever waits for another.
+// The roles are swapped relative to the tiled path ("swap-AB"): the TMEM lanes carry
+// rows of W (output columns n), the MMA's N side carries the M <= 16 rows of X.
+// W is cut into bands of tile_rows rows (a multiple of 8, at most 128; the MMA is
+// always 128 lanes tall, lanes past tile_rows compute on stale shared memory and
+// are never read).  Work is the flat list of (band, k-block) units, cut into one
+// contiguous, equal share per CTA, so every SM streams the same number of weight
+// bytes through a deep TMA ring.  A CTA whose share covers only part of a band's K
+// range writes its fp32 partial [16 x 128] to the workspace and takes a ticket; the
+// CTA that takes the band's last ticket adds the partials in slot order (so the
+// result does not depend on arrival order), applies bias and activation and
+// stores.  No CTA ever waits for another.
+//
+// PAIR mode (the common case: enough rows of W for half the SMs): the K range of every
+// band is split over the two CTAs of a thread-block cluster.  The odd CTA sends its
+// fp32 partial straight into the even CTA's shared memory (distributed shared memory
+// stores + one remote mbarrier arrive); the even CTA adds it to its own registers
+// (rank 0 + rank 1, always in that order), applies the epilogue and stores.  No
+// global partials, no tickets, no fences to global memory.
+//
+// What bounds this kernel is per-stage and per-launch overhead, not arithmetic:
+//  * a 128x16x16 MMA occupies the tensor pipe for about 70 clocks whatever N is, and
+//    the issuing thread spends a few hundred clocks per pipeline hand-off, so one
+//    ring stage carries KB_PER_STAGE k-blocks (2 x 16 KiB of W) per hand-off;
+//  * k-steps are dealt round-robin onto WAYS independent accumulators;
+//  * the producer starts its first loads before the rest of the CTA has finished
+//    setting up, and the epilogue fetches its bias before the accumulator is ready.
 #pragma once
 #include "gemm_tiled.cuh"
 
@@ -17,8 +34,10 @@ namespace mtmc {
 struct SkinnyParams {
     int M, N, K;
     int n_tiles, k_blocks;
+    int tile_rows;           // W rows per band (multiple of 8, <= 128)
+    int num_stages;          // TMA ring depth (<= SkinnyCfg::MAX_STAGES)
     long long total_units;   // n_tiles * k_blocks
-    int max_slots;           // partial slots per tile
+    int max_slots;           // partial slots per band
     int act;
     const float* bias;
     void* out;
@@ -28,37 +47,65 @@ struct SkinnyParams {
 };
 
 struct SkinnyCfg {
-    static constexpr int BNW = 128;                       // W rows per tile = TMEM lanes
+    static constexpr int LANES = 128;                     // MMA M = TMEM lanes
     static constexpr int MX = 16;                         // X rows = MMA N
-    static constexpr int BK = 64;
-    static constexpr int W_BYTES = BNW * BK * 2;          // 16 KiB
-    static constexpr int X_BYTES = MX * BK * 2;           // 2 KiB
-    static constexpr int STAGE_BYTES = W_BYTES + X_BYTES;
-    static constexpr int STAGES = 11;
-    static constexpr int TMEM_COLS = 64;                  // two 32-column accumulator buffers
-    static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int BK = 64;                         // k-block: one 128-byte swizzle row
+    static constexpr int KB_PER_STAGE = 2;                // k-blocks per ring stage
+    static constexpr int X_BYTES = MX * BK * 2;           // 2 KiB per k-block
+    static constexpr int MAX_STAGES = 16;
+    static constexpr int RING_BYTES = 200 * 1024;         // shared memory given to the TMA ring
+    static constexpr int WAYS = 8;                        // independent accumulators
+    static constexpr int ACC_COLS = WAYS * MX;            // 128 TMEM columns per accumulator set
+    static constexpr int TMEM_COLS = 2 * ACC_COLS;        // two sets: MMA on one, epilogue on the other
+    static constexpr int NUM_BARRIERS = 2 * MAX_STAGES + 5;   // ring, accumulator sets, pair reduction
+    static constexpr int REDUCE_BYTES = MX * LANES * 4;       // the peer CTA's partial (PAIR mode)
+    static constexpr int SMEM_BYTES = RING_BYTES + REDUCE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int stage_bytes(int tile_rows) { return KB_PER_STAGE * (tile_rows * BK * 2 + X_BYTES); }
+    // The MMA always reads a 128-row (16 KiB) A tile, also when the band is shorter, so the
+    // last W tile of the last stage must start at least 16 KiB before the end of the ring.
+    static constexpr int stages_for(int tile_rows) {
+        return (RING_BYTES - 2 * LANES * BK * 2) / stage_bytes(tile_rows) + 1 < MAX_STAGES
+                   ? (RING_BYTES - 2 * LANES * BK * 2) / stage_bytes(tile_rows) + 1
+                   : MAX_STAGES;
+    }
 };
+
+#ifdef MTMC_TRACE
+__device__ long long g_trace[8 * 16];
+__device__ unsigned long long g_span[2 * 1024];
+__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define TRACE(i) do { if (blockIdx.x >= 112 && blockIdx.x < 120) g_trace[(blockIdx.x - 112) * 16 + (i)] = clock64(); } while (0)
+#else
+#define TRACE(i) do { } while (0)
+#endif
 
 __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, int grid) {
     return static_cast<int>(((u + 1) * grid - 1) / total);
 }
 
-template <bool OUT_BF16>
+template <bool OUT_BF16, bool PAIR>
 __global__ void __launch_bounds__(192, 1)
 skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                      const SkinnyParams p) {
     using Cfg = SkinnyCfg;
-    constexpr int STAGES = Cfg::STAGES;
+    constexpr int MAXS = Cfg::MAX_STAGES;
+    constexpr int KPS = Cfg::KB_PER_STAGE;
+    const int STAGES = p.num_stages;
+    const int R = p.tile_rows;
+    const uint32_t w_bytes = static_cast<uint32_t>(R) * Cfg::BK * 2;      // one W k-block; multiple of 1024
+    const uint32_t x_off = KPS * w_bytes;                                  // X k-blocks follow the W k-blocks
+    const uint32_t stage_bytes = KPS * (w_bytes + Cfg::X_BYTES);
     extern __shared__ uint8_t smem_raw[];
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
-    const uint32_t bar_base = base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t reduce_base = base + Cfg::RING_BYTES;                  // [16][128] fp32, written by the peer CTA
+    const uint32_t bar_base = reduce_base + Cfg::REDUCE_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
-    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (MAXS + s); };
+    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * MAXS + b); };
+    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * MAXS + 2 + b); };
+    const uint32_t red_bar = bar_base + 8u * (2 * MAXS + 4);
     uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
@@ -66,28 +113,64 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TRACE(0);
+#ifdef MTMC_TRACE
+    if (threadIdx.x == 0 && blockIdx.x < 1024) g_span[2 * blockIdx.x] = gtimer();
+#endif
     const int KB = p.k_blocks;
-    const long long u_begin = p.total_units * blockIdx.x / gridDim.x;
-    const long long u_end = p.total_units * (blockIdx.x + 1) / gridDim.x;
+    // This CTA's share of the unit list.
+    int first_tile, first_kb, n_units;
+    uint32_t crank = 0;
+    if (PAIR) {
+        // cluster of two: both CTAs work on band blockIdx.x / 2, each on one half of K
+        crank = cluster_ctarank();
+        const int half = (KB + 1) >> 1;
+        first_tile = static_cast<int>(blockIdx.x >> 1);
+        first_kb = crank ? half : 0;
+        n_units = crank ? KB - half : half;
+    } else {
+        long long u_begin, u_end;
+        if (p.total_units * gridDim.x < (1ll << 31)) {      // 32-bit arithmetic when it cannot overflow
+            const uint32_t tot = static_cast<uint32_t>(p.total_units);
+            u_begin = tot * blockIdx.x / gridDim.x;
+            u_end = tot * (blockIdx.x + 1u) / gridDim.x;
+        } else {
+            u_begin = p.total_units * blockIdx.x / gridDim.x;
+            u_end = p.total_units * (blockIdx.x + 1) / gridDim.x;
+        }
+        first_tile = static_cast<int>(u_begin / KB);
+        first_kb = static_cast<int>(u_begin - static_cast<long long>(first_tile) * KB);
+        n_units = static_cast<int>(u_end - u_begin);
+    }
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
-        *abort_flag = 0u;
-        *last_flag = 0u;
-        fence_barrier_init();
-        fence_proxy_async_smem();
-        tma_prefetch_desc(&tmW);
-        tma_prefetch_desc(&tmX);
+    // Set-up.  Warp 0 initialises the barriers and goes straight on to issue loads; it only
+    // arrives on the set-up barrier.  The other warps wait there for the barrier
+    // initialisation and for warp 1's TMEM allocation.
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&tmW);
+            tma_prefetch_desc(&tmX);
+            for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+            for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+            mbar_init(red_bar, 4);
+            *abort_flag = 0u;
+            *last_flag = 0u;
+            fence_barrier_init();
+            fence_proxy_async_smem();
+        }
+        __syncwarp();
+        asm volatile("bar.arrive 2, 192;" ::: "memory");
+        if (PAIR) cluster_arrive();          // publishes red_bar's initialisation to the peer; waited for at the end
+    } else {
+        if (warp == 1) {
+            tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
+            tmem_relinquish();
+            tc_fence_before();
+        }
+        asm volatile("bar.sync 2, 192;" ::: "memory");
+        tc_fence_after();
+        if (PAIR) cluster_arrive();          // after bar.sync: this CTA's barriers are initialised
     }
-    if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -96,89 +179,189 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             const uint64_t pol_keep = l2_policy_evict_last();      // X is re-read by every CTA
             int s = 0;
             uint32_t ph = 0;
-            for (long long u = u_begin; u < u_end; ++u) {
-                const int tile = static_cast<int>(u / KB);
-                const int kb = static_cast<int>(u - static_cast<long long>(tile) * KB);
-                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 2u)) break;
-                const uint32_t w_dst = base + s * Cfg::STAGE_BYTES;
-                mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
-                tma_load_2d_hint(w_dst, &tmW, full_bar(s), kb * Cfg::BK, tile * Cfg::BNW, pol_stream);
-                tma_load_2d_hint(w_dst + Cfg::W_BYTES, &tmX, full_bar(s), kb * Cfg::BK, 0, pol_keep);
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            int tile = first_tile, kb = first_kb, left = n_units;
+            bool first = true;
+            while (left > 0) {
+                int seg = min(KB - kb, left);                      // k-blocks of this band still to load
+                left -= seg;
+                while (seg > 0) {
+                    const int nkb = min(KPS, seg);
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 2u)) { left = 0; break; }
+                    const uint32_t dst = base + s * stage_bytes;
+                    mbar_expect_tx(full_bar(s), nkb * (w_bytes + Cfg::X_BYTES));
+                    for (int i = 0; i < nkb; ++i) {
+                        tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * Cfg::BK, tile * R, pol_stream);
+                        tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * Cfg::BK, 0, pol_keep);
+                    }
+                    if (first) { TRACE(2); first = false; }
+                    kb += nkb;
+                    seg -= nkb;
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                ++tile;
+                kb = 0;
             }
+            TRACE(3);
         }
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
+        const uint32_t tmem_base = *tmem_slot;
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(Cfg::BNW, Cfg::MX);
+            constexpr uint32_t idesc = umma_idesc_bf16(Cfg::LANES, Cfg::MX);
             int s = 0;
-            uint32_t ph = 0;
-            uint32_t acc_ph[2] = {0u, 0u};
-            int seg = 0;
-            bool ok = true;
-            for (long long u = u_begin; u < u_end && ok; ++seg) {
-                const int tile = static_cast<int>(u / KB);
-                const int kb0 = static_cast<int>(u - static_cast<long long>(tile) * KB);
-                const int kb1 = static_cast<int>(min(static_cast<long long>(KB), kb0 + (u_end - u)));
-                const int buf = seg & 1;
-                if (!mbar_wait(acce_bar(buf), acc_ph[buf] ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 3u)) { ok = false; break; }
-                acc_ph[buf] ^= 1u;
+            uint32_t ph = 0, acc_ph = 0;                         // bit b of acc_ph: phase of accumulator set b
+            int kb = first_kb, left = n_units, seg_idx = 0;
+            bool ok = true, first = true;
+            while (left > 0 && ok) {
+                int seg = min(KB - kb, left);
+                left -= seg;
+                const int buf = seg_idx & 1;
+                if (!mbar_wait(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 3u)) { ok = false; break; }
+                acc_ph ^= 1u << buf;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * 32);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * Cfg::ACC_COLS);
+                uint32_t step = 0;                                // MMA count within this segment
+                while (seg > 0) {
+                    const int nkb = min(KPS, seg);
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 4u)) { ok = false; break; }
+                    if (first) { TRACE(4); first = false; }
                     tc_fence_after();
-                    const uint32_t w_src = base + s * Cfg::STAGE_BYTES;
-                    const uint64_t a_desc = umma_smem_desc_sw128(w_src);
-                    const uint64_t b_desc = umma_smem_desc_sw128(w_src + Cfg::W_BYTES);
+                    const uint32_t src = base + s * stage_bytes;
+                    for (int i = 0; i < nkb; ++i) {
+                        const uint64_t a_desc = umma_smem_desc_sw128(src + i * w_bytes);
+                        const uint64_t b_desc = umma_smem_desc_sw128(src + x_off + i * Cfg::X_BYTES);
 #pragma unroll
-                    for (int k = 0; k < Cfg::BK / 16; ++k)
-                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < Cfg::BK / 16; ++k, ++step)
+                            umma_bf16(d_tmem + (step % Cfg::WAYS) * Cfg::MX, a_desc + 2u * k, b_desc + 2u * k, idesc,
+                                      step >= Cfg::WAYS ? 1u : 0u);
+                    }
                     umma_commit(empty_bar(s));
+                    seg -= nkb;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(accf_bar(buf));
-                u += kb1 - kb0;
+                kb = 0;
+                ++seg_idx;
             }
+            TRACE(5);
         }
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ epilogue / fix-up
+        const uint32_t tmem_base = *tmem_slot;
         const int q = warp & 3;
-        const int nl = q * 32 + lane;                 // row of W inside the tile = TMEM lane
+        const int nl = q * 32 + lane;                 // row of W inside the band = TMEM lane
         const int epi_tid = (warp - 2) * 32 + lane;
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
-        uint32_t acc_ph[2] = {0u, 0u};
-        int seg = 0;
+        uint32_t acc_ph = 0;
+        int tile = first_tile, kb0 = first_kb, left = n_units, seg_idx = 0;
         bool ok = true;
-        for (long long u = u_begin; u < u_end && ok; ++seg) {
-            const int tile = static_cast<int>(u / KB);
-            const int kb0 = static_cast<int>(u - static_cast<long long>(tile) * KB);
-            const int kb1 = static_cast<int>(min(static_cast<long long>(KB), kb0 + (u_end - u)));
-            const int buf = seg & 1;
-            if (!mbar_wait(accf_bar(buf), acc_ph[buf], abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 2u)) { ok = false; break; }
-            acc_ph[buf] ^= 1u;
-            tc_fence_after();
-            uint32_t r[16];
-            tmem_ld_32x32b_x16(tmem_base + lane_base + static_cast<uint32_t>(buf * 32), r);
-            tmem_ld_wait();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(buf));     // registers hold the tile: free the buffer now
-
+        if (PAIR) {
+            left = 0;                                          // the generic loop below is not used
+            const int n = first_tile * R + nl;
+            const bool row_ok = nl < R && n < p.N;
+            const float bn = (crank == 0 && row_ok && p.bias) ? __ldg(p.bias + n) : 0.0f;
             float acc[16];
 #pragma unroll
-            for (int m = 0; m < 16; ++m) acc[m] = __uint_as_float(r[m]);
+            for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+            if (n_units > 0) ok = mbar_wait(accf_bar(0), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 3u);
+            if (epi_tid == 0) TRACE(6);
+            if (ok && n_units > 0) {
+                tc_fence_after();
+                const int ways_used = min(Cfg::WAYS, n_units * (Cfg::BK / 16));
+                const uint32_t set_addr = tmem_base + lane_base;
+#pragma unroll
+                for (int w = 0; w < Cfg::WAYS; w += 2) {
+                    if (w < ways_used) {
+                        uint32_t r[32];
+                        tmem_ld_32x32b_x32(set_addr + w * Cfg::MX, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[m]);
+                        if (w + 1 < ways_used) {
+#pragma unroll
+                            for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[16 + m]);
+                        }
+                    }
+                }
+                tc_fence_before();
+            }
+            cluster_wait();                                    // set-up phase: the peer's barriers exist
+            if (crank == 1) {
+                // hand the partial to the even CTA: [m][lane] floats in its shared memory
+                const uint32_t dst = cluster_map_shared(reduce_base, 0) + static_cast<uint32_t>(nl) * 4u;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) st_shared_cluster_f32(dst + m * (Cfg::LANES * 4), ok ? acc[m] : 0.0f);
+                fence_acq_rel_cluster();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(cluster_map_shared(red_bar, 0));
+            } else if (ok) {
+                if (mbar_wait_cluster(red_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 4u)) {
+                    const float* peer = reinterpret_cast<const float*>(smem_raw + (reduce_base - raw_addr)) + nl;
+#pragma unroll
+                    for (int m = 0; m < 16; ++m) acc[m] += peer[m * Cfg::LANES];       // rank 0 + rank 1
+                    if (row_ok) {
+#pragma unroll
+                        for (int m = 0; m < 16; ++m) {
+                            if (m < p.M) {
+                                const float y = apply_act(p.act, acc[m] + bn);
+                                if (OUT_BF16)
+                                    reinterpret_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
+                                else
+                                    reinterpret_cast<float*>(p.out)[static_cast<size_t>(m) * p.N + n] = y;
+                            }
+                        }
+                    }
+                }
+            }
+            if (epi_tid == 0) TRACE(7);
+        }
+        while (left > 0 && ok) {
+            const int seg = min(KB - kb0, left);
+            left -= seg;
+            const int buf = seg_idx & 1;
+            const int n = tile * R + nl;
+            const bool row_ok = nl < R && n < p.N;
+            // fetched before the accumulator is ready so that its latency is off the tail
+            const float bn = (row_ok && p.bias) ? __ldg(p.bias + n) : 0.0f;
+            if (!mbar_wait(accf_bar(buf), (acc_ph >> buf) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 2u)) { ok = false; break; }
+            acc_ph ^= 1u << buf;
+            if (epi_tid == 0) TRACE(6);
+            tc_fence_after();
+            // Sum the accumulator ways that this segment wrote, in way order.
+            const int ways_used = min(Cfg::WAYS, seg * (Cfg::BK / 16));
+            float acc[16];
+#pragma unroll
+            for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+            const uint32_t set_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::ACC_COLS);
+#pragma unroll
+            for (int w = 0; w < Cfg::WAYS; w += 2) {
+                if (w < ways_used) {                           // warp-uniform
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(set_addr + w * Cfg::MX, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[m]);
+                    if (w + 1 < ways_used) {
+#pragma unroll
+                        for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[16 + m]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(buf));     // registers hold the band: free the set now
 
-            bool finalize = (kb0 == 0 && kb1 == KB);       // this CTA covered the tile's whole K range
+            bool finalize = (seg == KB);                   // this CTA covered the band's whole K range
             if (!finalize) {
                 const long long t_first = static_cast<long long>(tile) * KB;
                 const int c_first = skinny_cta_of_unit(t_first, p.total_units, gridDim.x);
                 const int c_last = skinny_cta_of_unit(t_first + KB - 1, p.total_units, gridDim.x);
                 const int n_contrib = c_last - c_first + 1;
                 const int slot = static_cast<int>(blockIdx.x) - c_first;
-                float* my = p.partial + (static_cast<size_t>(tile) * p.max_slots + slot) * (16 * 128) + nl;
+                float* band = p.partial + static_cast<size_t>(tile) * p.max_slots * (16 * 128) + nl;
+                float* my = band + static_cast<size_t>(slot) * (16 * 128);
 #pragma unroll
                 for (int m = 0; m < 16; ++m) __stcg(my + m * 128, acc[m]);
                 __threadfence();
@@ -192,38 +375,62 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 named_barrier_sync(1, 128);
                 if (*last_flag != 0u) {
                     __threadfence();
-                    const float* src = p.partial + static_cast<size_t>(tile) * p.max_slots * (16 * 128) + nl;
+                    if (n_contrib == 2) {
+                        // a + b == b + a exactly: adding the other CTA's partial to the registers gives
+                        // the same bits whichever of the two arrives last
+                        const float* other = band + static_cast<size_t>(1 - slot) * (16 * 128);
+                        float o[16];
 #pragma unroll
-                    for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
-                    for (int sl = 0; sl < n_contrib; ++sl) {
+                        for (int m = 0; m < 16; ++m) o[m] = __ldcg(other + m * 128);
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) acc[m] += __ldcg(src + (static_cast<size_t>(sl) * 16 + m) * 128);
+                        for (int m = 0; m < 16; ++m) acc[m] += o[m];
+                    } else {
+#pragma unroll
+                        for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+                        for (int sl = 0; sl < n_contrib; sl += 2) {          // slot order, two slots in flight
+                            float a0[16], a1[16];
+                            const bool two = sl + 1 < n_contrib;
+#pragma unroll
+                            for (int m = 0; m < 16; ++m) {
+                                a0[m] = __ldcg(band + (static_cast<size_t>(sl) * 16 + m) * 128);
+                                a1[m] = two ? __ldcg(band + (static_cast<size_t>(sl + 1) * 16 + m) * 128) : 0.0f;
+                            }
+#pragma unroll
+                            for (int m = 0; m < 16; ++m) { acc[m] += a0[m]; if (two) acc[m] += a1[m]; }
+                        }
                     }
                     finalize = true;
                 }
             }
-            if (finalize) {
-                const int n = tile * Cfg::BNW + nl;
-                if (n < p.N) {
-                    const float bn = p.bias ? __ldg(p.bias + n) : 0.0f;
+            if (finalize && row_ok) {
 #pragma unroll
-                    for (int m = 0; m < 16; ++m) {
-                        if (m < p.M) {
-                            const float y = apply_act(p.act, acc[m] + bn);
-                            if (OUT_BF16)
-                                reinterpret_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
-                            else
-                                reinterpret_cast<float*>(p.out)[static_cast<size_t>(m) * p.N + n] = y;
-                        }
+                for (int m = 0; m < 16; ++m) {
+                    if (m < p.M) {
+                        const float y = apply_act(p.act, acc[m] + bn);
+                        if (OUT_BF16)
+                            reinterpret_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
+                        else
+                            reinterpret_cast<float*>(p.out)[static_cast<size_t>(m) * p.N + n] = y;
                     }
                 }
             }
-            u += kb1 - kb0;
+            ++tile;
+            kb0 = 0;
+            ++seg_idx;
+            if (epi_tid == 0) TRACE(7);
         }
     }
 
     tc_fence_before();
     __syncthreads();
+    if (PAIR) {
+        // Neither CTA may leave while its peer can still write into (or arrive on) its shared
+        // memory.  The epilogue warps consumed the set-up phase already; the others do it here.
+        if (warp < 2) cluster_wait();
+        cluster_arrive();
+        cluster_wait();
+    }
+    if (threadIdx.x == 0) TRACE(8);
     if (*abort_flag != 0u) {
         const long long t0 = clock64();
         while (clock64() - t0 < 400000ll) __nanosleep(1000);
@@ -231,7 +438,11 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
     }
     if (warp == 1) {
         tc_fence_after();
-        tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+        tmem_dealloc(*tmem_slot, Cfg::TMEM_COLS);
+        if (lane == 0) TRACE(9);
+#ifdef MTMC_TRACE
+        if (lane == 0 && blockIdx.x < 1024) g_span[2 * blockIdx.x + 1] = gtimer();
+#endif
     }
 }
 

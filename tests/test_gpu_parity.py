@@ -139,7 +139,11 @@ def test_linear_lse_shift_law():
 
 
 # ------------------------------------------------------------------ skinny / split-K path
-@pytest.mark.parametrize("M,N,K", [(16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392)])
+@pytest.mark.parametrize("M,N,K", [
+    (16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392),   # few rows: ticketed split-K
+    (16, 4096, 512), (7, 2400, 1096), (3, 9472, 72), (16, 2368, 128),                  # cluster-pair split-K
+    (16, 20000, 256), (2, 9480, 64),                                                   # many rows / one k-block
+])
 @pytest.mark.parametrize("odt", ["fp32", "bf16"])
 def test_skinny_small(M, N, K, odt):
     li, out = run_linear(M, N, K, "gelu_tanh", odt, seed=4000 + M + N)
