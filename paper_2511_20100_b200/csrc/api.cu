@@ -152,6 +152,12 @@ int get_workspace(DeviceState* d, size_t need, void** out) {
 
 size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
+// Scratch of mtmc_linear_lse: one (max, sum-exp) pair per row and column piece; sized for the
+// narrowest tile (128 columns) and the largest tail split (4), whatever the call then picks.
+size_t lse_workspace_bytes(int64_t M, int64_t N) {
+    return round256(static_cast<size_t>((N + 127) / 128) * 4 * static_cast<size_t>(M) * sizeof(float2));
+}
+
 int pick_tile_n(int64_t N) {
     if (t_tile_n == 128 || t_tile_n == 256) return t_tile_n;
     return N > 128 ? 256 : 128;
@@ -171,24 +177,41 @@ struct TimedRegion {
 };
 
 template <int EPI, int BN, bool OUT_BF16>
-int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, GemmParams p) {
+int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
+                 const CUtensorMap& tmBt, const CUtensorMap& tmB2t, GemmParams p) {
     using Cfg = TileCfg<EPI, BN>;
     auto kern = gemm_tiled_kernel<EPI, BN, OUT_BF16>;
     CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB2, p);
+    const int grid = p.num_items < d->sm_count ? p.num_items : d->sm_count;
+    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB2, tmBt, tmB2t, p);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;
 }
 
-void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n) {
+// Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
+// form a partial wave; cutting each of them into `tail_split` column pieces (2 or 4, pieces
+// at least 32 columns wide, all pieces fitting one wave) shortens that wave accordingly.
+void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail) {
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.m_tiles = static_cast<int>((M + 127) / 128);
     p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
     p.num_tiles = p.m_tiles * p.n_tiles;
     p.k_blocks = static_cast<int>((K + 63) / 64);
     p.group_m = pick_group_m(p.m_tiles);
+    p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1; p.tail_width = out_tile_n;
+    const int r = p.num_tiles % sm_count;
+    if (split_tail && r > 0) {
+        int s = 1;
+        for (int cand = 4; cand >= 2; cand /= 2)
+            if (r * cand <= sm_count && out_tile_n / cand >= 32) { s = cand; break; }
+        if (s > 1) {
+            p.n_full = p.num_tiles - r;
+            p.tail_split = s;
+            p.tail_width = out_tile_n / s;
+            p.num_items = p.n_full + r * s;
+        }
+    }
 }
 
 int skinny_cta_of_unit_host(long long u, long long total, int grid) {
@@ -405,7 +428,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
             return s.ticket_bytes + s.partial_bytes;
         }
         case MTMC_OP_SWIGLU: return 0;
-        case MTMC_OP_LINEAR_LSE: return round256(static_cast<size_t>((N + 127) / 128) * static_cast<size_t>(M) * sizeof(float2));
+        case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N);
         default: return static_cast<size_t>(-1);
     }
 }
@@ -439,20 +462,22 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, i
 
     const int bn = pick_tile_n(N);
     GemmParams p{};
-    fill_tiling(p, M, N, K, bn);
+    fill_tiling(p, M, N, K, bn, d->sm_count, true);
     p.act = act; p.bias = b; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmBt;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
     if (rc) return rc;
     rc = encode_bf16_2d(&tmB, W, N, K, bn);
     if (rc) return rc;
+    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
+    if (rc) return rc;
     TimedRegion tr(d);
     if (bn == 256) {
-        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, p)
-                                        : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, p);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
     } else {
-        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, p)
-                                        : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, p);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
     }
     tr.stop();
     return rc;
@@ -467,17 +492,21 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     rc = get_device(&d);
     if (rc) return rc;
     GemmParams p{};
-    fill_tiling(p, M, N, K, 128);               // 128 output columns = 128 gate + 128 up accumulator columns
+    fill_tiling(p, M, N, K, 128, d->sm_count, true);   // 128 output columns = 128 gate + 128 up accumulator columns
     p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-    CUtensorMap tmA, tmG, tmU;
+    CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
     if (rc) return rc;
     rc = encode_bf16_2d(&tmG, Wg, N, K, 128);
     if (rc) return rc;
     rc = encode_bf16_2d(&tmU, Wu, N, K, 128);
     if (rc) return rc;
+    rc = encode_bf16_2d(&tmGt, Wg, N, K, p.tail_width);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmUt, Wu, N, K, p.tail_width);
+    if (rc) return rc;
     TimedRegion tr(d);
-    rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, p);
+    rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
     tr.stop();
     return rc;
 }
@@ -491,23 +520,26 @@ int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int
     if (rc) return rc;
     const int bn = pick_tile_n(N);
     GemmParams p{};
-    fill_tiling(p, M, N, K, bn);
+    fill_tiling(p, M, N, K, bn, d->sm_count, true);
     void* ws = nullptr;
-    rc = get_workspace(d, round256(static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M) * sizeof(float2)), &ws);
+    rc = get_workspace(d, lse_workspace_bytes(M, N), &ws);
     if (rc) return rc;
     p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmBt;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
     if (rc) return rc;
     rc = encode_bf16_2d(&tmB, W, N, K, bn);
     if (rc) return rc;
+    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
+    if (rc) return rc;
     TimedRegion tr(d);
-    rc = bn == 256 ? launch_tiled<EPI_LSE, 256, false>(d, tmA, tmB, tmB, p) : launch_tiled<EPI_LSE, 128, false>(d, tmA, tmB, tmB, p);
+    rc = bn == 256 ? launch_tiled<EPI_LSE, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                   : launch_tiled<EPI_LSE, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
     tr.stop();
     if (rc) return rc;
     const int rows_per_block = 8;
     lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.n_tiles, lse_out);
+        p.lse_partial, p.M, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;
@@ -575,7 +607,7 @@ int launch_lse_noalloc(NoAllocDevice* d, const CUtensorMap& tmA, const CUtensorM
     auto kern = gemm_tiled_kernel<EPI_LSE, BN, false>;
     CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
-    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB, p);
+    kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB, tmB, tmB, p);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;
@@ -611,7 +643,7 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
     if (rc) return rc;
     const int bn = pick_tile_n(N);
     GemmParams p{};
-    fill_tiling(p, M, N, K, bn);
+    fill_tiling(p, M, N, K, bn, d->sm_count, false);      // whole tiles only: one partial per column tile
     const size_t need = static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M);
     if (need > NOALLOC_MAX_PARTIALS)
         return fail(MTMC_ERR_UNSUPPORTED_SHAPE,
@@ -640,7 +672,7 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
     if (rc) return rc;
     const int rows_per_block = 8;
     lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.n_tiles, lse_out);
+        p.lse_partial, p.M, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;

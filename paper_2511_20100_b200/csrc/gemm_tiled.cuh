@@ -22,10 +22,17 @@ struct GemmParams {
     int M, N, K;
     int m_tiles, n_tiles, num_tiles, k_blocks;
     int group_m;
+    // Wave-tail split: the tiles of the last, partial wave (indices >= n_full) are cut into
+    // tail_split column pieces of tail_width output columns each, so that the wave fills the
+    // SMs with shorter work items.  tail_split == 1: no split, every item is a whole tile.
+    int n_full;           // items [0, n_full) are whole tiles
+    int num_items;        // n_full + (num_tiles - n_full) * tail_split
+    int tail_split;
+    int tail_width;       // OUT_TILE_N / tail_split, a multiple of 32
     int act;
     const float* bias;    // [N] or null
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
-    float2* lse_partial;  // [n_tiles][M] (max, sum-exp) per row and column tile (EPI_LSE)
+    float2* lse_partial;  // [n_tiles * tail_split][M] (max, sum-exp) per row and column piece (EPI_LSE)
     uint32_t* status;     // device status word
 };
 
@@ -52,6 +59,28 @@ __device__ __forceinline__ void tile_coords(const GemmParams& p, int idx, int& m
     const int gm = min(p.group_m, p.m_tiles - m_first);
     nb = r / gm;
     mb = m_first + (r - nb * gm);
+}
+// The inverse: position of tile (mb, nb) in the walk order.
+__device__ __forceinline__ int tile_index(int group_m, int m_tiles, int n_tiles, int mb, int nb) {
+    const int g = mb / group_m;
+    const int m_first = g * group_m;
+    const int gm = min(group_m, m_tiles - m_first);
+    return g * group_m * n_tiles + nb * gm + (mb - m_first);
+}
+// Work item -> row block, column tile, piece within the tile and the piece's width in output columns.
+__device__ __forceinline__ void item_coords(const GemmParams& p, int item, int full_width, int& mb, int& nb, int& sub,
+                                            int& width) {
+    if (item < p.n_full) {
+        tile_coords(p, item, mb, nb);
+        sub = 0;
+        width = full_width;
+    } else {
+        const int j = item - p.n_full;
+        const int parent = p.n_full + j / p.tail_split;
+        tile_coords(p, parent, mb, nb);
+        sub = j - (j / p.tail_split) * p.tail_split;
+        width = p.tail_width;
+    }
 }
 
 // z / (1 + exp(-z))
@@ -142,7 +171,8 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
 template <int EPI, int BN, bool OUT_BF16>
 __global__ void __launch_bounds__(192, 1)
 gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                  const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
+                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmBt,
+                  const __grid_constant__ CUtensorMap tmB2t, const GemmParams p) {
     using Cfg = TileCfg<EPI, BN>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -186,23 +216,25 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x) {
-                int mb, nb;
-                tile_coords(p, t, mb, nb);
+            for (int t = blockIdx.x; t < p.num_items && ok; t += gridDim.x) {
+                int mb, nb, sub, width;
+                item_coords(p, t, Cfg::OUT_TILE_N, mb, nb, sub, width);
+                const bool whole = width == Cfg::OUT_TILE_N;
                 const int m0 = mb * Cfg::BM;
-                const int n0 = nb * Cfg::OUT_TILE_N;
+                const int n0 = nb * Cfg::OUT_TILE_N + sub * width;
+                const uint32_t b_rows_bytes = static_cast<uint32_t>(width) * Cfg::BK * 2;   // one W box of this item
+                const uint32_t tx = Cfg::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes;
+                const CUtensorMap* mapB = whole ? &tmB : &tmBt;
+                const CUtensorMap* mapB2 = whole ? &tmB2 : &tmB2t;
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 1u)) { ok = false; break; }
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
-                    mbar_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    mbar_expect_tx(full_bar(s), tx);
                     tma_load_2d(a_dst, &tmA, full_bar(s), kb * Cfg::BK, m0);
-                    if (EPI == EPI_SWIGLU) {
-                        tma_load_2d(b_dst, &tmB, full_bar(s), kb * Cfg::BK, n0);
-                        tma_load_2d(b_dst + Cfg::B_BYTES / 2, &tmB2, full_bar(s), kb * Cfg::BK, n0);
-                    } else {
-                        tma_load_2d(b_dst, &tmB, full_bar(s), kb * Cfg::BK, n0);
-                    }
+                    tma_load_2d(b_dst, mapB, full_bar(s), kb * Cfg::BK, n0);
+                    if (EPI == EPI_SWIGLU)      // the up rows follow the gate rows: one contiguous B operand
+                        tma_load_2d(b_dst + b_rows_bytes, mapB2, full_bar(s), kb * Cfg::BK, n0);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -211,16 +243,17 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(Cfg::BM, BN);
             int s = 0;
             uint32_t ph = 0;
-            uint32_t acc_ph[2] = {0u, 0u};
+            uint32_t acc_ph = 0;                         // bit b: phase of accumulator buffer b
             int it = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++it) {
+            for (int t = blockIdx.x; t < p.num_items && ok; t += gridDim.x, ++it) {
                 const int buf = it & 1;
-                if (!mbar_wait(acce_bar(buf), acc_ph[buf] ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 1u)) { ok = false; break; }
-                acc_ph[buf] ^= 1u;
+                const int width = t < p.n_full ? Cfg::OUT_TILE_N : p.tail_width;
+                const uint32_t idesc = umma_idesc_bf16(Cfg::BM, EPI == EPI_SWIGLU ? 2 * width : width);
+                if (!mbar_wait(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 1u)) { ok = false; break; }
+                acc_ph ^= 1u << buf;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * BN);
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
@@ -244,23 +277,24 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
-        uint32_t acc_ph[2] = {0u, 0u};
+        uint32_t acc_ph = 0;
         int it = 0;
         bool ok = true;
-        for (int t = blockIdx.x; t < p.num_tiles && ok; t += gridDim.x, ++it) {
+        for (int t = blockIdx.x; t < p.num_items && ok; t += gridDim.x, ++it) {
             const int buf = it & 1;
-            int mb, nb;
-            tile_coords(p, t, mb, nb);
+            int mb, nb, sub, width;
+            item_coords(p, t, Cfg::OUT_TILE_N, mb, nb, sub, width);
             const int row = mb * Cfg::BM + q * 32 + lane;
-            const int n_tile0 = nb * Cfg::OUT_TILE_N;
-            if (!mbar_wait(accf_bar(buf), acc_ph[buf], abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 1u)) { ok = false; break; }
-            acc_ph[buf] ^= 1u;
+            const int n_tile0 = nb * Cfg::OUT_TILE_N + sub * width;
+            const int chunks = width / 32;
+            if (!mbar_wait(accf_bar(buf), (acc_ph >> buf) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 1u)) { ok = false; break; }
+            acc_ph ^= 1u << buf;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * BN);
 
             if (EPI == EPI_ACT) {
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = 0; c < chunks; ++c) {
                     const int n0 = n_tile0 + c * 32;
                     if (n0 >= p.N) break;            // warp-uniform
                     uint32_t r[32];
@@ -275,12 +309,12 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 }
             } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-                for (int c = 0; c < BN / 64; ++c) {
+                for (int c = 0; c < chunks; ++c) {
                     const int n0 = n_tile0 + c * 32;
                     if (n0 >= p.N) break;
                     uint32_t g[32], u[32];
                     tmem_ld_32x32b_x32(t_addr + c * 32, g);                 // gate columns
-                    tmem_ld_32x32b_x32(t_addr + BN / 2 + c * 32, u);        // up columns
+                    tmem_ld_32x32b_x32(t_addr + width + c * 32, u);         // up columns follow the gate columns
                     tmem_ld_wait();
                     float y[32];
 #pragma unroll
@@ -292,7 +326,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                 constexpr float LOG2E = 1.4426950408889634f;
                 float mx = -INFINITY, sum = 0.0f;
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = 0; c < chunks; ++c) {
                     const int n0 = n_tile0 + c * 32;
                     if (n0 >= p.N) break;
                     uint32_t r[32];
@@ -314,8 +348,10 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     sum = sum * ex2_approx(mx - nm) + cs;
                     mx = nm;
                 }
+                // a piece that lies wholly past N (only possible in the last column tile) stays neutral
                 if (row < p.M)
-                    p.lse_partial[static_cast<size_t>(nb) * p.M + row] = make_float2(mx * 0.6931471805599453f, sum);
+                    p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] =
+                        make_float2(mx * 0.6931471805599453f, sum);
             }
             // accumulator buffer drained: hand it back to the MMA warp
             tc_fence_before();
@@ -349,17 +385,23 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
     m = nm;
 }
 
-// Merges the per-column-tile (max, sum-exp) partials of each row, in ascending
-// tile order, into lse[row] = max + ln(sum).  One warp per row; lanes stride over
-// the partials and combine with shuffles.
-__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int n_parts, float* __restrict__ lse) {
+// Merges the (max, sum-exp) partials of each row, in ascending column order, into
+// lse[row] = max + ln(sum).  One warp per row; lanes stride over the column tiles and
+// combine with shuffles.  A whole tile left one partial (piece 0), a tile of the split
+// wave tail left tail_split of them.
+__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int m_tiles, int n_tiles, int group_m,
+                                 int n_full, int tail_split, float* __restrict__ lse) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
+    const int mb = row >> 7;
     float mx = -INFINITY, sum = 0.0f;
-    for (int i = lane; i < n_parts; i += 32) {
-        const float2 v = __ldcg(partial + static_cast<size_t>(i) * M + row);
-        lse_combine(mx, sum, v.x, v.y);
+    for (int nb = lane; nb < n_tiles; nb += 32) {
+        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+        for (int sub = 0; sub < pieces; ++sub) {
+            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split + sub) * M + row);
+            lse_combine(mx, sum, v.x, v.y);
+        }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
