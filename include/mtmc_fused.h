@@ -168,11 +168,14 @@ int64_t mtmc_launch_count(void);
 int mtmc_set_timing(int enabled);
 float mtmc_last_kernel_ms(void);
 
-/* Tuning hooks (0 / negative = automatic).  They select among kernels of this
- * library only; results stay within tolerance of each other.
- *   split_k : number of K splits requested on the skinny path
- *   tile_n  : 128 or 256, accumulator tile width of the tiled path          */
-int mtmc_set_tuning(int split_k, int tile_n);
+/* Tuning hooks (0 = automatic).  They select among kernels of this library only; results
+ * stay within tolerance of each other.  Thread-local.
+ *   split_k  : > 0 forces the ticketed split-K plan of the skinny path with this many K
+ *              splits per 128-row band of W
+ *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
+ *   cta_pair : > 0 forces the CTA-pair (cta_group::2, 256-row tiles) tiled kernel,
+ *              < 0 forbids it; automatic = pairs when M >= 512 and N >= 256          */
+int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
 
 /* Library version: major * 10000 + minor * 100 + patch. */
 int mtmc_version(void);

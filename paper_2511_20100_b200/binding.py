@@ -61,7 +61,7 @@ def load() -> ctypes.CDLL:
     L.mtmc_launch_count.restype = i64
     L.mtmc_set_timing.argtypes = [ci]
     L.mtmc_last_kernel_ms.restype = ctypes.c_float
-    L.mtmc_set_tuning.argtypes = [ci, ci]
+    L.mtmc_set_tuning.argtypes = [ci, ci, ci]
     _lib = L
     return L
 
@@ -212,8 +212,8 @@ def mtmc_last_kernel_ms() -> float:
     return float(load().mtmc_last_kernel_ms())
 
 
-def mtmc_set_tuning(split_k: int = 0, tile_n: int = 0) -> None:
-    _check(load().mtmc_set_tuning(int(split_k), int(tile_n)))
+def mtmc_set_tuning(split_k: int = 0, tile_n: int = 0, cta_pair: int = 0) -> None:
+    _check(load().mtmc_set_tuning(int(split_k), int(tile_n), int(cta_pair)))
 
 
 def mtmc_version() -> int:

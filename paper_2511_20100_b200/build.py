@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmtmcfused.so")
 SOURCES = ["api.cu"]
-HEADERS = ["ptx.cuh", "gemm_tiled.cuh", "skinny.cuh"]
+HEADERS = ["ptx.cuh", "gemm_tiled.cuh", "gemm_pair.cuh", "skinny.cuh"]
 
 
 def _nvcc() -> str:
@@ -36,7 +36,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("MTMC_NVCC_FLAGS", "").split()
     cmd += [os.path.join(CSRC, f) for f in SOURCES]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

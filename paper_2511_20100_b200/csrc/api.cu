@@ -14,6 +14,7 @@
 #include <cstring>
 #include <mutex>
 
+#include "gemm_pair.cuh"
 #include "skinny.cuh"
 
 namespace {
@@ -37,6 +38,7 @@ struct DeviceState {
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     bool timed = false;
     int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
+    int max_gemm_pairs = -1;         // the same for the CTA-pair tiled kernel
 };
 
 std::mutex g_mutex;
@@ -48,6 +50,7 @@ thread_local void* t_user_ws = nullptr;
 thread_local size_t t_user_ws_bytes = 0;
 thread_local int t_split_k = 0;
 thread_local int t_tile_n = 0;
+thread_local int t_cta_pair = 0;   // 0 automatic, 1 force CTA pairs, -1 force single CTAs
 thread_local int t_timing = 0;
 thread_local char t_error[512] = "";
 
@@ -189,16 +192,74 @@ int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB,
     return MTMC_OK;
 }
 
+template <int EPI, bool OUT_BF16>
+int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
+                const CUtensorMap& tmBt, const CUtensorMap& tmB2t, const GemmParams& p) {
+    using Cfg = PairCfg<EPI>;
+    auto kern = gemm_pair_kernel<EPI, OUT_BF16>;
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    const int pairs = p.num_items < clusters ? p.num_items : clusters;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmBt, tmB2t, p));
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
+// How many CTA pairs of the pair kernel fit on the device at once (0: clusters unavailable).
+int gemm_pairs(DeviceState* d) {
+    if (d->max_gemm_pairs < 0) {
+        auto kern = gemm_pair_kernel<EPI_ACT, true>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2u * static_cast<unsigned>(d->sm_count), 1, 1);
+        cfg.blockDim = dim3(192, 1, 1);
+        cfg.dynamicSmemBytes = PairCfg<EPI_ACT>::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PairCfg<EPI_ACT>::SMEM_BYTES) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        d->max_gemm_pairs = n;
+    }
+    return d->max_gemm_pairs;
+}
+
+// Large problems go to CTA pairs (256-row tiles); small ones keep single-CTA 128-row tiles.
+bool use_pair(DeviceState* d, int64_t M, int64_t N) {
+    if (t_cta_pair < 0 || t_tile_n == 128 || gemm_pairs(d) <= 0) return false;
+    if (t_cta_pair > 0) return true;
+    return M >= 512 && N >= 256;
+}
+
 // Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
 // form a partial wave; cutting each of them into `tail_split` column pieces (2 or 4, pieces
 // at least 32 columns wide, all pieces fitting one wave) shortens that wave accordingly.
-void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail) {
+void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail, int bm = 128) {
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
-    p.m_tiles = static_cast<int>((M + 127) / 128);
+    p.m_tiles = static_cast<int>((M + bm - 1) / bm);
+    p.rows_per_tile = bm;
     p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
     p.num_tiles = p.m_tiles * p.n_tiles;
     p.k_blocks = static_cast<int>((K + 63) / 64);
-    p.group_m = pick_group_m(p.m_tiles);
+    p.group_m = bm == 256 ? (p.m_tiles < 8 ? p.m_tiles : 8) : pick_group_m(p.m_tiles);
     p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1; p.tail_width = out_tile_n;
     const int r = p.num_tiles % sm_count;
     if (split_tail && r > 0) {
@@ -245,15 +306,6 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
             s.tile_rows = static_cast<int>(rows);
             s.n_tiles = static_cast<int>((N + rows - 1) / rows);
             g = 2ll * s.n_tiles;
-        }
-    }
-    if (const char* e = getenv("MTMC_SKINNY")) {   // development knob: "rows,split" (ticket plan)
-        int r = 0, sp = 0;
-        if (sscanf(e, "%d,%d", &r, &sp) == 2 && r >= 8 && r <= 128 && r % 8 == 0) {
-            s.pair = 0;
-            s.tile_rows = r;
-            s.n_tiles = static_cast<int>((N + r - 1) / r);
-            g = sp > 0 ? static_cast<long long>(s.n_tiles) * sp : sm_count;
         }
     }
     s.total = static_cast<long long>(s.n_tiles) * s.k_blocks;
@@ -395,10 +447,11 @@ int mtmc_set_workspace(void* dptr, size_t bytes) {
     return MTMC_OK;
 }
 
-int mtmc_set_tuning(int split_k, int tile_n) {
+int mtmc_set_tuning(int split_k, int tile_n, int cta_pair) {
     if (tile_n > 0 && tile_n != 128 && tile_n != 256) return fail(MTMC_ERR_INVALID_ARG, "tile_n must be 128 or 256");
     t_split_k = split_k > 0 ? split_k : 0;
     t_tile_n = tile_n > 0 ? tile_n : 0;
+    t_cta_pair = cta_pair > 0 ? 1 : (cta_pair < 0 ? -1 : 0);
     return MTMC_OK;
 }
 
@@ -460,6 +513,20 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, i
     if (rc) return rc;
     if (use_skinny(M, N)) return run_skinny(d, X, W, b, M, N, K, act, out_dtype, out);
 
+    if (use_pair(d, M, N)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+        p.act = act; p.bias = b; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB, tmBt;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
+            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
+            return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+        tr.stop();
+        return rc;
+    }
     const int bn = pick_tile_n(N);
     GemmParams p{};
     fill_tiling(p, M, N, K, bn, d->sm_count, true);
@@ -491,6 +558,20 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
+    if (use_pair(d, M, N)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 128, gemm_pairs(d), true, 256);
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmG, Wg, N, K, 128)) ||
+            (rc = encode_bf16_2d(&tmU, Wu, N, K, 128)) || (rc = encode_bf16_2d(&tmGt, Wg, N, K, p.tail_width)) ||
+            (rc = encode_bf16_2d(&tmUt, Wu, N, K, p.tail_width)))
+            return rc;
+        TimedRegion tr(d);
+        rc = launch_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, tmGt, tmUt, p);
+        tr.stop();
+        return rc;
+    }
     GemmParams p{};
     fill_tiling(p, M, N, K, 128, d->sm_count, true);   // 128 output columns = 128 gate + 128 up accumulator columns
     p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
@@ -518,12 +599,30 @@ int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
-    const int bn = pick_tile_n(N);
+    const bool pair = use_pair(d, M, N);
+    const int bn = pair ? 256 : pick_tile_n(N);
     GemmParams p{};
-    fill_tiling(p, M, N, K, bn, d->sm_count, true);
+    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+    else fill_tiling(p, M, N, K, bn, d->sm_count, true);
     void* ws = nullptr;
     rc = get_workspace(d, lse_workspace_bytes(M, N), &ws);
     if (rc) return rc;
+    if (pair) {
+        p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
+        CUtensorMap tmA, tmB, tmBt;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
+            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
+            return rc;
+        TimedRegion tr(d);
+        rc = launch_pair<EPI_LSE, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+        tr.stop();
+        if (rc) return rc;
+        lse_merge_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, t_stream>>>(
+            p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
+        CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(1);
+        return MTMC_OK;
+    }
     p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
     CUtensorMap tmA, tmB, tmBt;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
@@ -539,7 +638,7 @@ int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int
     if (rc) return rc;
     const int rows_per_block = 8;
     lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
+        p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;
@@ -614,25 +713,6 @@ int launch_lse_noalloc(NoAllocDevice* d, const CUtensorMap& tmA, const CUtensorM
 }
 }  // namespace
 
-#ifdef MTMC_TRACE
-__global__ void __launch_bounds__(192, 1) null_kernel(const __grid_constant__ CUtensorMap a, const __grid_constant__ CUtensorMap b, int x) {
-    extern __shared__ uint8_t sm[];
-    if (x == 12345) sm[threadIdx.x] = reinterpret_cast<const uint8_t*>(&a)[threadIdx.x & 63] + reinterpret_cast<const uint8_t*>(&b)[0];
-}
-extern "C" int mtmc_debug_null(int grid, int smem) {
-    CUtensorMap m; memset(&m, 0, sizeof m);
-    cudaFuncSetAttribute(null_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    null_kernel<<<grid, 192, smem, t_stream>>>(m, m, 0);
-    return cudaGetLastError() == cudaSuccess ? 0 : 4;
-}
-extern "C" int mtmc_debug_span(unsigned long long* out) {
-    return cudaMemcpyFromSymbol(out, mtmc::g_span, sizeof(unsigned long long) * 2048) == cudaSuccess ? 0 : 4;
-}
-extern "C" int mtmc_debug_trace(long long* out) {
-    return cudaMemcpyFromSymbol(out, mtmc::g_trace, sizeof(long long) * 8 * 16) == cudaSuccess ? 0 : 4;
-}
-#endif
-
 extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K,
                                        float* lse_out) {
     int rc = check_common(X, W, lse_out, M, N, K);
@@ -672,7 +752,7 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
     if (rc) return rc;
     const int rows_per_block = 8;
     lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
+        p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;

@@ -21,6 +21,7 @@ enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
 struct GemmParams {
     int M, N, K;
     int m_tiles, n_tiles, num_tiles, k_blocks;
+    int rows_per_tile;    // 128 (one CTA per tile) or 256 (CTA pair)
     int group_m;
     // Wave-tail split: the tiles of the last, partial wave (indices >= n_full) are cut into
     // tail_split column pieces of tail_width output columns each, so that the wave fills the
@@ -168,6 +169,77 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
     }
 }
 
+// One work item's epilogue for one thread: this thread owns output row `row` (TMEM lane
+// of t_addr) and walks the item's columns [n_tile0, n_tile0 + 32 * chunks) in chunks of 32.
+//   EPI_ACT    : + bias, activation, store
+//   EPI_SWIGLU : silu(gate) * up with the up columns `width` columns after the gate columns
+//   EPI_LSE    : online (max, sum-exp) in base-2 units, one partial per (row, column piece)
+template <int EPI, bool OUT_BF16>
+__device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int chunks,
+                                              int width, int nb, int sub, bool vec_ok) {
+    if (EPI == EPI_ACT) {
+#pragma unroll 1
+        for (int c = 0; c < chunks; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            if (n0 >= p.N) break;            // warp-uniform
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + c * 32, r);
+            float bv[32], y[32];
+            load_bias_chunk(p.bias, n0, p.N, bv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
+            apply_act_chunk(p.act, y);
+            if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, vec_ok);
+        }
+    } else if (EPI == EPI_SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < chunks; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            if (n0 >= p.N) break;
+            uint32_t g[32], u[32];
+            tmem_ld_32x32b_x32(t_addr + c * 32, g);                 // gate columns
+            tmem_ld_32x32b_x32(t_addr + width + c * 32, u);         // up columns follow the gate columns
+            tmem_ld_wait();
+            float y[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+            if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, vec_ok);
+        }
+    } else {
+        // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
+        constexpr float LOG2E = 1.4426950408889634f;
+        float mx = -INFINITY, sum = 0.0f;
+#pragma unroll 1
+        for (int c = 0; c < chunks; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            if (n0 >= p.N) break;
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + c * 32, r);
+            float bv[32], tv[32];
+            load_bias_chunk(p.bias, n0, p.N, bv);
+            tmem_ld_wait();
+            float cm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                // columns past N are zero-filled weight rows: mask them out of the reduction
+                tv[j] = (n0 + j < p.N) ? (__uint_as_float(r[j]) + bv[j]) * LOG2E : -INFINITY;
+                cm = fmaxf(cm, tv[j]);
+            }
+            const float nm = fmaxf(mx, cm);
+            float cs = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) cs += ex2_approx(tv[j] - nm);
+            sum = sum * ex2_approx(mx - nm) + cs;
+            mx = nm;
+        }
+        // a piece that lies wholly past N (only possible in the last column tile) stays neutral
+        if (row < p.M)
+            p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] =
+                make_float2(mx * 0.6931471805599453f, sum);
+    }
+}
+
 template <int EPI, int BN, bool OUT_BF16>
 __global__ void __launch_bounds__(192, 1)
 gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -292,67 +364,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * BN);
 
-            if (EPI == EPI_ACT) {
-#pragma unroll 1
-                for (int c = 0; c < chunks; ++c) {
-                    const int n0 = n_tile0 + c * 32;
-                    if (n0 >= p.N) break;            // warp-uniform
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(t_addr + c * 32, r);
-                    float bv[32], y[32];
-                    load_bias_chunk(p.bias, n0, p.N, bv);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
-                    apply_act_chunk(p.act, y);
-                    if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, vec_ok);
-                }
-            } else if (EPI == EPI_SWIGLU) {
-#pragma unroll 1
-                for (int c = 0; c < chunks; ++c) {
-                    const int n0 = n_tile0 + c * 32;
-                    if (n0 >= p.N) break;
-                    uint32_t g[32], u[32];
-                    tmem_ld_32x32b_x32(t_addr + c * 32, g);                 // gate columns
-                    tmem_ld_32x32b_x32(t_addr + width + c * 32, u);         // up columns follow the gate columns
-                    tmem_ld_wait();
-                    float y[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
-                    if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, vec_ok);
-                }
-            } else {
-                // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
-                constexpr float LOG2E = 1.4426950408889634f;
-                float mx = -INFINITY, sum = 0.0f;
-#pragma unroll 1
-                for (int c = 0; c < chunks; ++c) {
-                    const int n0 = n_tile0 + c * 32;
-                    if (n0 >= p.N) break;
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(t_addr + c * 32, r);
-                    float bv[32], tv[32];
-                    load_bias_chunk(p.bias, n0, p.N, bv);
-                    tmem_ld_wait();
-                    float cm = -INFINITY;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        // columns past N are zero-filled weight rows: mask them out of the reduction
-                        tv[j] = (n0 + j < p.N) ? (__uint_as_float(r[j]) + bv[j]) * LOG2E : -INFINITY;
-                        cm = fmaxf(cm, tv[j]);
-                    }
-                    const float nm = fmaxf(mx, cm);
-                    float cs = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) cs += ex2_approx(tv[j] - nm);
-                    sum = sum * ex2_approx(mx - nm) + cs;
-                    mx = nm;
-                }
-                // a piece that lies wholly past N (only possible in the last column tile) stays neutral
-                if (row < p.M)
-                    p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] =
-                        make_float2(mx * 0.6931471805599453f, sum);
-            }
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, chunks, width, nb, sub, vec_ok);
             // accumulator buffer drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
@@ -389,12 +401,12 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
 // lse[row] = max + ln(sum).  One warp per row; lanes stride over the column tiles and
 // combine with shuffles.  A whole tile left one partial (piece 0), a tile of the split
 // wave tail left tail_split of them.
-__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int m_tiles, int n_tiles, int group_m,
+__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles, int group_m,
                                  int n_full, int tail_split, float* __restrict__ lse) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
-    const int mb = row >> 7;
+    const int mb = row / rows_per_tile;
     float mx = -INFINITY, sum = 0.0f;
     for (int nb = lane; nb < n_tiles; nb += 32) {
         const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;

@@ -70,14 +70,6 @@ struct SkinnyCfg {
     }
 };
 
-#ifdef MTMC_TRACE
-__device__ long long g_trace[8 * 16];
-__device__ unsigned long long g_span[2 * 1024];
-__device__ __forceinline__ unsigned long long gtimer() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define TRACE(i) do { if (blockIdx.x >= 112 && blockIdx.x < 120) g_trace[(blockIdx.x - 112) * 16 + (i)] = clock64(); } while (0)
-#else
-#define TRACE(i) do { } while (0)
-#endif
 
 __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, int grid) {
     return static_cast<int>(((u + 1) * grid - 1) / total);
@@ -113,10 +105,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) TRACE(0);
-#ifdef MTMC_TRACE
-    if (threadIdx.x == 0 && blockIdx.x < 1024) g_span[2 * blockIdx.x] = gtimer();
-#endif
     const int KB = p.k_blocks;
     // This CTA's share of the unit list.
     int first_tile, first_kb, n_units;
@@ -180,7 +168,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             int s = 0;
             uint32_t ph = 0;
             int tile = first_tile, kb = first_kb, left = n_units;
-            bool first = true;
             while (left > 0) {
                 int seg = min(KB - kb, left);                      // k-blocks of this band still to load
                 left -= seg;
@@ -193,7 +180,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                         tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * Cfg::BK, tile * R, pol_stream);
                         tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * Cfg::BK, 0, pol_keep);
                     }
-                    if (first) { TRACE(2); first = false; }
                     kb += nkb;
                     seg -= nkb;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -201,7 +187,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 ++tile;
                 kb = 0;
             }
-            TRACE(3);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -212,7 +197,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             int s = 0;
             uint32_t ph = 0, acc_ph = 0;                         // bit b of acc_ph: phase of accumulator set b
             int kb = first_kb, left = n_units, seg_idx = 0;
-            bool ok = true, first = true;
+            bool ok = true;
             while (left > 0 && ok) {
                 int seg = min(KB - kb, left);
                 left -= seg;
@@ -225,7 +210,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 while (seg > 0) {
                     const int nkb = min(KPS, seg);
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 4u)) { ok = false; break; }
-                    if (first) { TRACE(4); first = false; }
                     tc_fence_after();
                     const uint32_t src = base + s * stage_bytes;
                     for (int i = 0; i < nkb; ++i) {
@@ -244,7 +228,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 kb = 0;
                 ++seg_idx;
             }
-            TRACE(5);
         }
         __syncwarp();
     } else {
@@ -266,7 +249,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 #pragma unroll
             for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
             if (n_units > 0) ok = mbar_wait(accf_bar(0), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 3u);
-            if (epi_tid == 0) TRACE(6);
             if (ok && n_units > 0) {
                 tc_fence_after();
                 const int ways_used = min(Cfg::WAYS, n_units * (Cfg::BK / 16));
@@ -315,7 +297,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     }
                 }
             }
-            if (epi_tid == 0) TRACE(7);
         }
         while (left > 0 && ok) {
             const int seg = min(KB - kb0, left);
@@ -327,7 +308,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             const float bn = (row_ok && p.bias) ? __ldg(p.bias + n) : 0.0f;
             if (!mbar_wait(accf_bar(buf), (acc_ph >> buf) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 2u)) { ok = false; break; }
             acc_ph ^= 1u << buf;
-            if (epi_tid == 0) TRACE(6);
             tc_fence_after();
             // Sum the accumulator ways that this segment wrote, in way order.
             const int ways_used = min(Cfg::WAYS, seg * (Cfg::BK / 16));
@@ -417,7 +397,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             ++tile;
             kb0 = 0;
             ++seg_idx;
-            if (epi_tid == 0) TRACE(7);
         }
     }
 
@@ -430,7 +409,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         cluster_arrive();
         cluster_wait();
     }
-    if (threadIdx.x == 0) TRACE(8);
     if (*abort_flag != 0u) {
         const long long t0 = clock64();
         while (clock64() - t0 < 400000ll) __nanosleep(1000);
@@ -439,10 +417,6 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(*tmem_slot, Cfg::TMEM_COLS);
-        if (lane == 0) TRACE(9);
-#ifdef MTMC_TRACE
-        if (lane == 0 && blockIdx.x < 1024) g_span[2 * blockIdx.x + 1] = gtimer();
-#endif
     }
 }
 

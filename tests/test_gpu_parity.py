@@ -74,6 +74,31 @@ def test_fused_linear_both_tile_widths(tile_n):
     _assert_close(inputs.to_f64(out), want, TOL["fp32"], "tile_n %d" % tile_n)
 
 
+@pytest.mark.parametrize("cta_pair", [1, -1])
+def test_cta_pair_and_single_cta_kernels_agree_with_the_oracle(cta_pair):
+    """Both tiled kernels on the same ragged shapes: 256-row CTA-pair tiles and 128-row single-CTA tiles."""
+    B.mtmc_set_tuning(cta_pair=cta_pair)
+    try:
+        li, out = run_linear(600, 1000, 328, "gelu_tanh", "bf16", seed=81)
+        si = inputs.swiglu_inputs(520, 648, 256, seed=82)
+        sw = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+        ll = inputs.linear_inputs(700, 3000, 192, seed=83)
+        lse = B.mtmc_linear_lse(ll.X.cuda(), ll.W.cuda(), ll.b.cuda())
+        one = inputs.linear_inputs(129, 257, 72, seed=84)             # second CTA of the pair almost empty
+        o1 = B.mtmc_fused_linear(one.X.cuda(), one.W.cuda(), one.b.cuda(), "relu", "fp32")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(out), ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b),
+                                                       ref.ACT_GELU_TANH), TOL["bf16"], "fused_linear")
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "swiglu")
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(inputs.bf16_bits(ll.X), inputs.bf16_bits(ll.W), inputs.f32(ll.b)),
+                  TOL["fp32"], "linear_lse")
+    _assert_close(inputs.to_f64(o1), ref.fused_linear(inputs.bf16_bits(one.X), inputs.bf16_bits(one.W), inputs.f32(one.b),
+                                                      ref.ACT_RELU), TOL["fp32"], "129x257x72")
+
+
 def test_fused_linear_exact_integers_and_no_bias():
     # integer-valued operands: every product and fp32 partial sum is exact, so the result must be too
     g = torch.Generator().manual_seed(5)
