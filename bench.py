@@ -120,6 +120,15 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def reduce_max(dist, value: float, device) -> float:
+    """Max over ranks of a per-rank time (identity without a process group)."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 # --------------------------------------------------------------------------------------- our arm
 def make_device_problem(name, device):
     c = inputs.CONFIGS[name]
@@ -246,11 +255,7 @@ def run_ours(args, rank, world, local_rank):
         dist.barrier()
     launches = B.mtmc_launch_count() - launches0
     B.mtmc_check_status()
-    total_ms = ev[0].elapsed_time(ev[args.steps])
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = reduce_max(dist, ev[0].elapsed_time(ev[args.steps]), device)
     ms_per_step = total_ms / args.steps
 
     # ---- per configuration: the same call back to back, rotating over enough copies of the
@@ -314,15 +319,15 @@ def run_ours(args, rank, world, local_rank):
     dom = per_config[dom_name]
     roofline = dict(dom.get("roofline", {"bound": "tensor", "achieved": dom["tflops"], "peak": peaks["tflops_sustained"],
                                           "unit": "TFLOP/s", "frac": round(dom["tflops"] / peaks["tflops_sustained"], 4)}))
-    roofline["kernel"] = ("skinny_splitk_kernel" if dom_name == "C5" else "gemm_tiled_kernel") + " on " + dom_name
+    roofline["kernel"] = ("skinny_splitk_kernel" if dom_name == "C5" else "gemm_pair_kernel (tcgen05 cta_group::2)") + " on " + dom_name
     roofline["peak_source"] = peaks["source"] + (" copy bandwidth" if dom_name == "C5" else " sustained cuBLAS bf16")
     roofline["traffic"] = None
-    prof = os.path.join(ROOT, "profiles", "traffic.json")
+    prof = os.path.join(ROOT, "profiles", "traffic.txt")      # DRAM bytes per launch from the committed ncu summaries
     if os.path.exists(prof):
-        try:
-            roofline["traffic"] = json.load(open(prof)).get("%s_dram_bytes_per_launch" % dom_name)
-        except Exception:
-            pass
+        for ln in open(prof):
+            tok = ln.split()
+            if len(tok) == 2 and tok[0] == "%s_dram_bytes_per_launch" % dom_name:
+                roofline["traffic"] = int(tok[1])
 
     # ------------------------------------------------------------------ end to end through the host-pointer C ABI
     e2e = None
@@ -346,11 +351,7 @@ def run_ours(args, rank, world, local_rank):
             for pr, pn in zip(problems, pinned):
                 call_host(B, pr, pn, local_rank)
         torch.cuda.synchronize()
-        e2e_s = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([e2e_s], dtype=torch.float64, device=device)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = float(t.item())
+        e2e_s = reduce_max(dist, time.perf_counter() - t0, device)
         e2e = {"value": round(world * step_flops * e2e_steps / e2e_s / 1e12, 3), "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                "ms_per_step": round(e2e_s / e2e_steps * 1e3, 3),
