@@ -168,6 +168,19 @@ def call_host(B, pr, pinned, dev_index):
                                  out=pinned["out"], device=dev_index)
 
 
+def eager_call(pr, dev):
+    """The unfused PyTorch-eager sequence of the same operator (context only: it rounds the GEMM
+    result to bf16 before the epilogue, and it is not on the product path)."""
+    c = pr["cfg"]
+    if c["op"] == "swiglu":
+        return torch.nn.functional.silu(dev[0] @ dev[1].T) * (dev[0] @ dev[2].T)
+    if c["op"] == "linear_lse":
+        return torch.logsumexp((dev[0] @ dev[1].T).float() + dev[2], dim=-1)
+    z = (dev[0] @ dev[1].T).float() + dev[2]
+    z = torch.relu(z) if c["act"] == "relu" else torch.nn.functional.gelu(z, approximate="tanh")
+    return z if c["out_dtype"] == "fp32" else z.to(torch.bfloat16)
+
+
 def cpu_baseline_sample():
     """The oracle timed on a bounded sample: the first REF_ROWS rows of every configuration."""
     from oracle import ref
@@ -262,7 +275,7 @@ def run_ours(args, rank, world, local_rank):
     # operands that their total exceeds twice the L2 (so every launch reads its operands from HBM);
     # one event pair around the loop, so launch overhead is amortised as it is inside a step.
     L2_BYTES = 126e6
-    per_cfg_ms, per_cfg_reps, per_cfg_copies = {}, {}, {}
+    per_cfg_ms, per_cfg_reps, per_cfg_copies, per_cfg_eager = {}, {}, {}, {}
     for pr in problems:
         n, c = pr["name"], pr["cfg"]
         nbytes = sum(t.numel() * t.element_size() for t in pr["dev"] if t is not None)
@@ -286,6 +299,18 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         per_cfg_ms[n] = e0.elapsed_time(e1) / reps
         per_cfg_reps[n], per_cfg_copies[n] = reps, copies
+        if not args.no_eager:
+            # context: the unfused torch sequence (cuBLAS GEMM + elementwise kernels), same rotation
+            for v in variants:
+                eager_call(pr, v["dev"])
+            torch.cuda.synchronize()
+            ereps = max(5, reps // 4)
+            e0.record()
+            for r in range(ereps):
+                eager_call(pr, variants[r % copies]["dev"])
+            e1.record()
+            torch.cuda.synchronize()
+            per_cfg_eager[n] = e0.elapsed_time(e1) / ereps
         del variants
     B.mtmc_check_status()
     clocks = sampler.stop()
@@ -300,6 +325,9 @@ def run_ours(args, rank, world, local_rank):
         entry = {"call": c["op"], "M": c["M"], "N": c["N"], "K": c["K"], "ms": round(ms, 5),
                  "launches_timed": per_cfg_reps[n], "operand_copies_rotated": per_cfg_copies[n],
                  "tflops": round(flops(c) / (ms * 1e-3) / 1e12, 3), "gbs": round(algorithmic_bytes(c) / (ms * 1e-3) / 1e9, 2)}
+        if n in per_cfg_eager:
+            entry["eager_ms"] = round(per_cfg_eager[n], 5)
+            entry["speedup_vs_eager"] = round(per_cfg_eager[n] / ms, 3)
         if n == "C5":
             entry["roofline"] = {"bound": "hbm", "achieved": entry["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": round(entry["gbs"] / peaks["hbm_gbs"], 4), "of": peaks["source"],
@@ -422,6 +450,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loop-ms", type=float, default=150.0, help="target length of each per-configuration timing loop")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
+    ap.add_argument("--no-eager", action="store_true", help="skip the PyTorch-eager context timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-pointer end-to-end leg")
     ap.add_argument("--configs", default=",".join(ORDER), help="comma-separated subset of C1..C5 (profiling aid)")
     args = ap.parse_args()
