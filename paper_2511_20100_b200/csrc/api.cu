@@ -259,7 +259,7 @@ void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
     p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
     p.num_tiles = p.m_tiles * p.n_tiles;
     p.k_blocks = static_cast<int>((K + 63) / 64);
-    p.group_m = bm == 256 ? (p.m_tiles < 8 ? p.m_tiles : 8) : pick_group_m(p.m_tiles);
+    p.group_m = pick_group_m(p.m_tiles);      // 16 row blocks per group measured best for both tile heights
     p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1; p.tail_width = out_tile_n;
     const int r = p.num_tiles % sm_count;
     if (split_tail && r > 0) {
