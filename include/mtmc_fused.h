@@ -154,6 +154,13 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
  * status (MTMC_OK, MTMC_ERR_DEVICE_TIMEOUT or MTMC_ERR_CUDA). */
 int mtmc_check_status(void);
 
+/* Self-test of the failure-detection path (no counterpart in the paper): enqueues a
+ * one-thread kernel that waits, with a one-millisecond limit, on a barrier nothing will
+ * ever signal.  The wait gives up, the kernel returns normally, and the next
+ * mtmc_check_status() reports MTMC_ERR_DEVICE_TIMEOUT exactly as it would for a stalled
+ * pipeline in a real kernel.  Nothing faults or hangs; the context stays usable. */
+int mtmc_selftest_timeout(void);
+
 /* Text for the last non-OK status returned on this host thread ("" if none). */
 const char* mtmc_last_error(void);
 

@@ -16,6 +16,10 @@
 //   fused linear :  Y[m][n] = act(z[m][n]),  act in {identity, ReLU, GELU-tanh, SiLU}
 //   SwiGLU       :  out[m][n] = silu(g[m][n]) * u[m][n],  g = X.Wg^T, u = X.Wu^T (no bias)
 //   row LSE      :  lse[m] = log( sum_n exp(z[m][n]) ), computed two-pass (max, then sum)
+//   row max      :  mx[m] = max_n z[m][n], arg[m] = the lowest n attaining it
+//                   (the paper's own example of a fusion action joins a linear with a row max,
+//                   section "Training Process")
+//   cross entropy:  loss[m] = lse[m] - z[m][target[m]]   (softmax cross entropy of the logits row)
 //
 // Layouts: X [M,K], W [N,K], out [M,N]; all dense row-major.  X/W arrive as bf16 bit
 // patterns (uint16_t: the upper half of an IEEE-754 binary32), b as binary32 and
@@ -198,6 +202,39 @@ int mtmc_ref_linear_lse_rows(const uint16_t* X, const uint16_t* W, const float* 
         parallel_for(N, [=](int64_t n) { zp[n] = preact(X, W, b, K, m, n); });
         lse[r] = lse_of_row(zp, N);
     }
+    return 0;
+}
+
+// mx[m] = max_n z[m][n]; arg[m] = lowest column index attaining it.  arg may be null.
+int mtmc_ref_linear_rowmax(const uint16_t* X, const uint16_t* W, const float* b,
+                           int64_t M, int64_t N, int64_t K, double* mx, int64_t* arg) {
+    if (!X || !W || !mx || M <= 0 || N <= 0 || K <= 0) return 1;
+    parallel_for(M, [=](int64_t m) {
+        double best = preact(X, W, b, K, m, 0);
+        int64_t where = 0;
+        for (int64_t n = 1; n < N; ++n) {
+            double z = preact(X, W, b, K, m, n);
+            if (z > best) { best = z; where = n; }
+        }
+        mx[m] = best;
+        if (arg) arg[m] = where;
+    });
+    return 0;
+}
+
+// loss[m] = lse[m] - z[m][target[m]], lse as in mtmc_ref_linear_lse (two-pass).  lse_out may be null.
+int mtmc_ref_linear_cross_entropy(const uint16_t* X, const uint16_t* W, const float* b, const int64_t* target,
+                                  int64_t M, int64_t N, int64_t K, double* loss, double* lse_out) {
+    if (!X || !W || !target || !loss || M <= 0 || N <= 0 || K <= 0) return 1;
+    for (int64_t m = 0; m < M; ++m)
+        if (target[m] < 0 || target[m] >= N) return 1;
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n) z[n] = preact(X, W, b, K, m, n);
+        const double l = lse_of_row(z.data(), N);
+        loss[m] = l - z[target[m]];
+        if (lse_out) lse_out[m] = l;
+    });
     return 0;
 }
 

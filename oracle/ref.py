@@ -47,6 +47,8 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
         L.mtmc_ref_linear_lse.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
         L.mtmc_ref_linear_lse_rows.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
+        L.mtmc_ref_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
+        L.mtmc_ref_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
         L.mtmc_ref_lse_vector.argtypes = [vp, i64]
         L.mtmc_ref_lse_vector.restype = dbl
         L.mtmc_ref_compare.argtypes = [vp, vp, i64, dbl, dbl, vp]
@@ -161,6 +163,35 @@ def linear_lse_rows(X, W, b, rows) -> np.ndarray:
                                           rows.ctypes.data, rows.shape[0], lse.ctypes.data),
            "mtmc_ref_linear_lse_rows")
     return lse
+
+
+def linear_rowmax(X, W, b):
+    """(max over n of X.W^T + b, lowest index attaining it) per row."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    mx = np.empty(M, dtype=np.float64)
+    arg = np.empty(M, dtype=np.int64)
+    _check(lib().mtmc_ref_linear_rowmax(X.ctypes.data, W.ctypes.data, bp, M, N, K, mx.ctypes.data, arg.ctypes.data),
+           "mtmc_ref_linear_rowmax")
+    return mx, arg
+
+
+def linear_cross_entropy(X, W, b, target):
+    """(loss, lse) per row: loss = lse - logit[target]."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    target = _idx(target)
+    if target.shape != (M,):
+        raise TypeError("target must be int64 [M]")
+    loss = np.empty(M, dtype=np.float64)
+    lse = np.empty(M, dtype=np.float64)
+    _check(lib().mtmc_ref_linear_cross_entropy(X.ctypes.data, W.ctypes.data, bp, target.ctypes.data, M, N, K,
+                                               loss.ctypes.data, lse.ctypes.data), "mtmc_ref_linear_cross_entropy")
+    return loss, lse
 
 
 def lse_vector(z) -> float:

@@ -27,7 +27,7 @@ EXPORTS = [
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_set_tuning", "mtmc_version",
+    "mtmc_set_tuning", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -198,6 +198,13 @@ def mtmc_workspace_bytes(op: str, M: int, N: int, K: int) -> int:
 
 def mtmc_check_status() -> None:
     _check(load().mtmc_check_status())
+
+
+def mtmc_selftest_timeout() -> None:
+    """Enqueues the bounded-wait self-test kernel; the following mtmc_check_status() raises DEVICE_TIMEOUT."""
+    torch.cuda.set_device(torch.cuda.current_device())
+    load().mtmc_set_stream(ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    _check(load().mtmc_selftest_timeout())
 
 
 def mtmc_launch_count() -> int:

@@ -331,6 +331,19 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
 
 bool use_skinny(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 31) / 32 <= static_cast<int64_t>(TICKET_BYTES / 4); }
 
+// One thread waits, with a one-millisecond limit, on an mbarrier that nothing ever arrives on:
+// the bounded wait gives up, records the status word and the kernel returns normally.
+__global__ void timeout_probe_kernel(uint32_t* status) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0u;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+        mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, STATUS_TIMEOUT_EPILOGUE | 0xEEu, 2000000ll);
+    }
+}
+
 template <bool OUT_BF16, bool PAIR>
 int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap& tmX, const SkinnyParams& p) {
     auto kern = skinny_splitk_kernel<OUT_BF16, PAIR>;
@@ -484,6 +497,16 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
         case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N);
         default: return static_cast<size_t>(-1);
     }
+}
+
+int mtmc_selftest_timeout(void) {
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    timeout_probe_kernel<<<1, 32, 0, t_stream>>>(d->status);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
 }
 
 int mtmc_check_status(void) {

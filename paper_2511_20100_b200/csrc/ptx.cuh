@@ -58,7 +58,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait for the phase with the given parity.  Returns false if the CTA has
 // been aborted (by this or another thread); the caller must then leave its loop.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* status, uint32_t code) {
+                                          uint32_t* status, uint32_t code, long long limit = WAIT_LIMIT_CLOCKS) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -66,7 +66,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 31u) == 0u) {
             if (*abort_flag != 0u) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CLOCKS) {
+            if (clock64() - t0 > limit) {
                 *abort_flag = code;
                 atomicCAS(status, 0u, code);
                 return false;

@@ -297,6 +297,23 @@ def test_argument_errors_enqueue_nothing():
     B.mtmc_check_status()
 
 
+def test_bounded_wait_reports_a_timeout_and_the_context_stays_usable():
+    """Failure detection without a fault: a wait that nothing will satisfy gives up after its limit,
+    the kernel returns, the status surfaces once on the host, and the library keeps working."""
+    B.mtmc_check_status()
+    B.mtmc_selftest_timeout()
+    with pytest.raises(B.MtmcError) as e:
+        B.mtmc_check_status()
+    assert e.value.status == B.ERR_DEVICE_TIMEOUT
+    B.mtmc_check_status()                                   # sticky status was cleared by the report
+    li, out = run_linear(140, 264, 192, "relu", "fp32", seed=91)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_RELU)
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "after the self-test")
+    sk, so = run_linear(16, 640, 1024, "gelu_tanh", "bf16", seed=92)     # ticket path after tickets were marked dirty
+    _assert_close(inputs.to_f64(so), ref.fused_linear(inputs.bf16_bits(sk.X), inputs.bf16_bits(sk.W), inputs.f32(sk.b),
+                                                     ref.ACT_GELU_TANH), TOL["bf16"], "skinny after the self-test")
+
+
 def test_host_pointer_entry_points():
     li = inputs.linear_inputs(150, 264, 128, seed=61)
     out = B.mtmc_fused_linear_host(li.X, li.W, li.b, "relu", "fp32")

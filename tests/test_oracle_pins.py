@@ -262,6 +262,60 @@ def test_lse_expected_level_for_unit_variance_logits():
     assert np.all(np.abs(lse - (math.log(4000) + 0.5)) < 0.15)
 
 
+# ---------------------------------------------------------------- row max, cross entropy
+def test_rowmax_pins():
+    li = inputs.linear_inputs(7, 300, 48, seed=61)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    mx, arg = ref.linear_rowmax(X, W, b)
+    z = li.X.double() @ li.W.double().T + li.b.double()
+    tmax, targ = z.max(dim=-1)
+    np.testing.assert_allclose(mx, tmax.numpy(), rtol=0, atol=1e-12)
+    assert np.array_equal(arg, targ.numpy())
+    # zero weights: the row max is max(b), attained at argmax(b), for every row
+    mx0, arg0 = ref.linear_rowmax(X, np.zeros_like(W), b)
+    assert np.all(mx0 == float(b.max())) and np.all(arg0 == int(b.argmax()))
+    # ties go to the lowest index: two identical weight rows and biases
+    W2 = W.copy(); W2[200] = W2[17]; b2 = b.copy(); b2[200] = b2[17]
+    _, arg2 = ref.linear_rowmax(X, W2, b2)
+    assert not np.any(arg2 == 200)
+    # the maximum bounds logsumexp from below within ln N
+    lse = ref.linear_lse(X, W, b)
+    assert np.all(mx <= lse) and np.all(lse <= mx + math.log(300))
+    # permuting the columns permutes the argmax and leaves the max unchanged
+    perm = np.random.default_rng(2).permutation(300)
+    mxp, argp = ref.linear_rowmax(X, W[perm].copy(), b[perm].copy())
+    assert np.array_equal(mxp, mx) and np.array_equal(perm[argp], arg)
+
+
+def test_cross_entropy_pins():
+    li = inputs.linear_inputs(9, 250, 64, seed=62)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    tgt = np.random.default_rng(3).integers(0, 250, size=9)
+    loss, lse = ref.linear_cross_entropy(X, W, b, tgt)
+    z = li.X.double() @ li.W.double().T + li.b.double()
+    want = torch.nn.functional.cross_entropy(z, torch.from_numpy(tgt), reduction="none")
+    np.testing.assert_allclose(loss, want.numpy(), rtol=0, atol=1e-12)
+    np.testing.assert_array_equal(lse, ref.linear_lse(X, W, b))
+    assert np.all(loss >= 0.0)
+    # -log softmax: exp(-loss) is the softmax probability of the target, and the probabilities of a row sum to 1
+    row = [float(np.exp(-ref.linear_cross_entropy(X[:1], W, b, np.array([n]))[0][0])) for n in range(250)]
+    assert sum(row) == pytest.approx(1.0, abs=1e-12)
+    # all logits equal: loss = ln N whatever the target
+    l0, _ = ref.linear_cross_entropy(X, np.zeros_like(W), None, tgt)
+    np.testing.assert_allclose(l0, np.full(9, math.log(250)), rtol=1e-15)
+    # adding a constant to every bias changes lse but not the loss (2.0 keeps b's low bits only approximately: bound it)
+    b_shift = (li.b.double() + 2.0).float().numpy()
+    ls, _ = ref.linear_cross_entropy(X, W, b_shift, tgt)
+    assert np.all(np.abs(ls - loss) <= 2 * np.abs((b_shift.astype(np.float64) - b.astype(np.float64)) - 2.0).max() + 1e-12)
+    # target = argmax gives the smallest loss of the row: lse - max
+    mx, arg = ref.linear_rowmax(X, W, b)
+    la, _ = ref.linear_cross_entropy(X, W, b, arg)
+    np.testing.assert_allclose(la, lse - mx, rtol=0, atol=1e-12)
+    assert np.all(la <= loss + 1e-12)
+    with pytest.raises(ValueError):
+        ref.linear_cross_entropy(X, W, b, np.full(9, 250))
+
+
 # ---------------------------------------------------------------- sampled variants, threads, comparator
 def test_points_match_full_and_threads_do_not_matter():
     li = inputs.linear_inputs(20, 31, 72, seed=51)
