@@ -50,8 +50,9 @@ def algorithmic_bytes(c) -> float:
     M, N, K = c["M"], c["N"], c["K"]
     if c["op"] == "swiglu":
         return 2.0 * (M * K + 2 * N * K) + 2.0 * M * N
-    if c["op"] == "linear_lse":
-        return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M
+    if c["op"] in ("linear_lse", "linear_rowmax", "linear_cross_entropy"):
+        extra = {"linear_lse": 0.0, "linear_rowmax": 4.0 * M, "linear_cross_entropy": 8.0 * M}[c["op"]]
+        return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M + extra
     out_b = 2.0 if c["out_dtype"] == "bf16" else 4.0
     return 2.0 * (M * K + N * K) + 4.0 * N + out_b * M * N
 
@@ -131,15 +132,17 @@ def reduce_max(dist, value: float, device) -> float:
 
 # --------------------------------------------------------------------------------------- our arm
 def make_device_problem(name, device):
-    c = inputs.CONFIGS[name]
+    c = inputs.CONFIGS.get(name) or inputs.EXTRA_CONFIGS[name]
     if c["op"] == "swiglu":
         si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
         host = [si.X, si.Wg, si.Wu]
     else:
         li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
         host = [li.X, li.W, li.b]
+    if c["op"] == "linear_cross_entropy":
+        host.append(inputs.targets(c["M"], c["N"], c["seed"]))
     dev = [t.to(device) for t in host]
-    if c["op"] == "linear_lse":
+    if c["op"] in ("linear_lse", "linear_rowmax", "linear_cross_entropy"):
         out = torch.empty((c["M"],), dtype=torch.float32, device=device)
     else:
         odt = torch.bfloat16 if c.get("out_dtype", "bf16") == "bf16" else torch.float32
@@ -153,6 +156,10 @@ def call_device(B, pr):
         B.mtmc_swiglu(d[0], d[1], d[2], out=pr["out"])
     elif c["op"] == "linear_lse":
         B.mtmc_linear_lse(d[0], d[1], d[2], lse_out=pr["out"])
+    elif c["op"] == "linear_rowmax":
+        B.mtmc_linear_rowmax(d[0], d[1], d[2], max_out=pr["out"], want_argmax=False)
+    elif c["op"] == "linear_cross_entropy":
+        B.mtmc_linear_cross_entropy(d[0], d[1], d[2], d[3], loss_out=pr["out"])
     else:
         B.mtmc_fused_linear(d[0], d[1], d[2], c["act"], c["out_dtype"], out=pr["out"])
 
@@ -176,6 +183,10 @@ def eager_call(pr, dev):
         return torch.nn.functional.silu(dev[0] @ dev[1].T) * (dev[0] @ dev[2].T)
     if c["op"] == "linear_lse":
         return torch.logsumexp((dev[0] @ dev[1].T).float() + dev[2], dim=-1)
+    if c["op"] == "linear_rowmax":
+        return ((dev[0] @ dev[1].T).float() + dev[2]).max(dim=-1).values
+    if c["op"] == "linear_cross_entropy":
+        return torch.nn.functional.cross_entropy((dev[0] @ dev[1].T).float() + dev[2], dev[3], reduction="none")
     z = (dev[0] @ dev[1].T).float() + dev[2]
     z = torch.relu(z) if c["act"] == "relu" else torch.nn.functional.gelu(z, approximate="tanh")
     return z if c["out_dtype"] == "fp32" else z.to(torch.bfloat16)
@@ -276,7 +287,8 @@ def run_ours(args, rank, world, local_rank):
     # one event pair around the loop, so launch overhead is amortised as it is inside a step.
     L2_BYTES = 126e6
     per_cfg_ms, per_cfg_reps, per_cfg_copies, per_cfg_eager = {}, {}, {}, {}
-    for pr in problems:
+    extras = [] if (args.no_extras or ORDER != list(inputs.CONFIGS)) else [make_device_problem(n, device) for n in inputs.EXTRA_CONFIGS]
+    for pr in problems + extras:
         n, c = pr["name"], pr["cfg"]
         nbytes = sum(t.numel() * t.element_size() for t in pr["dev"] if t is not None)
         copies = 1 if n == "C1" else max(1, min(4, int(-(-2 * L2_BYTES // nbytes))))
@@ -319,12 +331,14 @@ def run_ours(args, rank, world, local_rank):
     value = world * step_flops / (ms_per_step * 1e-3) / 1e12
 
     per_config = {}
-    for n in ORDER:
-        c = inputs.CONFIGS[n]
+    for n in ORDER + [e["name"] for e in extras]:
+        c = inputs.CONFIGS.get(n) or inputs.EXTRA_CONFIGS[n]
         ms = per_cfg_ms[n]
         entry = {"call": c["op"], "M": c["M"], "N": c["N"], "K": c["K"], "ms": round(ms, 5),
                  "launches_timed": per_cfg_reps[n], "operand_copies_rotated": per_cfg_copies[n],
                  "tflops": round(flops(c) / (ms * 1e-3) / 1e12, 3), "gbs": round(algorithmic_bytes(c) / (ms * 1e-3) / 1e9, 2)}
+        if n in inputs.EXTRA_CONFIGS:
+            entry["note"] = "further row reduction on the LM-head shape; measured beside the step, not part of it"
         if n in per_cfg_eager:
             entry["eager_ms"] = round(per_cfg_eager[n], 5)
             entry["speedup_vs_eager"] = round(per_cfg_eager[n] / ms, 3)
@@ -450,6 +464,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--loop-ms", type=float, default=150.0, help="target length of each per-configuration timing loop")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
+    ap.add_argument("--no-extras", action="store_true", help="skip the row-max / cross-entropy measurements")
     ap.add_argument("--no-eager", action="store_true", help="skip the PyTorch-eager context timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-pointer end-to-end leg")
     ap.add_argument("--configs", default=",".join(ORDER), help="comma-separated subset of C1..C5 (profiling aid)")

@@ -61,6 +61,8 @@ extern "C" {
 #define MTMC_OP_FUSED_LINEAR 0
 #define MTMC_OP_SWIGLU 1
 #define MTMC_OP_LINEAR_LSE 2
+#define MTMC_OP_LINEAR_ROWMAX 3
+#define MTMC_OP_LINEAR_CROSS_ENTROPY 4
 
 /* out[m][n] = act( sum_k X[m][k] W[n][k] + b[n] ).
  * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
@@ -86,6 +88,23 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu,
  * Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_LSE, M, N, K) bytes of workspace. */
 int mtmc_linear_lse(const void* X, const void* W, const float* b,
                     int64_t M, int64_t N, int64_t K, float* lse_out);
+
+/* max_out[m] = max_n ( sum_k X[m][k] W[n][k] + b[n] ), fp32 [M]; argmax_out[m] (int32 [M], may
+ * be NULL) = the lowest column attaining it.  (The paper's example of a semantic action,
+ * fusing a linear with a row maximum, section "Training Process".)  Same machinery as
+ * mtmc_linear_lse: per-piece (max, column) partials in the workspace, merged per row.
+ * Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_ROWMAX, M, N, K) bytes of workspace. */
+int mtmc_linear_rowmax(const void* X, const void* W, const float* b,
+                       int64_t M, int64_t N, int64_t K, float* max_out, int32_t* argmax_out);
+
+/* Softmax cross entropy of the never-materialised logits:
+ *   loss_out[m] = lse[m] - ( sum_k X[m][k] W[targets[m]][k] + b[targets[m]] ),   fp32 [M];
+ * lse_out (fp32 [M], may be NULL) also receives the row logsumexp.  targets is int64 [M] on the
+ * device, 8-byte aligned; a target outside [0, N) makes that row's loss NaN.  (Fused LM-head
+ * loss: the tile that holds a row's target column sets the logit aside while it accumulates the
+ * row's (max, sum-exp).)  Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_CROSS_ENTROPY, M, N, K). */
+int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, const int64_t* targets,
+                              int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out);
 
 /* Allocation-free variant of mtmc_linear_lse: same arguments, same result (same
  * kernels), but the (max, sum-exp) partials live in an 8 MiB array that is part of

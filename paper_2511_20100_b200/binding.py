@@ -19,11 +19,11 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_WORKSPACE = 1, 2, 3, 4, 5, 6
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}
 OUT_DTYPE = {"fp32": 0, "bf16": 1}
-OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2}
+OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4}
 
 EXPORTS = [
     "mtmc_fused_linear", "mtmc_swiglu", "mtmc_linear_lse",
-    "mtmc_linear_lse_noalloc",
+    "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
@@ -53,6 +53,8 @@ def load() -> ctypes.CDLL:
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
+    L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
+    L.mtmc_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_set_stream.argtypes = [vp]
     L.mtmc_set_workspace.argtypes = [vp, sz]
     L.mtmc_workspace_bytes.argtypes = [ci, i64, i64, i64]
@@ -121,6 +123,39 @@ def mtmc_linear_lse(X, W, b, lse_out=None):
                                   None if b is None else _dev(b, torch.float32, (N,), "b"),
                                   M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
     return lse_out
+
+
+def mtmc_linear_rowmax(X, W, b, max_out=None, argmax_out=None, want_argmax=True):
+    """(max_n, argmax_n) of X @ W.T + b per row, fp32 [M] and int32 [M]; the logits are never materialised."""
+    M, K = X.shape
+    N = W.shape[0]
+    if max_out is None:
+        max_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    if argmax_out is None and want_argmax:
+        argmax_out = torch.empty((M,), dtype=torch.int32, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_linear_rowmax(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                     None if b is None else _dev(b, torch.float32, (N,), "b"), M, N, K,
+                                     _dev(max_out, torch.float32, (M,), "max_out"),
+                                     None if argmax_out is None else _dev(argmax_out, torch.int32, (M,), "argmax_out")))
+    return max_out, argmax_out
+
+
+def mtmc_linear_cross_entropy(X, W, b, targets, loss_out=None, lse_out=None, want_lse=False):
+    """loss[m] = logsumexp_n(z[m]) - z[m][targets[m]] with z = X @ W.T + b; targets int64 [M] on the device."""
+    M, K = X.shape
+    N = W.shape[0]
+    if loss_out is None:
+        loss_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_linear_cross_entropy(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                            None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                            _dev(targets, torch.int64, (M,), "targets"), M, N, K,
+                                            _dev(loss_out, torch.float32, (M,), "loss_out"),
+                                            None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return (loss_out, lse_out) if want_lse else loss_out
 
 
 def mtmc_linear_lse_noalloc(X, W, b, lse_out):

@@ -441,6 +441,54 @@ int stage_buffer(DeviceState* d, int i, size_t bytes, void** out) {
     return MTMC_OK;
 }
 
+// The three row reductions over the never-materialised logits share one driver: a tiled kernel
+// leaves one partial per (row, column piece) in the workspace, a merge kernel finishes the rows.
+//   EPI_LSE    : out_a = lse                     EPI_ROWMAX : out_a = max, out_i = argmax (may be null)
+//   EPI_XENT   : out_b = loss, out_a = lse (may be null); the target logits sit behind the partials
+template <int EPI>
+int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
+                      float* out_a, float* out_b, int32_t* out_i) {
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    const bool pair = use_pair(d, M, N);
+    const int bn = pair ? 256 : pick_tile_n(N);
+    GemmParams p{};
+    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+    else fill_tiling(p, M, N, K, bn, d->sm_count, true);
+    const size_t partial_bytes = lse_workspace_bytes(M, N);
+    const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
+    void* ws = nullptr;
+    rc = get_workspace(d, partial_bytes + extra, &ws);
+    if (rc) return rc;
+    p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
+    p.targets = reinterpret_cast<const long long*>(targets);
+    p.target_logit = EPI == EPI_XENT ? reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes) : nullptr;
+    // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
+    if (EPI == EPI_XENT) CUDA_TRY(cudaMemsetAsync(p.target_logit, 0xFF, static_cast<size_t>(M) * sizeof(float), t_stream));
+    CUtensorMap tmA, tmB, tmBt;
+    if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, pair ? 128 : bn)) ||
+        (rc = encode_bf16_2d(&tmBt, W, N, K, pair ? p.tail_width / 2 : p.tail_width)))
+        return rc;
+    TimedRegion tr(d);
+    if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+    else rc = bn == 256 ? launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                        : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    tr.stop();
+    if (rc) return rc;
+    const unsigned blocks = static_cast<unsigned>((M + 7) / 8);
+    if (EPI == EPI_ROWMAX)
+        rowmax_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
+                                                          p.n_full, p.tail_split, out_a, out_i);
+    else
+        lse_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
+                                                       p.n_full, p.tail_split, out_a, p.target_logit, out_b);
+    CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -495,6 +543,8 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
         }
         case MTMC_OP_SWIGLU: return 0;
         case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N);
+        case MTMC_OP_LINEAR_ROWMAX: return lse_workspace_bytes(M, N);
+        case MTMC_OP_LINEAR_CROSS_ENTROPY: return lse_workspace_bytes(M, N) + round256(static_cast<size_t>(M) * sizeof(float));
         default: return static_cast<size_t>(-1);
     }
 }
@@ -618,53 +668,24 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
 int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
     int rc = check_common(X, W, lse_out, M, N, K);
     if (rc) return rc;
-    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
-    DeviceState* d = nullptr;
-    rc = get_device(&d);
+    return run_row_reduction<EPI_LSE>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr);
+}
+
+int mtmc_linear_rowmax(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* max_out,
+                       int32_t* argmax_out) {
+    int rc = check_common(X, W, max_out, M, N, K);
     if (rc) return rc;
-    const bool pair = use_pair(d, M, N);
-    const int bn = pair ? 256 : pick_tile_n(N);
-    GemmParams p{};
-    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
-    else fill_tiling(p, M, N, K, bn, d->sm_count, true);
-    void* ws = nullptr;
-    rc = get_workspace(d, lse_workspace_bytes(M, N), &ws);
+    if (argmax_out && (reinterpret_cast<uintptr_t>(argmax_out) & 3u)) return fail(MTMC_ERR_INVALID_ARG, "argmax_out must be 4-byte aligned");
+    return run_row_reduction<EPI_ROWMAX>(X, W, b, nullptr, M, N, K, max_out, nullptr, argmax_out);
+}
+
+int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N,
+                              int64_t K, float* loss_out, float* lse_out) {
+    int rc = check_common(X, W, loss_out, M, N, K);
     if (rc) return rc;
-    if (pair) {
-        p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
-        CUtensorMap tmA, tmB, tmBt;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
-            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
-            return rc;
-        TimedRegion tr(d);
-        rc = launch_pair<EPI_LSE, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
-        tr.stop();
-        if (rc) return rc;
-        lse_merge_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, t_stream>>>(
-            p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
-        CUDA_TRY(cudaGetLastError());
-        g_launches.fetch_add(1);
-        return MTMC_OK;
-    }
-    p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
-    CUtensorMap tmA, tmB, tmBt;
-    rc = encode_bf16_2d(&tmA, X, M, K, 128);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmB, W, N, K, bn);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
-    if (rc) return rc;
-    TimedRegion tr(d);
-    rc = bn == 256 ? launch_tiled<EPI_LSE, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
-                   : launch_tiled<EPI_LSE, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
-    tr.stop();
-    if (rc) return rc;
-    const int rows_per_block = 8;
-    lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
-    CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return MTMC_OK;
+    if (!targets) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(targets) & 7u) return fail(MTMC_ERR_INVALID_ARG, "targets must be 8-byte aligned");
+    return run_row_reduction<EPI_XENT>(X, W, b, targets, M, N, K, lse_out, loss_out, nullptr);
 }
 
 }  // extern "C"
@@ -775,7 +796,7 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
     if (rc) return rc;
     const int rows_per_block = 8;
     lse_merge_kernel<<<static_cast<unsigned>((M + rows_per_block - 1) / rows_per_block), rows_per_block * 32, 0, t_stream>>>(
-        p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out);
+        p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse_out, nullptr, nullptr);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
     return MTMC_OK;

@@ -15,7 +15,7 @@
 
 namespace mtmc {
 
-enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2 };
+enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2, EPI_ROWMAX = 3, EPI_XENT = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
 
 struct GemmParams {
@@ -33,7 +33,10 @@ struct GemmParams {
     int act;
     const float* bias;    // [N] or null
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
-    float2* lse_partial;  // [n_tiles * tail_split][M] (max, sum-exp) per row and column piece (EPI_LSE)
+    float2* lse_partial;  // [n_tiles * tail_split][M] per row and column piece: (max, sum-exp) for EPI_LSE / EPI_XENT,
+                          // (max, index bits) for EPI_ROWMAX
+    const long long* targets;   // [M] target column per row (EPI_XENT)
+    float* target_logit;        // [M] logit at the target column, written by the one piece that holds it (EPI_XENT)
     uint32_t* status;     // device status word
 };
 
@@ -174,6 +177,8 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
 //   EPI_ACT    : + bias, activation, store
 //   EPI_SWIGLU : silu(gate) * up with the up columns `width` columns after the gate columns
 //   EPI_LSE    : online (max, sum-exp) in base-2 units, one partial per (row, column piece)
+//   EPI_XENT   : the same, and the logit at the row's target column is set aside
+//   EPI_ROWMAX : running (max, lowest column attaining it), one partial per (row, column piece)
 template <int EPI, bool OUT_BF16>
 __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int chunks,
                                               int width, int nb, int sub, bool vec_ok) {
@@ -206,10 +211,34 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
             if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, vec_ok);
         }
+    } else if (EPI == EPI_ROWMAX) {
+        float mx = -INFINITY;
+        int arg = 0x7fffffff;
+#pragma unroll 1
+        for (int c = 0; c < chunks; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            if (n0 >= p.N) break;
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + c * 32, r);
+            float bv[32];
+            load_bias_chunk(p.bias, n0, p.N, bv);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float z = (n0 + j < p.N) ? __uint_as_float(r[j]) + bv[j] : -INFINITY;
+                if (z > mx) { mx = z; arg = n0 + j; }        // strict: ties keep the lower column
+            }
+        }
+        if (row < p.M)
+            p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] = make_float2(mx, __int_as_float(arg));
     } else {
         // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
         constexpr float LOG2E = 1.4426950408889634f;
         float mx = -INFINITY, sum = 0.0f;
+        int tgt = -1;
+        float tz = 0.0f;
+        bool found = false;
+        if (EPI == EPI_XENT && row < p.M) tgt = static_cast<int>(p.targets[row]);
 #pragma unroll 1
         for (int c = 0; c < chunks; ++c) {
             const int n0 = n_tile0 + c * 32;
@@ -222,9 +251,25 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             float cm = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                // columns past N are zero-filled weight rows: mask them out of the reduction
-                tv[j] = (n0 + j < p.N) ? (__uint_as_float(r[j]) + bv[j]) * LOG2E : -INFINITY;
+                tv[j] = fmaf(__uint_as_float(r[j]), LOG2E, bv[j] * LOG2E);
                 cm = fmaxf(cm, tv[j]);
+            }
+            if (n0 + 32 > p.N) {      // ragged last chunk: columns past N are zero-filled weight rows, mask them out
+                cm = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if (n0 + j >= p.N) tv[j] = -INFINITY;
+                    cm = fmaxf(cm, tv[j]);
+                }
+            }
+            if (EPI == EPI_XENT) {
+                const int rel = tgt - n0;                    // the target's place in this chunk, if it is here
+                if (static_cast<unsigned>(rel) < 32u && tgt < p.N) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j == rel) tz = tv[j] * 0.6931471805599453f;
+                    found = true;
+                }
             }
             const float nm = fmaxf(mx, cm);
             float cs = 0.0f;
@@ -237,6 +282,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         if (row < p.M)
             p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] =
                 make_float2(mx * 0.6931471805599453f, sum);
+        if (EPI == EPI_XENT && found) p.target_logit[row] = tz;
     }
 }
 
@@ -400,9 +446,11 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
 // Merges the (max, sum-exp) partials of each row, in ascending column order, into
 // lse[row] = max + ln(sum).  One warp per row; lanes stride over the column tiles and
 // combine with shuffles.  A whole tile left one partial (piece 0), a tile of the split
-// wave tail left tail_split of them.
-__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles, int group_m,
-                                 int n_full, int tail_split, float* __restrict__ lse) {
+// wave tail left tail_split of them.  With target_logit / loss given it also writes the
+// softmax cross entropy loss[row] = lse[row] - logit[row][target[row]].
+__global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
+                                 int group_m, int n_full, int tail_split, float* __restrict__ lse,
+                                 const float* __restrict__ target_logit, float* __restrict__ loss) {
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -421,7 +469,41 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
         const float os = __shfl_xor_sync(0xffffffffu, sum, off);
         lse_combine(mx, sum, om, os);
     }
-    if (lane == 0) lse[row] = mx + __logf(sum);
+    if (lane == 0) {
+        const float l = mx + __logf(sum);
+        if (lse) lse[row] = l;
+        if (loss) loss[row] = l - __ldcg(target_logit + row);
+    }
+}
+
+// Merges the (max, column) partials of each row: the largest value, ties to the lowest column.
+__global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
+                                    int group_m, int n_full, int tail_split, float* __restrict__ max_out,
+                                    int* __restrict__ argmax_out) {
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    const int mb = row / rows_per_tile;
+    float mx = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int nb = lane; nb < n_tiles; nb += 32) {
+        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+        for (int sub = 0; sub < pieces; ++sub) {
+            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split + sub) * M + row);
+            const int a = __float_as_int(v.y);
+            if (v.x > mx || (v.x == mx && a < arg)) { mx = v.x; arg = a; }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, mx, off);
+        const int oa = __shfl_xor_sync(0xffffffffu, arg, off);
+        if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+    }
+    if (lane == 0) {
+        max_out[row] = mx;
+        if (argmax_out) argmax_out[row] = arg;
+    }
 }
 
 }  // namespace mtmc

@@ -27,6 +27,17 @@ CONFIGS = {
     "C5": dict(op="fused_linear", M=16, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=4),
 }
 
+# Further row reductions on the LM-head shape (measured beside the five, not part of the benchmark step).
+EXTRA_CONFIGS = {
+    "X1": dict(op="linear_rowmax", M=4096, N=32000, K=4096, seed=3),
+    "X2": dict(op="linear_cross_entropy", M=4096, N=32000, K=4096, seed=3),
+}
+
+
+def targets(M: int, N: int, seed: int) -> torch.Tensor:
+    """Seeded uniform target columns, int64 [M]."""
+    return torch.from_numpy(np.random.default_rng(seed).integers(0, N, size=M))
+
 
 @dataclass
 class LinearInputs:

@@ -163,6 +163,92 @@ def test_linear_lse_shift_law():
     assert torch.allclose(b - a, torch.full_like(a, 3.0), atol=2e-3)
 
 
+# ------------------------------------------------------------------ row max and cross entropy of the fused logits
+def _check_rowmax(li, mx_gpu, arg_gpu, what):
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    want_mx, want_arg = ref.linear_rowmax(X, W, b)
+    _assert_close(inputs.to_f64(mx_gpu), want_mx, TOL["fp32"], what + " max")
+    _, logits = ref.linear_lse(X, W, b, want_logits=True)
+    arg = arg_gpu.cpu().numpy().astype(np.int64)
+    assert np.all((arg >= 0) & (arg < logits.shape[1]))
+    # fp32 and fp64 may order near-ties differently: the column the GPU names must hold the maximum within
+    # tolerance, and wherever the runner-up is clearly lower the two must name the same column
+    picked = logits[np.arange(logits.shape[0]), arg]
+    assert np.all(np.abs(picked - want_mx) <= 1e-3 + 1e-3 * np.abs(want_mx)), what + " argmax validity"
+    if logits.shape[1] > 1:
+        second = np.partition(logits, -2, axis=1)[:, -2]
+        clear = (want_mx - second) > 1e-2
+        assert np.array_equal(arg[clear], want_arg[clear]), what + " argmax"
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 8, 64), (200, 1000, 256), (129, 257, 72), (64, 3000, 128), (600, 1100, 192)])
+def test_linear_rowmax_small(M, N, K):
+    li = inputs.linear_inputs(M, N, K, seed=5000 + M + N)
+    bufm, mx = _guarded((M,), torch.float32)
+    arg = torch.full((M,), -7, dtype=torch.int32, device="cuda")
+    B.mtmc_linear_rowmax(li.X.cuda(), li.W.cuda(), li.b.cuda(), max_out=mx, argmax_out=arg)
+    B.mtmc_check_status()
+    assert _canaries_intact(bufm, M)
+    _check_rowmax(li, mx, arg, "rowmax %dx%dx%d" % (M, N, K))
+    only_max, none = B.mtmc_linear_rowmax(li.X.cuda(), li.W.cuda(), li.b.cuda(), want_argmax=False)
+    assert none is None and torch.equal(only_max, mx)
+
+
+def test_linear_rowmax_ties_go_to_the_lowest_column():
+    li = inputs.linear_inputs(140, 700, 64, seed=5100)
+    W = li.W.clone(); b = li.b.clone()
+    W[650] = W[13]; b[650] = b[13]; W[300] = W[13]; b[300] = b[13]        # three identical columns
+    _, arg = B.mtmc_linear_rowmax(li.X.cuda(), W.cuda(), b.cuda())
+    B.mtmc_check_status()
+    a = arg.cpu().numpy()
+    assert not np.any((a == 650) | (a == 300))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 8, 64), (200, 1000, 256), (129, 257, 72), (64, 3000, 128), (600, 1100, 192)])
+def test_linear_cross_entropy_small(M, N, K):
+    li = inputs.linear_inputs(M, N, K, seed=5200 + M + N)
+    tgt = torch.from_numpy(np.random.default_rng(M + N).integers(0, N, size=M))
+    bufl, loss = _guarded((M,), torch.float32)
+    _, lse = B.mtmc_linear_cross_entropy(li.X.cuda(), li.W.cuda(), li.b.cuda(), tgt.cuda(), loss_out=loss, want_lse=True)
+    B.mtmc_check_status()
+    assert _canaries_intact(bufl, M)
+    want_loss, want_lse = ref.linear_cross_entropy(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), tgt.numpy())
+    _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "cross entropy %dx%dx%d" % (M, N, K))
+    _assert_close(inputs.to_f64(lse), want_lse, TOL["fp32"], "lse of cross entropy")
+    assert torch.equal(B.mtmc_linear_cross_entropy(li.X.cuda(), li.W.cuda(), li.b.cuda(), tgt.cuda()), loss)
+
+
+def test_cross_entropy_target_out_of_range_gives_nan_for_that_row_only():
+    li = inputs.linear_inputs(40, 300, 64, seed=5300)
+    tgt = torch.arange(40, dtype=torch.int64) % 300
+    tgt[7] = 300
+    tgt[19] = -1
+    loss = B.mtmc_linear_cross_entropy(li.X.cuda(), li.W.cuda(), li.b.cuda(), tgt.cuda())
+    B.mtmc_check_status()
+    bad = torch.isnan(loss).cpu().numpy()
+    assert bad[7] and bad[19] and bad.sum() == 2
+
+
+def test_rowmax_and_cross_entropy_at_lm_head_size_on_sampled_rows():
+    c = inputs.CONFIGS["C4"]
+    li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+    tgt = torch.from_numpy(np.random.default_rng(9).integers(0, c["N"], size=c["M"]))
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    mx, arg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+    loss, lse = B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt.cuda(), want_lse=True)
+    B.mtmc_check_status()
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, c["M"] - 1], np.random.default_rng(4).integers(0, c["M"], size=10)]))
+    sub = inputs.LinearInputs(li.X[rows].contiguous(), li.W, li.b)
+    idx = torch.from_numpy(rows).cuda()
+    _check_rowmax(sub, mx[idx], arg[idx], "C4 rowmax sampled rows")
+    want_loss, want_lse = ref.linear_cross_entropy(inputs.bf16_bits(sub.X), inputs.bf16_bits(sub.W), inputs.f32(sub.b), tgt.numpy()[rows])
+    _assert_close(inputs.to_f64(loss[idx]), want_loss, TOL["fp32"], "C4 cross entropy sampled rows")
+    _assert_close(inputs.to_f64(lse[idx]), want_lse, TOL["fp32"], "C4 lse sampled rows")
+    # properties at full size: max <= lse <= max + ln N and loss >= lse - max >= 0 for every row
+    assert bool((mx <= lse + 1e-3).all()) and bool((lse <= mx + np.log(c["N"]) + 1e-3).all())
+    assert bool((loss >= lse - mx - 2e-3).all())
+
+
 # ------------------------------------------------------------------ skinny / split-K path
 @pytest.mark.parametrize("M,N,K", [
     (16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392),   # few rows: ticketed split-K
