@@ -27,7 +27,7 @@ struct PairCfg {
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     static constexpr int TMEM_COLS = 2 * BN;
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int THREADS = 192;
 };
 
@@ -42,7 +42,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
-    const uint32_t bar_base = base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
+    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
@@ -156,7 +157,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             acc_ph ^= 1u << buf;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::BN);
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, width / 32, width, nb, sub, vec_ok);
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, width / 32, width, nb, sub, vec_ok,
+                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
             // this CTA's half of the accumulator is drained: tell the MMA issuer in the even CTA
             tc_fence_before();
             __syncwarp();

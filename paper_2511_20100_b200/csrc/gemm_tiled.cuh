@@ -18,6 +18,9 @@ namespace mtmc {
 enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2, EPI_ROWMAX = 3, EPI_XENT = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
 
+// Bytes of warp-private store staging per epilogue warp: one 32-row x 32-column chunk in fp32.
+constexpr int EPI_STAGE_BYTES_PER_WARP = 32 * 32 * 4;
+
 struct GemmParams {
     int M, N, K;
     int m_tiles, n_tiles, num_tiles, k_blocks;
@@ -51,7 +54,7 @@ struct TileCfg {
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
     static constexpr int TMEM_COLS = 2 * BN;             // two accumulator buffers
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;  // + alignment slack
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;  // + alignment slack
     static constexpr int THREADS = 192;
 };
 
@@ -154,6 +157,53 @@ __device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int 
     }
 }
 
+// Coalesced store of one 32-row x 32-column chunk held one row per lane.  The rows are
+// exchanged through a warp-private shared-memory buffer (16-byte units, XOR-swizzled so that
+// neither side has bank conflicts) so that every 128-bit store instruction of the warp
+// writes whole, contiguous row segments: 8 rows x 64 B for bf16, 4 rows x 128 B for fp32.
+// Requires the chunk to lie wholly inside [0, N) and 16-byte aligned rows; rows >= M are
+// not stored.  `row0` is the output row of lane 0.
+template <bool OUT_BF16>
+__device__ __forceinline__ void store_chunk_coalesced(uint8_t* stage, void* out, int row0, int n0, int M, int N,
+                                                      const float (&y)[32], int lane) {
+    constexpr int UNITS = OUT_BF16 ? 4 : 8;                  // 16-byte units per row of the chunk
+    constexpr int ROW_BYTES = UNITS * 16;
+    uint4* my_row = reinterpret_cast<uint4*>(stage + lane * ROW_BYTES);
+    const int wkey = OUT_BF16 ? ((lane >> 1) & 3) : (lane & 7);
+#pragma unroll
+    for (int u = 0; u < UNITS; ++u) {
+        uint4 q;
+        if (OUT_BF16) {
+            q.x = pack_bf16x2(y[8 * u + 0], y[8 * u + 1]);
+            q.y = pack_bf16x2(y[8 * u + 2], y[8 * u + 3]);
+            q.z = pack_bf16x2(y[8 * u + 4], y[8 * u + 5]);
+            q.w = pack_bf16x2(y[8 * u + 6], y[8 * u + 7]);
+        } else {
+            q.x = __float_as_uint(y[4 * u + 0]);
+            q.y = __float_as_uint(y[4 * u + 1]);
+            q.z = __float_as_uint(y[4 * u + 2]);
+            q.w = __float_as_uint(y[4 * u + 3]);
+        }
+        my_row[u ^ wkey] = q;
+    }
+    __syncwarp();
+    constexpr int ROWS_PER_STORE = 32 / UNITS;
+    const int sub_row = lane / UNITS;
+    const int unit = lane % UNITS;
+    const size_t elem = OUT_BF16 ? 2 : 4;
+#pragma unroll
+    for (int it = 0; it < UNITS; ++it) {
+        const int r = it * ROWS_PER_STORE + sub_row;
+        const int rkey = OUT_BF16 ? ((r >> 1) & 3) : (r & 7);
+        const uint4 q = *reinterpret_cast<const uint4*>(stage + r * ROW_BYTES + ((unit ^ rkey) * 16));
+        if (row0 + r < M) {
+            uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (static_cast<size_t>(row0 + r) * N + n0) * elem + unit * 16;
+            *reinterpret_cast<uint4*>(dst) = q;
+        }
+    }
+    __syncwarp();                                            // the buffer is reused by the next chunk
+}
+
 // Loads bias[n0 .. n0+32) into registers (zeros past N or without bias).
 __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N, float (&b)[32]) {
     if (bias == nullptr) {
@@ -181,7 +231,7 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
 //   EPI_ROWMAX : running (max, lowest column attaining it), one partial per (row, column piece)
 template <int EPI, bool OUT_BF16>
 __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int chunks,
-                                              int width, int nb, int sub, bool vec_ok) {
+                                              int width, int nb, int sub, bool vec_ok, uint8_t* stage, int lane) {
     if (EPI == EPI_ACT) {
 #pragma unroll 1
         for (int c = 0; c < chunks; ++c) {
@@ -195,7 +245,8 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
             apply_act_chunk(p.act, y);
-            if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, vec_ok);
+            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
+            else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, false);
         }
     } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
@@ -209,7 +260,8 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             float y[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
-            if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, vec_ok);
+            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<true>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
+            else if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, false);
         }
     } else if (EPI == EPI_ROWMAX) {
         float mx = -INFINITY;
@@ -297,7 +349,8 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
-    const uint32_t bar_base = base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
+    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
@@ -410,7 +463,8 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * BN);
 
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, chunks, width, nb, sub, vec_ok);
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, chunks, width, nb, sub, vec_ok,
+                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
             // accumulator buffer drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
