@@ -81,9 +81,16 @@ def _dev(t: torch.Tensor, dtype, shape, name: str) -> int:
     return t.data_ptr()
 
 
+_raw_stream = getattr(torch._C, "_cuda_getCurrentRawStream", None)
+
+
 def _use_current_stream(device) -> None:
-    torch.cuda.set_device(device)
-    load().mtmc_set_stream(ctypes.c_void_p(torch.cuda.current_stream(device).cuda_stream))
+    """Makes `device` current and hands torch's current stream on it to the library."""
+    idx = device.index if device.index is not None else torch.cuda.current_device()
+    if torch.cuda.current_device() != idx:
+        torch.cuda.set_device(idx)
+    handle = _raw_stream(idx) if _raw_stream is not None else torch.cuda.current_stream(idx).cuda_stream
+    load().mtmc_set_stream(ctypes.c_void_p(handle))
 
 
 def mtmc_fused_linear(X, W, b, act="none", out_dtype="bf16", out=None):

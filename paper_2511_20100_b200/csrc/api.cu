@@ -179,12 +179,35 @@ struct TimedRegion {
     }
 };
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and device instead of per call.
+// (Instantiations of one kernel template share a function-pointer type, so the record is keyed
+// on the pointer value, not on the type.)
+struct SmemAttrRecord { const void* fn; int dev; };
+SmemAttrRecord g_smem_attr[256];
+int g_smem_attr_count = 0;
+
+template <class Kernel>
+int ensure_smem_attr(Kernel kern, int bytes) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    const void* key = reinterpret_cast<const void*>(kern);
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        for (int i = 0; i < g_smem_attr_count; ++i)
+            if (g_smem_attr[i].fn == key && g_smem_attr[i].dev == dev) return MTMC_OK;
+    }
+    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (g_smem_attr_count < 256) g_smem_attr[g_smem_attr_count++] = SmemAttrRecord{key, dev};
+    return MTMC_OK;
+}
+
 template <int EPI, int BN, bool OUT_BF16>
 int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
                  const CUtensorMap& tmBt, const CUtensorMap& tmB2t, GemmParams p) {
     using Cfg = TileCfg<EPI, BN>;
     auto kern = gemm_tiled_kernel<EPI, BN, OUT_BF16>;
-    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
     const int grid = p.num_items < d->sm_count ? p.num_items : d->sm_count;
     kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB2, tmBt, tmB2t, p);
     CUDA_TRY(cudaGetLastError());
@@ -197,7 +220,7 @@ int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, co
                 const CUtensorMap& tmBt, const CUtensorMap& tmB2t, const GemmParams& p) {
     using Cfg = PairCfg<EPI>;
     auto kern = gemm_pair_kernel<EPI, OUT_BF16>;
-    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
     const int pairs = p.num_items < clusters ? p.num_items : clusters;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
@@ -347,7 +370,7 @@ __global__ void timeout_probe_kernel(uint32_t* status) {
 template <bool OUT_BF16, bool PAIR>
 int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap& tmX, const SkinnyParams& p) {
     auto kern = skinny_splitk_kernel<OUT_BF16, PAIR>;
-    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES));
+    if (int rc = ensure_smem_attr(kern, SkinnyCfg::SMEM_BYTES)) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(s.grid), 1, 1);
     cfg.blockDim = dim3(192, 1, 1);
