@@ -14,6 +14,7 @@
 //
 //   z[m][n]  = sum_{k=0..K-1} X[m][k] * W[n][k]  (+ b[n])        "X . W^T + b"
 //   fused linear :  Y[m][n] = act(z[m][n]),  act in {identity, ReLU, GELU-tanh, SiLU}
+//   + residual   :  Y[m][n] = act(z[m][n]) + R[m][n]   (the layer's skip connection joined to the epilogue)
 //   SwiGLU       :  out[m][n] = silu(g[m][n]) * u[m][n],  g = X.Wg^T, u = X.Wu^T (no bias)
 //   row LSE      :  lse[m] = log( sum_n exp(z[m][n]) ), computed two-pass (max, then sum)
 //   row max      :  mx[m] = max_n z[m][n], arg[m] = the lowest n attaining it
@@ -120,6 +121,20 @@ int mtmc_ref_fused_linear(const uint16_t* X, const uint16_t* W, const float* b,
     if (!X || !W || !out || M <= 0 || N <= 0 || K <= 0 || act < 0 || act > 3) return 1;
     parallel_for(M, [=](int64_t m) {
         for (int64_t n = 0; n < N; ++n) out[m * N + n] = act_apply(act, preact(X, W, b, K, m, n));
+    });
+    return 0;
+}
+
+// Y = act(X.W^T + b) + R.  R is [M,N], either bf16 bit patterns (r_is_bf16 != 0) or binary32.
+int mtmc_ref_fused_linear_residual(const uint16_t* X, const uint16_t* W, const float* b, const void* R, int r_is_bf16,
+                                   int64_t M, int64_t N, int64_t K, int act, double* out) {
+    if (!X || !W || !R || !out || M <= 0 || N <= 0 || K <= 0 || act < 0 || act > 3) return 1;
+    parallel_for(M, [=](int64_t m) {
+        for (int64_t n = 0; n < N; ++n) {
+            const double r = r_is_bf16 ? bf16_to_double(static_cast<const uint16_t*>(R)[m * N + n])
+                                       : static_cast<double>(static_cast<const float*>(R)[m * N + n]);
+            out[m * N + n] = act_apply(act, preact(X, W, b, K, m, n)) + r;
+        }
     });
     return 0;
 }

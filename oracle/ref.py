@@ -42,6 +42,7 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_act.argtypes = [ci, dbl]
         L.mtmc_ref_act.restype = dbl
         L.mtmc_ref_fused_linear.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp]
+        L.mtmc_ref_fused_linear_residual.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, ci, vp]
         L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
@@ -102,6 +103,21 @@ def fused_linear(X, W, b, act_kind: int) -> np.ndarray:
     out = np.empty((M, N), dtype=np.float64)
     _check(lib().mtmc_ref_fused_linear(X.ctypes.data, W.ctypes.data, bp, M, N, K, int(act_kind), out.ctypes.data),
            "mtmc_ref_fused_linear")
+    return out
+
+
+def fused_linear_residual(X, W, b, R, act_kind: int) -> np.ndarray:
+    """act(X.W^T + b) + R; R is [M,N] uint16 (bf16 bit patterns) or float32."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    R = np.ascontiguousarray(R)
+    if R.shape != (M, N) or R.dtype not in (np.uint16, np.float32):
+        raise TypeError("R must be [M,N] uint16 (bf16 bits) or float32")
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear_residual(X.ctypes.data, W.ctypes.data, bp, R.ctypes.data, int(R.dtype == np.uint16),
+                                                M, N, K, int(act_kind), out.ctypes.data), "mtmc_ref_fused_linear_residual")
     return out
 
 

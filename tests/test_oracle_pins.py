@@ -138,6 +138,23 @@ def test_against_torch_fp64_matmul(M, N, K, seed):
         np.testing.assert_allclose(got, fn(want).numpy(), rtol=1e-12, atol=1e-13)
 
 
+def test_residual_is_added_after_the_activation():
+    li = inputs.linear_inputs(6, 11, 40, seed=14)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    rng = np.random.default_rng(8)
+    R32 = rng.normal(size=(6, 11)).astype(np.float32)
+    Rb = bits(R32)
+    for kind in ACTS:
+        base = ref.fused_linear(X, W, b, kind)
+        assert np.array_equal(ref.fused_linear_residual(X, W, b, R32, kind), base + R32.astype(np.float64))
+        assert np.array_equal(ref.fused_linear_residual(X, W, b, Rb, kind), base + widen(Rb))
+        assert np.array_equal(ref.fused_linear_residual(X, W, b, np.zeros_like(R32), kind), base)
+    # torch: relu(z) + r, not relu(z + r)
+    z = li.X.double() @ li.W.double().T + li.b.double()
+    want = torch.relu(z) + torch.from_numpy(R32).double()
+    np.testing.assert_allclose(ref.fused_linear_residual(X, W, b, R32, ref.ACT_RELU), want.numpy(), rtol=0, atol=1e-12)
+
+
 # ---------------------------------------------------------------- activations
 def _closed_forms():
     rows = []
