@@ -54,7 +54,8 @@ def algorithmic_bytes(c) -> float:
         extra = {"linear_lse": 0.0, "linear_rowmax": 4.0 * M, "linear_cross_entropy": 8.0 * M}[c["op"]]
         return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M + extra
     out_b = 2.0 if c["out_dtype"] == "bf16" else 4.0
-    return 2.0 * (M * K + N * K) + 4.0 * N + out_b * M * N
+    res = out_b * M * N if c["op"] == "fused_linear_residual" else 0.0
+    return 2.0 * (M * K + N * K) + 4.0 * N + out_b * M * N + res
 
 
 def measured_peaks():
@@ -141,6 +142,8 @@ def make_device_problem(name, device):
         host = [li.X, li.W, li.b]
     if c["op"] == "linear_cross_entropy":
         host.append(inputs.targets(c["M"], c["N"], c["seed"]))
+    if c["op"] == "fused_linear_residual":
+        host.append(inputs.residual(c["M"], c["N"], c["seed"]))
     dev = [t.to(device) for t in host]
     if c["op"] in ("linear_lse", "linear_rowmax", "linear_cross_entropy"):
         out = torch.empty((c["M"],), dtype=torch.float32, device=device)
@@ -160,6 +163,8 @@ def call_device(B, pr):
         B.mtmc_linear_rowmax(d[0], d[1], d[2], max_out=pr["out"], want_argmax=False)
     elif c["op"] == "linear_cross_entropy":
         B.mtmc_linear_cross_entropy(d[0], d[1], d[2], d[3], loss_out=pr["out"])
+    elif c["op"] == "fused_linear_residual":
+        B.mtmc_fused_linear_residual(d[0], d[1], d[2], d[3], c["act"], c["out_dtype"], out=pr["out"])
     else:
         B.mtmc_fused_linear(d[0], d[1], d[2], c["act"], c["out_dtype"], out=pr["out"])
 
@@ -188,6 +193,8 @@ def eager_call(pr, dev):
     if c["op"] == "linear_cross_entropy":
         return torch.nn.functional.cross_entropy((dev[0] @ dev[1].T).float() + dev[2], dev[3], reduction="none")
     z = (dev[0] @ dev[1].T).float() + dev[2]
+    if c["op"] == "fused_linear_residual":
+        return (z + dev[3].float()).to(torch.bfloat16)
     z = torch.relu(z) if c["act"] == "relu" else torch.nn.functional.gelu(z, approximate="tanh")
     return z if c["out_dtype"] == "fp32" else z.to(torch.bfloat16)
 
@@ -338,7 +345,7 @@ def run_ours(args, rank, world, local_rank):
                  "launches_timed": per_cfg_reps[n], "operand_copies_rotated": per_cfg_copies[n],
                  "tflops": round(flops(c) / (ms * 1e-3) / 1e12, 3), "gbs": round(algorithmic_bytes(c) / (ms * 1e-3) / 1e9, 2)}
         if n in inputs.EXTRA_CONFIGS:
-            entry["note"] = "further row reduction on the LM-head shape; measured beside the step, not part of it"
+            entry["note"] = "further operator of the same family; measured beside the step, not part of it"
         if n in per_cfg_eager:
             entry["eager_ms"] = round(per_cfg_eager[n], 5)
             entry["speedup_vs_eager"] = round(per_cfg_eager[n] / ms, 3)

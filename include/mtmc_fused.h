@@ -74,6 +74,15 @@ extern "C" {
 int mtmc_fused_linear(const void* X, const void* W, const float* b,
                       int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 
+/* out[m][n] = act( sum_k X[m][k] W[n][k] + b[n] ) + R[m][n].
+ * (The layer's skip connection joined to the epilogue, e.g. the MLP down-projection that
+ * follows mtmc_swiglu: one more elementwise pass over [M,N] that never happens.)  R is [M,N]
+ * in the OUTPUT's element type (fp32 or bf16 according to out_dtype), 16-byte aligned; the
+ * sum is formed in fp32 and rounded once.  out may be the same buffer as R (in-place
+ * update of the residual stream); any other overlap is not allowed. */
+int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, const void* R,
+                               int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+
 /* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
  * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate
  * product fused in one kernel; neither GEMM result is written to memory.) */

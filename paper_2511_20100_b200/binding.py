@@ -22,7 +22,7 @@ OUT_DTYPE = {"fp32": 0, "bf16": 1}
 OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4}
 
 EXPORTS = [
-    "mtmc_fused_linear", "mtmc_swiglu", "mtmc_linear_lse",
+    "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_swiglu", "mtmc_linear_lse",
     "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
@@ -51,6 +51,7 @@ def load() -> ctypes.CDLL:
     vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
     for name in ("mtmc_fused_linear", "mtmc_fused_linear_host"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
@@ -104,6 +105,21 @@ def mtmc_fused_linear(X, W, b, act="none", out_dtype="bf16", out=None):
     _check(load().mtmc_fused_linear(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
                                     None if b is None else _dev(b, torch.float32, (N,), "b"),
                                     M, N, K, ACT[act], OUT_DTYPE[out_dtype], _dev(out, odt, (M, N), "out")))
+    return out
+
+
+def mtmc_fused_linear_residual(X, W, b, R, act="none", out_dtype="bf16", out=None):
+    """out = act(X @ W.T + b) + R; R [M,N] in the output dtype; `out` may be R itself (in-place)."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_fused_linear_residual(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                             None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                             _dev(R, odt, (M, N), "R"), M, N, K, ACT[act], OUT_DTYPE[out_dtype],
+                                             _dev(out, odt, (M, N), "out")))
     return out
 
 

@@ -415,14 +415,14 @@ int skinny_pairs(DeviceState* d) {
     return d->max_pairs;
 }
 
-int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
-               int out_dtype, void* out) {
+int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K,
+               int act, int out_dtype, void* out) {
     SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), N, K);
     SkinnyParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
     p.tile_rows = s.tile_rows; p.num_stages = s.stages;
-    p.act = act; p.bias = b; p.out = out; p.status = d->status;
+    p.act = act; p.bias = b; p.residual = R; p.out = out; p.status = d->status;
     void* ws = nullptr;
     if (t_user_ws) {
         int rc = get_workspace(d, s.ticket_bytes + s.partial_bytes, &ws);
@@ -514,6 +514,11 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
 
 }  // namespace
 
+namespace {
+int fused_linear_impl(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K, int act,
+                      int out_dtype, void* out);
+}
+
 extern "C" {
 
 int mtmc_version(void) { return 100; }
@@ -599,6 +604,21 @@ int mtmc_check_status(void) {
 
 int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
                       int out_dtype, void* out) {
+    return fused_linear_impl(X, W, b, nullptr, M, N, K, act, out_dtype, out);
+}
+
+int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N,
+                               int64_t K, int act, int out_dtype, void* out) {
+    if (!R) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(R)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    return fused_linear_impl(X, W, b, R, M, N, K, act, out_dtype, out);
+}
+
+}  // extern "C"
+
+namespace {
+int fused_linear_impl(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K, int act,
+                      int out_dtype, void* out) {
     int rc = check_common(X, W, out, M, N, K);
     if (rc) return rc;
     if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
@@ -607,12 +627,12 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, i
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(M, N)) return run_skinny(d, X, W, b, M, N, K, act, out_dtype, out);
+    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out);
 
     if (use_pair(d, M, N)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
-        p.act = act; p.bias = b; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB, tmBt;
         if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
             (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
@@ -626,7 +646,7 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, i
     const int bn = pick_tile_n(N);
     GemmParams p{};
     fill_tiling(p, M, N, K, bn, d->sm_count, true);
-    p.act = act; p.bias = b; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
     CUtensorMap tmA, tmB, tmBt;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
     if (rc) return rc;
@@ -645,6 +665,9 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, i
     tr.stop();
     return rc;
 }
+}  // namespace
+
+extern "C" {
 
 int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
     int rc = check_common(X, Wg, out, M, N, K);

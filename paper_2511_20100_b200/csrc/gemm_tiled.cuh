@@ -35,6 +35,7 @@ struct GemmParams {
     int tail_width;       // OUT_TILE_N / tail_split, a multiple of 32
     int act;
     const float* bias;    // [N] or null
+    const void* residual; // [M,N] in the output's element type, added after the activation, or null (EPI_ACT)
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
     float2* lse_partial;  // [n_tiles * tail_split][M] per row and column piece: (max, sum-exp) for EPI_LSE / EPI_XENT,
                           // (max, index bits) for EPI_ROWMAX
@@ -204,6 +205,43 @@ __device__ __forceinline__ void store_chunk_coalesced(uint8_t* stage, void* out,
     __syncwarp();                                            // the buffer is reused by the next chunk
 }
 
+// y[j] += R[row][n0 + j] for the 32 columns of one chunk of one row (R in the output's type).
+template <bool OUT_BF16>
+__device__ __forceinline__ void add_residual_chunk(const void* residual, int row, int n0, int N, float (&y)[32], bool vec_ok) {
+    if (OUT_BF16) {
+        const __nv_bfloat16* r = reinterpret_cast<const __nv_bfloat16*>(residual) + static_cast<size_t>(row) * N + n0;
+        if (vec_ok && n0 + 32 <= N) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const uint4 q = *reinterpret_cast<const uint4*>(r + 8 * v);
+                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    y[8 * v + 2 * h] += __uint_as_float(w[h] << 16);
+                    y[8 * v + 2 * h + 1] += __uint_as_float(w[h] & 0xffff0000u);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (n0 + j < N) y[j] += __bfloat162float(r[j]);
+        }
+    } else {
+        const float* r = reinterpret_cast<const float*>(residual) + static_cast<size_t>(row) * N + n0;
+        if (vec_ok && n0 + 32 <= N) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                const float4 q = *reinterpret_cast<const float4*>(r + 4 * v);
+                y[4 * v] += q.x; y[4 * v + 1] += q.y; y[4 * v + 2] += q.z; y[4 * v + 3] += q.w;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (n0 + j < N) y[j] += r[j];
+        }
+    }
+}
+
 // Loads bias[n0 .. n0+32) into registers (zeros past N or without bias).
 __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N, float (&b)[32]) {
     if (bias == nullptr) {
@@ -245,6 +283,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
             apply_act_chunk(p.act, y);
+            if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
             else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, false);
         }

@@ -40,6 +40,7 @@ struct SkinnyParams {
     int max_slots;           // partial slots per band
     int act;
     const float* bias;
+    const void* residual;    // [M,N] in the output's element type, added after the activation, or null
     void* out;
     float* partial;          // [n_tiles][max_slots][16][128] fp32
     uint32_t* tickets;       // [n_tiles], zero between launches
@@ -73,6 +74,19 @@ struct SkinnyCfg {
 
 __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, int grid) {
     return static_cast<int>(((u + 1) * grid - 1) / total);
+}
+
+// out[m][n] = y (+ R[m][n]), rounded once to the output type.
+template <bool OUT_BF16>
+__device__ __forceinline__ void skinny_store(const SkinnyParams& p, int m, int n, float y) {
+    const size_t idx = static_cast<size_t>(m) * p.N + n;
+    if (OUT_BF16) {
+        if (p.residual) y += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.residual)[idx]);
+        reinterpret_cast<__nv_bfloat16*>(p.out)[idx] = __float2bfloat16_rn(y);
+    } else {
+        if (p.residual) y += reinterpret_cast<const float*>(p.residual)[idx];
+        reinterpret_cast<float*>(p.out)[idx] = y;
+    }
 }
 
 template <bool OUT_BF16, bool PAIR>
@@ -286,13 +300,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     if (row_ok) {
 #pragma unroll
                         for (int m = 0; m < 16; ++m) {
-                            if (m < p.M) {
-                                const float y = apply_act(p.act, acc[m] + bn);
-                                if (OUT_BF16)
-                                    reinterpret_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
-                                else
-                                    reinterpret_cast<float*>(p.out)[static_cast<size_t>(m) * p.N + n] = y;
-                            }
+                            if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
                         }
                     }
                 }
@@ -385,13 +393,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             if (finalize && row_ok) {
 #pragma unroll
                 for (int m = 0; m < 16; ++m) {
-                    if (m < p.M) {
-                        const float y = apply_act(p.act, acc[m] + bn);
-                        if (OUT_BF16)
-                            reinterpret_cast<__nv_bfloat16*>(p.out)[static_cast<size_t>(m) * p.N + n] = __float2bfloat16_rn(y);
-                        else
-                            reinterpret_cast<float*>(p.out)[static_cast<size_t>(m) * p.N + n] = y;
-                    }
+                    if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
                 }
             }
             ++tile;

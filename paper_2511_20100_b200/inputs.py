@@ -27,11 +27,18 @@ CONFIGS = {
     "C5": dict(op="fused_linear", M=16, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=4),
 }
 
-# Further row reductions on the LM-head shape (measured beside the five, not part of the benchmark step).
+# Further operators of the same family (measured beside the five, not part of the benchmark step).
 EXTRA_CONFIGS = {
     "X1": dict(op="linear_rowmax", M=4096, N=32000, K=4096, seed=3),
     "X2": dict(op="linear_cross_entropy", M=4096, N=32000, K=4096, seed=3),
+    # the MLP down-projection that follows C3, with the skip connection joined to the epilogue
+    "X3": dict(op="fused_linear_residual", M=8192, N=4096, K=11008, act="none", out_dtype="bf16", seed=5),
 }
+
+
+def residual(M: int, N: int, seed: int, dtype=torch.bfloat16) -> torch.Tensor:
+    """Seeded N(0,1) residual stream [M,N] in the output dtype."""
+    return torch.randn(M, N, generator=_gen(seed + 1000), dtype=torch.float32).to(dtype)
 
 
 def targets(M: int, N: int, seed: int) -> torch.Tensor:

@@ -99,6 +99,26 @@ def test_cta_pair_and_single_cta_kernels_agree_with_the_oracle(cta_pair):
                                                       ref.ACT_RELU), TOL["fp32"], "129x257x72")
 
 
+@pytest.mark.parametrize("M,N,K", [(9, 520, 392), (16, 4096, 512), (129, 257, 72), (300, 520, 200), (600, 1000, 328)])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_fused_linear_residual(M, N, K, odt):
+    """Skip connection joined to the epilogue, on the skinny, single-CTA and CTA-pair paths; also in place."""
+    li = inputs.linear_inputs(M, N, K, seed=6000 + M + N)
+    tdt = torch.bfloat16 if odt == "bf16" else torch.float32
+    R = torch.randn(M, N, generator=torch.Generator().manual_seed(M * N)).to(tdt)
+    Rnp = inputs.bf16_bits(R) if odt == "bf16" else R.numpy()
+    want = ref.fused_linear_residual(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), Rnp, ref.ACT_SILU)
+    buf, out = _guarded((M, N), tdt)
+    Xd, Wd, bd, Rd = li.X.cuda(), li.W.cuda(), li.b.cuda(), R.cuda()
+    B.mtmc_fused_linear_residual(Xd, Wd, bd, Rd, "silu", odt, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "residual %dx%dx%d %s" % (M, N, K, odt))
+    B.mtmc_fused_linear_residual(Xd, Wd, bd, Rd, "silu", odt, out=Rd)          # in place
+    B.mtmc_check_status()
+    assert torch.equal(Rd, out)
+
+
 def test_fused_linear_exact_integers_and_no_bias():
     # integer-valued operands: every product and fp32 partial sum is exact, so the result must be too
     g = torch.Generator().manual_seed(5)
