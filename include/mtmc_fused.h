@@ -68,9 +68,10 @@ extern "C" {
  * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
  * the bias add and activation happen in fp32 on the fp32 accumulator, with no
  * intermediate rounding.)  X, W bf16; b fp32 or NULL; out fp32 or bf16 [M,N]
- * according to out_dtype.  Shapes with M <= 16 and a long K take the split-K
- * weight-streaming path (HBM-bound decode shape); all others the tiled
- * tensor-core path.  Needs workspace only on the split-K path. */
+ * according to out_dtype.  Shapes with M <= 64 (decode batches) take the split-K
+ * weight-streaming path (HBM-bound); all others the tiled tensor-core path.
+ * Needs workspace only on the ticketed variant of the split-K path (few rows of W,
+ * or a forced split; see mtmc_workspace_bytes). */
 int mtmc_fused_linear(const void* X, const void* W, const float* b,
                       int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 

@@ -23,7 +23,7 @@ using namespace mtmc;
 
 constexpr int MAX_DEVICES = 64;
 constexpr size_t TICKET_BYTES = 64 * 1024;   // library-owned split-K tickets: 16384 tiles
-constexpr int SKINNY_MAX_M = 16;
+constexpr int SKINNY_MAX_M = 64;              // rows of X the weight-streaming path takes (MMA N = 16, 32 or 64)
 
 struct DeviceState {
     bool ready = false;
@@ -303,7 +303,7 @@ int skinny_cta_of_unit_host(long long u, long long total, int grid) {
 }
 
 struct SkinnyPlan {
-    int n_tiles, k_blocks, grid, max_slots, tile_rows, stages, pair;
+    int n_tiles, k_blocks, grid, max_slots, tile_rows, stages, pair, mx;
     long long total;
     size_t ticket_bytes, partial_bytes;
 };
@@ -314,8 +314,9 @@ struct SkinnyPlan {
 //    pair reduces through distributed shared memory.
 //  * ticket plan (few rows, or a forced split): 128-row bands, the (band, k-block) list cut
 //    evenly over the SMs or over n_tiles * split_k CTAs; partials and tickets in the workspace.
-SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
+SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t M, int64_t N, int64_t K) {
     SkinnyPlan s;
+    s.mx = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
     s.k_blocks = static_cast<int>((K + 63) / 64);
     s.tile_rows = 128;
     s.n_tiles = static_cast<int>((N + 127) / 128);
@@ -337,7 +338,8 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
         if (g > 65535 * 16) g = 65535 * 16;
     }
     s.grid = static_cast<int>(g);
-    s.stages = SkinnyCfg::stages_for(s.tile_rows);
+    s.stages = s.mx == 16 ? SkinnyCfg<16>::stages_for(s.tile_rows)
+                          : (s.mx == 32 ? SkinnyCfg<32>::stages_for(s.tile_rows) : SkinnyCfg<64>::stages_for(s.tile_rows));
     int mx = 1;
     if (!s.pair) {
         for (int t = 0; t < s.n_tiles; ++t) {
@@ -348,7 +350,7 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t N, int64_t K) {
     }
     s.max_slots = mx;
     s.ticket_bytes = s.pair ? 0 : round256(static_cast<size_t>(s.n_tiles) * 4);
-    s.partial_bytes = mx > 1 ? static_cast<size_t>(s.n_tiles) * s.max_slots * 16 * 128 * 4 : 0;
+    s.partial_bytes = mx > 1 ? static_cast<size_t>(s.n_tiles) * s.max_slots * s.mx * 128 * 4 : 0;
     return s;
 }
 
@@ -367,14 +369,14 @@ __global__ void timeout_probe_kernel(uint32_t* status) {
     }
 }
 
-template <bool OUT_BF16, bool PAIR>
+template <bool OUT_BF16, bool PAIR, int MX>
 int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap& tmX, const SkinnyParams& p) {
-    auto kern = skinny_splitk_kernel<OUT_BF16, PAIR>;
-    if (int rc = ensure_smem_attr(kern, SkinnyCfg::SMEM_BYTES)) return rc;
+    auto kern = skinny_splitk_kernel<OUT_BF16, PAIR, MX>;
+    if (int rc = ensure_smem_attr(kern, SkinnyCfg<MX>::SMEM_BYTES)) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(s.grid), 1, 1);
     cfg.blockDim = dim3(192, 1, 1);
-    cfg.dynamicSmemBytes = SkinnyCfg::SMEM_BYTES;
+    cfg.dynamicSmemBytes = SkinnyCfg<MX>::SMEM_BYTES;
     cfg.stream = t_stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -392,12 +394,12 @@ int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap
 // cannot be scheduled): the pair plan sizes its bands to this.
 int skinny_pairs(DeviceState* d) {
     if (d->max_pairs < 0) {
-        auto kern = skinny_splitk_kernel<true, true>;
+        auto kern = skinny_splitk_kernel<true, true, 16>;
         int n = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2u * static_cast<unsigned>(d->sm_count), 1, 1);
         cfg.blockDim = dim3(192, 1, 1);
-        cfg.dynamicSmemBytes = SkinnyCfg::SMEM_BYTES;
+        cfg.dynamicSmemBytes = SkinnyCfg<16>::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -405,7 +407,7 @@ int skinny_pairs(DeviceState* d) {
         attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg::SMEM_BYTES) != cudaSuccess ||
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SkinnyCfg<16>::SMEM_BYTES) != cudaSuccess ||
             cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
             (void)cudaGetLastError();
             n = 0;
@@ -417,7 +419,7 @@ int skinny_pairs(DeviceState* d) {
 
 int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K,
                int act, int out_dtype, void* out) {
-    SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), N, K);
+    SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
     SkinnyParams p;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
@@ -443,11 +445,17 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
     CUtensorMap tmW, tmX;
     int rc = encode_bf16_2d(&tmW, W, N, K, s.tile_rows);
     if (rc) return rc;
-    rc = encode_bf16_2d(&tmX, X, M, K, SkinnyCfg::MX);
+    rc = encode_bf16_2d(&tmX, X, M, K, s.mx);
     if (rc) return rc;
     TimedRegion tr(d);
-    rc = out_dtype == MTMC_OUT_BF16 ? (s.pair ? launch_skinny<true, true>(s, tmW, tmX, p) : launch_skinny<true, false>(s, tmW, tmX, p))
-                                    : (s.pair ? launch_skinny<false, true>(s, tmW, tmX, p) : launch_skinny<false, false>(s, tmW, tmX, p));
+    const bool bf = out_dtype == MTMC_OUT_BF16;
+#define MTMC_SKINNY_DISPATCH(MXV)                                                                         \
+    rc = bf ? (s.pair ? launch_skinny<true, true, MXV>(s, tmW, tmX, p) : launch_skinny<true, false, MXV>(s, tmW, tmX, p)) \
+            : (s.pair ? launch_skinny<false, true, MXV>(s, tmW, tmX, p) : launch_skinny<false, false, MXV>(s, tmW, tmX, p))
+    if (s.mx == 16) { MTMC_SKINNY_DISPATCH(16); }
+    else if (s.mx == 32) { MTMC_SKINNY_DISPATCH(32); }
+    else { MTMC_SKINNY_DISPATCH(64); }
+#undef MTMC_SKINNY_DISPATCH
     tr.stop();
     return rc;
 }
@@ -566,7 +574,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
             if (!use_skinny(M, N)) return 0;
             DeviceState* d = nullptr;
             if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
-            SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), N, K);
+            SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
             return s.ticket_bytes + s.partial_bytes;
         }
         case MTMC_OP_SWIGLU: return 0;

@@ -35,31 +35,32 @@ struct SkinnyParams {
     int M, N, K;
     int n_tiles, k_blocks;
     int tile_rows;           // W rows per band (multiple of 8, <= 128)
-    int num_stages;          // TMA ring depth (<= SkinnyCfg::MAX_STAGES)
+    int num_stages;          // TMA ring depth (<= SkinnyCfg<MX>::MAX_STAGES)
     long long total_units;   // n_tiles * k_blocks
     int max_slots;           // partial slots per band
     int act;
     const float* bias;
     const void* residual;    // [M,N] in the output's element type, added after the activation, or null
     void* out;
-    float* partial;          // [n_tiles][max_slots][16][128] fp32
+    float* partial;          // [n_tiles][max_slots][MX][128] fp32
     uint32_t* tickets;       // [n_tiles], zero between launches
     uint32_t* status;
 };
 
+template <int MX_>
 struct SkinnyCfg {
     static constexpr int LANES = 128;                     // MMA M = TMEM lanes
-    static constexpr int MX = 16;                         // X rows = MMA N
+    static constexpr int MX = MX_;                        // X rows = MMA N: 16, 32 or 64
     static constexpr int BK = 64;                         // k-block: one 128-byte swizzle row
     static constexpr int KB_PER_STAGE = 2;                // k-blocks per ring stage
-    static constexpr int X_BYTES = MX * BK * 2;           // 2 KiB per k-block
+    static constexpr int X_BYTES = MX * BK * 2;           // 2 / 4 / 8 KiB per k-block
     static constexpr int MAX_STAGES = 16;
-    static constexpr int RING_BYTES = 200 * 1024;         // shared memory given to the TMA ring
-    static constexpr int WAYS = 8;                        // independent accumulators
-    static constexpr int ACC_COLS = WAYS * MX;            // 128 TMEM columns per accumulator set
+    static constexpr int WAYS = MX == 64 ? 4 : 8;         // independent accumulators
+    static constexpr int ACC_COLS = WAYS * MX;            // TMEM columns per accumulator set (128 / 256 / 256)
     static constexpr int TMEM_COLS = 2 * ACC_COLS;        // two sets: MMA on one, epilogue on the other
     static constexpr int NUM_BARRIERS = 2 * MAX_STAGES + 5;   // ring, accumulator sets, pair reduction
     static constexpr int REDUCE_BYTES = MX * LANES * 4;       // the peer CTA's partial (PAIR mode)
+    static constexpr int RING_BYTES = 208 * 1024 - REDUCE_BYTES;   // shared memory given to the TMA ring
     static constexpr int SMEM_BYTES = RING_BYTES + REDUCE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int stage_bytes(int tile_rows) { return KB_PER_STAGE * (tile_rows * BK * 2 + X_BYTES); }
     // The MMA always reads a 128-row (16 KiB) A tile, also when the band is shorter, so the
@@ -71,6 +72,24 @@ struct SkinnyCfg {
     }
 };
 
+// acc[m] += the accumulator ways that were written, in way order (TMEM -> registers).
+template <int MX, int WAYS>
+__device__ __forceinline__ void skinny_sum_ways(uint32_t set_addr, int ways_used, float (&acc)[MX]) {
+#pragma unroll
+    for (int l = 0; l < WAYS * MX / 32; ++l) {                // 32 TMEM columns per load
+        const int first_way = (32 * l) / MX;
+        if (first_way < ways_used) {                          // warp-uniform
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(set_addr + 32 * l, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int way = (32 * l + j) / MX;            // differs from first_way only when MX == 16
+                if (MX >= 32 || way < ways_used) acc[(32 * l + j) % MX] += __uint_as_float(r[j]);
+            }
+        }
+    }
+}
 
 __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, int grid) {
     return static_cast<int>(((u + 1) * grid - 1) / total);
@@ -89,11 +108,11 @@ __device__ __forceinline__ void skinny_store(const SkinnyParams& p, int m, int n
     }
 }
 
-template <bool OUT_BF16, bool PAIR>
+template <bool OUT_BF16, bool PAIR, int MX>
 __global__ void __launch_bounds__(192, 1)
 skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                      const SkinnyParams p) {
-    using Cfg = SkinnyCfg;
+    using Cfg = SkinnyCfg<MX>;
     constexpr int MAXS = Cfg::MAX_STAGES;
     constexpr int KPS = Cfg::KB_PER_STAGE;
     const int STAGES = p.num_stages;
@@ -105,7 +124,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
-    const uint32_t reduce_base = base + Cfg::RING_BYTES;                  // [16][128] fp32, written by the peer CTA
+    const uint32_t reduce_base = base + Cfg::RING_BYTES;                  // [MX][128] fp32, written by the peer CTA
     const uint32_t bar_base = reduce_base + Cfg::REDUCE_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (MAXS + s); };
@@ -259,28 +278,13 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             const int n = first_tile * R + nl;
             const bool row_ok = nl < R && n < p.N;
             const float bn = (crank == 0 && row_ok && p.bias) ? __ldg(p.bias + n) : 0.0f;
-            float acc[16];
+            float acc[MX];
 #pragma unroll
-            for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
+            for (int m = 0; m < MX; ++m) acc[m] = 0.0f;
             if (n_units > 0) ok = mbar_wait(accf_bar(0), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 3u);
             if (ok && n_units > 0) {
                 tc_fence_after();
-                const int ways_used = min(Cfg::WAYS, n_units * (Cfg::BK / 16));
-                const uint32_t set_addr = tmem_base + lane_base;
-#pragma unroll
-                for (int w = 0; w < Cfg::WAYS; w += 2) {
-                    if (w < ways_used) {
-                        uint32_t r[32];
-                        tmem_ld_32x32b_x32(set_addr + w * Cfg::MX, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[m]);
-                        if (w + 1 < ways_used) {
-#pragma unroll
-                            for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[16 + m]);
-                        }
-                    }
-                }
+                skinny_sum_ways<MX, Cfg::WAYS>(tmem_base + lane_base, min(Cfg::WAYS, n_units * (Cfg::BK / 16)), acc);
                 tc_fence_before();
             }
             cluster_wait();                                    // set-up phase: the peer's barriers exist
@@ -288,7 +292,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 // hand the partial to the even CTA: [m][lane] floats in its shared memory
                 const uint32_t dst = cluster_map_shared(reduce_base, 0) + static_cast<uint32_t>(nl) * 4u;
 #pragma unroll
-                for (int m = 0; m < 16; ++m) st_shared_cluster_f32(dst + m * (Cfg::LANES * 4), ok ? acc[m] : 0.0f);
+                for (int m = 0; m < MX; ++m) st_shared_cluster_f32(dst + m * (Cfg::LANES * 4), ok ? acc[m] : 0.0f);
                 fence_acq_rel_cluster();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_remote(cluster_map_shared(red_bar, 0));
@@ -296,10 +300,10 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 if (mbar_wait_cluster(red_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 4u)) {
                     const float* peer = reinterpret_cast<const float*>(smem_raw + (reduce_base - raw_addr)) + nl;
 #pragma unroll
-                    for (int m = 0; m < 16; ++m) acc[m] += peer[m * Cfg::LANES];       // rank 0 + rank 1
+                    for (int m = 0; m < MX; ++m) acc[m] += peer[m * Cfg::LANES];       // rank 0 + rank 1
                     if (row_ok) {
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) {
+                        for (int m = 0; m < MX; ++m) {
                             if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
                         }
                     }
@@ -318,25 +322,11 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             acc_ph ^= 1u << buf;
             tc_fence_after();
             // Sum the accumulator ways that this segment wrote, in way order.
-            const int ways_used = min(Cfg::WAYS, seg * (Cfg::BK / 16));
-            float acc[16];
+            float acc[MX];
 #pragma unroll
-            for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
-            const uint32_t set_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::ACC_COLS);
-#pragma unroll
-            for (int w = 0; w < Cfg::WAYS; w += 2) {
-                if (w < ways_used) {                           // warp-uniform
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(set_addr + w * Cfg::MX, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[m]);
-                    if (w + 1 < ways_used) {
-#pragma unroll
-                        for (int m = 0; m < 16; ++m) acc[m] += __uint_as_float(r[16 + m]);
-                    }
-                }
-            }
+            for (int m = 0; m < MX; ++m) acc[m] = 0.0f;
+            skinny_sum_ways<MX, Cfg::WAYS>(tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::ACC_COLS),
+                                           min(Cfg::WAYS, seg * (Cfg::BK / 16)), acc);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acce_bar(buf));     // registers hold the band: free the set now
@@ -348,10 +338,10 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 const int c_last = skinny_cta_of_unit(t_first + KB - 1, p.total_units, gridDim.x);
                 const int n_contrib = c_last - c_first + 1;
                 const int slot = static_cast<int>(blockIdx.x) - c_first;
-                float* band = p.partial + static_cast<size_t>(tile) * p.max_slots * (16 * 128) + nl;
-                float* my = band + static_cast<size_t>(slot) * (16 * 128);
+                float* band = p.partial + static_cast<size_t>(tile) * p.max_slots * (MX * 128) + nl;
+                float* my = band + static_cast<size_t>(slot) * (MX * 128);
 #pragma unroll
-                for (int m = 0; m < 16; ++m) __stcg(my + m * 128, acc[m]);
+                for (int m = 0; m < MX; ++m) __stcg(my + m * 128, acc[m]);
                 __threadfence();
                 named_barrier_sync(1, 128);
                 if (epi_tid == 0) {
@@ -366,25 +356,21 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     if (n_contrib == 2) {
                         // a + b == b + a exactly: adding the other CTA's partial to the registers gives
                         // the same bits whichever of the two arrives last
-                        const float* other = band + static_cast<size_t>(1 - slot) * (16 * 128);
-                        float o[16];
+                        const float* other = band + static_cast<size_t>(1 - slot) * (MX * 128);
+                        float o[MX];
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) o[m] = __ldcg(other + m * 128);
+                        for (int m = 0; m < MX; ++m) o[m] = __ldcg(other + m * 128);
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) acc[m] += o[m];
+                        for (int m = 0; m < MX; ++m) acc[m] += o[m];
                     } else {
 #pragma unroll
-                        for (int m = 0; m < 16; ++m) acc[m] = 0.0f;
-                        for (int sl = 0; sl < n_contrib; sl += 2) {          // slot order, two slots in flight
-                            float a0[16], a1[16];
-                            const bool two = sl + 1 < n_contrib;
+                        for (int m = 0; m < MX; ++m) acc[m] = 0.0f;
+                        for (int sl = 0; sl < n_contrib; ++sl) {             // slot order
+                            float a0[MX];
 #pragma unroll
-                            for (int m = 0; m < 16; ++m) {
-                                a0[m] = __ldcg(band + (static_cast<size_t>(sl) * 16 + m) * 128);
-                                a1[m] = two ? __ldcg(band + (static_cast<size_t>(sl + 1) * 16 + m) * 128) : 0.0f;
-                            }
+                            for (int m = 0; m < MX; ++m) a0[m] = __ldcg(band + (static_cast<size_t>(sl) * MX + m) * 128);
 #pragma unroll
-                            for (int m = 0; m < 16; ++m) { acc[m] += a0[m]; if (two) acc[m] += a1[m]; }
+                            for (int m = 0; m < MX; ++m) acc[m] += a0[m];
                         }
                     }
                     finalize = true;
@@ -392,7 +378,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             }
             if (finalize && row_ok) {
 #pragma unroll
-                for (int m = 0; m < 16; ++m) {
+                for (int m = 0; m < MX; ++m) {
                     if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
                 }
             }

@@ -274,12 +274,30 @@ def test_rowmax_and_cross_entropy_at_lm_head_size_on_sampled_rows():
     (16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392),   # few rows: ticketed split-K
     (16, 4096, 512), (7, 2400, 1096), (3, 9472, 72), (16, 2368, 128),                  # cluster-pair split-K
     (16, 20000, 256), (2, 9480, 64),                                                   # many rows / one k-block
+    (17, 520, 392), (32, 4096, 512), (33, 2400, 1096), (64, 9472, 136), (50, 300, 2048), (64, 20000, 128),   # decode batches up to 64
 ])
 @pytest.mark.parametrize("odt", ["fp32", "bf16"])
 def test_skinny_small(M, N, K, odt):
     li, out = run_linear(M, N, K, "gelu_tanh", odt, seed=4000 + M + N)
     want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
     _assert_close(inputs.to_f64(out), want, TOL[odt], "skinny %dx%dx%d %s" % (M, N, K, odt))
+
+
+@pytest.mark.parametrize("M", [24, 64])
+@pytest.mark.parametrize("split_k", [1, 3])
+def test_skinny_decode_batch_forced_split(M, split_k):
+    li = inputs.linear_inputs(M, 640, 2048, seed=46)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_SILU)
+    B.mtmc_set_tuning(split_k=split_k)
+    try:
+        Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+        first = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
+        again = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(first), want, TOL["fp32"], "M %d split_k %d" % (M, split_k))
+    assert torch.equal(first, again)
 
 
 @pytest.mark.parametrize("split_k", [1, 2, 8, 37])
