@@ -303,6 +303,7 @@ def run_ours(args, rank, world, local_rank):
         for v in variants:
             call_device(B, v)
         torch.cuda.synchronize()
+        time.sleep(args.settle_s)      # let the power/clock state left by the previous loop settle: each loop describes its own kernel
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(3):
@@ -419,7 +420,7 @@ def run_ours(args, rank, world, local_rank):
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "+".join(ORDER) + " (one call each per step)",
                        "l2": "inputs larger than L2: a step reads ~1.0 GB of distinct operands (L2 126 MB), every call starts cold; "
-                             "per_config loops rotate operand copies totalling > 2x L2",
+                             "per_config loops rotate operand copies totalling > 2x L2 and start after 0.5 s of idle",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "per_config": per_config, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
@@ -469,6 +470,7 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--settle-s", type=float, default=0.5, help="idle time before each per-configuration loop")
     ap.add_argument("--loop-ms", type=float, default=150.0, help="target length of each per-configuration timing loop")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
     ap.add_argument("--no-extras", action="store_true", help="skip the row-max / cross-entropy measurements")

@@ -419,6 +419,8 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_launch_dependents();     // the next kernel in the stream may begin its own set-up
+    pdl_wait();                  // everything before this line touched only shared and tensor memory
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
