@@ -399,7 +399,7 @@ int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;      // no programmatic dependent launch here: measured slower for this 30 us kernel
+    cfg.numAttrs = 1 + pdl_attribute(attr + 1);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmW, tmX, p));
     g_launches.fetch_add(1);
     return MTMC_OK;

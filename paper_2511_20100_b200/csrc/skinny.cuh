@@ -182,6 +182,8 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         __syncwarp();
         asm volatile("bar.arrive 2, 192;" ::: "memory");
         if (PAIR) cluster_arrive();          // publishes red_bar's initialisation to the peer; waited for at the end
+        pdl_launch_dependents();
+        pdl_wait();                          // before the first load from global memory
     } else {
         if (warp == 1) {
             tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
@@ -191,6 +193,8 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         asm volatile("bar.sync 2, 192;" ::: "memory");
         tc_fence_after();
         if (PAIR) cluster_arrive();          // after bar.sync: this CTA's barriers are initialised
+        pdl_launch_dependents();
+        pdl_wait();                          // before the first access to global memory
     }
 
     if (warp == 0) {
