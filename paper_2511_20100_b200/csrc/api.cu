@@ -535,12 +535,57 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     return MTMC_OK;
 }
 
-}  // namespace
-
-namespace {
+// out = act(X.W^T + b) (+ R): picks the weight-streaming path for decode batches, CTA pairs for
+// large shapes and single-CTA tiles otherwise.
 int fused_linear_impl(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K, int act,
-                      int out_dtype, void* out);
+                      int out_dtype, void* out) {
+    int rc = check_common(X, W, out, M, N, K);
+    if (rc) return rc;
+    if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    rc = get_device(&d);
+    if (rc) return rc;
+    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out);
+
+    if (use_pair(d, M, N)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB, tmBt;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
+            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
+            return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+        tr.stop();
+        return rc;
+    }
+    const int bn = pick_tile_n(N);
+    GemmParams p{};
+    fill_tiling(p, M, N, K, bn, d->sm_count, true);
+    p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    CUtensorMap tmA, tmB, tmBt;
+    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmB, W, N, K, bn);
+    if (rc) return rc;
+    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    if (bn == 256) {
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    } else {
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                        : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    }
+    tr.stop();
+    return rc;
 }
+}  // namespace
 
 extern "C" {
 
@@ -636,61 +681,6 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
     if (!aligned16(R)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
     return fused_linear_impl(X, W, b, R, M, N, K, act, out_dtype, out);
 }
-
-}  // extern "C"
-
-namespace {
-int fused_linear_impl(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K, int act,
-                      int out_dtype, void* out) {
-    int rc = check_common(X, W, out, M, N, K);
-    if (rc) return rc;
-    if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
-    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
-    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
-    DeviceState* d = nullptr;
-    rc = get_device(&d);
-    if (rc) return rc;
-    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out);
-
-    if (use_pair(d, M, N)) {
-        GemmParams p{};
-        fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
-        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-        CUtensorMap tmA, tmB, tmBt;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
-            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
-            return rc;
-        TimedRegion tr(d);
-        rc = out_dtype == MTMC_OUT_BF16 ? launch_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
-                                        : launch_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
-        tr.stop();
-        return rc;
-    }
-    const int bn = pick_tile_n(N);
-    GemmParams p{};
-    fill_tiling(p, M, N, K, bn, d->sm_count, true);
-    p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-    CUtensorMap tmA, tmB, tmBt;
-    rc = encode_bf16_2d(&tmA, X, M, K, 128);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmB, W, N, K, bn);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
-    if (rc) return rc;
-    TimedRegion tr(d);
-    if (bn == 256) {
-        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
-                                        : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
-    } else {
-        rc = out_dtype == MTMC_OUT_BF16 ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
-                                        : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
-    }
-    tr.stop();
-    return rc;
-}
-}  // namespace
-
-extern "C" {
 
 int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
     int rc = check_common(X, Wg, out, M, N, K);
