@@ -15,6 +15,9 @@
 //   z[m][n]  = sum_{k=0..K-1} X[m][k] * W[n][k]  (+ b[n])        "X . W^T + b"
 //   fused linear :  Y[m][n] = act(z[m][n]),  act in {identity, ReLU, GELU-tanh, SiLU}
 //   + residual   :  Y[m][n] = act(z[m][n]) + R[m][n]   (the layer's skip connection joined to the epilogue)
+//   FP8 linear   :  Y[m][n] = act( sx*sw * sum_k Xq[m][k] Wq[n][k] + b[n] ),  Xq, Wq 8-bit floats
+//                   (E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities),
+//                   sx, sw per-tensor scales: the lower-precision variant of the same layer
 //   SwiGLU       :  out[m][n] = silu(g[m][n]) * u[m][n],  g = X.Wg^T, u = X.Wu^T (no bias)
 //   row LSE      :  lse[m] = log( sum_n exp(z[m][n]) ), computed two-pass (max, then sum)
 //   row max      :  mx[m] = max_n z[m][n], arg[m] = the lowest n attaining it
@@ -56,6 +59,17 @@ double bf16_to_double(uint16_t bits) {
     float f;
     std::memcpy(&f, &u, sizeof f);
     return static_cast<double>(f);
+}
+
+// E4M3 bit pattern -> double, exactly.  exponent field 0: subnormal m/8 * 2^-6; otherwise
+// (1 + m/8) * 2^(e-7); the pattern S.1111.111 is NaN (the format has no infinities).
+double e4m3_to_double(uint8_t bits) {
+    const int sign = bits >> 7, e = (bits >> 3) & 15, m = bits & 7;
+    double v;
+    if (e == 15 && m == 7) v = std::numeric_limits<double>::quiet_NaN();
+    else if (e == 0) v = std::ldexp(static_cast<double>(m) / 8.0, -6);
+    else v = std::ldexp(1.0 + static_cast<double>(m) / 8.0, e - 7);
+    return sign ? -v : v;
 }
 
 // One pre-activation value: ascending k, one double accumulator, bias added last.
@@ -135,6 +149,45 @@ int mtmc_ref_fused_linear_residual(const uint16_t* X, const uint16_t* W, const f
                                        : static_cast<double>(static_cast<const float*>(R)[m * N + n]);
             out[m * N + n] = act_apply(act, preact(X, W, b, K, m, n)) + r;
         }
+    });
+    return 0;
+}
+
+// Scalar decode of one E4M3 pattern (for the pins).
+double mtmc_ref_e4m3(uint8_t bits) { return e4m3_to_double(bits); }
+
+// Y = act(sx*sw * Xq.Wq^T + b) with E4M3 operands (one byte per element), full output in double.
+int mtmc_ref_fused_linear_fp8(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                              int64_t M, int64_t N, int64_t K, int act, double* out) {
+    if (!X || !W || !out || M <= 0 || N <= 0 || K <= 0 || act < 0 || act > 3) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(M, [=](int64_t m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k) acc += e4m3_to_double(X[m * K + k]) * e4m3_to_double(W[n * K + k]);
+            double z = scale * acc;
+            if (b) z += static_cast<double>(b[n]);
+            out[m * N + n] = act_apply(act, z);
+        }
+    });
+    return 0;
+}
+
+// The same at P listed (row, col) positions.
+int mtmc_ref_fused_linear_fp8_points(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                                     int64_t M, int64_t N, int64_t K, int act,
+                                     const int64_t* rows, const int64_t* cols, int64_t P, double* out) {
+    if (!X || !W || !out || !rows || !cols || M <= 0 || N <= 0 || K <= 0 || act < 0 || act > 3) return 1;
+    for (int64_t p = 0; p < P; ++p)
+        if (rows[p] < 0 || rows[p] >= M || cols[p] < 0 || cols[p] >= N) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(P, [=](int64_t p) {
+        const int64_t m = rows[p], n = cols[p];
+        double acc = 0.0;
+        for (int64_t k = 0; k < K; ++k) acc += e4m3_to_double(X[m * K + k]) * e4m3_to_double(W[n * K + k]);
+        double z = scale * acc;
+        if (b) z += static_cast<double>(b[n]);
+        out[p] = act_apply(act, z);
     });
     return 0;
 }

@@ -43,6 +43,10 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_act.restype = dbl
         L.mtmc_ref_fused_linear.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp]
         L.mtmc_ref_fused_linear_residual.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, ci, vp]
+        L.mtmc_ref_e4m3.argtypes = [ctypes.c_uint8]
+        L.mtmc_ref_e4m3.restype = dbl
+        L.mtmc_ref_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp]
+        L.mtmc_ref_fused_linear_fp8_points.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
@@ -118,6 +122,42 @@ def fused_linear_residual(X, W, b, R, act_kind: int) -> np.ndarray:
     out = np.empty((M, N), dtype=np.float64)
     _check(lib().mtmc_ref_fused_linear_residual(X.ctypes.data, W.ctypes.data, bp, R.ctypes.data, int(R.dtype == np.uint16),
                                                 M, N, K, int(act_kind), out.ctypes.data), "mtmc_ref_fused_linear_residual")
+    return out
+
+
+def e4m3(bits: int) -> float:
+    return float(lib().mtmc_ref_e4m3(int(bits) & 0xFF))
+
+
+def _fp8(a, shape) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint8 or tuple(a.shape) != tuple(shape):
+        raise TypeError("fp8 operand must be a uint8 bit-pattern array of shape %r" % (shape,))
+    return a
+
+
+def fused_linear_fp8(X, W, b, scale_x: float, scale_w: float, act_kind: int) -> np.ndarray:
+    """act(scale_x*scale_w * Xq.Wq^T + b) with E4M3 bit patterns (uint8) for Xq [M,K] and Wq [N,K]."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
+                                           int(act_kind), out.ctypes.data), "mtmc_ref_fused_linear_fp8")
+    return out
+
+
+def fused_linear_fp8_points(X, W, b, scale_x: float, scale_w: float, act_kind: int, rows, cols) -> np.ndarray:
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    rows, cols = _idx(rows), _idx(cols)
+    out = np.empty(rows.shape[0], dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear_fp8_points(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
+                                                  int(act_kind), rows.ctypes.data, cols.ctypes.data, rows.shape[0],
+                                                  out.ctypes.data), "mtmc_ref_fused_linear_fp8_points")
     return out
 
 

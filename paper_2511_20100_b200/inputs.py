@@ -82,6 +82,32 @@ def swiglu_inputs(M: int, N: int, K: int, seed: int) -> SwigluInputs:
     return SwigluInputs(X, Wg, Wu)
 
 
+@dataclass
+class Fp8LinearInputs:
+    X: torch.Tensor            # [M, K] float8_e4m3fn, CPU
+    W: torch.Tensor            # [N, K] float8_e4m3fn, CPU
+    b: torch.Tensor | None     # [N] fp32
+    scale_x: float             # per-tensor scales: real value = scale * stored value
+    scale_w: float
+
+
+def fp8_linear_inputs(M: int, N: int, K: int, seed: int, bias: bool = True) -> Fp8LinearInputs:
+    """The bf16 recipe's draws, quantised per tensor to E4M3 with the scale that maps the largest
+    magnitude to 448 (the format's maximum); scales are rounded to fp32."""
+    li = linear_inputs(M, N, K, seed, bias)
+    out = []
+    for t in (li.X.float(), li.W.float()):
+        scale = float(torch.tensor(float(t.abs().max()) / 448.0, dtype=torch.float32)) or 1.0
+        out.append(((t / scale).to(torch.float8_e4m3fn), scale))
+    return Fp8LinearInputs(out[0][0], out[1][0], li.b, out[0][1], out[1][1])
+
+
+def fp8_bits(t: torch.Tensor) -> np.ndarray:
+    """float8_e4m3fn tensor (CPU) -> uint8 numpy array of the raw bit patterns."""
+    assert t.dtype == torch.float8_e4m3fn
+    return t.detach().cpu().contiguous().view(torch.uint8).numpy()
+
+
 def bf16_bits(t: torch.Tensor) -> np.ndarray:
     """bf16 tensor (CPU) -> uint16 numpy array of the same shape holding the raw bit patterns."""
     assert t.dtype == torch.bfloat16

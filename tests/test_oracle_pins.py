@@ -155,6 +155,47 @@ def test_residual_is_added_after_the_activation():
     np.testing.assert_allclose(ref.fused_linear_residual(X, W, b, R32, ref.ACT_RELU), want.numpy(), rtol=0, atol=1e-12)
 
 
+# ---------------------------------------------------------------- FP8 (E4M3) operands
+def test_e4m3_decode_every_pattern():
+    # known values of the format: 0x38 = 1, 0x7E = 448 (largest), 0x01 = 2^-9 (smallest subnormal), 0x08 = 2^-6
+    assert ref.e4m3(0x38) == 1.0 and ref.e4m3(0x7E) == 448.0 and ref.e4m3(0x01) == 2.0 ** -9 and ref.e4m3(0x08) == 2.0 ** -6
+    assert ref.e4m3(0xB8) == -1.0 and ref.e4m3(0x00) == 0.0 and math.isnan(ref.e4m3(0x7F)) and math.isnan(ref.e4m3(0xFF))
+    # and all 256 against torch's float8_e4m3fn conversion
+    pats = torch.arange(256, dtype=torch.int32).to(torch.uint8)
+    want = pats.view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    for i in range(256):
+        got = ref.e4m3(i)
+        assert (math.isnan(got) and math.isnan(want[i])) or got == want[i], i
+    # monotone in the positive half
+    vals = [ref.e4m3(i) for i in range(0x7F)]
+    assert all(a < b for a, b in zip(vals, vals[1:]))
+
+
+def test_fp8_linear_pins():
+    fi = inputs.fp8_linear_inputs(7, 13, 96, seed=71)
+    X8, W8, b = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    got = ref.fused_linear_fp8(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_NONE)
+    scale = float(np.float32(fi.scale_x)) * float(np.float32(fi.scale_w))
+    want = scale * (fi.X.to(torch.float64) @ fi.W.to(torch.float64).T) + fi.b.double()
+    np.testing.assert_allclose(got, want.numpy(), rtol=1e-13, atol=1e-13)
+    # exact brute force: every E4M3 value is a multiple of 2^-9, so products are multiples of 2^-18
+    xi = (fi.X.to(torch.float64) * 512).numpy().astype(np.int64)
+    wi = (fi.W.to(torch.float64) * 512).numpy().astype(np.int64)
+    raw = ref.fused_linear_fp8(X8, W8, None, 1.0, 1.0, ref.ACT_NONE)
+    for m in range(7):
+        for n in range(13):
+            assert Fraction(raw[m, n]) == Fraction(int((xi[m] * wi[n]).sum()), 512 * 512)
+    # scales multiply the sum, not the bias; activation applied last
+    twice = ref.fused_linear_fp8(X8, W8, b, 2.0 * fi.scale_x, fi.scale_w, ref.ACT_NONE)
+    np.testing.assert_allclose(twice - b.astype(np.float64), 2.0 * (got - b.astype(np.float64)), rtol=1e-13, atol=1e-13)
+    g = ref.fused_linear_fp8(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH)
+    np.testing.assert_allclose(g, torch.nn.functional.gelu(want, approximate="tanh").numpy(), rtol=1e-12, atol=1e-13)
+    rows, cols = np.array([0, 6, 3]), np.array([12, 0, 5])
+    assert np.array_equal(ref.fused_linear_fp8_points(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH, rows, cols), g[rows, cols])
+    # quantisation recipe: the largest magnitude lands on the format's maximum
+    assert float(fi.X.to(torch.float32).abs().max()) == 448.0 and float(fi.W.to(torch.float32).abs().max()) == 448.0
+
+
 # ---------------------------------------------------------------- activations
 def _closed_forms():
     rows = []
