@@ -50,6 +50,8 @@ def algorithmic_bytes(c) -> float:
     M, N, K = c["M"], c["N"], c["K"]
     if c["op"] == "swiglu":
         return 2.0 * (M * K + 2 * N * K) + 2.0 * M * N
+    if c["op"] == "fused_linear_fp8":
+        return 1.0 * (M * K + N * K) + 4.0 * N + 2.0 * M * N
     if c["op"] in ("linear_lse", "linear_rowmax", "linear_cross_entropy"):
         extra = {"linear_lse": 0.0, "linear_rowmax": 4.0 * M, "linear_cross_entropy": 8.0 * M}[c["op"]]
         return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M + extra
@@ -134,6 +136,11 @@ def reduce_max(dist, value: float, device) -> float:
 # --------------------------------------------------------------------------------------- our arm
 def make_device_problem(name, device):
     c = inputs.CONFIGS.get(name) or inputs.EXTRA_CONFIGS[name]
+    if c["op"] == "fused_linear_fp8":
+        fi = inputs.fp8_linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+        dev = [fi.X.to(device), fi.W.to(device), fi.b.to(device)]
+        out = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=device)
+        return {"name": name, "cfg": c, "host": [], "dev": dev, "out": out, "scales": (fi.scale_x, fi.scale_w)}
     if c["op"] == "swiglu":
         si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
         host = [si.X, si.Wg, si.Wu]
@@ -165,6 +172,8 @@ def call_device(B, pr):
         B.mtmc_linear_cross_entropy(d[0], d[1], d[2], d[3], loss_out=pr["out"])
     elif c["op"] == "fused_linear_residual":
         B.mtmc_fused_linear_residual(d[0], d[1], d[2], d[3], c["act"], c["out_dtype"], out=pr["out"])
+    elif c["op"] == "fused_linear_fp8":
+        B.mtmc_fused_linear_fp8(d[0], d[1], d[2], pr["scales"][0], pr["scales"][1], c["act"], c["out_dtype"], out=pr["out"])
     else:
         B.mtmc_fused_linear(d[0], d[1], d[2], c["act"], c["out_dtype"], out=pr["out"])
 
@@ -319,7 +328,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         per_cfg_ms[n] = e0.elapsed_time(e1) / reps
         per_cfg_reps[n], per_cfg_copies[n] = reps, copies
-        if not args.no_eager:
+        if not args.no_eager and c["op"] != "fused_linear_fp8":
             # context: the unfused torch sequence (cuBLAS GEMM + elementwise kernels), same rotation
             for v in variants:
                 eager_call(pr, v["dev"])
@@ -354,6 +363,12 @@ def run_ours(args, rank, world, local_rank):
             entry["roofline"] = {"bound": "hbm", "achieved": entry["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": round(entry["gbs"] / peaks["hbm_gbs"], 4), "of": peaks["source"],
                                  "frac_of_nominal_8000": round(entry["gbs"] / 8000.0, 4)}
+        elif c["op"] == "fused_linear_fp8":
+            peak8 = 2.0 * peaks["tflops_sustained"]       # E4M3 peak = measured bf16 peak x the nominal 2:1 ratio
+            entry["roofline"] = {"bound": "tensor", "achieved": entry["tflops"], "peak": peak8, "unit": "TFLOP/s",
+                                 "frac": round(entry["tflops"] / peak8, 4),
+                                 "of": peaks["source"] + " sustained cuBLAS bf16 x 2 (nominal fp8:bf16 ratio)",
+                                 "frac_of_nominal_4500": round(entry["tflops"] / 4500.0, 4)}
         elif n != "C1":
             entry["roofline"] = {"bound": "tensor", "achieved": entry["tflops"], "peak": peaks["tflops_sustained"],
                                  "unit": "TFLOP/s", "frac": round(entry["tflops"] / peaks["tflops_sustained"], 4),

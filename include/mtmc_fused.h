@@ -84,6 +84,17 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b,
 int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, const void* R,
                                int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 
+/* The same layer with 8-bit floating-point operands:
+ *   out[m][n] = act( scale_x * scale_w * sum_k X8[m][k] W8[n][k] + b[n] ).
+ * X8 [M,K] and W8 [N,K] hold E4M3 values (1 sign, 4 exponent bits with bias 7, 3 mantissa
+ * bits, no infinities; one byte per element, dense row-major); scale_x, scale_w are the
+ * per-tensor scales (real value = scale * stored value), passed by value.  Products are
+ * exact and accumulate in fp32 on the tensor cores (tcgen05 kind::f8f6f4, K = 32 per MMA,
+ * twice the bf16 rate); the epilogue is the one of mtmc_fused_linear.  K % 16 == 0.  All M
+ * take the tiled kernels (no weight-streaming variant yet). */
+int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                          int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+
 /* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
  * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate
  * product fused in one kernel; neither GEMM result is written to memory.) */

@@ -22,7 +22,7 @@ OUT_DTYPE = {"fp32": 0, "bf16": 1}
 OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4}
 
 EXPORTS = [
-    "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_swiglu", "mtmc_linear_lse",
+    "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_fused_linear_fp8", "mtmc_swiglu", "mtmc_linear_lse",
     "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
@@ -44,13 +44,19 @@ def load() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError("libmtmcfused.so is missing at %s: build it with "
-                           "`python -m paper_2511_20100_b200.build` (there is no fallback path)" % LIB_PATH)
+    from . import build as _build
+    if _build.needs_build():
+        # missing or older than its sources: compile it in-tree (nvcc); there is no other code path to fall back on
+        try:
+            _build.build()
+        except Exception as e:
+            raise RuntimeError("libmtmcfused.so is missing or stale at %s and could not be built (%s); "
+                               "there is no fallback path" % (LIB_PATH, e))
     L = ctypes.CDLL(LIB_PATH)
     vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
     for name in ("mtmc_fused_linear", "mtmc_fused_linear_host"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
@@ -120,6 +126,21 @@ def mtmc_fused_linear_residual(X, W, b, R, act="none", out_dtype="bf16", out=Non
                                              None if b is None else _dev(b, torch.float32, (N,), "b"),
                                              _dev(R, odt, (M, N), "R"), M, N, K, ACT[act], OUT_DTYPE[out_dtype],
                                              _dev(out, odt, (M, N), "out")))
+    return out
+
+
+def mtmc_fused_linear_fp8(X8, W8, b, scale_x, scale_w, act="none", out_dtype="bf16", out=None):
+    """out = act(scale_x * scale_w * X8 @ W8.T + b) with float8_e4m3fn operands X8 [M,K], W8 [N,K]."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt, device=X8.device)
+    _use_current_stream(X8.device)
+    _check(load().mtmc_fused_linear_fp8(_dev(X8, torch.float8_e4m3fn, (M, K), "X8"), _dev(W8, torch.float8_e4m3fn, (N, K), "W8"),
+                                        None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                        float(scale_x), float(scale_w), M, N, K, ACT[act], OUT_DTYPE[out_dtype],
+                                        _dev(out, odt, (M, N), "out")))
     return out
 
 

@@ -120,6 +120,19 @@ int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols
     return MTMC_OK;
 }
 
+// 2-D E4M3 row-major [rows, cols] tensor (one byte per element), box = 128 columns x box_rows rows.
+int encode_u8_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols)};
+    cuuint32_t box[2] = {128u, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+    return MTMC_OK;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_common(const void* X, const void* W, const void* out, int64_t M, int64_t N, int64_t K) {
@@ -290,13 +303,17 @@ bool use_pair(DeviceState* d, int64_t M, int64_t N) {
 // Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
 // form a partial wave; cutting each of them into `tail_split` column pieces (2 or 4, pieces
 // at least 32 columns wide, all pieces fitting one wave) shortens that wave accordingly.
-void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail, int bm = 128) {
+void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail, int bm = 128,
+                 bool fp8 = false) {
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.m_tiles = static_cast<int>((M + bm - 1) / bm);
     p.rows_per_tile = bm;
     p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
     p.num_tiles = p.m_tiles * p.n_tiles;
-    p.k_blocks = static_cast<int>((K + 63) / 64);
+    p.fp8 = fp8 ? 1 : 0;
+    p.bk_elems = fp8 ? 128 : 64;               // one 128-byte swizzle row of K per ring stage
+    p.acc_scale = 1.0f;
+    p.k_blocks = static_cast<int>((K + p.bk_elems - 1) / p.bk_elems);
     p.group_m = pick_group_m(p.m_tiles);      // 16 row blocks per group measured best for both tile heights
     p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1; p.tail_width = out_tile_n;
     const int r = p.num_tiles % sm_count;
@@ -680,6 +697,41 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
     if (!R) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
     if (!aligned16(R)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
     return fused_linear_impl(X, W, b, R, M, N, K, act, out_dtype, out);
+}
+
+int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,
+                          int64_t K, int act, int out_dtype, void* out) {
+    if (!X8 || !W8 || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "dimensions must be below 2^31");
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for one-byte operands (16-byte rows for TMA)", (long long)K);
+    if (!aligned16(X8) || !aligned16(W8) || !aligned16(out) || (b && !aligned16(b))) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    const bool pair = use_pair(d, M, N);
+    const int bn = pair ? 256 : pick_tile_n(N);
+    GemmParams p{};
+    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, true);
+    else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, true);
+    p.acc_scale = scale_x * scale_w;
+    p.act = act; p.bias = b; p.residual = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    CUtensorMap tmA, tmB, tmBt;
+    if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, pair ? 128 : bn)) ||
+        (rc = encode_u8_2d(&tmBt, W8, N, K, pair ? p.tail_width / 2 : p.tail_width)))
+        return rc;
+    const bool bf = out_dtype == MTMC_OUT_BF16;
+    TimedRegion tr(d);
+    if (pair) rc = bf ? launch_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
+                      : launch_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+    else if (bn == 256) rc = bf ? launch_tiled<EPI_ACT, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                : launch_tiled<EPI_ACT, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    else rc = bf ? launch_tiled<EPI_ACT, 128, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                 : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    tr.stop();
+    return rc;
 }
 
 int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {

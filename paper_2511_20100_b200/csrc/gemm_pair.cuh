@@ -102,8 +102,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = cluster_map_shared(full_bar(s), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2u * cta_bytes);     // both CTAs' bytes
-                    tma_load_2d_pair(a_dst, &tmA, full0, kb * Cfg::BK, m0);
-                    tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kb * Cfg::BK, n_row0);
+                    tma_load_2d_pair(a_dst, &tmA, full0, kb * p.bk_elems, m0);
+                    tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kb * p.bk_elems, n_row0);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -120,7 +120,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int t = pair_id; t < p.num_items && ok; t += num_pairs, ++it) {
                 const int buf = it & 1;
                 const int width = t < p.n_full ? Cfg::OUT_TILE_N : p.tail_width;
-                const uint32_t idesc = umma_idesc_bf16(Cfg::BM, EPI == EPI_SWIGLU ? 2 * width : width);
+                const int mma_n = EPI == EPI_SWIGLU ? 2 * width : width;
+                const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(Cfg::BM, mma_n) : umma_idesc_bf16(Cfg::BM, mma_n);
                 if (!mbar_wait_cluster(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 5u)) { ok = false; break; }
                 acc_ph ^= 1u << buf;
                 tc_fence_after();
@@ -131,9 +132,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                     const uint64_t a_desc = umma_smem_desc_sw128(a_src);
                     const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
+                    // four MMAs per 128-byte row either way: 4 x 16 bf16 or 4 x 32 E4M3, 32 bytes apart
+                    if (p.fp8) {
 #pragma unroll
-                    for (int k = 0; k < Cfg::BK / 16; ++k)
-                        umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k)
+                            umma_fp8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
                     umma_commit_pair(empty_bar(s), 3);           // frees the stage in both CTAs
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }

@@ -34,6 +34,9 @@ struct GemmParams {
     int tail_split;
     int tail_width;       // OUT_TILE_N / tail_split, a multiple of 32
     int act;
+    int fp8;              // 0: bf16 operands (64 per 128-byte row, K = 16 per MMA); 1: E4M3 operands (128 per row, K = 32)
+    int bk_elems;         // elements of K per ring stage: 64 or 128
+    float acc_scale;      // multiplies the accumulator before the bias (product of the FP8 per-tensor scales; 1 otherwise)
     const float* bias;    // [N] or null
     const void* residual; // [M,N] in the output's element type, added after the activation, or null (EPI_ACT)
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
@@ -281,7 +284,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             load_bias_chunk(p.bias, n0, p.N, bv);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(r[j]) + bv[j];
+            for (int j = 0; j < 32; ++j) y[j] = fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]);
             apply_act_chunk(p.act, y);
             if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
@@ -443,10 +446,10 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t b_dst = a_dst + Cfg::A_BYTES;
                     mbar_expect_tx(full_bar(s), tx);
-                    tma_load_2d(a_dst, &tmA, full_bar(s), kb * Cfg::BK, m0);
-                    tma_load_2d(b_dst, mapB, full_bar(s), kb * Cfg::BK, n0);
+                    tma_load_2d(a_dst, &tmA, full_bar(s), kb * p.bk_elems, m0);
+                    tma_load_2d(b_dst, mapB, full_bar(s), kb * p.bk_elems, n0);
                     if (EPI == EPI_SWIGLU)      // the up rows follow the gate rows: one contiguous B operand
-                        tma_load_2d(b_dst + b_rows_bytes, mapB2, full_bar(s), kb * Cfg::BK, n0);
+                        tma_load_2d(b_dst + b_rows_bytes, mapB2, full_bar(s), kb * p.bk_elems, n0);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -463,7 +466,8 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             for (int t = blockIdx.x; t < p.num_items && ok; t += gridDim.x, ++it) {
                 const int buf = it & 1;
                 const int width = t < p.n_full ? Cfg::OUT_TILE_N : p.tail_width;
-                const uint32_t idesc = umma_idesc_bf16(Cfg::BM, EPI == EPI_SWIGLU ? 2 * width : width);
+                const int mma_n = EPI == EPI_SWIGLU ? 2 * width : width;
+                const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(Cfg::BM, mma_n) : umma_idesc_bf16(Cfg::BM, mma_n);
                 if (!mbar_wait(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 1u)) { ok = false; break; }
                 acc_ph ^= 1u << buf;
                 tc_fence_after();
@@ -474,9 +478,16 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                     const uint64_t a_desc = umma_smem_desc_sw128(a_src);
                     const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
+                    // four MMAs per 128-byte row either way: 4 x 16 bf16 or 4 x 32 E4M3, 32 bytes apart
+                    if (p.fp8) {
 #pragma unroll
-                    for (int k = 0; k < Cfg::BK / 16; ++k)
-                        umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < 4; ++k)
+                            umma_fp8(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
                     umma_commit(empty_bar(s));      // frees the stage once these MMAs have read it
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }

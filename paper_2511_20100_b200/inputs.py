@@ -33,6 +33,9 @@ EXTRA_CONFIGS = {
     "X2": dict(op="linear_cross_entropy", M=4096, N=32000, K=4096, seed=3),
     # the MLP down-projection that follows C3, with the skip connection joined to the epilogue
     "X3": dict(op="fused_linear_residual", M=8192, N=4096, K=11008, act="none", out_dtype="bf16", seed=5),
+    # C2 and the SwiGLU-sized GEMM with E4M3 operands (tensor peak is twice the bf16 one)
+    "X4": dict(op="fused_linear_fp8", M=4096, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=1),
+    "X5": dict(op="fused_linear_fp8", M=8192, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=6),
 }
 
 

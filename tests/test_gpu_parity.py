@@ -119,6 +119,43 @@ def test_fused_linear_residual(M, N, K, odt):
     assert torch.equal(Rd, out)
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 16, 16), (17, 8, 128), (100, 72, 144), (129, 257, 272), (300, 520, 400),
+                                   (600, 1000, 656), (1024, 2048, 1024)])
+@pytest.mark.parametrize("act,odt", [("none", "fp32"), ("gelu_tanh", "bf16"), ("relu", "fp32")])
+def test_fused_linear_fp8(M, N, K, act, odt):
+    """E4M3 operands with per-tensor scales on the single-CTA and CTA-pair kernels (K = 32 per MMA)."""
+    fi = inputs.fp8_linear_inputs(M, N, K, seed=7000 + M + N)
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, act, odt, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    want = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, B.ACT[act])
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "fp8 %dx%dx%d %s %s" % (M, N, K, act, odt))
+
+
+def test_fused_linear_fp8_exact_small_integers():
+    # operands in {-2..2} are exact in E4M3 and every fp32 partial sum is exact: the result must be exact too
+    g = torch.Generator().manual_seed(6)
+    X = torch.randint(-2, 3, (200, 256), generator=g).float().to(torch.float8_e4m3fn)
+    W = torch.randint(-2, 3, (264, 256), generator=g).float().to(torch.float8_e4m3fn)
+    out = B.mtmc_fused_linear_fp8(X.cuda(), W.cuda(), None, 1.0, 1.0, "none", "fp32")
+    B.mtmc_check_status()
+    want = ref.fused_linear_fp8(inputs.fp8_bits(X), inputs.fp8_bits(W), None, 1.0, 1.0, ref.ACT_NONE)
+    assert np.array_equal(inputs.to_f64(out), want)
+
+
+def test_fused_linear_fp8_at_full_size_on_sampled_points():
+    fi = inputs.fp8_linear_inputs(4096, 4096, 4096, seed=1)
+    out = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "gelu_tanh", "bf16")
+    B.mtmc_check_status()
+    rows, cols = inputs.sample_points(4096, 4096, 4000, seed=5, tile_m=256, tile_n=256)
+    want = ref.fused_linear_fp8_points(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w,
+                                       ref.ACT_GELU_TANH, rows, cols)
+    got = inputs.to_f64(out[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()])
+    _assert_close(got, want, TOL["bf16"], "fp8 4096^3 sampled")
+    assert bool(torch.isfinite(out.float()).all())
+
+
 def test_fused_linear_exact_integers_and_no_bias():
     # integer-valued operands: every product and fp32 partial sum is exact, so the result must be too
     g = torch.Generator().manual_seed(5)
