@@ -168,10 +168,10 @@ int get_workspace(DeviceState* d, size_t need, void** out) {
 
 size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
-// Scratch of mtmc_linear_lse: one (max, sum-exp) pair per row and column piece; sized for the
-// narrowest tile (128 columns) and the largest tail split (4), whatever the call then picks.
+// Scratch of mtmc_linear_lse: one (max, sum-exp) pair per row and column piece (per epilogue warp share); sized for
+// the narrowest tile (128 columns) and the largest tail split (4), whatever the call then picks.
 size_t lse_workspace_bytes(int64_t M, int64_t N) {
-    return round256(static_cast<size_t>((N + 127) / 128) * 4 * static_cast<size_t>(M) * sizeof(float2));
+    return round256(static_cast<size_t>((N + 127) / 128) * 4 * EPI_HALVES * static_cast<size_t>(M) * sizeof(float2));
 }
 
 int pick_tile_n(int64_t N) {
@@ -274,7 +274,7 @@ int gemm_pairs(DeviceState* d) {
         int n = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2u * static_cast<unsigned>(d->sm_count), 1, 1);
-        cfg.blockDim = dim3(192, 1, 1);
+        cfg.blockDim = dim3(PairCfg<EPI_ACT>::THREADS, 1, 1);
         cfg.dynamicSmemBytes = PairCfg<EPI_ACT>::SMEM_BYTES;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -807,7 +807,7 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
 // the library carries these 8 MiB until the process exits.  In host code the names
 // below are host-side stand-ins, not device addresses; the device addresses are
 // fetched once per device with cudaGetSymbolAddress and cached.
-constexpr size_t NOALLOC_MAX_PARTIALS = 1u << 20;           // float2 entries = 8 MiB
+constexpr size_t NOALLOC_MAX_PARTIALS = (1u << 20) * EPI_HALVES;   // float2 entries = 8 MiB with one epilogue warp per quadrant
 static __device__ __align__(256) float2 g_noalloc_partials[NOALLOC_MAX_PARTIALS];
 static __device__ __align__(256) uint32_t g_noalloc_status[64];
 
@@ -879,7 +879,7 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
     const int bn = pick_tile_n(N);
     GemmParams p{};
     fill_tiling(p, M, N, K, bn, d->sm_count, false);      // whole tiles only: one partial per column tile
-    const size_t need = static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M);
+    const size_t need = EPI_HALVES * static_cast<size_t>(p.n_tiles) * static_cast<size_t>(M);
     if (need > NOALLOC_MAX_PARTIALS)
         return fail(MTMC_ERR_UNSUPPORTED_SHAPE,
                     "mtmc_linear_lse_noalloc: ceil(N/%d) * M = %zu partials exceed the built-in scratch of %zu "

@@ -27,12 +27,12 @@ struct PairCfg {
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     static constexpr int TMEM_COLS = 2 * BN;
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
-    static constexpr int THREADS = 192;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
 };
 
 template <int EPI, bool OUT_BF16>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                  const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmBt,
                  const __grid_constant__ CUtensorMap tmB2t, const GemmParams p) {
@@ -43,7 +43,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
-    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
+    const uint32_t bar_base = epi_stage_base + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
@@ -60,7 +60,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 8); }   // 4 warps x 2 CTAs
+        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 2 * EPI_WARPS); }   // every epilogue warp of both CTAs
         *abort_flag = 0u;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -86,6 +86,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            const uint32_t full0_base = cluster_map_shared(full_bar(0), 0);   // the even CTA's full barriers
             for (int t = pair_id; t < p.num_items && ok; t += num_pairs) {
                 int mb, nb, sub, width;
                 item_coords(p, t, Cfg::OUT_TILE_N, mb, nb, sub, width);
@@ -97,13 +98,16 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n_row0 = nb * Cfg::OUT_TILE_N + sub * width + ((EPI == EPI_SWIGLU) ? 0 : static_cast<int>(rank) * b_rows);
                 const CUtensorMap* mapB = (EPI == EPI_SWIGLU && rank == 1) ? (whole ? &tmB2 : &tmB2t) : (whole ? &tmB : &tmBt);
                 const uint32_t cta_bytes = Cfg::A_BYTES + static_cast<uint32_t>(b_rows) * Cfg::BK * 2;
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                int kx = 0;                                              // K coordinate of the next k-block
+                for (int kb = 0; kb < p.k_blocks; ++kb, kx += p.bk_elems) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 3u)) { ok = false; break; }
+                    // loads first, bookkeeping after: the time from "slot free" to "load issued" is on the ring's
+                    // critical path (a transaction count may run ahead of its expect_tx within a phase)
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
-                    const uint32_t full0 = cluster_map_shared(full_bar(s), 0);
+                    const uint32_t full0 = full0_base + 8u * s;
+                    tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
+                    tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kx, n_row0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2u * cta_bytes);     // both CTAs' bytes
-                    tma_load_2d_pair(a_dst, &tmA, full0, kb * p.bk_elems, m0);
-                    tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kb * p.bk_elems, n_row0);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -151,7 +155,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         __syncwarp();
     } else {
         // ------------------------------------------------------------------ epilogue (both CTAs)
-        const int q = warp & 3;
+        const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;            // which half of the item's columns this warp takes
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
         uint32_t acc_ph = 0;
@@ -167,8 +172,9 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             acc_ph ^= 1u << buf;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::BN);
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, width / 32, width, nb, sub, vec_ok,
-                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
+            const int chunks = width / 32, split_at = EPI_HALVES == 2 ? (chunks + 1) / 2 : chunks;      // two warps per lane quadrant share the columns
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, half ? split_at : 0, half ? chunks : split_at, width, nb, sub, half,
+                                         vec_ok, smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
             // this CTA's half of the accumulator is drained: tell the MMA issuer in the even CTA
             tc_fence_before();
             __syncwarp();

@@ -18,6 +18,15 @@ namespace mtmc {
 enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2, EPI_ROWMAX = 3, EPI_XENT = 4 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
 
+// Epilogue warps per CTA: EPI_HALVES per TMEM lane quadrant, each draining its share of an item's
+// columns.  Measured on C2-C4: eight warps (two per quadrant) shorten the last, exposed epilogue of a
+// CTA but cost as much again in the steady state, so the default is one warp per quadrant.
+#ifndef MTMC_EPI_WARPS
+#define MTMC_EPI_WARPS 4
+#endif
+constexpr int EPI_WARPS = MTMC_EPI_WARPS;
+constexpr int EPI_HALVES = EPI_WARPS / 4;
+static_assert(EPI_WARPS == 4 || EPI_WARPS == 8, "one or two epilogue warps per TMEM lane quadrant");
 // Bytes of warp-private store staging per epilogue warp: one 32-row x 32-column chunk in fp32.
 constexpr int EPI_STAGE_BYTES_PER_WARP = 32 * 32 * 4;
 
@@ -40,7 +49,7 @@ struct GemmParams {
     const float* bias;    // [N] or null
     const void* residual; // [M,N] in the output's element type, added after the activation, or null (EPI_ACT)
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
-    float2* lse_partial;  // [n_tiles * tail_split][M] per row and column piece: (max, sum-exp) for EPI_LSE / EPI_XENT,
+    float2* lse_partial;  // [n_tiles * tail_split * EPI_HALVES][M] per row, column piece and share of the piece: (max, sum-exp) for EPI_LSE / EPI_XENT,
                           // (max, index bits) for EPI_ROWMAX
     const long long* targets;   // [M] target column per row (EPI_XENT)
     float* target_logit;        // [M] logit at the target column, written by the one piece that holds it (EPI_XENT)
@@ -58,8 +67,8 @@ struct TileCfg {
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;   // output columns per tile
     static constexpr int TMEM_COLS = 2 * BN;             // two accumulator buffers
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;  // + alignment slack
-    static constexpr int THREADS = 192;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;  // + alignment slack
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
 };
 
 __device__ __forceinline__ void tile_coords(const GemmParams& p, int idx, int& mb, int& nb) {
@@ -103,6 +112,16 @@ __device__ __forceinline__ float gelu_tanh_f(float z) {
     const float u2 = 1.5957691216057308f * z * fmaf(0.044715f * z, z, 1.0f);   // 2u
     return z * rcp_approx(1.0f + ex2_approx(-1.4426950408889634f * u2));
 }
+// The same through the hardware tanh (one special-function op instead of two).  Its absolute
+// error of about 5e-4 is far inside a bf16 result's rounding, so bf16 outputs use it; fp32
+// outputs keep the exp/reciprocal form above.
+__device__ __forceinline__ float gelu_tanh_fast(float z) {
+    const float u = 0.7978845608028654f * z * fmaf(0.044715f * z, z, 1.0f);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float hz = 0.5f * z;
+    return fmaf(hz, t, hz);
+}
 __device__ __forceinline__ float apply_act(int act, float z) {
     switch (act) {
         case ACT_RELU: return fmaxf(z, 0.0f);
@@ -112,13 +131,14 @@ __device__ __forceinline__ float apply_act(int act, float z) {
     }
 }
 
+template <bool OUT_BF16>
 __device__ __forceinline__ void apply_act_chunk(int act, float (&y)[32]) {
     if (act == ACT_RELU) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) y[j] = fmaxf(y[j], 0.0f);
     } else if (act == ACT_GELU_TANH) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) y[j] = gelu_tanh_f(y[j]);
+        for (int j = 0; j < 32; ++j) y[j] = OUT_BF16 ? gelu_tanh_fast(y[j]) : gelu_tanh_f(y[j]);
     } else if (act == ACT_SILU) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) y[j] = silu_f(y[j]);
@@ -264,35 +284,47 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
 }
 
 // One work item's epilogue for one thread: this thread owns output row `row` (TMEM lane
-// of t_addr) and walks the item's columns [n_tile0, n_tile0 + 32 * chunks) in chunks of 32.
+// of t_addr) and walks chunks [c_begin, c_end) of 32 columns of the item that starts at column n_tile0
+// (the other half of the chunks belongs to the second warp of this lane quadrant).
 //   EPI_ACT    : + bias, activation, store
 //   EPI_SWIGLU : silu(gate) * up with the up columns `width` columns after the gate columns
 //   EPI_LSE    : online (max, sum-exp) in base-2 units, one partial per (row, column piece)
 //   EPI_XENT   : the same, and the logit at the row's target column is set aside
 //   EPI_ROWMAX : running (max, lowest column attaining it), one partial per (row, column piece)
 template <int EPI, bool OUT_BF16>
-__device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int chunks,
-                                              int width, int nb, int sub, bool vec_ok, uint8_t* stage, int lane) {
+__device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int c_begin,
+                                              int c_end, int width, int nb, int sub, int half, bool vec_ok, uint8_t* stage,
+                                              int lane) {
     if (EPI == EPI_ACT) {
+        // Two chunks in flight: while chunk c is being activated and stored, the TMEM load and the
+        // bias fetch of chunk c + 1 are already under way.
+        int live = c_end;                                    // chunks that start inside [0, N)
+        if (n_tile0 + c_end * 32 > p.N) live = (p.N - n_tile0 + 31) / 32;
+        uint32_t r[32];
+        float bv[32];
+        if (c_begin < live) {
+            tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
+            load_bias_chunk(p.bias, n_tile0 + c_begin * 32, p.N, bv);
+        }
 #pragma unroll 1
-        for (int c = 0; c < chunks; ++c) {
+        for (int c = c_begin; c < live; ++c) {
             const int n0 = n_tile0 + c * 32;
-            if (n0 >= p.N) break;            // warp-uniform
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_addr + c * 32, r);
-            float bv[32], y[32];
-            load_bias_chunk(p.bias, n0, p.N, bv);
-            tmem_ld_wait();
+            tmem_ld_wait();                                  // chunk c has landed in r
+            float y[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]);
-            apply_act_chunk(p.act, y);
+            if (c + 1 < live) {                              // r and bv are free again: refill them for chunk c + 1
+                tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
+                load_bias_chunk(p.bias, n0 + 32, p.N, bv);
+            }
+            apply_act_chunk<OUT_BF16>(p.act, y);
             if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
             else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, false);
         }
     } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
-        for (int c = 0; c < chunks; ++c) {
+        for (int c = c_begin; c < c_end; ++c) {
             const int n0 = n_tile0 + c * 32;
             if (n0 >= p.N) break;
             uint32_t g[32], u[32];
@@ -309,7 +341,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         float mx = -INFINITY;
         int arg = 0x7fffffff;
 #pragma unroll 1
-        for (int c = 0; c < chunks; ++c) {
+        for (int c = c_begin; c < c_end; ++c) {
             const int n0 = n_tile0 + c * 32;
             if (n0 >= p.N) break;
             uint32_t r[32];
@@ -324,7 +356,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             }
         }
         if (row < p.M)
-            p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] = make_float2(mx, __int_as_float(arg));
+            p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] = make_float2(mx, __int_as_float(arg));
     } else {
         // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
         constexpr float LOG2E = 1.4426950408889634f;
@@ -334,7 +366,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         bool found = false;
         if (EPI == EPI_XENT && row < p.M) tgt = static_cast<int>(p.targets[row]);
 #pragma unroll 1
-        for (int c = 0; c < chunks; ++c) {
+        for (int c = c_begin; c < c_end; ++c) {
             const int n0 = n_tile0 + c * 32;
             if (n0 >= p.N) break;
             uint32_t r[32];
@@ -374,14 +406,14 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         }
         // a piece that lies wholly past N (only possible in the last column tile) stays neutral
         if (row < p.M)
-            p.lse_partial[static_cast<size_t>(nb * p.tail_split + sub) * p.M + row] =
+            p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] =
                 make_float2(mx * 0.6931471805599453f, sum);
         if (EPI == EPI_XENT && found) p.target_logit[row] = tz;
     }
 }
 
 template <int EPI, int BN, bool OUT_BF16>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
 gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                   const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmBt,
                   const __grid_constant__ CUtensorMap tmB2t, const GemmParams p) {
@@ -392,7 +424,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
-    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
+    const uint32_t bar_base = epi_stage_base + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
@@ -406,7 +438,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), EPI_WARPS); }
         *abort_flag = 0u;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -498,6 +530,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
     } else {
         // ------------------------------------------------------------------ epilogue
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;            // which half of the item's columns this warp takes
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
         uint32_t acc_ph = 0;
@@ -515,8 +548,9 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * BN);
 
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, chunks, width, nb, sub, vec_ok,
-                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
+            const int split_at = EPI_HALVES == 2 ? (chunks + 1) / 2 : chunks;   // the warps of a lane quadrant share the columns
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, half ? split_at : 0, half ? chunks : split_at, width, nb, sub, half,
+                                         vec_ok, smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
             // accumulator buffer drained: hand it back to the MMA warp
             tc_fence_before();
             __syncwarp();
@@ -551,8 +585,8 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
 
 // Merges the (max, sum-exp) partials of each row, in ascending column order, into
 // lse[row] = max + ln(sum).  One warp per row; lanes stride over the column tiles and
-// combine with shuffles.  A whole tile left one partial (piece 0), a tile of the split
-// wave tail left tail_split of them.  With target_logit / loss given it also writes the
+// combine with shuffles.  Every piece left EPI_HALVES partials; a whole tile is one piece, a tile
+// of the split wave tail is tail_split pieces.  With target_logit / loss given it also writes the
 // softmax cross entropy loss[row] = lse[row] - logit[row][target[row]].
 __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
                                  int group_m, int n_full, int tail_split, float* __restrict__ lse,
@@ -564,8 +598,8 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
     float mx = -INFINITY, sum = 0.0f;
     for (int nb = lane; nb < n_tiles; nb += 32) {
         const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
-        for (int sub = 0; sub < pieces; ++sub) {
-            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split + sub) * M + row);
+        for (int sl = 0; sl < EPI_HALVES * pieces; ++sl) {    // ascending columns
+            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
             lse_combine(mx, sum, v.x, v.y);
         }
     }
@@ -594,8 +628,8 @@ __global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, i
     int arg = 0x7fffffff;
     for (int nb = lane; nb < n_tiles; nb += 32) {
         const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
-        for (int sub = 0; sub < pieces; ++sub) {
-            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split + sub) * M + row);
+        for (int sl = 0; sl < EPI_HALVES * pieces; ++sl) {
+            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
             const int a = __float_as_int(v.y);
             if (v.x > mx || (v.x == mx && a < arg)) { mx = v.x; arg = a; }
         }
