@@ -359,7 +359,7 @@ def run_ours(args, rank, world, local_rank):
         if n in per_cfg_eager:
             entry["eager_ms"] = round(per_cfg_eager[n], 5)
             entry["speedup_vs_eager"] = round(per_cfg_eager[n] / ms, 3)
-        if n == "C5":
+        if n == "C5" or (n in inputs.EXTRA_CONFIGS and c["M"] <= 64):      # weight streaming: bound by HBM
             entry["roofline"] = {"bound": "hbm", "achieved": entry["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                  "frac": round(entry["gbs"] / peaks["hbm_gbs"], 4), "of": peaks["source"],
                                  "frac_of_nominal_8000": round(entry["gbs"] / 8000.0, 4)}

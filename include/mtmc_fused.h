@@ -90,8 +90,9 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
  * bits, no infinities; one byte per element, dense row-major); scale_x, scale_w are the
  * per-tensor scales (real value = scale * stored value), passed by value.  Products are
  * exact and accumulate in fp32 on the tensor cores (tcgen05 kind::f8f6f4, K = 32 per MMA,
- * twice the bf16 rate); the epilogue is the one of mtmc_fused_linear.  K % 16 == 0.  All M
- * take the tiled kernels (no weight-streaming variant yet). */
+ * twice the bf16 rate); the epilogue is the one of mtmc_fused_linear.  K % 16 == 0.  As
+ * for bf16, M <= 64 takes the weight-streaming split-K path (half the bytes of bf16
+ * weights), larger M the tiled kernels. */
 int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
                           int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 

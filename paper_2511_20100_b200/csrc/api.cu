@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
@@ -346,10 +347,10 @@ struct SkinnyPlan {
 //    pair reduces through distributed shared memory.
 //  * ticket plan (few rows, or a forced split): 128-row bands, the (band, k-block) list cut
 //    evenly over the SMs or over n_tiles * split_k CTAs; partials and tickets in the workspace.
-SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t M, int64_t N, int64_t K) {
+SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t M, int64_t N, int64_t K, int bk_elems = 64) {
     SkinnyPlan s;
     s.mx = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
-    s.k_blocks = static_cast<int>((K + 63) / 64);
+    s.k_blocks = static_cast<int>((K + bk_elems - 1) / bk_elems);
     s.tile_rows = 128;
     s.n_tiles = static_cast<int>((N + 127) / 128);
     s.pair = 0;
@@ -401,9 +402,9 @@ __global__ void timeout_probe_kernel(uint32_t* status) {
     }
 }
 
-template <bool OUT_BF16, bool PAIR, int MX>
+template <bool OUT_BF16, bool PAIR, int MX, bool FP8>
 int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap& tmX, const SkinnyParams& p) {
-    auto kern = skinny_splitk_kernel<OUT_BF16, PAIR, MX>;
+    auto kern = skinny_splitk_kernel<OUT_BF16, PAIR, MX, FP8>;
     if (int rc = ensure_smem_attr(kern, SkinnyCfg<MX>::SMEM_BYTES)) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(s.grid), 1, 1);
@@ -450,9 +451,10 @@ int skinny_pairs(DeviceState* d) {
 }
 
 int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K,
-               int act, int out_dtype, void* out) {
-    SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
+               int act, int out_dtype, void* out, bool fp8 = false, float acc_scale = 1.0f) {
+    SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, fp8 ? 128 : 64);
     SkinnyParams p;
+    p.acc_scale = acc_scale;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
     p.tile_rows = s.tile_rows; p.num_stages = s.stages;
@@ -475,18 +477,24 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
         }
     }
     CUtensorMap tmW, tmX;
-    int rc = encode_bf16_2d(&tmW, W, N, K, s.tile_rows);
+    int rc = fp8 ? encode_u8_2d(&tmW, W, N, K, s.tile_rows) : encode_bf16_2d(&tmW, W, N, K, s.tile_rows);
     if (rc) return rc;
-    rc = encode_bf16_2d(&tmX, X, M, K, s.mx);
+    rc = fp8 ? encode_u8_2d(&tmX, X, M, K, s.mx) : encode_bf16_2d(&tmX, X, M, K, s.mx);
     if (rc) return rc;
     TimedRegion tr(d);
     const bool bf = out_dtype == MTMC_OUT_BF16;
-#define MTMC_SKINNY_DISPATCH(MXV)                                                                         \
-    rc = bf ? (s.pair ? launch_skinny<true, true, MXV>(s, tmW, tmX, p) : launch_skinny<true, false, MXV>(s, tmW, tmX, p)) \
-            : (s.pair ? launch_skinny<false, true, MXV>(s, tmW, tmX, p) : launch_skinny<false, false, MXV>(s, tmW, tmX, p))
-    if (s.mx == 16) { MTMC_SKINNY_DISPATCH(16); }
-    else if (s.mx == 32) { MTMC_SKINNY_DISPATCH(32); }
-    else { MTMC_SKINNY_DISPATCH(64); }
+#define MTMC_SKINNY_DISPATCH(MXV, F8)                                                                         \
+    rc = bf ? (s.pair ? launch_skinny<true, true, MXV, F8>(s, tmW, tmX, p) : launch_skinny<true, false, MXV, F8>(s, tmW, tmX, p)) \
+            : (s.pair ? launch_skinny<false, true, MXV, F8>(s, tmW, tmX, p) : launch_skinny<false, false, MXV, F8>(s, tmW, tmX, p))
+    if (fp8) {
+        if (s.mx == 16) { MTMC_SKINNY_DISPATCH(16, true); }
+        else if (s.mx == 32) { MTMC_SKINNY_DISPATCH(32, true); }
+        else { MTMC_SKINNY_DISPATCH(64, true); }
+    } else {
+        if (s.mx == 16) { MTMC_SKINNY_DISPATCH(16, false); }
+        else if (s.mx == 32) { MTMC_SKINNY_DISPATCH(32, false); }
+        else { MTMC_SKINNY_DISPATCH(64, false); }
+    }
 #undef MTMC_SKINNY_DISPATCH
     tr.stop();
     return rc;
@@ -651,8 +659,10 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
             if (!use_skinny(M, N)) return 0;
             DeviceState* d = nullptr;
             if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
+            // the larger of the bf16 and the E4M3 plan: mtmc_fused_linear_fp8 shares this op id
             SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
-            return s.ticket_bytes + s.partial_bytes;
+            SkinnyPlan s8 = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, 128);
+            return std::max(s.ticket_bytes + s.partial_bytes, s8.ticket_bytes + s8.partial_bytes);
         }
         case MTMC_OP_SWIGLU: return 0;
         case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N);
@@ -711,6 +721,7 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
+    if (use_skinny(M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
     const bool pair = use_pair(d, M, N);
     const int bn = pair ? 256 : pick_tile_n(N);
     GemmParams p{};

@@ -39,6 +39,7 @@ struct SkinnyParams {
     long long total_units;   // n_tiles * k_blocks
     int max_slots;           // partial slots per band
     int act;
+    float acc_scale;         // multiplies the accumulator before the bias (FP8 per-tensor scales; 1 otherwise)
     const float* bias;
     const void* residual;    // [M,N] in the output's element type, added after the activation, or null
     void* out;
@@ -108,11 +109,14 @@ __device__ __forceinline__ void skinny_store(const SkinnyParams& p, int m, int n
     }
 }
 
-template <bool OUT_BF16, bool PAIR, int MX>
+// FP8: E4M3 operands (128 per 128-byte row, K = 32 per MMA) instead of bf16 (64 per row, K = 16);
+// the bytes per stage, the ring and the four MMAs per row are the same for both.
+template <bool OUT_BF16, bool PAIR, int MX, bool FP8 = false>
 __global__ void __launch_bounds__(192, 1)
 skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmX,
                      const SkinnyParams p) {
     using Cfg = SkinnyCfg<MX>;
+    constexpr int BKE = FP8 ? 128 : 64;                      // elements of K per k-block
     constexpr int MAXS = Cfg::MAX_STAGES;
     constexpr int KPS = Cfg::KB_PER_STAGE;
     const int STAGES = p.num_stages;
@@ -214,8 +218,8 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     const uint32_t dst = base + s * stage_bytes;
                     mbar_expect_tx(full_bar(s), nkb * (w_bytes + Cfg::X_BYTES));
                     for (int i = 0; i < nkb; ++i) {
-                        tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * Cfg::BK, tile * R, pol_stream);
-                        tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * Cfg::BK, 0, pol_keep);
+                        tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * BKE, tile * R, pol_stream);
+                        tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * BKE, 0, pol_keep);
                     }
                     kb += nkb;
                     seg -= nkb;
@@ -230,7 +234,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         // ------------------------------------------------------------------ MMA issuer
         const uint32_t tmem_base = *tmem_slot;
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(Cfg::LANES, Cfg::MX);
+            constexpr uint32_t idesc = FP8 ? umma_idesc_e4m3(Cfg::LANES, Cfg::MX) : umma_idesc_bf16(Cfg::LANES, Cfg::MX);
             int s = 0;
             uint32_t ph = 0, acc_ph = 0;                         // bit b of acc_ph: phase of accumulator set b
             int kb = first_kb, left = n_units, seg_idx = 0;
@@ -253,9 +257,11 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                         const uint64_t a_desc = umma_smem_desc_sw128(src + i * w_bytes);
                         const uint64_t b_desc = umma_smem_desc_sw128(src + x_off + i * Cfg::X_BYTES);
 #pragma unroll
-                        for (int k = 0; k < Cfg::BK / 16; ++k, ++step)
-                            umma_bf16(d_tmem + (step % Cfg::WAYS) * Cfg::MX, a_desc + 2u * k, b_desc + 2u * k, idesc,
-                                      step >= Cfg::WAYS ? 1u : 0u);
+                        for (int k = 0; k < Cfg::BK / 16; ++k, ++step) {      // four MMAs per 128-byte row either way
+                            const uint32_t d = d_tmem + (step % Cfg::WAYS) * Cfg::MX;
+                            if constexpr (FP8) umma_fp8(d, a_desc + 2u * k, b_desc + 2u * k, idesc, step >= Cfg::WAYS ? 1u : 0u);
+                            else umma_bf16(d, a_desc + 2u * k, b_desc + 2u * k, idesc, step >= Cfg::WAYS ? 1u : 0u);
+                        }
                     }
                     umma_commit(empty_bar(s));
                     seg -= nkb;
@@ -308,7 +314,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     if (row_ok) {
 #pragma unroll
                         for (int m = 0; m < MX; ++m) {
-                            if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
+                            if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn));
                         }
                     }
                 }
@@ -383,7 +389,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             if (finalize && row_ok) {
 #pragma unroll
                 for (int m = 0; m < MX; ++m) {
-                    if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, acc[m] + bn));
+                    if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn));
                 }
             }
             ++tile;

@@ -36,6 +36,8 @@ EXTRA_CONFIGS = {
     # C2 and the SwiGLU-sized GEMM with E4M3 operands (tensor peak is twice the bf16 one)
     "X4": dict(op="fused_linear_fp8", M=4096, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=1),
     "X5": dict(op="fused_linear_fp8", M=8192, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=6),
+    # the decode GEMM of C5 with E4M3 weights and activations: half the bytes to stream
+    "X6": dict(op="fused_linear_fp8", M=16, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=4),
 }
 
 

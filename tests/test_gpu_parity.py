@@ -133,6 +133,25 @@ def test_fused_linear_fp8(M, N, K, act, odt):
     _assert_close(inputs.to_f64(out), want, TOL[odt], "fp8 %dx%dx%d %s %s" % (M, N, K, act, odt))
 
 
+@pytest.mark.parametrize("M,N,K,split_k", [(1, 4096, 4096, 0), (8, 8192, 2064, 0), (16, 4736, 1024, 0), (17, 5000, 4112, 0),
+                                           (33, 9472, 528, 0), (64, 16384, 4096, 0), (4, 1024, 4096, 4), (48, 640, 2192, 3),
+                                           (2, 300, 16, 0), (64, 96, 8192, 0)])
+@pytest.mark.parametrize("act,odt", [("none", "fp32"), ("silu", "bf16")])
+def test_fused_linear_fp8_skinny(M, N, K, split_k, act, odt):
+    """E4M3 weights streamed once on the split-K path (M <= 64): CTA-pair and ticket plans, ragged K and N."""
+    fi = inputs.fp8_linear_inputs(M, N, K, seed=7100 + M + N)
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    B.mtmc_set_tuning(split_k=split_k)
+    try:
+        B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, act, odt, out=out)
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    assert _canaries_intact(buf, M * N)
+    want = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, B.ACT[act])
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "fp8 skinny %dx%dx%d %s %s" % (M, N, K, act, odt))
+
+
 def test_fused_linear_fp8_exact_small_integers():
     # operands in {-2..2} are exact in E4M3 and every fp32 partial sum is exact: the result must be exact too
     g = torch.Generator().manual_seed(6)
