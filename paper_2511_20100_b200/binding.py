@@ -27,7 +27,7 @@ EXPORTS = [
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_set_tuning", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -71,6 +71,7 @@ def load() -> ctypes.CDLL:
     L.mtmc_set_timing.argtypes = [ci]
     L.mtmc_last_kernel_ms.restype = ctypes.c_float
     L.mtmc_set_tuning.argtypes = [ci, ci, ci]
+    L.mtmc_set_static_weights.argtypes = [ci]
     _lib = L
     return L
 
@@ -300,6 +301,11 @@ def mtmc_last_kernel_ms() -> float:
 
 def mtmc_set_tuning(split_k: int = 0, tile_n: int = 0, cta_pair: int = 0) -> None:
     _check(load().mtmc_set_tuning(int(split_k), int(tile_n), int(cta_pair)))
+
+
+def mtmc_set_static_weights(enabled: bool = True) -> None:
+    """Promise that no work in flight writes W: the weight-streaming path may start its W loads early."""
+    _check(load().mtmc_set_static_weights(1 if enabled else 0))
 
 
 def mtmc_version() -> int:

@@ -52,6 +52,7 @@ thread_local size_t t_user_ws_bytes = 0;
 thread_local int t_split_k = 0;
 thread_local int t_tile_n = 0;
 thread_local int t_cta_pair = 0;   // 0 automatic, 1 force CTA pairs, -1 force single CTAs
+thread_local int t_static_weights = 0;   // caller's promise that no work in flight writes W (see mtmc_set_static_weights)
 thread_local int t_timing = 0;
 thread_local char t_error[512] = "";
 
@@ -455,6 +456,7 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
     SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, fp8 ? 128 : 64);
     SkinnyParams p;
     p.acc_scale = acc_scale;
+    p.early_w = t_static_weights;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
     p.tile_rows = s.tile_rows; p.num_stages = s.stages;
@@ -636,6 +638,8 @@ int mtmc_set_tuning(int split_k, int tile_n, int cta_pair) {
     t_cta_pair = cta_pair > 0 ? 1 : (cta_pair < 0 ? -1 : 0);
     return MTMC_OK;
 }
+
+int mtmc_set_static_weights(int enabled) { t_static_weights = enabled ? 1 : 0; return MTMC_OK; }
 
 int mtmc_set_timing(int enabled) { t_timing = enabled ? 1 : 0; return MTMC_OK; }
 

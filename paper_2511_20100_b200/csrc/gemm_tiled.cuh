@@ -591,6 +591,7 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
 __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
                                  int group_m, int n_full, int tail_split, float* __restrict__ lse,
                                  const float* __restrict__ target_logit, float* __restrict__ loss) {
+    pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -620,6 +621,7 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
 __global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
                                     int group_m, int n_full, int tail_split, float* __restrict__ max_out,
                                     int* __restrict__ argmax_out) {
+    pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;

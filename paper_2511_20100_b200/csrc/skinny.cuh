@@ -40,6 +40,8 @@ struct SkinnyParams {
     int max_slots;           // partial slots per band
     int act;
     float acc_scale;         // multiplies the accumulator before the bias (FP8 per-tensor scales; 1 otherwise)
+    int early_w;             // 1: W is not written by any work still in flight, so its first ring of loads may
+                             // go out before the wait on the preceding kernel (X, bias and outputs still wait)
     const float* bias;
     const void* residual;    // [M,N] in the output's element type, added after the activation, or null
     void* out;
@@ -61,15 +63,22 @@ struct SkinnyCfg {
     static constexpr int TMEM_COLS = 2 * ACC_COLS;        // two sets: MMA on one, epilogue on the other
     static constexpr int NUM_BARRIERS = 2 * MAX_STAGES + 5;   // ring, accumulator sets, pair reduction
     static constexpr int REDUCE_BYTES = MX * LANES * 4;       // the peer CTA's partial (PAIR mode)
+    // One CTA per SM with the whole shared memory: splitting an SM between the running kernel and the next
+    // launch (two CTAs of 111 KiB, dependents released after the last load) was measured slower, 28.7-29.2 us
+    // against 26.8-27.4 us at 16 x 8192 x 8192, because the ring is then only three stages deep.
     static constexpr int RING_BYTES = 208 * 1024 - REDUCE_BYTES;   // shared memory given to the TMA ring
     static constexpr int SMEM_BYTES = RING_BYTES + REDUCE_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int stage_bytes(int tile_rows) { return KB_PER_STAGE * (tile_rows * BK * 2 + X_BYTES); }
-    // The MMA always reads a 128-row (16 KiB) A tile, also when the band is shorter, so the
-    // last W tile of the last stage must start at least 16 KiB before the end of the ring.
+    // The MMA always reads a 128-row (16 KiB) A tile, also when the band is shorter, so the last W
+    // k-block of the last stage must start at least 16 KiB before the end of the ring.
+    static constexpr int last_w_end(int tile_rows, int stages) {
+        return (stages - 1) * stage_bytes(tile_rows) + (KB_PER_STAGE - 1) * tile_rows * BK * 2 + LANES * BK * 2;
+    }
     static constexpr int stages_for(int tile_rows) {
-        return (RING_BYTES - 2 * LANES * BK * 2) / stage_bytes(tile_rows) + 1 < MAX_STAGES
-                   ? (RING_BYTES - 2 * LANES * BK * 2) / stage_bytes(tile_rows) + 1
-                   : MAX_STAGES;
+        int s = RING_BYTES / stage_bytes(tile_rows);
+        if (s > MAX_STAGES) s = MAX_STAGES;
+        while (s > 1 && last_w_end(tile_rows, s) > RING_BYTES) --s;
+        return s;
     }
 };
 
@@ -168,6 +177,45 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         n_units = static_cast<int>(u_end - u_begin);
     }
 
+    // The TMA producer's walk over this CTA's k-blocks (one lane of warp 0 runs it).
+    //   early = true : only the first ring-full of stages, only their W k-blocks (weights nobody is writing),
+    //                  before the wait on the preceding kernel; each stage's full byte count is announced here.
+    //   early = false: the whole walk; stages that the early pass already started get only their X k-blocks.
+    auto produce = [&](bool early) {
+        const uint64_t pol_stream = l2_policy_evict_first();   // W is read exactly once
+        const uint64_t pol_keep = l2_policy_evict_last();      // X is re-read by every CTA
+        const int pre = p.early_w ? STAGES : 0;                // stages begun by the early pass
+        int s = 0, idx = 0;
+        uint32_t ph = 0;
+        int tile = first_tile, kb = first_kb, left = n_units;
+        while (left > 0) {
+            int seg = min(KB - kb, left);                      // k-blocks of this band still to load
+            left -= seg;
+            while (seg > 0) {
+                if (early && idx >= pre) return;
+                const int nkb = min(KPS, seg);
+                const bool begun = !early && idx < pre;        // W already on its way, bytes already announced
+                const uint32_t dst = base + s * stage_bytes;
+                if (!begun) {
+                    if (!early && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 2u)) return;
+                    mbar_expect_tx(full_bar(s), nkb * (w_bytes + Cfg::X_BYTES));
+                    for (int i = 0; i < nkb; ++i)
+                        tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * BKE, tile * R, pol_stream);
+                }
+                if (!early) {
+                    for (int i = 0; i < nkb; ++i)
+                        tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * BKE, 0, pol_keep);
+                }
+                kb += nkb;
+                seg -= nkb;
+                ++idx;
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            ++tile;
+            kb = 0;
+        }
+    };
+
     // Set-up.  Warp 0 initialises the barriers and goes straight on to issue loads; it only
     // arrives on the set-up barrier.  The other warps wait there for the barrier
     // initialisation and for warp 1's TMEM allocation.
@@ -186,8 +234,9 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         __syncwarp();
         asm volatile("bar.arrive 2, 192;" ::: "memory");
         if (PAIR) cluster_arrive();          // publishes red_bar's initialisation to the peer; waited for at the end
+        if (lane == 0 && p.early_w) produce(true);
         pdl_launch_dependents();
-        pdl_wait();                          // before the first load from global memory
+        pdl_wait();                          // before the first load of anything a preceding kernel may have written
     } else {
         if (warp == 1) {
             tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
@@ -203,32 +252,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
-            const uint64_t pol_stream = l2_policy_evict_first();   // W is read exactly once
-            const uint64_t pol_keep = l2_policy_evict_last();      // X is re-read by every CTA
-            int s = 0;
-            uint32_t ph = 0;
-            int tile = first_tile, kb = first_kb, left = n_units;
-            while (left > 0) {
-                int seg = min(KB - kb, left);                      // k-blocks of this band still to load
-                left -= seg;
-                while (seg > 0) {
-                    const int nkb = min(KPS, seg);
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 2u)) { left = 0; break; }
-                    const uint32_t dst = base + s * stage_bytes;
-                    mbar_expect_tx(full_bar(s), nkb * (w_bytes + Cfg::X_BYTES));
-                    for (int i = 0; i < nkb; ++i) {
-                        tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * BKE, tile * R, pol_stream);
-                        tma_load_2d_hint(dst + x_off + i * Cfg::X_BYTES, &tmX, full_bar(s), (kb + i) * BKE, 0, pol_keep);
-                    }
-                    kb += nkb;
-                    seg -= nkb;
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
-                }
-                ++tile;
-                kb = 0;
-            }
-        }
+        if (lane == 0) produce(false);
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer

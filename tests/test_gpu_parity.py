@@ -339,6 +339,31 @@ def test_skinny_small(M, N, K, odt):
     _assert_close(inputs.to_f64(out), want, TOL[odt], "skinny %dx%dx%d %s" % (M, N, K, odt))
 
 
+@pytest.mark.parametrize("M,N,K,split_k", [(16, 8192, 8192, 0), (1, 4096, 1024, 0), (64, 9472, 136, 0), (5, 300, 2048, 0),
+                                           (16, 512, 1024, 4), (33, 2400, 1096, 0), (7, 128, 64, 0)])
+def test_skinny_static_weights_same_bits(M, N, K, split_k):
+    """With the static-weights promise the first ring of W loads goes out before the wait on the preceding kernel:
+    same bits as without it, launch after launch (each launch follows one of this library's own kernels)."""
+    li = inputs.linear_inputs(M, N, K, seed=4100 + M + N)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    B.mtmc_set_tuning(split_k=split_k)
+    try:
+        plain = B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32")
+        B.mtmc_set_static_weights(True)
+        outs = [B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32") for _ in range(12)]
+        lse = B.mtmc_linear_lse(Xd, Wd, bd)                      # a merge kernel right before the next skinny launch
+        after_merge = B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_static_weights(False)
+        B.mtmc_set_tuning()
+    for o in outs + [after_merge]:
+        assert torch.equal(o, plain)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(plain), want, TOL["fp32"], "static weights %dx%dx%d" % (M, N, K))
+    assert torch.isfinite(lse).all()
+
+
 @pytest.mark.parametrize("M", [24, 64])
 @pytest.mark.parametrize("split_k", [1, 3])
 def test_skinny_decode_batch_forced_split(M, split_k):
