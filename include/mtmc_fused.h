@@ -218,8 +218,9 @@ float mtmc_last_kernel_ms(void);
 
 /* Tuning hooks (0 = automatic).  They select among kernels of this library only; results
  * stay within tolerance of each other.  Thread-local.
- *   split_k  : > 0 forces the ticketed split-K plan of the skinny path with this many K
- *              splits per 128-row band of W
+ *   split_k  : > 0 forces the ticketed split-K plan of the skinny path (M <= 64) with this
+ *              many K splits per 128-row band of W; for larger M it caps the cluster
+ *              size of the cluster split-K kernel (1 = never use that kernel)
  *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
  *   cta_pair : > 0 forces the CTA-pair (cta_group::2, 256-row tiles) tiled kernel,
  *              < 0 forbids it; automatic = pairs when M >= 512 and N >= 256          */

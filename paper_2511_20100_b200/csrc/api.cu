@@ -16,6 +16,7 @@
 #include <mutex>
 
 #include "gemm_pair.cuh"
+#include "gemm_ksplit.cuh"
 #include "skinny.cuh"
 
 namespace {
@@ -40,6 +41,7 @@ struct DeviceState {
     bool timed = false;
     int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
     int max_gemm_pairs = -1;         // the same for the CTA-pair tiled kernel
+    int max_ksplit[3] = {-1, -1, -1};   // co-resident clusters of two / four / eight CTAs of the cluster split-K kernel
 };
 
 std::mutex g_mutex;
@@ -295,6 +297,86 @@ int gemm_pairs(DeviceState* d) {
     return d->max_gemm_pairs;
 }
 
+template <int EPI, bool OUT_BF16, int KS>
+int launch_ksplit_ks(int tiles, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
+    using Cfg = KSplitCfg<EPI, KS>;
+    auto kern = gemm_ksplit_kernel<EPI, OUT_BF16, KS>;
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles * KS), 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = KS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1 + pdl_attribute(attr + 1);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+template <int EPI, bool OUT_BF16>
+int launch_ksplit(int ks, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
+    if constexpr (EPI != EPI_SWIGLU) {
+        if (ks == 8) return launch_ksplit_ks<EPI, OUT_BF16, 8>(p.num_tiles, tmA, tmB, tmB2, p);
+    }
+    return ks == 4 ? launch_ksplit_ks<EPI, OUT_BF16, 4>(p.num_tiles, tmA, tmB, tmB2, p)
+                   : launch_ksplit_ks<EPI, OUT_BF16, 2>(p.num_tiles, tmA, tmB, tmB2, p);
+}
+
+// How many clusters of `ks` CTAs of the cluster split-K kernel the device holds at once (0: none).
+template <int KS>
+int ksplit_clusters_ks(DeviceState* d) {
+    int& cached = d->max_ksplit[KS == 8 ? 2 : (KS == 4 ? 1 : 0)];
+    if (cached < 0) {
+        using Cfg = KSplitCfg<EPI_ACT, KS>;
+        auto kern = gemm_ksplit_kernel<EPI_ACT, true, KS>;
+        int n = 0;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(KS * d->sm_count), 1, 1);
+        cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+        cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = KS;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess ||
+            cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) {
+            (void)cudaGetLastError();
+            n = 0;
+        }
+        cached = n;
+    }
+    return cached;
+}
+
+// Cluster split-K (2, 4 or 8 CTAs per 128 x 256 tile) for problems of at most half a wave of tiles whose K is
+// long enough to cut (at least 8 k-blocks per CTA): the widest cluster whose tiles all run at once.  0: not this path.
+// The tuning hook split_k = 1 turns it off; 2 or 4 cap the cluster size.  SwiGLU tiles have four output chunks,
+// so their clusters stop at four.
+int pick_ksplit(DeviceState* d, int64_t M, int64_t N, int64_t K, int out_tile_n, bool fp8) {
+    if (EPI_HALVES != 1 || t_split_k == 1 || t_tile_n != 0 || t_cta_pair > 0) return 0;
+    if (N <= 128) return 0;                                   // those take 128-column tiles
+    const int64_t tiles = ((M + 127) / 128) * ((N + out_tile_n - 1) / out_tile_n);
+    const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
+    const int cap = t_split_k > 0 ? t_split_k : 8;
+    if (tiles > d->sm_count / 2) return 0;
+    if (cap >= 8 && out_tile_n == 256 && k_blocks >= 64 && tiles <= ksplit_clusters_ks<8>(d) && tiles * 8 <= d->sm_count) return 8;
+    if (cap >= 4 && k_blocks >= 32 && tiles <= ksplit_clusters_ks<4>(d) && tiles * 4 <= d->sm_count) return 4;
+    if (k_blocks >= 16 && tiles <= ksplit_clusters_ks<2>(d)) return 2;
+    return 0;
+}
+
+// The schedule of a cluster split-K launch: one whole tile per cluster; row-reduction partials are laid out as
+// for a tile cut into `ks` column pieces (each CTA finishes its own columns).
+void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int ks, bool fp8);
+
 // Large problems go to CTA pairs (256-row tiles); small ones keep single-CTA 128-row tiles.
 bool use_pair(DeviceState* d, int64_t M, int64_t N) {
     if (t_cta_pair < 0 || t_tile_n == 128 || gemm_pairs(d) <= 0) return false;
@@ -330,6 +412,12 @@ void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
             p.num_items = p.n_full + r * s;
         }
     }
+}
+
+void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int ks, bool fp8) {
+    fill_tiling(p, M, N, K, out_tile_n, 1, false, 128, fp8);
+    p.n_full = 0;
+    p.tail_split = ks;
 }
 
 int skinny_cta_of_unit_host(long long u, long long total, int grid) {
@@ -525,10 +613,12 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    const bool pair = use_pair(d, M, N);
-    const int bn = pair ? 256 : pick_tile_n(N);
+    const int ks = pick_ksplit(d, M, N, K, 256, false);
+    const bool pair = !ks && use_pair(d, M, N);
+    const int bn = (pair || ks) ? 256 : pick_tile_n(N);
     GemmParams p{};
-    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+    if (ks) fill_ksplit(p, M, N, K, 256, ks, false);
+    else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
     else fill_tiling(p, M, N, K, bn, d->sm_count, true);
     const size_t partial_bytes = lse_workspace_bytes(M, N);
     const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
@@ -545,7 +635,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
         (rc = encode_bf16_2d(&tmBt, W, N, K, pair ? p.tail_width / 2 : p.tail_width)))
         return rc;
     TimedRegion tr(d);
-    if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+    if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
+    else if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
     else rc = bn == 256 ? launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
                         : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
     tr.stop();
@@ -576,6 +667,17 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     if (rc) return rc;
     if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out);
 
+    if (const int ks = pick_ksplit(d, M, N, K, 256, false)) {
+        GemmParams p{};
+        fill_ksplit(p, M, N, K, 256, ks, false);
+        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 256))) return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
+        tr.stop();
+        return rc;
+    }
     if (use_pair(d, M, N)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
@@ -726,6 +828,18 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     int rc = get_device(&d);
     if (rc) return rc;
     if (use_skinny(M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
+    if (const int ks = pick_ksplit(d, M, N, K, 256, true)) {
+        GemmParams p{};
+        fill_ksplit(p, M, N, K, 256, ks, true);
+        p.acc_scale = scale_x * scale_w;
+        p.act = act; p.bias = b; p.residual = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB;
+        if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, 256))) return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
+        tr.stop();
+        return rc;
+    }
     const bool pair = use_pair(d, M, N);
     const int bn = pair ? 256 : pick_tile_n(N);
     GemmParams p{};
@@ -757,6 +871,19 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
+    if (const int ks = pick_ksplit(d, M, N, K, 128, false)) {
+        GemmParams p{};
+        fill_ksplit(p, M, N, K, 128, ks, false);
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmG, tmU;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmG, Wg, N, K, 128)) ||
+            (rc = encode_bf16_2d(&tmU, Wu, N, K, 128)))
+            return rc;
+        TimedRegion tr(d);
+        rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
+        tr.stop();
+        return rc;
+    }
     if (use_pair(d, M, N)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 128, gemm_pairs(d), true, 256);

@@ -1,0 +1,251 @@
+// Split-K over a thread-block cluster, for problems with far fewer output tiles than SMs
+// (decode / small-prefill batches of 65 ... a few hundred rows against a large weight matrix).
+//
+// There the tiled kernels leave most SMs idle and every busy CTA walks the whole K range, so
+// the time is one CTA's k-walk.  Here a cluster of KS CTAs (2, 4 or 8) owns one 128 x 256 tile:
+// CTA r multiplies k-blocks [r KB/KS, (r+1) KB/KS) into its own TMEM accumulator (the same
+// TMA ring and tcgen05 mainloop as the tiled kernel), then the cluster does a reduce-scatter
+// through distributed shared memory: CTA r receives, from every peer, the peer's partial of
+// the 256 / KS accumulator columns that r will finish, adds the KS partials in rank order
+// (so the bits do not depend on timing), writes the sum back to its TMEM and runs the usual
+// epilogue on its columns.  The partials never touch L2 or HBM and the epilogue is shared
+// out over the cluster as well.
+//
+// The receive buffer is the CTA's TMA ring, idle once its last MMA has completed; a CTA tells
+// its peers so (remote arrive on their `ready` barrier) and sends only when every peer is
+// ready.  All waits are on CTAs of the same cluster, which the hardware schedules together,
+// and all are bounded.
+#pragma once
+#include "gemm_tiled.cuh"
+
+namespace mtmc {
+
+template <int EPI, int KS>
+struct KSplitCfg {
+    static_assert(KS == 2 || KS == 4 || KS == 8, "cluster of two, four or eight CTAs (eight: not for SwiGLU, whose tile has four output chunks)");
+    using Tile = TileCfg<EPI, 256>;
+    static constexpr int BN = 256;
+    static constexpr int STAGES = Tile::STAGES;
+    static constexpr int STAGE_BYTES = Tile::STAGE_BYTES;
+    static constexpr int OUT_TILE_N = Tile::OUT_TILE_N;
+    static constexpr int AC = BN / 32;                    // 32-column chunks of the accumulator
+    static constexpr int OC = OUT_TILE_N / 32;            // 32-column chunks of the output tile (SwiGLU: half of AC)
+    static constexpr int OWN_OC = OC / KS;                // output chunks this CTA finishes
+    static constexpr int OWN_AC = AC / KS;                // accumulator chunks it receives from each peer
+    static constexpr int BLOCK_BYTES = 32 * 32 * 4;       // one chunk of one lane quadrant: 32 rows x 128 bytes
+    static constexpr int RECV_BYTES = (KS - 1) * OWN_AC * 4 * BLOCK_BYTES;
+    static_assert(RECV_BYTES <= STAGES * STAGE_BYTES, "the ring holds the peers' partials");
+    static_assert(OWN_OC >= 1, "at least one output chunk per CTA");
+    static constexpr int NUM_BARRIERS = 2 * STAGES + 3;   // ring, accumulator full, ready, received
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int THREADS = 192;                   // producer, MMA issuer, four epilogue warps
+    static constexpr int TMEM_COLS = BN;                  // one accumulator: a CTA has exactly one work item
+};
+
+__device__ __forceinline__ void st_shared_cluster_v4(uint32_t caddr, float a, float b, float c, float d) {
+    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+template <int EPI, bool OUT_BF16, int KS>
+__global__ void __launch_bounds__(192, 1)
+gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                   const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
+    using Cfg = KSplitCfg<EPI, KS>;
+    using Tile = typename Cfg::Tile;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    const uint32_t accf_bar = bar_base + 8u * (2 * STAGES);
+    const uint32_t ready_bar = bar_base + 8u * (2 * STAGES + 1);      // peers that are ready to receive (their ring is idle)
+    const uint32_t recv_bar = bar_base + 8u * (2 * STAGES + 2);       // peers' epilogue warps that have delivered to me
+    uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int tile = static_cast<int>(blockIdx.x) / KS;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(accf_bar, 1);
+        mbar_init(ready_bar, KS - 1);             // one arrival per peer CTA
+        mbar_init(recv_bar, (KS - 1) * 4);        // one per epilogue warp of every peer
+        *abort_flag = 0u;
+        fence_barrier_init();
+        fence_proxy_async_smem();
+        tma_prefetch_desc(&tmA);
+        tma_prefetch_desc(&tmB);
+        if (EPI == EPI_SWIGLU) tma_prefetch_desc(&tmB2);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();        // every CTA's barriers exist before any peer arrives on them
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_launch_dependents();
+    pdl_wait();
+
+    int mb, nb;
+    tile_coords(p, tile, mb, nb);
+    const int kb0 = static_cast<int>(static_cast<long long>(rank) * p.k_blocks / KS);
+    const int kb1 = static_cast<int>(static_cast<long long>(rank + 1) * p.k_blocks / KS);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            const int m0 = mb * 128;
+            const int n0 = nb * Cfg::OUT_TILE_N;
+            constexpr uint32_t b_rows_bytes = static_cast<uint32_t>(Cfg::OUT_TILE_N) * Tile::BK * 2;
+            constexpr uint32_t tx = Tile::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 7u)) break;
+                const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
+                const uint32_t b_dst = a_dst + Tile::A_BYTES;
+                mbar_expect_tx(full_bar(s), tx);
+                tma_load_2d(a_dst, &tmA, full_bar(s), kb * p.bk_elems, m0);
+                tma_load_2d(b_dst, &tmB, full_bar(s), kb * p.bk_elems, n0);
+                if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), kb * p.bk_elems, n0);
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(128, Cfg::BN) : umma_idesc_bf16(128, Cfg::BN);
+            for (int kb = kb0; kb < kb1; ++kb) {
+                if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 7u)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
+                const uint64_t a_desc = umma_smem_desc_sw128(a_src);
+                const uint64_t b_desc = umma_smem_desc_sw128(a_src + Tile::A_BYTES);
+                if (p.fp8) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_fp8(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_bf16(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+                }
+                umma_commit(empty_bar(s));
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            }
+            if (ok) umma_commit(accf_bar);           // my part of the sum is complete and my ring is idle
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ reduce-scatter + epilogue
+        const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
+        const uint32_t t_addr = tmem_base + lane_base;
+        const int sw = lane & 7;                     // the eight 16-byte pieces of a row sit at piece ^ (row & 7)
+        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        // Accumulator chunk held at place `loc` of the receive buffer of CTA `owner`: output chunk
+        // owner * OWN_OC + loc % OWN_OC of the gate / only half (loc < OWN_OC) or of the up half.
+        auto acc_chunk = [&](int owner, int loc) { return (loc / Cfg::OWN_OC) * Cfg::OC + owner * Cfg::OWN_OC + loc % Cfg::OWN_OC; };
+        bool ok = mbar_wait(accf_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 7u);
+        if (ok) {
+            tc_fence_after();
+            // my ring is idle (every MMA that read it has completed): the peers may write their partials into it
+            if (warp == 2 && lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(ready_bar, lane));
+            ok = mbar_wait_cluster(ready_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 8u);
+        }
+        if (ok) {
+#pragma unroll 1
+            for (int i = 1; i < KS; ++i) {
+                const int peer = (static_cast<int>(rank) + i) % KS;
+                const int sidx = static_cast<int>(rank) < peer ? static_cast<int>(rank) : static_cast<int>(rank) - 1;   // my place among the peer's senders
+                const uint32_t peer_ring = cluster_map_shared(base, peer);
+#pragma unroll 1
+                for (int loc = 0; loc < Cfg::OWN_AC; ++loc) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(t_addr + acc_chunk(peer, loc) * 32, r);
+                    tmem_ld_wait();
+                    const uint32_t dst = peer_ring + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 128);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        st_shared_cluster_v4(dst + ((v ^ sw) << 4), __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                             __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                }
+                fence_acq_rel_cluster();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(cluster_map_shared(recv_bar, peer));
+            }
+            ok = mbar_wait_cluster(recv_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 9u);
+        }
+        if (ok) {
+            // sum of the KS partials of my columns, in rank order, back into TMEM
+#pragma unroll 1
+            for (int loc = 0; loc < Cfg::OWN_AC; ++loc) {
+                const int a = acc_chunk(static_cast<int>(rank), loc);
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(t_addr + a * 32, r);
+                tmem_ld_wait();
+                float acc[32];
+#pragma unroll
+                for (int s = 0; s < KS; ++s) {
+                    if (s == static_cast<int>(rank)) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) acc[j] = (s == 0) ? __uint_as_float(r[j]) : acc[j] + __uint_as_float(r[j]);
+                    } else {
+                        const int sidx = s < static_cast<int>(rank) ? s : s - 1;
+                        const uint32_t src = base + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 128);
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const float4 t = ld_shared_v4(src + ((g ^ sw) << 4));
+                            acc[4 * g] = (s == 0) ? t.x : acc[4 * g] + t.x;
+                            acc[4 * g + 1] = (s == 0) ? t.y : acc[4 * g + 1] + t.y;
+                            acc[4 * g + 2] = (s == 0) ? t.z : acc[4 * g + 2] + t.z;
+                            acc[4 * g + 3] = (s == 0) ? t.w : acc[4 * g + 3] + t.w;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(acc[j]);
+                tmem_st_32x32b_x32(t_addr + a * 32, r);
+            }
+            tmem_st_wait();
+            const int row = mb * 128 + q * 32 + lane;
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, static_cast<int>(rank) * Cfg::OWN_OC,
+                                         (static_cast<int>(rank) + 1) * Cfg::OWN_OC, Cfg::OUT_TILE_N, nb, static_cast<int>(rank), 0, vec_ok,
+                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    // No CTA frees its TMEM or leaves while a peer can still write into its ring or arrive on its barriers.
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();
+    if (*abort_flag != 0u) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 400000ll) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace mtmc

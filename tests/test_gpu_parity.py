@@ -325,6 +325,68 @@ def test_rowmax_and_cross_entropy_at_lm_head_size_on_sampled_rows():
     assert bool((loss >= lse - mx - 2e-3).all())
 
 
+# ------------------------------------------------------------------ cluster split-K (few tiles, long K)
+# Problems of at most half a wave of 128 x 256 tiles: a cluster of 2, 4 or 8 CTAs per tile, reduce-scatter through
+# distributed shared memory.  Ragged in every dimension, k-blocks that do not divide evenly among the CTAs,
+# column groups that lie wholly past N.
+KSPLIT = [(128, 1024, 4096), (100, 520, 1096), (300, 1000, 2056), (512, 2048, 2048), (700, 1100, 1160), (65, 8192, 1024),
+          (128, 300, 2048), (200, 4096, 4096)]
+
+
+@pytest.mark.parametrize("M,N,K", KSPLIT)
+@pytest.mark.parametrize("act,odt", [("gelu_tanh", "bf16"), ("none", "fp32")])
+def test_cluster_split_k_fused_linear(M, N, K, act, odt):
+    li = inputs.linear_inputs(M, N, K, seed=8000 + M + N)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[act])
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    B.mtmc_fused_linear(Xd, Wd, bd, act, odt, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "cluster split-K %dx%dx%d %s" % (M, N, K, odt))
+    # the partials are added in rank order: every launch gives the same bits
+    for _ in range(5):
+        assert torch.equal(B.mtmc_fused_linear(Xd, Wd, bd, act, odt), out)
+    # smaller clusters, and the tiled kernel without any split, stay within tolerance as well
+    for cap in (4, 2, 1):
+        B.mtmc_set_tuning(split_k=cap)
+        try:
+            other = B.mtmc_fused_linear(Xd, Wd, bd, act, odt)
+            B.mtmc_check_status()
+        finally:
+            B.mtmc_set_tuning()
+        _assert_close(inputs.to_f64(other), want, TOL[odt], "split_k cap %d %dx%dx%d %s" % (cap, M, N, K, odt))
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 1024, 4096), (300, 1000, 2056), (512, 2048, 2048), (700, 1100, 1160), (128, 300, 2048)])
+def test_cluster_split_k_other_epilogues(M, N, K):
+    li = inputs.linear_inputs(M, N, K, seed=8100 + M + N)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    lse = B.mtmc_linear_lse(Xd, Wd, bd)
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "split-K lse %dx%dx%d" % (M, N, K))
+    mx, arg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+    _check_rowmax(li, mx, arg, "split-K rowmax %dx%dx%d" % (M, N, K))
+    tgt = torch.from_numpy(np.random.default_rng(M + N).integers(0, N, size=M))
+    loss = B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt.cuda())
+    want_loss, _ = ref.linear_cross_entropy(Xb, Wb, bf, tgt.numpy())
+    _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "split-K cross entropy")
+    R = torch.randn(M, N, generator=torch.Generator().manual_seed(M * N)).bfloat16()
+    res = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "silu", "bf16")
+    _assert_close(inputs.to_f64(res), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_SILU), TOL["bf16"],
+                  "split-K residual")
+    B.mtmc_check_status()
+    si = inputs.swiglu_inputs(M, N, K, seed=8200 + M)
+    sw = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "split-K swiglu")
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=8300 + M)
+    f8 = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "gelu_tanh", "bf16")
+    want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(f8), want8, TOL["bf16"], "split-K fp8")
+    B.mtmc_check_status()
+
+
 # ------------------------------------------------------------------ skinny / split-K path
 @pytest.mark.parametrize("M,N,K", [
     (16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392),   # few rows: ticketed split-K
