@@ -25,7 +25,10 @@ using namespace mtmc;
 
 constexpr int MAX_DEVICES = 64;
 constexpr size_t TICKET_BYTES = 64 * 1024;   // library-owned split-K tickets: 16384 tiles
-constexpr int SKINNY_MAX_M = 64;              // rows of X the weight-streaming path takes (MMA N = 16, 32 or 64)
+#ifndef MTMC_SKINNY_MAX_M
+#define MTMC_SKINNY_MAX_M 64
+#endif
+constexpr int SKINNY_MAX_M = MTMC_SKINNY_MAX_M;   // rows of X the weight-streaming path takes (MMA N = 16, 32 or 64)
 
 struct DeviceState {
     bool ready = false;

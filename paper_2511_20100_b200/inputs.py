@@ -38,6 +38,9 @@ EXTRA_CONFIGS = {
     "X5": dict(op="fused_linear_fp8", M=8192, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=6),
     # the decode GEMM of C5 with E4M3 weights and activations: half the bytes to stream
     "X6": dict(op="fused_linear_fp8", M=16, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=4),
+    # a decode batch of 128 rows against the same weights: too many rows for the weight-streaming kernel, one
+    # row block of 32 tiles for the tiled one -> clusters of four CTAs per tile, split along K
+    "X7": dict(op="fused_linear", M=128, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=7),
 }
 
 
