@@ -231,6 +231,27 @@ int mtmc_ref_swiglu_points(const uint16_t* X, const uint16_t* Wg, const uint16_t
     return 0;
 }
 
+// out = silu(sx*sg * Xq.Wgq^T) * (sx*su * Xq.Wuq^T) with E4M3 operands: the SwiGLU gate of an FP8 layer whose
+// gate and up projections carry their own per-tensor scales.
+int mtmc_ref_swiglu_fp8(const uint8_t* X, const uint8_t* Wg, const uint8_t* Wu, float scale_x, float scale_g, float scale_u,
+                        int64_t M, int64_t N, int64_t K, double* out) {
+    if (!X || !Wg || !Wu || !out || M <= 0 || N <= 0 || K <= 0) return 1;
+    const double sg = static_cast<double>(scale_x) * static_cast<double>(scale_g);
+    const double su = static_cast<double>(scale_x) * static_cast<double>(scale_u);
+    parallel_for(M, [=](int64_t m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double g = 0.0, u = 0.0;
+            for (int64_t k = 0; k < K; ++k) {
+                const double x = e4m3_to_double(X[m * K + k]);
+                g += x * e4m3_to_double(Wg[n * K + k]);
+                u += x * e4m3_to_double(Wu[n * K + k]);
+            }
+            out[m * N + n] = act_apply(3, sg * g) * (su * u);
+        }
+    });
+    return 0;
+}
+
 // One row of logits -> its logsumexp, two passes: the maximum, then the sum of
 // exp(z - max) in ascending n, then max + log(sum).
 static double lse_of_row(const double* z, int64_t N) {
@@ -249,6 +270,24 @@ int mtmc_ref_linear_lse(const uint16_t* X, const uint16_t* W, const float* b,
     parallel_for(M, [=](int64_t m) {
         std::vector<double> z(static_cast<size_t>(N));
         for (int64_t n = 0; n < N; ++n) z[n] = preact(X, W, b, K, m, n);
+        if (logits) std::copy(z.begin(), z.end(), logits + m * N);
+        lse[m] = lse_of_row(z.data(), N);
+    });
+    return 0;
+}
+
+// lse[m] = log sum_n exp(sx*sw * Xq.Wq^T + b) with E4M3 operands; logits as above.
+int mtmc_ref_linear_lse_fp8(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                            int64_t M, int64_t N, int64_t K, double* lse, double* logits) {
+    if (!X || !W || !lse || M <= 0 || N <= 0 || K <= 0) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int64_t k = 0; k < K; ++k) acc += e4m3_to_double(X[m * K + k]) * e4m3_to_double(W[n * K + k]);
+            z[n] = scale * acc + (b ? static_cast<double>(b[n]) : 0.0);
+        }
         if (logits) std::copy(z.begin(), z.end(), logits + m * N);
         lse[m] = lse_of_row(z.data(), N);
     });

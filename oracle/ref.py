@@ -47,6 +47,8 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_e4m3.restype = dbl
         L.mtmc_ref_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp]
         L.mtmc_ref_fused_linear_fp8_points.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp, vp, i64, vp]
+        L.mtmc_ref_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
+        L.mtmc_ref_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
         L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
@@ -159,6 +161,31 @@ def fused_linear_fp8_points(X, W, b, scale_x: float, scale_w: float, act_kind: i
                                                   int(act_kind), rows.ctypes.data, cols.ctypes.data, rows.shape[0],
                                                   out.ctypes.data), "mtmc_ref_fused_linear_fp8_points")
     return out
+
+
+def swiglu_fp8(X, Wg, Wu, scale_x: float, scale_g: float, scale_u: float) -> np.ndarray:
+    """silu(scale_x*scale_g * Xq.Wgq^T) * (scale_x*scale_u * Xq.Wuq^T) with E4M3 bit patterns (uint8)."""
+    M, K = X.shape
+    N = Wg.shape[0]
+    X, Wg, Wu = _fp8(X, (M, K)), _fp8(Wg, (N, K)), _fp8(Wu, (N, K))
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_swiglu_fp8(X.ctypes.data, Wg.ctypes.data, Wu.ctypes.data, float(scale_x), float(scale_g),
+                                     float(scale_u), M, N, K, out.ctypes.data), "mtmc_ref_swiglu_fp8")
+    return out
+
+
+def linear_lse_fp8(X, W, b, scale_x: float, scale_w: float, want_logits: bool = False):
+    """Row logsumexp of scale_x*scale_w * Xq.Wq^T + b with E4M3 bit patterns (uint8)."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    lse = np.empty(M, dtype=np.float64)
+    logits = np.empty((M, N), dtype=np.float64) if want_logits else None
+    _check(lib().mtmc_ref_linear_lse_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
+                                         lse.ctypes.data, logits.ctypes.data if want_logits else None),
+           "mtmc_ref_linear_lse_fp8")
+    return (lse, logits) if want_logits else lse
 
 
 def fused_linear_points(X, W, b, act_kind: int, rows, cols) -> np.ndarray:

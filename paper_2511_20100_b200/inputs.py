@@ -110,6 +110,16 @@ def fp8_linear_inputs(M: int, N: int, K: int, seed: int, bias: bool = True) -> F
     return Fp8LinearInputs(out[0][0], out[1][0], li.b, out[0][1], out[1][1])
 
 
+def fp8_swiglu_inputs(M: int, N: int, K: int, seed: int):
+    """The SwiGLU recipe's draws quantised per tensor to E4M3: (X8, Wg8, Wu8, scale_x, scale_g, scale_u)."""
+    si = swiglu_inputs(M, N, K, seed)
+    out = []
+    for t in (si.X.float(), si.Wg.float(), si.Wu.float()):
+        scale = float(torch.tensor(float(t.abs().max()) / 448.0, dtype=torch.float32)) or 1.0
+        out.append(((t / scale).to(torch.float8_e4m3fn), scale))
+    return out[0][0], out[1][0], out[2][0], out[0][1], out[1][1], out[2][1]
+
+
 def fp8_bits(t: torch.Tensor) -> np.ndarray:
     """float8_e4m3fn tensor (CPU) -> uint8 numpy array of the raw bit patterns."""
     assert t.dtype == torch.float8_e4m3fn

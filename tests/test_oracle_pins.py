@@ -196,6 +196,51 @@ def test_fp8_linear_pins():
     assert float(fi.X.to(torch.float32).abs().max()) == 448.0 and float(fi.W.to(torch.float32).abs().max()) == 448.0
 
 
+def _as_bf16_bits(t8, factor):
+    """E4M3 tensor times a power of two, as bf16 bit patterns: exact, every E4M3 value has 4 significant bits."""
+    v = t8.to(torch.float32) * factor
+    b = v.to(torch.bfloat16)
+    assert torch.equal(b.to(torch.float32), v)
+    return inputs.bf16_bits(b)
+
+
+def test_fp8_swiglu_pins():
+    X8, Wg8, Wu8, sx, sg, su = inputs.fp8_swiglu_inputs(6, 11, 80, seed=72)
+    xb, gb, ub = inputs.fp8_bits(X8), inputs.fp8_bits(Wg8), inputs.fp8_bits(Wu8)
+    got = ref.swiglu_fp8(xb, gb, ub, sx, sg, su)
+    f = lambda v: float(np.float32(v))
+    g = f(sx) * f(sg) * (X8.to(torch.float64) @ Wg8.to(torch.float64).T)
+    u = f(sx) * f(su) * (X8.to(torch.float64) @ Wu8.to(torch.float64).T)
+    np.testing.assert_allclose(got, (torch.nn.functional.silu(g) * u).numpy(), rtol=1e-12, atol=1e-13)
+    # gate and up carry their own scales: the product of the two linear layers, each pinned on its own
+    prod = ref.fused_linear_fp8(xb, gb, None, sx, sg, ref.ACT_SILU) * ref.fused_linear_fp8(xb, ub, None, sx, su, ref.ACT_NONE)
+    np.testing.assert_allclose(got, prod, rtol=1e-14, atol=0)
+    # with power-of-two scales folded into bf16 copies of the operands it is the bf16 function, bit for bit
+    folded = ref.swiglu(_as_bf16_bits(X8, 2.0 ** -3), _as_bf16_bits(Wg8, 2.0 ** -7), _as_bf16_bits(Wu8, 2.0 ** -5))
+    assert np.array_equal(ref.swiglu_fp8(xb, gb, ub, 2.0 ** -3, 2.0 ** -7, 2.0 ** -5), folded)
+    # linear in the up scale, zero for a zero up projection, and the gate scale is inside the silu
+    np.testing.assert_allclose(ref.swiglu_fp8(xb, gb, ub, sx, sg, 2.0 * su), 2.0 * got, rtol=1e-14, atol=0)
+    assert not np.any(ref.swiglu_fp8(xb, gb, np.zeros_like(ub), sx, sg, su))
+    assert not np.allclose(ref.swiglu_fp8(xb, gb, ub, sx, 2.0 * sg, su), 2.0 * got)
+
+
+def test_fp8_linear_lse_pins():
+    fi = inputs.fp8_linear_inputs(5, 37, 64, seed=73)
+    X8, W8, b = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    lse, logits = ref.linear_lse_fp8(X8, W8, b, fi.scale_x, fi.scale_w, want_logits=True)
+    scale = float(np.float32(fi.scale_x)) * float(np.float32(fi.scale_w))
+    z = scale * (fi.X.to(torch.float64) @ fi.W.to(torch.float64).T) + fi.b.double()
+    np.testing.assert_allclose(logits, z.numpy(), rtol=1e-13, atol=1e-13)
+    np.testing.assert_allclose(lse, torch.logsumexp(z, dim=-1).numpy(), rtol=1e-13, atol=0)
+    # the logits are those of the pinned FP8 linear layer, and the row reduction is the pinned one
+    assert np.array_equal(logits, ref.fused_linear_fp8(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_NONE))
+    assert np.array_equal(lse, np.array([ref.lse_vector(row) for row in logits]))
+    # shift law through the bias, and the bf16 function on operands with the power-of-two scales folded in
+    np.testing.assert_allclose(ref.linear_lse_fp8(X8, W8, b + np.float32(0.5), fi.scale_x, fi.scale_w), lse + 0.5, rtol=0, atol=2e-7)   # b + 0.5 rounds in fp32
+    folded = ref.linear_lse(_as_bf16_bits(fi.X, 2.0 ** -4), _as_bf16_bits(fi.W, 2.0 ** -8), b)
+    assert np.array_equal(ref.linear_lse_fp8(X8, W8, b, 2.0 ** -4, 2.0 ** -8), folded)
+
+
 # ---------------------------------------------------------------- activations
 def _closed_forms():
     rows = []
