@@ -96,6 +96,18 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
 int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
                           int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 
+/* The SwiGLU gate and the row logsumexp with E4M3 operands, on the same kernels as their bf16
+ * forms (layout, K % 16 == 0 and scale conventions as for mtmc_fused_linear_fp8):
+ *   mtmc_swiglu_fp8     : out = silu(scale_x*scale_g * X8.Wg8^T) * (scale_x*scale_u * X8.Wu8^T),
+ *                         bf16 [M,N]; gate and up projection carry their own per-tensor scales
+ *   mtmc_linear_lse_fp8 : lse_out[m] = log sum_n exp(scale_x*scale_w * X8.W8^T + b), fp32 [M]
+ * The paper's operators are bf16/fp16/fp32; these are the lower-precision forms of the same
+ * fused epilogues. */
+int mtmc_swiglu_fp8(const void* X8, const void* Wg8, const void* Wu8, float scale_x, float scale_g, float scale_u,
+                    int64_t M, int64_t N, int64_t K, void* out);
+int mtmc_linear_lse_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                        int64_t M, int64_t N, int64_t K, float* lse_out);
+
 /* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
  * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate
  * product fused in one kernel; neither GEMM result is written to memory.) */

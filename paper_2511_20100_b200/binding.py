@@ -27,7 +27,7 @@ EXPORTS = [
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -58,6 +58,8 @@ def load() -> ctypes.CDLL:
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    L.mtmc_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
+    L.mtmc_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
@@ -143,6 +145,33 @@ def mtmc_fused_linear_fp8(X8, W8, b, scale_x, scale_w, act="none", out_dtype="bf
                                         float(scale_x), float(scale_w), M, N, K, ACT[act], OUT_DTYPE[out_dtype],
                                         _dev(out, odt, (M, N), "out")))
     return out
+
+
+def mtmc_swiglu_fp8(X8, Wg8, Wu8, scale_x, scale_g, scale_u, out=None):
+    """out = silu(scale_x*scale_g * X8 @ Wg8.T) * (scale_x*scale_u * X8 @ Wu8.T), float8_e4m3fn operands, bf16 [M,N]."""
+    M, K = X8.shape
+    N = Wg8.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_swiglu_fp8(_dev(X8, f8, (M, K), "X8"), _dev(Wg8, f8, (N, K), "Wg8"), _dev(Wu8, f8, (N, K), "Wu8"),
+                                  float(scale_x), float(scale_g), float(scale_u), M, N, K, _dev(out, torch.bfloat16, (M, N), "out")))
+    return out
+
+
+def mtmc_linear_lse_fp8(X8, W8, b, scale_x, scale_w, lse_out=None):
+    """lse_out[m] = logsumexp_n(scale_x*scale_w * X8 @ W8.T + b) with float8_e4m3fn operands, fp32 [M]."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    if lse_out is None:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_linear_lse_fp8(_dev(X8, f8, (M, K), "X8"), _dev(W8, f8, (N, K), "W8"),
+                                      None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                      float(scale_x), float(scale_w), M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
 
 
 def mtmc_swiglu(X, Wg, Wu, out=None):

@@ -400,6 +400,7 @@ void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
     p.fp8 = fp8 ? 1 : 0;
     p.bk_elems = fp8 ? 128 : 64;               // one 128-byte swizzle row of K per ring stage
     p.acc_scale = 1.0f;
+    p.acc_scale2 = 1.0f;
     p.k_blocks = static_cast<int>((K + p.bk_elems - 1) / p.bk_elems);
     p.group_m = pick_group_m(p.m_tiles);      // 16 row blocks per group measured best for both tile heights
     p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1; p.tail_width = out_tile_n;
@@ -611,18 +612,20 @@ int stage_buffer(DeviceState* d, int i, size_t bytes, void** out) {
 //   EPI_XENT   : out_b = loss, out_a = lse (may be null); the target logits sit behind the partials
 template <int EPI>
 int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
-                      float* out_a, float* out_b, int32_t* out_i) {
+                      float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f) {
+    auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
     if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    const int ks = pick_ksplit(d, M, N, K, 256, false);
+    const int ks = pick_ksplit(d, M, N, K, 256, fp8);
     const bool pair = !ks && use_pair(d, M, N);
     const int bn = (pair || ks) ? 256 : pick_tile_n(N);
     GemmParams p{};
-    if (ks) fill_ksplit(p, M, N, K, 256, ks, false);
-    else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
-    else fill_tiling(p, M, N, K, bn, d->sm_count, true);
+    if (ks) fill_ksplit(p, M, N, K, 256, ks, fp8);
+    else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, fp8);
+    else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, fp8);
+    p.acc_scale = acc_scale;
     const size_t partial_bytes = lse_workspace_bytes(M, N);
     const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
     void* ws = nullptr;
@@ -634,8 +637,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
     if (EPI == EPI_XENT) CUDA_TRY(cudaMemsetAsync(p.target_logit, 0xFF, static_cast<size_t>(M) * sizeof(float), t_stream));
     CUtensorMap tmA, tmB, tmBt;
-    if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, pair ? 128 : bn)) ||
-        (rc = encode_bf16_2d(&tmBt, W, N, K, pair ? p.tail_width / 2 : p.tail_width)))
+    if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmB, W, N, K, pair ? 128 : bn)) ||
+        (rc = encode(&tmBt, W, N, K, pair ? p.tail_width / 2 : p.tail_width)))
         return rc;
     TimedRegion tr(d);
     if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
@@ -717,6 +720,66 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     tr.stop();
     return rc;
 }
+// out = silu(sg * X.Wg^T) * (su * X.Wu^T): bf16 operands (sg = su = 1) or E4M3 operands with the scale products.
+int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out, bool fp8, float sg, float su) {
+    auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
+    int rc = check_common(X, Wg, out, M, N, K);
+    if (rc) return rc;
+    if (!Wu) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(Wu)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    DeviceState* d = nullptr;
+    rc = get_device(&d);
+    if (rc) return rc;
+    if (const int ks = pick_ksplit(d, M, N, K, 128, fp8)) {
+        GemmParams p{};
+        fill_ksplit(p, M, N, K, 128, ks, fp8);
+        p.acc_scale = sg; p.acc_scale2 = su;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmG, tmU;
+        if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmG, Wg, N, K, 128)) ||
+            (rc = encode(&tmU, Wu, N, K, 128)))
+            return rc;
+        TimedRegion tr(d);
+        rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
+        tr.stop();
+        return rc;
+    }
+    if (use_pair(d, M, N)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 128, gemm_pairs(d), true, 256, fp8);
+        p.acc_scale = sg; p.acc_scale2 = su;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
+        if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmG, Wg, N, K, 128)) ||
+            (rc = encode(&tmU, Wu, N, K, 128)) || (rc = encode(&tmGt, Wg, N, K, p.tail_width)) ||
+            (rc = encode(&tmUt, Wu, N, K, p.tail_width)))
+            return rc;
+        TimedRegion tr(d);
+        rc = launch_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, tmGt, tmUt, p);
+        tr.stop();
+        return rc;
+    }
+    GemmParams p{};
+    fill_tiling(p, M, N, K, 128, d->sm_count, true, 128, fp8);   // 128 output columns = 128 gate + 128 up accumulator columns
+    p.acc_scale = sg; p.acc_scale2 = su;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
+    rc = encode(&tmA, X, M, K, 128);
+    if (rc) return rc;
+    rc = encode(&tmG, Wg, N, K, 128);
+    if (rc) return rc;
+    rc = encode(&tmU, Wu, N, K, 128);
+    if (rc) return rc;
+    rc = encode(&tmGt, Wg, N, K, p.tail_width);
+    if (rc) return rc;
+    rc = encode(&tmUt, Wu, N, K, p.tail_width);
+    if (rc) return rc;
+    TimedRegion tr(d);
+    rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
+    tr.stop();
+    return rc;
+}
+
 }  // namespace
 
 extern "C" {
@@ -867,64 +930,27 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
 }
 
 int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
-    int rc = check_common(X, Wg, out, M, N, K);
-    if (rc) return rc;
-    if (!Wu) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
-    if (!aligned16(Wu)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
-    DeviceState* d = nullptr;
-    rc = get_device(&d);
-    if (rc) return rc;
-    if (const int ks = pick_ksplit(d, M, N, K, 128, false)) {
-        GemmParams p{};
-        fill_ksplit(p, M, N, K, 128, ks, false);
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-        CUtensorMap tmA, tmG, tmU;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmG, Wg, N, K, 128)) ||
-            (rc = encode_bf16_2d(&tmU, Wu, N, K, 128)))
-            return rc;
-        TimedRegion tr(d);
-        rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
-        tr.stop();
-        return rc;
-    }
-    if (use_pair(d, M, N)) {
-        GemmParams p{};
-        fill_tiling(p, M, N, K, 128, gemm_pairs(d), true, 256);
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-        CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmG, Wg, N, K, 128)) ||
-            (rc = encode_bf16_2d(&tmU, Wu, N, K, 128)) || (rc = encode_bf16_2d(&tmGt, Wg, N, K, p.tail_width)) ||
-            (rc = encode_bf16_2d(&tmUt, Wu, N, K, p.tail_width)))
-            return rc;
-        TimedRegion tr(d);
-        rc = launch_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, tmGt, tmUt, p);
-        tr.stop();
-        return rc;
-    }
-    GemmParams p{};
-    fill_tiling(p, M, N, K, 128, d->sm_count, true);   // 128 output columns = 128 gate + 128 up accumulator columns
-    p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
-    CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-    rc = encode_bf16_2d(&tmA, X, M, K, 128);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmG, Wg, N, K, 128);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmU, Wu, N, K, 128);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmGt, Wg, N, K, p.tail_width);
-    if (rc) return rc;
-    rc = encode_bf16_2d(&tmUt, Wu, N, K, p.tail_width);
-    if (rc) return rc;
-    TimedRegion tr(d);
-    rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
-    tr.stop();
-    return rc;
+    return swiglu_impl(X, Wg, Wu, M, N, K, out, false, 1.0f, 1.0f);
+}
+
+int mtmc_swiglu_fp8(const void* X8, const void* Wg8, const void* Wu8, float scale_x, float scale_g, float scale_u,
+                    int64_t M, int64_t N, int64_t K, void* out) {
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
+    return swiglu_impl(X8, Wg8, Wu8, M, N, K, out, true, scale_x * scale_g, scale_x * scale_u);
 }
 
 int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
     int rc = check_common(X, W, lse_out, M, N, K);
     if (rc) return rc;
     return run_row_reduction<EPI_LSE>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr);
+}
+
+int mtmc_linear_lse_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,
+                        int64_t K, float* lse_out) {
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
+    int rc = check_common(X8, W8, lse_out, M, N, K);
+    if (rc) return rc;
+    return run_row_reduction<EPI_LSE>(X8, W8, b, nullptr, M, N, K, lse_out, nullptr, nullptr, true, scale_x * scale_w);
 }
 
 int mtmc_linear_rowmax(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* max_out,

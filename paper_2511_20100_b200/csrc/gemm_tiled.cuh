@@ -46,6 +46,7 @@ struct GemmParams {
     int fp8;              // 0: bf16 operands (64 per 128-byte row, K = 16 per MMA); 1: E4M3 operands (128 per row, K = 32)
     int bk_elems;         // elements of K per ring stage: 64 or 128
     float acc_scale;      // multiplies the accumulator before the bias (product of the FP8 per-tensor scales; 1 otherwise)
+    float acc_scale2;     // the same for the up half of a SwiGLU accumulator (acc_scale is then the gate half's)
     const float* bias;    // [N] or null
     const void* residual; // [M,N] in the output's element type, added after the activation, or null (EPI_ACT)
     void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
@@ -332,6 +333,13 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tmem_ld_32x32b_x32(t_addr + width + c * 32, u);         // up columns follow the gate columns
             tmem_ld_wait();
             float y[32];
+            if (p.fp8) {                                            // E4M3 operands: the per-tensor scales of gate and up
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    g[j] = __float_as_uint(__uint_as_float(g[j]) * p.acc_scale);
+                    u[j] = __float_as_uint(__uint_as_float(u[j]) * p.acc_scale2);
+                }
+            }
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<true>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
@@ -351,7 +359,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                const float z = (n0 + j < p.N) ? __uint_as_float(r[j]) + bv[j] : -INFINITY;
+                const float z = (n0 + j < p.N) ? fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]) : -INFINITY;   // scale 1: the same bits as r + b
                 if (z > mx) { mx = z; arg = n0 + j; }        // strict: ties keep the lower column
             }
         }
@@ -360,6 +368,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
     } else {
         // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
         constexpr float LOG2E = 1.4426950408889634f;
+        const float zscale = LOG2E * p.acc_scale;            // accumulator -> base-2 logit units (acc_scale is 1 for bf16 operands)
         float mx = -INFINITY, sum = 0.0f;
         int tgt = -1;
         float tz = 0.0f;
@@ -377,7 +386,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             float cm = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                tv[j] = fmaf(__uint_as_float(r[j]), LOG2E, bv[j] * LOG2E);
+                tv[j] = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);
                 cm = fmaxf(cm, tv[j]);
             }
             if (n0 + 32 > p.N) {      // ragged last chunk: columns past N are zero-filled weight rows, mask them out

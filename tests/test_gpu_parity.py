@@ -152,6 +152,30 @@ def test_fused_linear_fp8_skinny(M, N, K, split_k, act, odt):
     _assert_close(inputs.to_f64(out), want, TOL[odt], "fp8 skinny %dx%dx%d %s %s" % (M, N, K, act, odt))
 
 
+@pytest.mark.parametrize("M,N,K", [(1, 16, 16), (100, 72, 144), (300, 392, 272), (128, 1024, 4096), (600, 1000, 656), (1024, 2048, 1024)])
+def test_swiglu_fp8(M, N, K):
+    """E4M3 SwiGLU with separate gate / up scales on the single-CTA, cluster split-K and CTA-pair kernels."""
+    X8, Wg8, Wu8, sx, sg, su = inputs.fp8_swiglu_inputs(M, N, K, seed=7200 + M + N)
+    buf, out = _guarded((M, N), torch.bfloat16)
+    B.mtmc_swiglu_fp8(X8.cuda(), Wg8.cuda(), Wu8.cuda(), sx, sg, su, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    want = ref.swiglu_fp8(inputs.fp8_bits(X8), inputs.fp8_bits(Wg8), inputs.fp8_bits(Wu8), sx, sg, su)
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "swiglu fp8 %dx%dx%d" % (M, N, K))
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 16), (5, 8, 64), (200, 1000, 256), (129, 257, 80), (128, 1024, 4096), (600, 3000, 128),
+                                   (1024, 4096, 512)])
+def test_linear_lse_fp8(M, N, K):
+    fi = inputs.fp8_linear_inputs(M, N, K, seed=7300 + M + N)
+    buf, out = _guarded((M,), torch.float32)
+    B.mtmc_linear_lse_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, lse_out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M)
+    want = ref.linear_lse_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w)
+    _assert_close(inputs.to_f64(out), want, TOL["fp32"], "lse fp8 %dx%dx%d" % (M, N, K))
+
+
 def test_fused_linear_fp8_exact_small_integers():
     # operands in {-2..2} are exact in E4M3 and every fp32 partial sum is exact: the result must be exact too
     g = torch.Generator().manual_seed(6)
