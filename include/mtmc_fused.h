@@ -234,8 +234,10 @@ float mtmc_last_kernel_ms(void);
  *              many K splits per 128-row band of W; for larger M it caps the cluster
  *              size of the cluster split-K kernel (1 = never use that kernel)
  *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
- *   cta_pair : > 0 forces the CTA-pair (cta_group::2, 256-row tiles) tiled kernel,
- *              < 0 forbids it; automatic = pairs when M >= 512 and N >= 256          */
+ *   cta_pair : 1 forces the CTA-pair (cta_group::2) kernel with 256 x 256 tiles and overlapped
+ *              epilogues, 2 the one with 512 x 256 tiles (activation epilogues; the other
+ *              operators then take the 256 x 256 pair kernel), < 0 forbids both;
+ *              automatic = pairs when M >= 512 and N >= 256, the large tiles for long K */
 int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
 
 /* Static weights (thread-local, default 0 = off).  With enabled != 0 the caller promises, for

@@ -17,6 +17,7 @@
 
 #include "gemm_pair.cuh"
 #include "gemm_ksplit.cuh"
+#include "gemm_big.cuh"
 #include "skinny.cuh"
 
 namespace {
@@ -274,6 +275,29 @@ int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, co
     return MTMC_OK;
 }
 
+template <int EPI, bool OUT_BF16>
+int launch_big(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
+    using Cfg = BigCfg<EPI>;
+    auto kern = gemm_big_kernel<EPI, OUT_BF16>;
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
+    const int pairs = p.num_tiles < clusters ? p.num_tiles : clusters;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1 + pdl_attribute(attr + 1);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
 // How many CTA pairs of the pair kernel fit on the device at once (0: clusters unavailable).
 int gemm_pairs(DeviceState* d) {
     if (d->max_gemm_pairs < 0) {
@@ -385,6 +409,25 @@ bool use_pair(DeviceState* d, int64_t M, int64_t N) {
     if (t_cta_pair < 0 || t_tile_n == 128 || gemm_pairs(d) <= 0) return false;
     if (t_cta_pair > 0) return true;
     return M >= 512 && N >= 256;
+}
+
+// The 512 x 256 pair tiles (gemm_big.cuh) against the 256 x 256 ones with overlapped epilogues (gemm_pair.cuh).
+// Measured on plain and GELU epilogues: per FLOP the large tiles are on a par at K = 4096 and 5-15 % ahead from
+// K = 8192 on (a quarter less operand traffic, and the exposed epilogue shrinks against the k-walk); their
+// tiles are twice as large, so with few waves they can lose more to the last, partial wave.  Hence: always
+// from 96 k-blocks on, from 64 k-blocks on when their waves cost no more than the pair kernel's, counted in
+// 256-row tile waves.  Tuning hook: cta_pair = 2 forces them, 1 forces the 256 x 256 pair tiles.
+bool use_big(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
+    const int pairs = gemm_pairs(d);
+    if (pairs <= 0 || EPI_HALVES != 1 || t_tile_n != 0 || t_cta_pair < 0 || t_cta_pair == 1) return false;
+    if (t_cta_pair == 2) return true;
+    if (M < 512 || N < 256) return false;
+    const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
+    if (k_blocks >= 96) return true;
+    if (k_blocks < 64) return false;
+    const int64_t n_tiles = (N + 255) / 256;
+    const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
+    return 2 * ((t_big + pairs - 1) / pairs) <= (t_pair + pairs - 1) / pairs;
 }
 
 // Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
@@ -684,6 +727,18 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
         tr.stop();
         return rc;
     }
+    if (use_big(d, M, N, K, false)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512);
+        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 256)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128))) return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_big<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, p)
+                                        : launch_big<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, p);
+        tr.stop();
+        return rc;
+    }
     if (use_pair(d, M, N)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
@@ -803,7 +858,7 @@ int mtmc_set_tuning(int split_k, int tile_n, int cta_pair) {
     if (tile_n > 0 && tile_n != 128 && tile_n != 256) return fail(MTMC_ERR_INVALID_ARG, "tile_n must be 128 or 256");
     t_split_k = split_k > 0 ? split_k : 0;
     t_tile_n = tile_n > 0 ? tile_n : 0;
-    t_cta_pair = cta_pair > 0 ? 1 : (cta_pair < 0 ? -1 : 0);
+    t_cta_pair = cta_pair > 1 ? 2 : (cta_pair > 0 ? 1 : (cta_pair < 0 ? -1 : 0));
     return MTMC_OK;
 }
 
@@ -903,6 +958,19 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
         if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, 256))) return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
+        tr.stop();
+        return rc;
+    }
+    if (use_big(d, M, N, K, true)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512, true);
+        p.acc_scale = scale_x * scale_w;
+        p.act = act; p.bias = b; p.residual = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmB;
+        if ((rc = encode_u8_2d(&tmA, X8, M, K, 256)) || (rc = encode_u8_2d(&tmB, W8, N, K, 128))) return rc;
+        TimedRegion tr(d);
+        rc = out_dtype == MTMC_OUT_BF16 ? launch_big<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, p)
+                                        : launch_big<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, p);
         tr.stop();
         return rc;
     }

@@ -99,6 +99,51 @@ def test_cta_pair_and_single_cta_kernels_agree_with_the_oracle(cta_pair):
                                                       ref.ACT_RELU), TOL["fp32"], "129x257x72")
 
 
+
+@pytest.mark.parametrize("M,N,K", [(100, 72, 136), (512, 256, 64), (600, 520, 328), (1100, 1300, 1024), (2048, 1000, 200)])
+@pytest.mark.parametrize("act,odt", [("gelu_tanh", "bf16"), ("relu", "fp32")])
+def test_large_tile_pair_kernel_forced(M, N, K, act, odt):
+    """The CTA-pair kernel with 512 x 256 tiles (two 128-row halves per CTA, eight epilogue warps), forced by the
+    tuning hook on shapes that leave rows, columns and k-blocks ragged."""
+    li = inputs.linear_inputs(M, N, K, seed=8800 + M + N)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[act])
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    B.mtmc_set_tuning(cta_pair=2)
+    try:
+        B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), act, odt, out=out)
+        B.mtmc_check_status()
+        again = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), act, odt)
+    finally:
+        B.mtmc_set_tuning()
+    assert _canaries_intact(buf, M * N)
+    assert torch.equal(again, out)
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "512-row tiles %dx%dx%d %s %s" % (M, N, K, act, odt))
+
+
+def test_large_tile_pair_kernel_chosen_for_long_k():
+    """From 96 k-blocks on the 512 x 256 tiles are the default for M >= 512, N >= 256: bf16, residual and FP8 forms."""
+    M, N, K = 600, 520, 6144
+    li = inputs.linear_inputs(M, N, K, seed=8900)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    out = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
+    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, ref.ACT_SILU), TOL["fp32"], "long K, default path")
+    B.mtmc_set_tuning(cta_pair=1)
+    try:
+        small_tiles = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(small_tiles), ref.fused_linear(Xb, Wb, bf, ref.ACT_SILU), TOL["fp32"], "long K, 256-row tiles")
+    R = torch.randn(M, N, generator=torch.Generator().manual_seed(5)).bfloat16()
+    res = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "none", "bf16")
+    _assert_close(inputs.to_f64(res), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_NONE), TOL["bf16"],
+                  "long K residual")
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=8901)
+    f8 = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "gelu_tanh", "bf16")
+    want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(f8), want8, TOL["bf16"], "long K fp8")
+    B.mtmc_check_status()
+
 @pytest.mark.parametrize("M,N,K", [(9, 520, 392), (16, 4096, 512), (129, 257, 72), (300, 520, 200), (600, 1000, 328)])
 @pytest.mark.parametrize("odt", ["fp32", "bf16"])
 def test_fused_linear_residual(M, N, K, odt):
