@@ -279,12 +279,13 @@ template <int EPI, bool OUT_BF16>
 int launch_big(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
     using Cfg = BigCfg<EPI>;
     auto kern = gemm_big_kernel<EPI, OUT_BF16>;
-    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
+    constexpr int SMEM = Cfg::smem_bytes(OUT_BF16);
+    if (int rc = ensure_smem_attr(kern, SMEM)) return rc;
     const int pairs = p.num_tiles < clusters ? p.num_tiles : clusters;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
     cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
-    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.dynamicSmemBytes = SMEM;
     cfg.stream = t_stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -425,6 +426,24 @@ bool use_big(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
     if (k_blocks >= 96) return true;
     if (k_blocks < 64) return false;
+    const int64_t n_tiles = (N + 255) / 256;
+    const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
+    return 2 * ((t_big + pairs - 1) / pairs) <= (t_pair + pairs - 1) / pairs;
+}
+
+// The same choice for the row reductions (logsumexp, row max, cross entropy).  Their epilogues store one partial
+// per row, so little is exposed when it is not overlapped: the large tiles are 4-5 % ahead at K = 4096 already
+// (C4: 680-714 us against 710-750 us).  From 32 k-blocks on when their waves cost no more, always from 96 on.
+// SwiGLU stays on the 256 x 256 tiles: its epilogue (two MUFU operations per element plus the stores) is too long
+// to expose (measured on C3: 2-3 % slower on the large tiles).
+bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
+    const int pairs = gemm_pairs(d);
+    if (pairs <= 0 || EPI_HALVES != 1 || t_tile_n != 0 || t_cta_pair < 0 || t_cta_pair == 1) return false;
+    if (t_cta_pair == 2) return true;
+    if (M < 512 || N < 256) return false;
+    const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
+    if (k_blocks >= 96) return true;
+    if (k_blocks < 32) return false;
     const int64_t n_tiles = (N + 255) / 256;
     const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
     return 2 * ((t_big + pairs - 1) / pairs) <= (t_pair + pairs - 1) / pairs;
@@ -662,10 +681,12 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     int rc = get_device(&d);
     if (rc) return rc;
     const int ks = pick_ksplit(d, M, N, K, 256, fp8);
-    const bool pair = !ks && use_pair(d, M, N);
-    const int bn = (pair || ks) ? 256 : pick_tile_n(N);
+    const bool big = !ks && use_big_rowred(d, M, N, K, fp8);
+    const bool pair = !ks && !big && use_pair(d, M, N);
+    const int bn = (pair || ks || big) ? 256 : pick_tile_n(N);
     GemmParams p{};
     if (ks) fill_ksplit(p, M, N, K, 256, ks, fp8);
+    else if (big) fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512, fp8);
     else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, fp8);
     else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, fp8);
     p.acc_scale = acc_scale;
@@ -680,11 +701,12 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
     if (EPI == EPI_XENT) CUDA_TRY(cudaMemsetAsync(p.target_logit, 0xFF, static_cast<size_t>(M) * sizeof(float), t_stream));
     CUtensorMap tmA, tmB, tmBt;
-    if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmB, W, N, K, pair ? 128 : bn)) ||
-        (rc = encode(&tmBt, W, N, K, pair ? p.tail_width / 2 : p.tail_width)))
+    if ((rc = encode(&tmA, X, M, K, big ? 256 : 128)) || (rc = encode(&tmB, W, N, K, (pair || big) ? 128 : bn)) ||
+        (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width)))
         return rc;
     TimedRegion tr(d);
     if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
+    else if (big) rc = launch_big<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, p);
     else if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
     else rc = bn == 256 ? launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
                         : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);

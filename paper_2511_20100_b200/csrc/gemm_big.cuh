@@ -36,10 +36,19 @@ struct BigCfg {
     static constexpr int TMEM_COLS = 2 * BN;             // the two row halves of one tile: all of tensor memory
     static constexpr int NUM_BARRIERS = 2 * STAGES + 2;  // ring, accumulator full, accumulator empty
     static constexpr bool STORES = (EPI == EPI_ACT || EPI == EPI_SWIGLU);
-    static constexpr int EPI_STAGING_BYTES = STORES ? WARPS_EPI * EPI_STAGE_BYTES_PER_WARP : 0;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_STAGING_BYTES + NUM_BARRIERS * 8 + 16 + 1024;
+    // Store staging per epilogue warp: a 32 x 32 chunk, 2 KiB as bf16, 4 KiB as fp32.
+    __host__ __device__ static constexpr int stage_bytes_per_warp(bool out_bf16) { return out_bf16 ? 2048 : 4096; }
+    __host__ __device__ static constexpr int staging_bytes(bool out_bf16) { return STORES ? WARPS_EPI * stage_bytes_per_warp(out_bf16) : 0; }
+    // Two copies of the tile's 256 bias values (the tile in its epilogue and the next one), where they fit:
+    // not beside the fp32 store staging.
+    static constexpr bool HAS_BIAS = (EPI != EPI_SWIGLU);
+    __host__ __device__ static constexpr bool bias_in_smem(bool out_bf16) { return HAS_BIAS && (!STORES || out_bf16); }
+    __host__ __device__ static constexpr int bias_bytes(bool out_bf16) { return bias_in_smem(out_bf16) ? 2 * BN * 4 : 0; }
+    __host__ __device__ static constexpr int smem_bytes(bool out_bf16) {
+        return STAGES * STAGE_BYTES + staging_bytes(out_bf16) + NUM_BARRIERS * 8 + 16 + bias_bytes(out_bf16) + 1024;
+    }
     static constexpr int THREADS = 64 + 32 * WARPS_EPI;
-    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory per CTA");
+    static_assert(smem_bytes(true) <= 227 * 1024 && smem_bytes(false) <= 227 * 1024, "shared memory per CTA");
     static_assert(EPI_HALVES == 1, "the epilogue's partial layout assumes one warp per quadrant and tile half");
 };
 
@@ -54,7 +63,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
-    const uint32_t bar_base = epi_stage_base + Cfg::EPI_STAGING_BYTES;
+    const uint32_t bar_base = epi_stage_base + Cfg::staging_bytes(OUT_BF16);
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     const uint32_t accf_bar = bar_base + 8u * (2 * STAGES);
@@ -62,6 +71,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
+    float* bias_s = reinterpret_cast<float*>(ctrl + 16);                      // [2][BN], if Cfg::bias_in_smem
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -165,17 +175,30 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(hh * Cfg::BN);
         const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        constexpr bool BIAS_S = Cfg::bias_in_smem(OUT_BF16);
+        const int et = static_cast<int>(threadIdx.x) - 64;       // 0 .. 255: this thread's column of the tile's bias
         uint32_t acc_ph = 0;
         bool ok = true;
         for (int t = pair_id; t < p.num_tiles && ok; t += num_pairs) {
             int mb, nb;
             tile_coords(p, t, mb, nb);
             const int row = mb * Cfg::BM + static_cast<int>(rank) * 256 + hh * 128 + q * 32 + lane;
+            float* bias_tile = nullptr;
+            if (BIAS_S) {
+                // while the mainloop runs: the tile's bias into shared memory (the other copy may still be read by a
+                // warp that is finishing the previous tile; nobody is more than one tile ahead, see the barrier below)
+                bias_tile = bias_s + acc_ph * Cfg::BN;
+                const int n = nb * Cfg::OUT_TILE_N + et;
+                bias_tile[et] = (p.bias != nullptr && n < p.N) ? __ldg(p.bias + n) : 0.0f;
+            }
             if (!mbar_wait(accf_bar, acc_ph, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 6u)) { ok = false; break; }
             acc_ph ^= 1u;
             tc_fence_after();
+            // every epilogue warp has passed the same accumulator-full wait, so all of them reach this barrier
+            if (BIAS_S) asm volatile("bar.sync 1, 256;" ::: "memory");
             epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, 0, Cfg::OUT_TILE_N / 32, Cfg::OUT_TILE_N, nb, 0, 0, vec_ok,
-                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
+                                         smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * Cfg::stage_bytes_per_warp(OUT_BF16), lane,
+                                         bias_tile);
             // this warp's share of the accumulators is drained: tell the MMA issuer in the even CTA
             tc_fence_before();
             __syncwarp();

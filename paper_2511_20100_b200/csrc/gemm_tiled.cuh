@@ -284,6 +284,22 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
     }
 }
 
+// The same from a copy of the tile's bias in shared memory (bias_tile[j] = bias of the tile's column j, zeros
+// past N), when the kernel keeps one: a global load costs the exposed epilogue of gemm_big.cuh several hundred
+// clocks per chunk, a broadcast shared-memory load a few tens.
+__device__ __forceinline__ void tile_bias_chunk(const GemmParams& p, const float* bias_tile, int n_tile0, int n0, float (&b)[32]) {
+    if (bias_tile == nullptr) {
+        load_bias_chunk(p.bias, n0, p.N, b);
+    } else {
+        const float4* b4 = reinterpret_cast<const float4*>(bias_tile + (n0 - n_tile0));
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+            const float4 t = b4[v];
+            b[4 * v] = t.x; b[4 * v + 1] = t.y; b[4 * v + 2] = t.z; b[4 * v + 3] = t.w;
+        }
+    }
+}
+
 // One work item's epilogue for one thread: this thread owns output row `row` (TMEM lane
 // of t_addr) and walks chunks [c_begin, c_end) of 32 columns of the item that starts at column n_tile0
 // (the other half of the chunks belongs to the second warp of this lane quadrant).
@@ -295,7 +311,7 @@ __device__ __forceinline__ void load_bias_chunk(const float* bias, int n0, int N
 template <int EPI, bool OUT_BF16>
 __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int c_begin,
                                               int c_end, int width, int nb, int sub, int half, bool vec_ok, uint8_t* stage,
-                                              int lane) {
+                                              int lane, const float* bias_tile = nullptr) {
     if (EPI == EPI_ACT) {
         // Two chunks in flight: while chunk c is being activated and stored, the TMEM load and the
         // bias fetch of chunk c + 1 are already under way.
@@ -305,7 +321,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         float bv[32];
         if (c_begin < live) {
             tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
-            load_bias_chunk(p.bias, n_tile0 + c_begin * 32, p.N, bv);
+            tile_bias_chunk(p, bias_tile, n_tile0, n_tile0 + c_begin * 32, bv);
         }
 #pragma unroll 1
         for (int c = c_begin; c < live; ++c) {
@@ -316,7 +332,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             for (int j = 0; j < 32; ++j) y[j] = fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]);
             if (c + 1 < live) {                              // r and bv are free again: refill them for chunk c + 1
                 tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
-                load_bias_chunk(p.bias, n0 + 32, p.N, bv);
+                tile_bias_chunk(p, bias_tile, n_tile0, n0 + 32, bv);
             }
             apply_act_chunk<OUT_BF16>(p.act, y);
             if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
@@ -355,7 +371,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             uint32_t r[32];
             tmem_ld_32x32b_x32(t_addr + c * 32, r);
             float bv[32];
-            load_bias_chunk(p.bias, n0, p.N, bv);
+            tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -381,7 +397,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             uint32_t r[32];
             tmem_ld_32x32b_x32(t_addr + c * 32, r);
             float bv[32], tv[32];
-            load_bias_chunk(p.bias, n0, p.N, bv);
+            tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
             float cm = -INFINITY;
 #pragma unroll

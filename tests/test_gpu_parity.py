@@ -120,6 +120,29 @@ def test_large_tile_pair_kernel_forced(M, N, K, act, odt):
     _assert_close(inputs.to_f64(out), want, TOL[odt], "512-row tiles %dx%dx%d %s %s" % (M, N, K, act, odt))
 
 
+@pytest.mark.parametrize("M,N,K", [(100, 72, 136), (600, 520, 328), (1100, 1300, 1024)])
+def test_large_tile_pair_kernel_row_reductions(M, N, K):
+    """logsumexp, row max and cross entropy on the 512 x 256 tiles (forced), bias staged in shared memory."""
+    li = inputs.linear_inputs(M, N, K, seed=8950 + M)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    tgt = torch.from_numpy(np.random.default_rng(M).integers(0, N, size=M))
+    B.mtmc_set_tuning(cta_pair=2)
+    try:
+        lse = B.mtmc_linear_lse(Xd, Wd, bd)
+        lse_nobias = B.mtmc_linear_lse(Xd, Wd, None)
+        mx, arg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+        loss = B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt.cuda())
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "lse, 512-row tiles")
+    _assert_close(inputs.to_f64(lse_nobias), ref.linear_lse(Xb, Wb, None), TOL["fp32"], "lse without bias, 512-row tiles")
+    _check_rowmax(li, mx, arg, "rowmax, 512-row tiles")
+    want_loss, _ = ref.linear_cross_entropy(Xb, Wb, bf, tgt.numpy())
+    _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "cross entropy, 512-row tiles")
+
+
 def test_large_tile_pair_kernel_chosen_for_long_k():
     """From 96 k-blocks on the 512 x 256 tiles are the default for M >= 512, N >= 256: bf16, residual and FP8 forms."""
     M, N, K = 600, 520, 6144
