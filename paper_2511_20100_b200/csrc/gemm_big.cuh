@@ -34,7 +34,7 @@ struct BigCfg {
     static constexpr int WARPS_EPI = 8;                  // quadrant = warp % 4, row half = (warp - 2) / 4
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     static constexpr int TMEM_COLS = 2 * BN;             // the two row halves of one tile: all of tensor memory
-    static constexpr int NUM_BARRIERS = 2 * STAGES + 2;  // ring, accumulator full, accumulator empty
+    static constexpr int NUM_BARRIERS = 2 * STAGES + 3;  // ring, accumulator full, accumulator empty, bias copy written
     static constexpr bool STORES = (EPI == EPI_ACT || EPI == EPI_SWIGLU);
     // Store staging per epilogue warp: a 32 x 32 chunk, 2 KiB as bf16, 4 KiB as fp32.
     __host__ __device__ static constexpr int stage_bytes_per_warp(bool out_bf16) { return out_bf16 ? 2048 : 4096; }
@@ -44,8 +44,9 @@ struct BigCfg {
     static constexpr bool HAS_BIAS = (EPI != EPI_SWIGLU);
     __host__ __device__ static constexpr bool bias_in_smem(bool out_bf16) { return HAS_BIAS && (!STORES || out_bf16); }
     __host__ __device__ static constexpr int bias_bytes(bool out_bf16) { return bias_in_smem(out_bf16) ? 2 * BN * 4 : 0; }
+    static constexpr int BIAS_OFFSET = (NUM_BARRIERS * 8 + 16 + 15) / 16 * 16;     // from the first barrier
     __host__ __device__ static constexpr int smem_bytes(bool out_bf16) {
-        return STAGES * STAGE_BYTES + staging_bytes(out_bf16) + NUM_BARRIERS * 8 + 16 + bias_bytes(out_bf16) + 1024;
+        return STAGES * STAGE_BYTES + staging_bytes(out_bf16) + BIAS_OFFSET + bias_bytes(out_bf16) + 1024;
     }
     static constexpr int THREADS = 64 + 32 * WARPS_EPI;
     static_assert(smem_bytes(true) <= 227 * 1024 && smem_bytes(false) <= 227 * 1024, "shared memory per CTA");
@@ -68,10 +69,13 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     const uint32_t accf_bar = bar_base + 8u * (2 * STAGES);
     const uint32_t acce_bar = bar_base + 8u * (2 * STAGES + 1);
+    const uint32_t bias_bar = bar_base + 8u * (2 * STAGES + 2);      // every epilogue warp has written its part of the tile's bias
     uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
-    float* bias_s = reinterpret_cast<float*>(ctrl + 16);                      // [2][BN], if Cfg::bias_in_smem
+    // [2][BN] floats if Cfg::bias_in_smem, read as float4: on the next 16-byte boundary after the control words
+    float* bias_s = reinterpret_cast<float*>(smem_raw + (bar_base - raw_addr) + Cfg::BIAS_OFFSET);
+    static_assert(Cfg::BIAS_OFFSET % 16 == 0 && Cfg::BIAS_OFFSET >= 8 * Cfg::NUM_BARRIERS + 16, "bias copy: aligned, after the control words");
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -83,6 +87,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(accf_bar, 1);
         mbar_init(acce_bar, 2 * Cfg::WARPS_EPI);         // every epilogue warp of both CTAs
+        mbar_init(bias_bar, Cfg::WARPS_EPI);
         *abort_flag = 0u;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -186,16 +191,19 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             float* bias_tile = nullptr;
             if (BIAS_S) {
                 // while the mainloop runs: the tile's bias into shared memory (the other copy may still be read by a
-                // warp that is finishing the previous tile; nobody is more than one tile ahead, see the barrier below)
+                // warp that is finishing the previous tile; nobody gets more than one tile ahead: the wait on `bias_bar`
+                // below needs every warp's arrival for this tile)
                 bias_tile = bias_s + acc_ph * Cfg::BN;
                 const int n = nb * Cfg::OUT_TILE_N + et;
                 bias_tile[et] = (p.bias != nullptr && n < p.N) ? __ldg(p.bias + n) : 0.0f;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bias_bar);
             }
             if (!mbar_wait(accf_bar, acc_ph, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 6u)) { ok = false; break; }
             acc_ph ^= 1u;
             tc_fence_after();
-            // every epilogue warp has passed the same accumulator-full wait, so all of them reach this barrier
-            if (BIAS_S) asm volatile("bar.sync 1, 256;" ::: "memory");
+            // the other warps' parts of the bias copy (an mbarrier, so that this wait is bounded like every other)
+            if (BIAS_S && !mbar_wait(bias_bar, acc_ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 0xAu)) { ok = false; break; }
             epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, 0, Cfg::OUT_TILE_N / 32, Cfg::OUT_TILE_N, nb, 0, 0, vec_ok,
                                          smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * Cfg::stage_bytes_per_warp(OUT_BF16), lane,
                                          bias_tile);

@@ -362,22 +362,32 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             else if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, false);
         }
     } else if (EPI == EPI_ROWMAX) {
+        // Four interleaved (max, column) chains per chunk, merged with the tie rule (the lower column wins), and
+        // the next chunk's TMEM load in flight meanwhile.
         float mx = -INFINITY;
         int arg = 0x7fffffff;
+        const int live = min(c_end, (p.N - n_tile0 + 31) / 32);
+        uint32_t r[32];
+        if (c_begin < live) tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
 #pragma unroll 1
-        for (int c = c_begin; c < c_end; ++c) {
+        for (int c = c_begin; c < live; ++c) {
             const int n0 = n_tile0 + c * 32;
-            if (n0 >= p.N) break;
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_addr + c * 32, r);
             float bv[32];
             tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
+            float z[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float z = (n0 + j < p.N) ? fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]) : -INFINITY;   // scale 1: the same bits as r + b
-                if (z > mx) { mx = z; arg = n0 + j; }        // strict: ties keep the lower column
-            }
+            for (int j = 0; j < 32; ++j)
+                z[j] = (n0 + j < p.N) ? fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]) : -INFINITY;   // scale 1: the same bits as r + b
+            if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            int a4[4] = {0x7fffffff, 0x7fffffff, 0x7fffffff, 0x7fffffff};
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (z[j] > m4[j & 3]) { m4[j & 3] = z[j]; a4[j & 3] = n0 + j; }      // strict: ties keep the lower column of the chain
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (m4[k] > mx || (m4[k] == mx && a4[k] < arg)) { mx = m4[k]; arg = a4[k]; }
         }
         if (row < p.M)
             p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] = make_float2(mx, __int_as_float(arg));
@@ -390,27 +400,32 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         float tz = 0.0f;
         bool found = false;
         if (EPI == EPI_XENT && row < p.M) tgt = static_cast<int>(p.targets[row]);
+        // Chunks that start inside [0, N); the TMEM load of chunk c + 1 is issued as soon as chunk c has been
+        // turned into logits, and the maxima and sums run as four interleaved chains (32-long dependent chains
+        // are what an epilogue warp otherwise spends its time on, visibly so when the epilogue is not overlapped).
+        int live = min(c_end, (p.N - n_tile0 + 31) / 32);
+        uint32_t r[32];
+        if (c_begin < live) tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
 #pragma unroll 1
-        for (int c = c_begin; c < c_end; ++c) {
+        for (int c = c_begin; c < live; ++c) {
             const int n0 = n_tile0 + c * 32;
-            if (n0 >= p.N) break;
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_addr + c * 32, r);
             float bv[32], tv[32];
             tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
-            float cm = -INFINITY;
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
                 tv[j] = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);
-                cm = fmaxf(cm, tv[j]);
+                m4[j & 3] = fmaxf(m4[j & 3], tv[j]);
             }
+            if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);      // r is free again
             if (n0 + 32 > p.N) {      // ragged last chunk: columns past N are zero-filled weight rows, mask them out
-                cm = -INFINITY;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) m4[k] = -INFINITY;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     if (n0 + j >= p.N) tv[j] = -INFINITY;
-                    cm = fmaxf(cm, tv[j]);
+                    m4[j & 3] = fmaxf(m4[j & 3], tv[j]);
                 }
             }
             if (EPI == EPI_XENT) {
@@ -422,11 +437,11 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
                     found = true;
                 }
             }
-            const float nm = fmaxf(mx, cm);
-            float cs = 0.0f;
+            const float nm = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) cs += ex2_approx(tv[j] - nm);
-            sum = sum * ex2_approx(mx - nm) + cs;
+            for (int j = 0; j < 32; ++j) s4[j & 3] += ex2_approx(tv[j] - nm);
+            sum = sum * ex2_approx(mx - nm) + ((s4[0] + s4[1]) + (s4[2] + s4[3]));
             mx = nm;
         }
         // a piece that lies wholly past N (only possible in the last column tile) stays neutral
