@@ -84,6 +84,16 @@ int mtmc_fused_linear(const void* X, const void* W, const float* b,
 int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, const void* R,
                                int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 
+/* mtmc_fused_linear on row-major views that are not dense: rows of X, W and out lie ldx, ldw
+ * and ldo elements apart (a column slice of a wider matrix, one projection inside a fused
+ * QKV weight, an output written straight into a concatenated buffer).  ldx, ldw >= K and
+ * multiples of 8 (TMA wants 16-byte row pitches); ldo >= N, any value -- vector stores need
+ * ldo % 8 == 0 (bf16) or ldo % 4 == 0 (fp32), otherwise rows are written element by element.
+ * Everything else as for mtmc_fused_linear: same kernels, same results.  The paper's operators
+ * take framework tensors, which may be such views. */
+int mtmc_fused_linear_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b,
+                              int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out, int64_t ldo);
+
 /* The same layer with 8-bit floating-point operands:
  *   out[m][n] = act( scale_x * scale_w * sum_k X8[m][k] W8[n][k] + b[n] ).
  * X8 [M,K] and W8 [N,K] hold E4M3 values (1 sign, 4 exponent bits with bias 7, 3 mantissa

@@ -27,7 +27,7 @@ EXPORTS = [
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -58,6 +58,7 @@ def load() -> ctypes.CDLL:
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    L.mtmc_fused_linear_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, i64]
     L.mtmc_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     L.mtmc_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
@@ -129,6 +130,31 @@ def mtmc_fused_linear_residual(X, W, b, R, act="none", out_dtype="bf16", out=Non
                                              None if b is None else _dev(b, torch.float32, (N,), "b"),
                                              _dev(R, odt, (M, N), "R"), M, N, K, ACT[act], OUT_DTYPE[out_dtype],
                                              _dev(out, odt, (M, N), "out")))
+    return out
+
+
+def _view2d(t: torch.Tensor, dtype, shape, name: str):
+    """Device pointer and row pitch (elements) of a 2-D CUDA tensor whose rows are contiguous."""
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype or tuple(t.shape) != tuple(shape) or t.stride(1) != 1 or t.stride(0) < t.shape[1]:
+        raise TypeError("%s must be %s of shape %r with unit column stride (got %s %r, strides %r)" % (
+            name, dtype, tuple(shape), t.dtype, tuple(t.shape), tuple(t.stride())))
+    return t.data_ptr(), t.stride(0)
+
+
+def mtmc_fused_linear_strided(X, W, b, act="none", out_dtype="bf16", out=None):
+    """mtmc_fused_linear on views: X [M,K], W [N,K] and out [M,N] may be column slices of wider row-major tensors."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (wp, ldw), (op, ldo) = _view2d(X, torch.bfloat16, (M, K), "X"), _view2d(W, torch.bfloat16, (N, K), "W"), \
+        _view2d(out, odt, (M, N), "out")
+    _check(load().mtmc_fused_linear_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                            M, N, K, ACT[act], OUT_DTYPE[out_dtype], op, ldo))
     return out
 
 

@@ -116,9 +116,9 @@ int get_device(DeviceState** out, int* dev_out = nullptr) {
 }
 
 // 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
-int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
+int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
     cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld > 0 ? ld : cols) * 2};      // row pitch in bytes
     cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -129,9 +129,9 @@ int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols
 }
 
 // 2-D E4M3 row-major [rows, cols] tensor (one byte per element), box = 128 columns x box_rows rows.
-int encode_u8_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows) {
+int encode_u8_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
     cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld > 0 ? ld : cols)};
     cuuint32_t box[2] = {128u, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
@@ -455,6 +455,7 @@ bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
 void fill_tiling(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int sm_count, bool split_tail, int bm = 128,
                  bool fp8 = false) {
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.ldo = p.N;
     p.m_tiles = static_cast<int>((M + bm - 1) / bm);
     p.rows_per_tile = bm;
     p.n_tiles = static_cast<int>((N + out_tile_n - 1) / out_tile_n);
@@ -606,12 +607,14 @@ int skinny_pairs(DeviceState* d) {
 }
 
 int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K,
-               int act, int out_dtype, void* out, bool fp8 = false, float acc_scale = 1.0f) {
+               int act, int out_dtype, void* out, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0,
+               int64_t ldo = 0) {
     SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, fp8 ? 128 : 64);
     SkinnyParams p;
     p.acc_scale = acc_scale;
     p.early_w = t_static_weights;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
+    p.ldo = static_cast<int>(ldo > 0 ? ldo : N);
     p.n_tiles = s.n_tiles; p.k_blocks = s.k_blocks; p.total_units = s.total; p.max_slots = s.max_slots;
     p.tile_rows = s.tile_rows; p.num_stages = s.stages;
     p.act = act; p.bias = b; p.residual = R; p.out = out; p.status = d->status;
@@ -633,9 +636,9 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
         }
     }
     CUtensorMap tmW, tmX;
-    int rc = fp8 ? encode_u8_2d(&tmW, W, N, K, s.tile_rows) : encode_bf16_2d(&tmW, W, N, K, s.tile_rows);
+    int rc = fp8 ? encode_u8_2d(&tmW, W, N, K, s.tile_rows) : encode_bf16_2d(&tmW, W, N, K, s.tile_rows, ldw);
     if (rc) return rc;
-    rc = fp8 ? encode_u8_2d(&tmX, X, M, K, s.mx) : encode_bf16_2d(&tmX, X, M, K, s.mx);
+    rc = fp8 ? encode_u8_2d(&tmX, X, M, K, s.mx) : encode_bf16_2d(&tmX, X, M, K, s.mx, ldx);
     if (rc) return rc;
     TimedRegion tr(d);
     const bool bf = out_dtype == MTMC_OUT_BF16;
@@ -701,8 +704,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
     if (EPI == EPI_XENT) CUDA_TRY(cudaMemsetAsync(p.target_logit, 0xFF, static_cast<size_t>(M) * sizeof(float), t_stream));
     CUtensorMap tmA, tmB, tmBt;
-    if ((rc = encode(&tmA, X, M, K, big ? 256 : 128)) || (rc = encode(&tmB, W, N, K, (pair || big) ? 128 : bn)) ||
-        (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width)))
+    if ((rc = encode(&tmA, X, M, K, big ? 256 : 128, 0)) || (rc = encode(&tmB, W, N, K, (pair || big) ? 128 : bn, 0)) ||
+        (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width, 0)))
         return rc;
     TimedRegion tr(d);
     if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
@@ -727,7 +730,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
 // out = act(X.W^T + b) (+ R): picks the weight-streaming path for decode batches, CTA pairs for
 // large shapes and single-CTA tiles otherwise.
 int fused_linear_impl(const void* X, const void* W, const float* b, const void* R, int64_t M, int64_t N, int64_t K, int act,
-                      int out_dtype, void* out) {
+                      int out_dtype, void* out, int64_t ldx = 0, int64_t ldw = 0, int64_t ldo = 0) {
     int rc = check_common(X, W, out, M, N, K);
     if (rc) return rc;
     if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
@@ -736,14 +739,14 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out);
+    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
 
     if (const int ks = pick_ksplit(d, M, N, K, 256, false)) {
         GemmParams p{};
         fill_ksplit(p, M, N, K, 256, ks, false);
-        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 256))) return rc;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, 256, ldw))) return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
         tr.stop();
@@ -752,9 +755,9 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     if (use_big(d, M, N, K, false)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512);
-        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 256)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128))) return rc;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 256, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128, ldw))) return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_big<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, p)
                                         : launch_big<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB, p);
@@ -764,10 +767,10 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     if (use_pair(d, M, N)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
-        p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB, tmBt;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128)) ||
-            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2)))
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128, ldw)) ||
+            (rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width / 2, ldw)))
             return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
@@ -778,13 +781,13 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     const int bn = pick_tile_n(N);
     GemmParams p{};
     fill_tiling(p, M, N, K, bn, d->sm_count, true);
-    p.act = act; p.bias = b; p.residual = R; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+    p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
     CUtensorMap tmA, tmB, tmBt;
-    rc = encode_bf16_2d(&tmA, X, M, K, 128);
+    rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx);
     if (rc) return rc;
-    rc = encode_bf16_2d(&tmB, W, N, K, bn);
+    rc = encode_bf16_2d(&tmB, W, N, K, bn, ldw);
     if (rc) return rc;
-    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width);
+    rc = encode_bf16_2d(&tmBt, W, N, K, p.tail_width, ldw);
     if (rc) return rc;
     TimedRegion tr(d);
     if (bn == 256) {
@@ -813,8 +816,8 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         p.acc_scale = sg; p.acc_scale2 = su;
         p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU;
-        if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmG, Wg, N, K, 128)) ||
-            (rc = encode(&tmU, Wu, N, K, 128)))
+        if ((rc = encode(&tmA, X, M, K, 128, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) ||
+            (rc = encode(&tmU, Wu, N, K, 128, 0)))
             return rc;
         TimedRegion tr(d);
         rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
@@ -827,9 +830,9 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         p.acc_scale = sg; p.acc_scale2 = su;
         p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-        if ((rc = encode(&tmA, X, M, K, 128)) || (rc = encode(&tmG, Wg, N, K, 128)) ||
-            (rc = encode(&tmU, Wu, N, K, 128)) || (rc = encode(&tmGt, Wg, N, K, p.tail_width)) ||
-            (rc = encode(&tmUt, Wu, N, K, p.tail_width)))
+        if ((rc = encode(&tmA, X, M, K, 128, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) ||
+            (rc = encode(&tmU, Wu, N, K, 128, 0)) || (rc = encode(&tmGt, Wg, N, K, p.tail_width, 0)) ||
+            (rc = encode(&tmUt, Wu, N, K, p.tail_width, 0)))
             return rc;
         TimedRegion tr(d);
         rc = launch_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, tmGt, tmUt, p);
@@ -841,15 +844,15 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     p.acc_scale = sg; p.acc_scale2 = su;
         p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
     CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-    rc = encode(&tmA, X, M, K, 128);
+    rc = encode(&tmA, X, M, K, 128, 0);
     if (rc) return rc;
-    rc = encode(&tmG, Wg, N, K, 128);
+    rc = encode(&tmG, Wg, N, K, 128, 0);
     if (rc) return rc;
-    rc = encode(&tmU, Wu, N, K, 128);
+    rc = encode(&tmU, Wu, N, K, 128, 0);
     if (rc) return rc;
-    rc = encode(&tmGt, Wg, N, K, p.tail_width);
+    rc = encode(&tmGt, Wg, N, K, p.tail_width, 0);
     if (rc) return rc;
-    rc = encode(&tmUt, Wu, N, K, p.tail_width);
+    rc = encode(&tmUt, Wu, N, K, p.tail_width, 0);
     if (rc) return rc;
     TimedRegion tr(d);
     rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
@@ -956,6 +959,14 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
     if (!R) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
     if (!aligned16(R)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
     return fused_linear_impl(X, W, b, R, M, N, K, act, out_dtype, out);
+}
+
+int mtmc_fused_linear_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, int64_t M, int64_t N,
+                              int64_t K, int act, int out_dtype, void* out, int64_t ldo) {
+    if (ldx < K || ldw < K || ldo < N) return fail(MTMC_ERR_INVALID_ARG, "row pitches must cover the rows (ldx, ldw >= K, ldo >= N)");
+    if (ldx % 8 != 0 || ldw % 8 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "ldx and ldw must be multiples of 8 elements (16-byte rows for TMA)");
+    if (ldx >= (1ll << 31) || ldw >= (1ll << 31) || ldo >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "row pitches must be below 2^31");
+    return fused_linear_impl(X, W, b, nullptr, M, N, K, act, out_dtype, out, ldx, ldw, ldo);
 }
 
 int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,

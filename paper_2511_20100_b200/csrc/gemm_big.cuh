@@ -179,7 +179,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int hh = (warp - 2) >> 2;              // row half of the CTA's 256 rows = accumulator column block
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(hh * Cfg::BN);
-        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);
         constexpr bool BIAS_S = Cfg::bias_in_smem(OUT_BF16);
         const int et = static_cast<int>(threadIdx.x) - 64;       // 0 .. 255: this thread's column of the tile's bias
         uint32_t acc_ph = 0;

@@ -158,7 +158,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t t_addr = tmem_base + lane_base;
         const int sw = lane & 7;                     // the eight 16-byte pieces of a row sit at piece ^ (row & 7)
-        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);
         // Accumulator chunk held at place `loc` of the receive buffer of CTA `owner`: output chunk
         // owner * OWN_OC + loc % OWN_OC of the gate / only half (loc < OWN_OC) or of the up half.
         auto acc_chunk = [&](int owner, int loc) { return (loc / Cfg::OWN_OC) * Cfg::OC + owner * Cfg::OWN_OC + loc % Cfg::OWN_OC; };

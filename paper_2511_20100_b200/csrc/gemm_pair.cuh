@@ -158,7 +158,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;            // which half of the item's columns this warp takes
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
-        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);
         uint32_t acc_ph = 0;
         int it = 0;
         bool ok = true;

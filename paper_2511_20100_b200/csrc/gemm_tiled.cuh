@@ -49,7 +49,8 @@ struct GemmParams {
     float acc_scale2;     // the same for the up half of a SwiGLU accumulator (acc_scale is then the gate half's)
     const float* bias;    // [N] or null
     const void* residual; // [M,N] in the output's element type, added after the activation, or null (EPI_ACT)
-    void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU)
+    void* out;            // [M,N] fp32 / bf16 (EPI_ACT, EPI_SWIGLU), rows `ldo` elements apart
+    int ldo;              // row pitch of out in elements (N for a dense output)
     float2* lse_partial;  // [n_tiles * tail_split * EPI_HALVES][M] per row, column piece and share of the piece: (max, sum-exp) for EPI_LSE / EPI_XENT,
                           // (max, index bits) for EPI_ROWMAX
     const long long* targets;   // [M] target column per row (EPI_XENT)
@@ -149,9 +150,9 @@ __device__ __forceinline__ void apply_act_chunk(int act, float (&y)[32]) {
 // Stores 32 consecutive columns [n0, n0+32) of one output row; 128-bit stores when
 // the row segment is whole and 16-byte aligned, predicated scalar stores otherwise.
 template <bool OUT_BF16>
-__device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int N, const float (&y)[32], bool vec_ok) {
+__device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int N, int ld, const float (&y)[32], bool vec_ok) {
     if (OUT_BF16) {
-        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * N + n0;
+        __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(out) + static_cast<size_t>(row) * ld + n0;
         if (vec_ok && n0 + 32 <= N) {
             uint4* o4 = reinterpret_cast<uint4*>(o);
 #pragma unroll
@@ -169,7 +170,7 @@ __device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int 
                 if (n0 + j < N) o[j] = __float2bfloat16_rn(y[j]);
         }
     } else {
-        float* o = reinterpret_cast<float*>(out) + static_cast<size_t>(row) * N + n0;
+        float* o = reinterpret_cast<float*>(out) + static_cast<size_t>(row) * ld + n0;
         if (vec_ok && n0 + 32 <= N) {
             float4* o4 = reinterpret_cast<float4*>(o);
 #pragma unroll
@@ -189,7 +190,7 @@ __device__ __forceinline__ void store_row_chunk(void* out, int row, int n0, int 
 // Requires the chunk to lie wholly inside [0, N) and 16-byte aligned rows; rows >= M are
 // not stored.  `row0` is the output row of lane 0.
 template <bool OUT_BF16>
-__device__ __forceinline__ void store_chunk_coalesced(uint8_t* stage, void* out, int row0, int n0, int M, int N,
+__device__ __forceinline__ void store_chunk_coalesced(uint8_t* stage, void* out, int row0, int n0, int M, int ld,
                                                       const float (&y)[32], int lane) {
     constexpr int UNITS = OUT_BF16 ? 4 : 8;                  // 16-byte units per row of the chunk
     constexpr int ROW_BYTES = UNITS * 16;
@@ -222,7 +223,7 @@ __device__ __forceinline__ void store_chunk_coalesced(uint8_t* stage, void* out,
         const int rkey = OUT_BF16 ? ((r >> 1) & 3) : (r & 7);
         const uint4 q = *reinterpret_cast<const uint4*>(stage + r * ROW_BYTES + ((unit ^ rkey) * 16));
         if (row0 + r < M) {
-            uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (static_cast<size_t>(row0 + r) * N + n0) * elem + unit * 16;
+            uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (static_cast<size_t>(row0 + r) * ld + n0) * elem + unit * 16;
             *reinterpret_cast<uint4*>(dst) = q;
         }
     }
@@ -336,8 +337,8 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             }
             apply_act_chunk<OUT_BF16>(p.act, y);
             if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
-            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
-            else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, y, false);
+            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.ldo, y, lane);
+            else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, p.ldo, y, false);
         }
     } else if (EPI == EPI_SWIGLU) {
 #pragma unroll 1
@@ -358,8 +359,8 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             }
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
-            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<true>(stage, p.out, row - lane, n0, p.M, p.N, y, lane);
-            else if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, y, false);
+            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<true>(stage, p.out, row - lane, n0, p.M, p.ldo, y, lane);
+            else if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, p.ldo, y, false);
         }
     } else if (EPI == EPI_ROWMAX) {
         // Four interleaved (max, column) chains per chunk, merged with the tie rule (the lower column wins), and
@@ -572,7 +573,7 @@ gemm_tiled_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const int half = (warp - 2) >> 2;            // which half of the item's columns this warp takes
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
-        const bool vec_ok = OUT_BF16 ? (p.N % 8 == 0) : (p.N % 4 == 0);
+        const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);       // 16-byte aligned rows of out (and of a dense residual)
         uint32_t acc_ph = 0;
         int it = 0;
         bool ok = true;

@@ -45,6 +45,7 @@ struct SkinnyParams {
     const float* bias;
     const void* residual;    // [M,N] in the output's element type, added after the activation, or null
     void* out;
+    int ldo;                 // row pitch of out (and of the residual) in elements; N when dense
     float* partial;          // [n_tiles][max_slots][MX][128] fp32
     uint32_t* tickets;       // [n_tiles], zero between launches
     uint32_t* status;
@@ -108,7 +109,7 @@ __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, 
 // out[m][n] = y (+ R[m][n]), rounded once to the output type.
 template <bool OUT_BF16>
 __device__ __forceinline__ void skinny_store(const SkinnyParams& p, int m, int n, float y) {
-    const size_t idx = static_cast<size_t>(m) * p.N + n;
+    const size_t idx = static_cast<size_t>(m) * p.ldo + n;
     if (OUT_BF16) {
         if (p.residual) y += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.residual)[idx]);
         reinterpret_cast<__nv_bfloat16*>(p.out)[idx] = __float2bfloat16_rn(y);

@@ -143,6 +143,29 @@ def test_large_tile_pair_kernel_row_reductions(M, N, K):
     _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "cross entropy, 512-row tiles")
 
 
+@pytest.mark.parametrize("M,N,K,padx,padw,pado", [(5, 300, 512, 64, 8, 20), (100, 72, 136, 8, 24, 3), (300, 520, 328, 16, 8, 8),
+                                                  (128, 1024, 4096, 64, 64, 1024), (1100, 1300, 1024, 8, 8, 4), (600, 520, 6144, 8, 16, 0)])
+@pytest.mark.parametrize("act,odt", [("gelu_tanh", "bf16"), ("none", "fp32")])
+def test_fused_linear_strided_views(M, N, K, padx, padw, pado, act, odt):
+    """Column slices of wider matrices as X, W and out, on the weight-streaming, single-CTA, cluster split-K and
+    CTA-pair kernels; the columns of the wide output outside the slice must stay untouched."""
+    li = inputs.linear_inputs(M, N, K, seed=9000 + M + N)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[act])
+    tdt = torch.bfloat16 if odt == "bf16" else torch.float32
+    Xw = torch.full((M, K + padx), 3.0, dtype=torch.bfloat16, device="cuda")
+    Ww = torch.full((N, K + padw), -2.0, dtype=torch.bfloat16, device="cuda")
+    Ow = torch.full((M, N + pado), 7.0, dtype=tdt, device="cuda")
+    offx, offw, offo = (8 if padx >= 16 else 0), (8 if padw >= 16 else 0), (8 if pado >= 16 else 0)
+    Xv, Wv, Ov = Xw[:, offx:offx + K], Ww[:, offw:offw + K], Ow[:, offo:offo + N]
+    Xv.copy_(li.X.cuda()); Wv.copy_(li.W.cuda())
+    B.mtmc_fused_linear_strided(Xv, Wv, li.b.cuda(), act, odt, out=Ov)
+    B.mtmc_check_status()
+    _assert_close(inputs.to_f64(Ov.contiguous()), want, TOL[odt], "strided %dx%dx%d %s" % (M, N, K, odt))
+    assert bool((Ow[:, :offo] == 7.0).all()) and bool((Ow[:, offo + N:] == 7.0).all())
+    dense = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), act, odt)
+    assert torch.equal(dense, Ov.contiguous())              # the same kernels on the same values
+
+
 def test_large_tile_pair_kernel_chosen_for_long_k():
     """From 96 k-blocks on the 512 x 256 tiles are the default for M >= 512, N >= 256: bf16, residual and FP8 forms."""
     M, N, K = 600, 520, 6144
