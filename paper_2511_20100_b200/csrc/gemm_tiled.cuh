@@ -341,13 +341,17 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, p.ldo, y, false);
         }
     } else if (EPI == EPI_SWIGLU) {
+        // As for the activation epilogue: the gate and up loads of chunk c + 1 go out as soon as chunk c has been
+        // combined, so that they are under way during its stores.
+        const int live = min(c_end, (p.N - n_tile0 + 31) / 32);
+        uint32_t g[32], u[32];
+        if (c_begin < live) {
+            tmem_ld_32x32b_x32(t_addr + c_begin * 32, g);            // gate columns
+            tmem_ld_32x32b_x32(t_addr + width + c_begin * 32, u);    // up columns follow the gate columns
+        }
 #pragma unroll 1
-        for (int c = c_begin; c < c_end; ++c) {
+        for (int c = c_begin; c < live; ++c) {
             const int n0 = n_tile0 + c * 32;
-            if (n0 >= p.N) break;
-            uint32_t g[32], u[32];
-            tmem_ld_32x32b_x32(t_addr + c * 32, g);                 // gate columns
-            tmem_ld_32x32b_x32(t_addr + width + c * 32, u);         // up columns follow the gate columns
             tmem_ld_wait();
             float y[32];
             if (p.fp8) {                                            // E4M3 operands: the per-tensor scales of gate and up
@@ -359,6 +363,10 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             }
 #pragma unroll
             for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+            if (c + 1 < live) {
+                tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, g);
+                tmem_ld_32x32b_x32(t_addr + width + (c + 1) * 32, u);
+            }
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<true>(stage, p.out, row - lane, n0, p.M, p.ldo, y, lane);
             else if (row < p.M) store_row_chunk<true>(p.out, row, n0, p.N, p.ldo, y, false);
         }
