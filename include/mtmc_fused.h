@@ -69,9 +69,12 @@ extern "C" {
  * the bias add and activation happen in fp32 on the fp32 accumulator, with no
  * intermediate rounding.)  X, W bf16; b fp32 or NULL; out fp32 or bf16 [M,N]
  * according to out_dtype.  Shapes with M <= 64 (decode batches) take the split-K
- * weight-streaming path (HBM-bound); all others the tiled tensor-core path.
- * Needs workspace only on the ticketed variant of the split-K path (few rows of W,
- * or a forced split; see mtmc_workspace_bytes). */
+ * weight-streaming path (HBM-bound); problems of at most half a wave of 128 x 256
+ * tiles with a long K a cluster split-K kernel (2, 4 or 8 CTAs per tile, reduction
+ * through distributed shared memory); all others the tiled tensor-core kernels
+ * (CTA pairs on 256 x 256 or 512 x 256 tiles for M >= 512 and N >= 256, single
+ * CTAs otherwise).  Needs workspace only on the ticketed variant of the
+ * weight-streaming path (few rows of W, or a forced split; see mtmc_workspace_bytes). */
 int mtmc_fused_linear(const void* X, const void* W, const float* b,
                       int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
 
@@ -245,9 +248,10 @@ float mtmc_last_kernel_ms(void);
  *              size of the cluster split-K kernel (1 = never use that kernel)
  *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
  *   cta_pair : 1 forces the CTA-pair (cta_group::2) kernel with 256 x 256 tiles and overlapped
- *              epilogues, 2 the one with 512 x 256 tiles (activation epilogues; the other
- *              operators then take the 256 x 256 pair kernel), < 0 forbids both;
- *              automatic = pairs when M >= 512 and N >= 256, the large tiles for long K */
+ *              epilogues, 2 the one with 512 x 256 tiles (activation epilogues and row
+ *              reductions; SwiGLU then takes the 256 x 256 pair kernel), < 0 forbids both;
+ *              automatic = pairs when M >= 512 and N >= 256; the large tiles for the row
+ *              reductions and for activation epilogues with a long K */
 int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
 
 /* Static weights (thread-local, default 0 = off).  With enabled != 0 the caller promises, for
