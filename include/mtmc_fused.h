@@ -190,7 +190,7 @@ int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b,
 /* Same three operations with every pointer a HOST pointer (pageable or pinned).
  * The library copies the operands to device buffers it owns (cudaMalloc,
  * grow-only, per device), runs the device entry point on the current stream,
- * copies the result back and synchronises the stream before returning.  These
+ * copies the result back and waits for it before returning.  These
  * allocate and synchronise; they are a convenience for callers without device
  * memory management and the end-to-end leg of the benchmark.  (No counterpart in
  * the paper: its measurements are device-resident.) */
@@ -200,6 +200,23 @@ int mtmc_swiglu_host(const void* X, const void* Wg, const void* Wu,
                      int64_t M, int64_t N, int64_t K, void* out);
 int mtmc_linear_lse_host(const void* X, const void* W, const float* b,
                          int64_t M, int64_t N, int64_t K, float* lse_out);
+
+/* The same without waiting for the result: the call enqueues the copy in (on a copy stream of
+ * the library's), the kernels (on the current stream) and the copy out (on a second copy
+ * stream), chained by events, and returns.  Consecutive calls overlap -- the next call's
+ * operands travel to the device while this call computes and its result travels back --
+ * which is what a host-resident pipeline needs from a PCIe link that is slower than the
+ * kernels.  Host buffers should be pinned (pageable memory makes the copies synchronous)
+ * and must stay valid, and the result unread, until mtmc_host_sync() returns; at most six
+ * calls are in flight (a seventh first waits for the oldest).  mtmc_host_sync() waits for
+ * every call issued so far on the current device.  (No counterpart in the paper.) */
+int mtmc_fused_linear_host_async(const void* X, const void* W, const float* b,
+                                 int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+int mtmc_swiglu_host_async(const void* X, const void* Wg, const void* Wu,
+                           int64_t M, int64_t N, int64_t K, void* out);
+int mtmc_linear_lse_host_async(const void* X, const void* W, const float* b,
+                               int64_t M, int64_t N, int64_t K, float* lse_out);
+int mtmc_host_sync(void);
 
 /* Stream on which later calls from this host thread enqueue (a cudaStream_t;
  * NULL = legacy default stream).  Thread-local. */

@@ -25,6 +25,7 @@ EXPORTS = [
     "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_fused_linear_fp8", "mtmc_swiglu", "mtmc_linear_lse",
     "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
+    "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
     "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
@@ -54,14 +55,15 @@ def load() -> ctypes.CDLL:
                                "there is no fallback path" % (LIB_PATH, e))
     L = ctypes.CDLL(LIB_PATH)
     vp, i64, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
-    for name in ("mtmc_fused_linear", "mtmc_fused_linear_host"):
+    for name in ("mtmc_fused_linear", "mtmc_fused_linear_host", "mtmc_fused_linear_host_async"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, i64]
     L.mtmc_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     L.mtmc_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
-    for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_linear_lse", "mtmc_linear_lse_host", "mtmc_linear_lse_noalloc"):
+    for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_swiglu_host_async", "mtmc_linear_lse", "mtmc_linear_lse_host",
+                 "mtmc_linear_lse_host_async", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
@@ -283,41 +285,63 @@ def _host(t: torch.Tensor, dtype, shape, name: str) -> int:
     return t.data_ptr()
 
 
-def mtmc_fused_linear_host(X, W, b, act="none", out_dtype="bf16", out=None, device=0):
-    """Host-pointer variant: CPU tensors in, CPU tensor out; copies and synchronises inside the library."""
+def mtmc_fused_linear_host(X, W, b, act="none", out_dtype="bf16", out=None, device=0, blocking=True):
+    """Host-pointer variant: CPU tensors in, CPU tensor out; copies inside the library.  blocking=False returns at once
+    (pinned tensors; the result is valid after mtmc_host_sync())."""
     M, K = X.shape
     N = W.shape[0]
     odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
     if out is None:
         out = torch.empty((M, N), dtype=odt)
     _use_current_stream(torch.device("cuda", device))
-    _check(load().mtmc_fused_linear_host(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
-                                         None if b is None else _host(b, torch.float32, (N,), "b"),
-                                         M, N, K, ACT[act], OUT_DTYPE[out_dtype], _host(out, odt, (M, N), "out")))
+    fn = load().mtmc_fused_linear_host if blocking else load().mtmc_fused_linear_host_async
+    _check(fn(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
+              None if b is None else _host(b, torch.float32, (N,), "b"),
+              M, N, K, ACT[act], OUT_DTYPE[out_dtype], _host(out, odt, (M, N), "out")))
     return out
 
 
-def mtmc_swiglu_host(X, Wg, Wu, out=None, device=0):
+def mtmc_swiglu_host(X, Wg, Wu, out=None, device=0, blocking=True):
     M, K = X.shape
     N = Wg.shape[0]
     if out is None:
         out = torch.empty((M, N), dtype=torch.bfloat16)
     _use_current_stream(torch.device("cuda", device))
-    _check(load().mtmc_swiglu_host(_host(X, torch.bfloat16, (M, K), "X"), _host(Wg, torch.bfloat16, (N, K), "Wg"),
-                                   _host(Wu, torch.bfloat16, (N, K), "Wu"), M, N, K, _host(out, torch.bfloat16, (M, N), "out")))
+    fn = load().mtmc_swiglu_host if blocking else load().mtmc_swiglu_host_async
+    _check(fn(_host(X, torch.bfloat16, (M, K), "X"), _host(Wg, torch.bfloat16, (N, K), "Wg"),
+              _host(Wu, torch.bfloat16, (N, K), "Wu"), M, N, K, _host(out, torch.bfloat16, (M, N), "out")))
     return out
 
 
-def mtmc_linear_lse_host(X, W, b, lse_out=None, device=0):
+def mtmc_linear_lse_host(X, W, b, lse_out=None, device=0, blocking=True):
     M, K = X.shape
     N = W.shape[0]
     if lse_out is None:
         lse_out = torch.empty((M,), dtype=torch.float32)
     _use_current_stream(torch.device("cuda", device))
-    _check(load().mtmc_linear_lse_host(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
-                                       None if b is None else _host(b, torch.float32, (N,), "b"),
-                                       M, N, K, _host(lse_out, torch.float32, (M,), "lse_out")))
+    fn = load().mtmc_linear_lse_host if blocking else load().mtmc_linear_lse_host_async
+    _check(fn(_host(X, torch.bfloat16, (M, K), "X"), _host(W, torch.bfloat16, (N, K), "W"),
+              None if b is None else _host(b, torch.float32, (N,), "b"),
+              M, N, K, _host(lse_out, torch.float32, (M,), "lse_out")))
     return lse_out
+
+
+def mtmc_fused_linear_host_async(X, W, b, act="none", out_dtype="bf16", out=None, device=0):
+    """mtmc_fused_linear_host without waiting for the result (valid after mtmc_host_sync())."""
+    return mtmc_fused_linear_host(X, W, b, act, out_dtype, out=out, device=device, blocking=False)
+
+
+def mtmc_swiglu_host_async(X, Wg, Wu, out=None, device=0):
+    return mtmc_swiglu_host(X, Wg, Wu, out=out, device=device, blocking=False)
+
+
+def mtmc_linear_lse_host_async(X, W, b, lse_out=None, device=0):
+    return mtmc_linear_lse_host(X, W, b, lse_out=lse_out, device=device, blocking=False)
+
+
+def mtmc_host_sync() -> None:
+    """Waits for every non-blocking host-pointer call issued so far on the current device."""
+    _check(load().mtmc_host_sync())
 
 
 def mtmc_set_workspace(t: torch.Tensor | None) -> None:

@@ -39,8 +39,19 @@ struct DeviceState {
     bool tickets_dirty = false;
     void* ws = nullptr;              // library-owned workspace (grow-only)
     size_t ws_bytes = 0;
-    void* stage[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // device copies for the *_host calls
-    size_t stage_bytes[5] = {0, 0, 0, 0, 0};
+    // The *_host entry points: a ring of slots, each with device copies of one call's operands and result and
+    // the events that order its three phases (copy in, kernels, copy out) across three streams.
+    struct HostSlot {
+        void* buf[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+        size_t bytes[5] = {0, 0, 0, 0, 0};
+        cudaEvent_t in_done = nullptr, k_done = nullptr, out_done = nullptr;
+        bool busy = false;
+    };
+    static constexpr int HOST_SLOTS = 6;
+    HostSlot hslot[HOST_SLOTS];
+    int hnext = 0;
+    size_t hwm[5] = {0, 0, 0, 0, 0};
+    cudaStream_t s_in = nullptr, s_out = nullptr;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     bool timed = false;
     int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
@@ -412,28 +423,34 @@ bool use_pair(DeviceState* d, int64_t M, int64_t N) {
     return M >= 512 && N >= 256;
 }
 
+// Waves of 512 x 256 tiles against waves of 256 x 256 tiles, both counted in 256-row tile waves: the large tiles
+// must not lose to the last, partial wave more than they gain per FLOP (nothing at moderate K, up to a tenth
+// when K is long).  A problem of 32 large tiles on 74 pairs, say, stays on the small ones.
+bool big_waves_ok(int64_t M, int64_t N, int pairs, bool long_k) {
+    const int64_t n_tiles = (N + 255) / 256;
+    const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
+    const int64_t w_pair = (t_pair + pairs - 1) / pairs, w_big = 2 * ((t_big + pairs - 1) / pairs);
+    return long_k ? 10 * w_big <= 11 * w_pair : w_big <= w_pair;
+}
+
 // The 512 x 256 pair tiles (gemm_big.cuh) against the 256 x 256 ones with overlapped epilogues (gemm_pair.cuh).
 // Measured on plain and GELU epilogues: per FLOP the large tiles are on a par at K = 4096 and 5-15 % ahead from
 // K = 8192 on (a quarter less operand traffic, and the exposed epilogue shrinks against the k-walk); their
-// tiles are twice as large, so with few waves they can lose more to the last, partial wave.  Hence: always
-// from 96 k-blocks on, from 64 k-blocks on when their waves cost no more than the pair kernel's, counted in
-// 256-row tile waves.  Tuning hook: cta_pair = 2 forces them, 1 forces the 256 x 256 pair tiles.
+// tiles are twice as large, so with few waves they can lose more to the last, partial wave.  Hence: from 64
+// k-blocks on when their waves cost no more than the pair kernel's (a tenth more from 96 k-blocks on).  Tuning hook: cta_pair = 2 forces them, 1 forces the 256 x 256 pair tiles.
 bool use_big(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     const int pairs = gemm_pairs(d);
     if (pairs <= 0 || EPI_HALVES != 1 || t_tile_n != 0 || t_cta_pair < 0 || t_cta_pair == 1) return false;
     if (t_cta_pair == 2) return true;
     if (M < 512 || N < 256) return false;
     const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
-    if (k_blocks >= 96) return true;
     if (k_blocks < 64) return false;
-    const int64_t n_tiles = (N + 255) / 256;
-    const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
-    return 2 * ((t_big + pairs - 1) / pairs) <= (t_pair + pairs - 1) / pairs;
+    return big_waves_ok(M, N, pairs, k_blocks >= 96);
 }
 
 // The same choice for the row reductions (logsumexp, row max, cross entropy).  Their epilogues store one partial
 // per row, so little is exposed when it is not overlapped: the large tiles are 4-5 % ahead at K = 4096 already
-// (C4: 680-714 us against 710-750 us).  From 32 k-blocks on when their waves cost no more, always from 96 on.
+// (C4: 680-714 us against 710-750 us).  From 32 k-blocks on, under the same wave rule.
 // SwiGLU stays on the 256 x 256 tiles: its epilogue (two MUFU operations per element plus the stores) is too long
 // to expose (measured on C3: 2-3 % slower on the large tiles).
 bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
@@ -442,11 +459,8 @@ bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     if (t_cta_pair == 2) return true;
     if (M < 512 || N < 256) return false;
     const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
-    if (k_blocks >= 96) return true;
     if (k_blocks < 32) return false;
-    const int64_t n_tiles = (N + 255) / 256;
-    const int64_t t_pair = ((M + 255) / 256) * n_tiles, t_big = ((M + 511) / 512) * n_tiles;
-    return 2 * ((t_big + pairs - 1) / pairs) <= (t_pair + pairs - 1) / pairs;
+    return big_waves_ok(M, N, pairs, k_blocks >= 96);
 }
 
 // Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
@@ -659,17 +673,66 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
     return rc;
 }
 
-// Device buffer i of the *_host entry points, at least `bytes` large.
-int stage_buffer(DeviceState* d, int i, size_t bytes, void** out) {
-    std::lock_guard<std::mutex> lock(g_mutex);
-    if (d->stage_bytes[i] < bytes) {
-        if (d->stage[i]) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(d->stage[i])); d->stage[i] = nullptr; d->stage_bytes[i] = 0; }
-        CUDA_TRY(cudaMalloc(&d->stage[i], bytes));
-        d->stage_bytes[i] = bytes;
+// One call through host pointers.  `in[i]` / `out` give host address and size of each operand (a null address
+// skips it); `launch` enqueues the device entry point on the compute stream given the device copies.  The copy in
+// runs on its own stream, the kernels on the caller's stream, the copy out on a third, chained by events, so
+// consecutive calls overlap: the next call's operands travel while this call computes and its result travels
+// back.  A slot is reused only after its previous copy out has finished.  blocking: wait for the result.
+// Host threads that share a device should not interleave asynchronous calls (they would share slots).
+struct HostOperand { const void* host; size_t bytes; };
+template <class Launch>
+int host_call(const HostOperand (&in)[4], void* out_host, size_t out_bytes, bool blocking, Launch launch) {
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    DeviceState::HostSlot* slot = nullptr;
+    {   // the ring position is the only state shared between host threads; the device entry point takes the lock itself
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!d->s_in) {
+            CUDA_TRY(cudaStreamCreateWithFlags(&d->s_in, cudaStreamNonBlocking));
+            CUDA_TRY(cudaStreamCreateWithFlags(&d->s_out, cudaStreamNonBlocking));
+        }
+        slot = &d->hslot[d->hnext];
+        d->hnext = (d->hnext + 1) % DeviceState::HOST_SLOTS;
     }
-    *out = d->stage[i];
+    DeviceState::HostSlot& s = *slot;
+    if (!s.in_done) {
+        CUDA_TRY(cudaEventCreateWithFlags(&s.in_done, cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&s.k_done, cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&s.out_done, cudaEventDisableTiming));
+    }
+    if (s.busy) { CUDA_TRY(cudaEventSynchronize(s.out_done)); s.busy = false; }
+    void* dev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    for (int i = 0; i < 5; ++i) {
+        const size_t need = i < 4 ? (in[i].host ? in[i].bytes : 0) : out_bytes;
+        if (need == 0) continue;
+        if (d->hwm[i] < need) d->hwm[i] = need;      // largest operand seen in this position, by any slot
+        if (s.bytes[i] < need) {        // the slot is idle: nothing on the device still uses its buffers
+            if (s.buf[i]) { CUDA_TRY(cudaFree(s.buf[i])); s.buf[i] = nullptr; s.bytes[i] = 0; }
+            CUDA_TRY(cudaMalloc(&s.buf[i], d->hwm[i]));     // sized for the largest, so that a steady workload stops reallocating
+            s.bytes[i] = d->hwm[i];
+        }
+        dev[i] = s.buf[i];
+    }
+    for (int i = 0; i < 4; ++i)
+        if (dev[i]) CUDA_TRY(cudaMemcpyAsync(dev[i], in[i].host, in[i].bytes, cudaMemcpyHostToDevice, d->s_in));
+    CUDA_TRY(cudaEventRecord(s.in_done, d->s_in));
+    CUDA_TRY(cudaStreamWaitEvent(t_stream, s.in_done, 0));
+    rc = launch(dev);
+    if (rc) return rc;
+    CUDA_TRY(cudaEventRecord(s.k_done, t_stream));
+    CUDA_TRY(cudaStreamWaitEvent(d->s_out, s.k_done, 0));
+    CUDA_TRY(cudaMemcpyAsync(out_host, dev[4], out_bytes, cudaMemcpyDeviceToHost, d->s_out));
+    CUDA_TRY(cudaEventRecord(s.out_done, d->s_out));
+    s.busy = true;
+    if (blocking) { CUDA_TRY(cudaEventSynchronize(s.out_done)); s.busy = false; }
     return MTMC_OK;
 }
+
+int fused_linear_host_impl(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act, int out_dtype,
+                           void* out, bool blocking);
+int swiglu_host_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out, bool blocking);
+int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out, bool blocking);
 
 // The three row reductions over the never-materialised logits share one driver: a tiled kernel
 // leaves one partial per (row, column piece) in the workspace, a merge kernel finishes the rows.
@@ -858,6 +921,37 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
     tr.stop();
     return rc;
+}
+
+int fused_linear_host_impl(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act, int out_dtype,
+                           void* out, bool blocking) {
+    if (!X || !W || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
+    const size_t ob = static_cast<size_t>(M) * N * (out_dtype == MTMC_OUT_BF16 ? 2 : 4);
+    const HostOperand in[4] = {{X, xb}, {W, wb}, {nullptr, 0}, {b, bb}};
+    return host_call(in, out, ob, blocking, [&](void* const* dev) {
+        return mtmc_fused_linear(dev[0], dev[1], static_cast<const float*>(dev[3]), M, N, K, act, out_dtype, dev[4]);
+    });
+}
+
+int swiglu_host_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out, bool blocking) {
+    if (!X || !Wg || !Wu || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, ob = static_cast<size_t>(M) * N * 2;
+    const HostOperand in[4] = {{X, xb}, {Wg, wb}, {Wu, wb}, {nullptr, 0}};
+    return host_call(in, out, ob, blocking, [&](void* const* dev) { return mtmc_swiglu(dev[0], dev[1], dev[2], M, N, K, dev[4]); });
+}
+
+int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out, bool blocking) {
+    if (!X || !W || !lse_out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
+    const HostOperand in[4] = {{X, xb}, {W, wb}, {nullptr, 0}, {b, bb}};
+    return host_call(in, lse_out, static_cast<size_t>(M) * 4, blocking, [&](void* const* dev) {
+        return mtmc_linear_lse(dev[0], dev[1], static_cast<const float*>(dev[3]), M, N, K, static_cast<float*>(dev[4]));
+    });
 }
 
 }  // namespace
@@ -1190,66 +1284,31 @@ extern "C" {
 // ---------------------------------------------------------------------------- host-pointer variants
 int mtmc_fused_linear_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
                            int out_dtype, void* out) {
-    if (!X || !W || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
-    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
-    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
-    DeviceState* d = nullptr;
-    int rc = get_device(&d);
-    if (rc) return rc;
-    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
-    const size_t ob = static_cast<size_t>(M) * N * (out_dtype == MTMC_OUT_BF16 ? 2 : 4);
-    void *dX, *dW, *dB = nullptr, *dO;
-    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dW)) || (rc = stage_buffer(d, 4, ob, &dO))) return rc;
-    if (b && (rc = stage_buffer(d, 3, bb, &dB))) return rc;
-    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
-    CUDA_TRY(cudaMemcpyAsync(dW, W, wb, cudaMemcpyHostToDevice, t_stream));
-    if (b) CUDA_TRY(cudaMemcpyAsync(dB, b, bb, cudaMemcpyHostToDevice, t_stream));
-    rc = mtmc_fused_linear(dX, dW, static_cast<const float*>(dB), M, N, K, act, out_dtype, dO);
-    if (rc) return rc;
-    CUDA_TRY(cudaMemcpyAsync(out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
-    CUDA_TRY(cudaStreamSynchronize(t_stream));
-    return MTMC_OK;
+    return fused_linear_host_impl(X, W, b, M, N, K, act, out_dtype, out, true);
 }
-
 int mtmc_swiglu_host(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
-    if (!X || !Wg || !Wu || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
-    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
-    DeviceState* d = nullptr;
-    int rc = get_device(&d);
-    if (rc) return rc;
-    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, ob = static_cast<size_t>(M) * N * 2;
-    void *dX, *dG, *dU, *dO;
-    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dG)) || (rc = stage_buffer(d, 2, wb, &dU)) ||
-        (rc = stage_buffer(d, 4, ob, &dO)))
-        return rc;
-    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
-    CUDA_TRY(cudaMemcpyAsync(dG, Wg, wb, cudaMemcpyHostToDevice, t_stream));
-    CUDA_TRY(cudaMemcpyAsync(dU, Wu, wb, cudaMemcpyHostToDevice, t_stream));
-    rc = mtmc_swiglu(dX, dG, dU, M, N, K, dO);
-    if (rc) return rc;
-    CUDA_TRY(cudaMemcpyAsync(out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
-    CUDA_TRY(cudaStreamSynchronize(t_stream));
-    return MTMC_OK;
+    return swiglu_host_impl(X, Wg, Wu, M, N, K, out, true);
+}
+int mtmc_linear_lse_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
+    return linear_lse_host_impl(X, W, b, M, N, K, lse_out, true);
+}
+int mtmc_fused_linear_host_async(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
+                                 int out_dtype, void* out) {
+    return fused_linear_host_impl(X, W, b, M, N, K, act, out_dtype, out, false);
+}
+int mtmc_swiglu_host_async(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {
+    return swiglu_host_impl(X, Wg, Wu, M, N, K, out, false);
+}
+int mtmc_linear_lse_host_async(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
+    return linear_lse_host_impl(X, W, b, M, N, K, lse_out, false);
 }
 
-int mtmc_linear_lse_host(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, float* lse_out) {
-    if (!X || !W || !lse_out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
-    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+int mtmc_host_sync(void) {
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    const size_t xb = static_cast<size_t>(M) * K * 2, wb = static_cast<size_t>(N) * K * 2, bb = static_cast<size_t>(N) * 4;
-    const size_t ob = static_cast<size_t>(M) * 4;
-    void *dX, *dW, *dB = nullptr, *dO;
-    if ((rc = stage_buffer(d, 0, xb, &dX)) || (rc = stage_buffer(d, 1, wb, &dW)) || (rc = stage_buffer(d, 4, ob, &dO))) return rc;
-    if (b && (rc = stage_buffer(d, 3, bb, &dB))) return rc;
-    CUDA_TRY(cudaMemcpyAsync(dX, X, xb, cudaMemcpyHostToDevice, t_stream));
-    CUDA_TRY(cudaMemcpyAsync(dW, W, wb, cudaMemcpyHostToDevice, t_stream));
-    if (b) CUDA_TRY(cudaMemcpyAsync(dB, b, bb, cudaMemcpyHostToDevice, t_stream));
-    rc = mtmc_linear_lse(dX, dW, static_cast<const float*>(dB), M, N, K, static_cast<float*>(dO));
-    if (rc) return rc;
-    CUDA_TRY(cudaMemcpyAsync(lse_out, dO, ob, cudaMemcpyDeviceToHost, t_stream));
-    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    for (auto& s : d->hslot)
+        if (s.busy) { CUDA_TRY(cudaEventSynchronize(s.out_done)); s.busy = false; }
     return MTMC_OK;
 }
 

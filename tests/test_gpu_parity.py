@@ -708,3 +708,34 @@ def test_host_pointer_entry_points():
     sw = B.mtmc_swiglu_host(si.X, si.Wg, si.Wu)
     _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
                   TOL["bf16"], "swiglu_host")
+
+
+def test_host_pointer_calls_without_waiting():
+    """Ten calls of mixed shapes through the host-pointer pipeline without waiting in between (more than its six slots,
+    so slots are reused while earlier calls are in flight), one wait at the end; every result against the oracle."""
+    shapes = [(150, 264, 128), (64, 1024, 512), (300, 520, 200), (16, 512, 1024), (129, 257, 72)]
+    jobs = []
+    for rep in range(2):
+        for i, (M, N, K) in enumerate(shapes):
+            li = inputs.linear_inputs(M, N, K, seed=9100 + 10 * rep + i)
+            X, W, b = li.X.pin_memory(), li.W.pin_memory(), li.b.pin_memory()
+            if i % 3 == 2:
+                out = torch.full((M,), float("nan")).pin_memory()
+                B.mtmc_linear_lse_host(X, W, b, lse_out=out, blocking=False)
+                want, tol = ref.linear_lse(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)), TOL["fp32"]
+            else:
+                out = torch.full((M, N), float("nan")).pin_memory()
+                B.mtmc_fused_linear_host(X, W, b, "silu", "fp32", out=out, blocking=False)
+                want, tol = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_SILU), TOL["fp32"]
+            jobs.append((out, want, tol, (X, W, b)))
+    si = inputs.swiglu_inputs(200, 392, 256, seed=9190)
+    sX, sG, sU = si.X.pin_memory(), si.Wg.pin_memory(), si.Wu.pin_memory()
+    sw = torch.zeros((200, 392), dtype=torch.bfloat16).pin_memory()
+    B.mtmc_swiglu_host(sX, sG, sU, out=sw, blocking=False)
+    B.mtmc_host_sync()
+    B.mtmc_check_status()
+    for n, (out, want, tol, _) in enumerate(jobs):
+        _assert_close(inputs.to_f64(out), want, tol, "pipelined host call %d" % n)
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "pipelined swiglu_host")
+
