@@ -136,6 +136,15 @@ def test_large_tile_pair_kernel_row_reductions(M, N, K):
         B.mtmc_check_status()
     finally:
         B.mtmc_set_tuning()
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=8960 + M)           # E4M3 operands through the same kernel
+    B.mtmc_set_tuning(cta_pair=2)
+    try:
+        lse8 = B.mtmc_linear_lse_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w)
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(lse8), ref.linear_lse_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b),
+                                                          fi.scale_x, fi.scale_w), TOL["fp32"], "fp8 lse, 512-row tiles")
     _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "lse, 512-row tiles")
     _assert_close(inputs.to_f64(lse_nobias), ref.linear_lse(Xb, Wb, None), TOL["fp32"], "lse without bias, 512-row tiles")
     _check_rowmax(li, mx, arg, "rowmax, 512-row tiles")
