@@ -748,3 +748,55 @@ def test_host_pointer_calls_without_waiting():
     _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
                   TOL["bf16"], "pipelined swiglu_host")
 
+
+def test_random_shapes_all_operators_and_kernels():
+    """Seeded sweep: 60 random shapes (ragged M, N, K; K a multiple of 8), each through a randomly chosen operator and
+    kernel choice (automatic, 256 x 256 pairs, 512 x 256 pairs, single-CTA tiles of either width), against the oracle."""
+    rng = np.random.default_rng(20251125)
+    tunings = [dict(), dict(cta_pair=1), dict(cta_pair=2), dict(cta_pair=-1), dict(tile_n=128), dict(split_k=2)]
+    for case in range(60):
+        M = int(rng.integers(1, 700))
+        N = int(rng.integers(1, 900))
+        K = 8 * int(rng.integers(1, 260))
+        while M * N * K > 4e8:
+            K = max(8, K // 2 // 8 * 8)
+        op = ["linear", "lse", "swiglu", "rowmax", "xent", "residual"][case % 6]
+        tune = tunings[int(rng.integers(0, len(tunings)))]
+        what = "case %d: %s %dx%dx%d %r" % (case, op, M, N, K, tune)
+        li = inputs.linear_inputs(M, N, K, seed=9300 + case)
+        Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+        Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+        B.mtmc_set_tuning(**tune)
+        try:
+            if op == "linear":
+                act = ["none", "relu", "gelu_tanh", "silu"][case // 6 % 4]
+                odt = "bf16" if case % 2 else "fp32"
+                buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+                B.mtmc_fused_linear(Xd, Wd, bd, act, odt, out=out)
+                B.mtmc_check_status()
+                assert _canaries_intact(buf, M * N), what
+                _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, B.ACT[act]), TOL[odt], what)
+            elif op == "lse":
+                _assert_close(inputs.to_f64(B.mtmc_linear_lse(Xd, Wd, bd)), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], what)
+            elif op == "swiglu":
+                si = inputs.swiglu_inputs(M, N, K, seed=9400 + case)
+                got = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+                _assert_close(inputs.to_f64(got), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                              TOL["bf16"], what)
+            elif op == "rowmax":
+                mx, arg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+                _check_rowmax(li, mx, arg, what)
+            elif op == "xent":
+                tgt = torch.from_numpy(rng.integers(0, N, size=M))
+                loss = B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt.cuda())
+                want, _ = ref.linear_cross_entropy(Xb, Wb, bf, tgt.numpy())
+                _assert_close(inputs.to_f64(loss), want, TOL["fp32"], what)
+            else:
+                R = torch.randn(M, N, generator=torch.Generator().manual_seed(case)).bfloat16()
+                got = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "silu", "bf16")
+                _assert_close(inputs.to_f64(got), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_SILU),
+                              TOL["bf16"], what)
+            B.mtmc_check_status()
+        finally:
+            B.mtmc_set_tuning()
+
