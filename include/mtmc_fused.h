@@ -265,10 +265,10 @@ float mtmc_last_kernel_ms(void);
  *              size of the cluster split-K kernel (1 = never use that kernel)
  *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
  *   cta_pair : 1 forces the CTA-pair (cta_group::2) kernel with 256 x 256 tiles and overlapped
- *              epilogues, 2 the one with 512 x 256 tiles (activation epilogues and row
- *              reductions; SwiGLU then takes the 256 x 256 pair kernel), < 0 forbids both;
+ *              epilogues, 2 the one with 512 x 256 tiles, < 0 forbids both;
  *              automatic = pairs when M >= 512 and N >= 256; the large tiles for the row
- *              reductions and for activation epilogues with a long K */
+ *              reductions and for activation epilogues with a long K, never for SwiGLU
+ *              (measured on a par at best) */
 int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
 
 /* Static weights (thread-local, default 0 = off).  With enabled != 0 the caller promises, for

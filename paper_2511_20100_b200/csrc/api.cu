@@ -463,6 +463,12 @@ bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     return big_waves_ok(M, N, pairs, k_blocks >= 96);
 }
 
+// SwiGLU on the 512 x 256 tiles: only when the tuning hook forces them (cta_pair = 2); measured slower by default.
+bool use_big_swiglu(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
+    (void)M; (void)N; (void)K; (void)fp8;
+    return gemm_pairs(d) > 0 && EPI_HALVES == 1 && t_tile_n == 0 && t_cta_pair == 2;
+}
+
 // Tiling of the output and the split of the wave tail.  With G CTAs, the last T % G tiles
 // form a partial wave; cutting each of them into `tail_split` column pieces (2 or 4, pieces
 // at least 32 columns wide, all pieces fitting one wave) shortens that wave accordingly.
@@ -884,6 +890,18 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
             return rc;
         TimedRegion tr(d);
         rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
+        tr.stop();
+        return rc;
+    }
+    if (use_big_swiglu(d, M, N, K, fp8)) {
+        GemmParams p{};
+        fill_tiling(p, M, N, K, 128, gemm_pairs(d), false, 512, fp8);
+        p.acc_scale = sg; p.acc_scale2 = su;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        CUtensorMap tmA, tmG, tmU;
+        if ((rc = encode(&tmA, X, M, K, 256, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) || (rc = encode(&tmU, Wu, N, K, 128, 0))) return rc;
+        TimedRegion tr(d);
+        rc = launch_big<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, p);
         tr.stop();
         return rc;
     }

@@ -145,6 +145,15 @@ def test_large_tile_pair_kernel_row_reductions(M, N, K):
         B.mtmc_set_tuning()
     _assert_close(inputs.to_f64(lse8), ref.linear_lse_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b),
                                                           fi.scale_x, fi.scale_w), TOL["fp32"], "fp8 lse, 512-row tiles")
+    si = inputs.swiglu_inputs(M, N, K, seed=8970 + M)                   # and the SwiGLU gate, which only the hook sends there
+    B.mtmc_set_tuning(cta_pair=2)
+    try:
+        sw = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "swiglu, 512-row tiles")
     _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "lse, 512-row tiles")
     _assert_close(inputs.to_f64(lse_nobias), ref.linear_lse(Xb, Wb, None), TOL["fp32"], "lse without bias, 512-row tiles")
     _check_rowmax(li, mx, arg, "rowmax, 512-row tiles")
