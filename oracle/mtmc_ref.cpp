@@ -345,6 +345,48 @@ int mtmc_ref_linear_cross_entropy(const uint16_t* X, const uint16_t* W, const fl
     return 0;
 }
 
+// One pre-activation of the E4M3 layer: sx*sw * sum_k xq[m][k] wq[n][k] + b[n].
+static double preact_fp8(const uint8_t* X, const uint8_t* W, const float* b, double scale, int64_t K, int64_t m, int64_t n) {
+    double acc = 0.0;
+    for (int64_t k = 0; k < K; ++k) acc += e4m3_to_double(X[m * K + k]) * e4m3_to_double(W[n * K + k]);
+    return scale * acc + (b ? static_cast<double>(b[n]) : 0.0);
+}
+
+// Row maximum and the lowest column attaining it, E4M3 operands.
+int mtmc_ref_linear_rowmax_fp8(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                               int64_t M, int64_t N, int64_t K, double* mx, int64_t* arg) {
+    if (!X || !W || !mx || M <= 0 || N <= 0 || K <= 0) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(M, [=](int64_t m) {
+        double best = preact_fp8(X, W, b, scale, K, m, 0);
+        int64_t where = 0;
+        for (int64_t n = 1; n < N; ++n) {
+            const double z = preact_fp8(X, W, b, scale, K, m, n);
+            if (z > best) { best = z; where = n; }
+        }
+        mx[m] = best;
+        if (arg) arg[m] = where;
+    });
+    return 0;
+}
+
+// loss[m] = lse[m] - z[m][target[m]], E4M3 operands; lse_out may be null.
+int mtmc_ref_linear_cross_entropy_fp8(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                                      const int64_t* target, int64_t M, int64_t N, int64_t K, double* loss, double* lse_out) {
+    if (!X || !W || !target || !loss || M <= 0 || N <= 0 || K <= 0) return 1;
+    for (int64_t m = 0; m < M; ++m)
+        if (target[m] < 0 || target[m] >= N) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n) z[n] = preact_fp8(X, W, b, scale, K, m, n);
+        const double l = lse_of_row(z.data(), N);
+        loss[m] = l - z[target[m]];
+        if (lse_out) lse_out[m] = l;
+    });
+    return 0;
+}
+
 // logsumexp of a plain vector of doubles (pins: closed forms, shift law).
 double mtmc_ref_lse_vector(const double* z, int64_t N) { return lse_of_row(z, N); }
 

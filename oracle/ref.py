@@ -49,6 +49,8 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_fused_linear_fp8_points.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
         L.mtmc_ref_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
+        L.mtmc_ref_linear_rowmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
+        L.mtmc_ref_linear_cross_entropy_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, i64, i64, i64, vp, vp]
         L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
@@ -274,6 +276,36 @@ def linear_cross_entropy(X, W, b, target):
     lse = np.empty(M, dtype=np.float64)
     _check(lib().mtmc_ref_linear_cross_entropy(X.ctypes.data, W.ctypes.data, bp, target.ctypes.data, M, N, K,
                                                loss.ctypes.data, lse.ctypes.data), "mtmc_ref_linear_cross_entropy")
+    return loss, lse
+
+
+def linear_rowmax_fp8(X, W, b, scale_x: float, scale_w: float):
+    """(row maximum, lowest column attaining it) of scale_x*scale_w * Xq.Wq^T + b with E4M3 bit patterns (uint8)."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    mx = np.empty(M, dtype=np.float64)
+    arg = np.empty(M, dtype=np.int64)
+    _check(lib().mtmc_ref_linear_rowmax_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
+                                            mx.ctypes.data, arg.ctypes.data), "mtmc_ref_linear_rowmax_fp8")
+    return mx, arg
+
+
+def linear_cross_entropy_fp8(X, W, b, scale_x: float, scale_w: float, target):
+    """(loss, lse) per row of the E4M3 layer: loss = lse - logit[target]."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    target = _idx(target)
+    if target.shape != (M,):
+        raise TypeError("target must be int64 [M]")
+    loss = np.empty(M, dtype=np.float64)
+    lse = np.empty(M, dtype=np.float64)
+    _check(lib().mtmc_ref_linear_cross_entropy_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w),
+                                                   target.ctypes.data, M, N, K, loss.ctypes.data, lse.ctypes.data),
+           "mtmc_ref_linear_cross_entropy_fp8")
     return loss, lse
 
 

@@ -241,6 +241,36 @@ def test_fp8_linear_lse_pins():
     assert np.array_equal(ref.linear_lse_fp8(X8, W8, b, 2.0 ** -4, 2.0 ** -8), folded)
 
 
+def test_fp8_rowmax_and_cross_entropy_pins():
+    fi = inputs.fp8_linear_inputs(6, 41, 48, seed=74)
+    X8, W8, b = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    z = ref.fused_linear_fp8(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_NONE)          # the pinned FP8 logits
+    mx, arg = ref.linear_rowmax_fp8(X8, W8, b, fi.scale_x, fi.scale_w)
+    assert np.array_equal(mx, z.max(axis=1)) and np.array_equal(arg, z.argmax(axis=1))
+    tv, ti = torch.from_numpy(z).max(dim=1)
+    assert np.array_equal(mx, tv.numpy()) and np.array_equal(arg, ti.numpy())
+    # ties go to the lowest column: duplicate the winning weight row (and its bias) further right
+    W2, b2 = W8.copy(), b.copy()
+    for m in range(1):
+        src, dst = int(arg[0]), 40 if arg[0] != 40 else 39
+        W2[dst], b2[dst] = W2[src], b2[src]
+    mx2, arg2 = ref.linear_rowmax_fp8(X8, W2, b2, fi.scale_x, fi.scale_w)
+    assert mx2[0] == mx[0] and arg2[0] == min(int(arg[0]), dst)
+    tgt = np.array([0, 40, 7, 7, 13, 22])
+    loss, lse = ref.linear_cross_entropy_fp8(X8, W8, b, fi.scale_x, fi.scale_w, tgt)
+    assert np.array_equal(lse, ref.linear_lse_fp8(X8, W8, b, fi.scale_x, fi.scale_w))
+    assert np.array_equal(loss, lse - z[np.arange(6), tgt])
+    want = torch.nn.functional.cross_entropy(torch.from_numpy(z), torch.from_numpy(tgt), reduction="none")
+    np.testing.assert_allclose(loss, want.numpy(), rtol=1e-12, atol=1e-12)
+    # with power-of-two scales folded into bf16 copies of the operands: the bf16 functions, bit for bit
+    fmx, farg = ref.linear_rowmax(_as_bf16_bits(fi.X, 2.0 ** -4), _as_bf16_bits(fi.W, 2.0 ** -8), b)
+    gmx, garg = ref.linear_rowmax_fp8(X8, W8, b, 2.0 ** -4, 2.0 ** -8)
+    assert np.array_equal(fmx, gmx) and np.array_equal(farg, garg)
+    floss, _ = ref.linear_cross_entropy(_as_bf16_bits(fi.X, 2.0 ** -4), _as_bf16_bits(fi.W, 2.0 ** -8), b, tgt)
+    gloss, _ = ref.linear_cross_entropy_fp8(X8, W8, b, 2.0 ** -4, 2.0 ** -8, tgt)
+    assert np.array_equal(floss, gloss)
+
+
 # ---------------------------------------------------------------- activations
 def _closed_forms():
     rows = []
