@@ -120,6 +120,12 @@ int mtmc_swiglu_fp8(const void* X8, const void* Wg8, const void* Wu8, float scal
                     int64_t M, int64_t N, int64_t K, void* out);
 int mtmc_linear_lse_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
                         int64_t M, int64_t N, int64_t K, float* lse_out);
+/* mtmc_linear_rowmax and mtmc_linear_cross_entropy (below) with E4M3 operands, same conventions:
+ * the logits are scale_x*scale_w * X8.W8^T + b. */
+int mtmc_linear_rowmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                           int64_t M, int64_t N, int64_t K, float* max_out, int32_t* argmax_out);
+int mtmc_linear_cross_entropy_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                                  const int64_t* targets, int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out);
 
 /* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
  * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate

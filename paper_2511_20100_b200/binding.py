@@ -28,7 +28,7 @@ EXPORTS = [
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -62,6 +62,8 @@ def load() -> ctypes.CDLL:
     L.mtmc_fused_linear_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, i64]
     L.mtmc_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     L.mtmc_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
+    L.mtmc_linear_rowmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
+    L.mtmc_linear_cross_entropy_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, i64, i64, i64, vp, vp]
     for name in ("mtmc_swiglu", "mtmc_swiglu_host", "mtmc_swiglu_host_async", "mtmc_linear_lse", "mtmc_linear_lse_host",
                  "mtmc_linear_lse_host_async", "mtmc_linear_lse_noalloc"):
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
@@ -257,6 +259,41 @@ def mtmc_linear_cross_entropy(X, W, b, targets, loss_out=None, lse_out=None, wan
                                             _dev(targets, torch.int64, (M,), "targets"), M, N, K,
                                             _dev(loss_out, torch.float32, (M,), "loss_out"),
                                             None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return (loss_out, lse_out) if want_lse else loss_out
+
+
+def mtmc_linear_rowmax_fp8(X8, W8, b, scale_x, scale_w, max_out=None, argmax_out=None, want_argmax=True):
+    """mtmc_linear_rowmax with float8_e4m3fn operands and per-tensor scales."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    if max_out is None:
+        max_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    if argmax_out is None and want_argmax:
+        argmax_out = torch.empty((M,), dtype=torch.int32, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_linear_rowmax_fp8(_dev(X8, f8, (M, K), "X8"), _dev(W8, f8, (N, K), "W8"),
+                                         None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                         float(scale_x), float(scale_w), M, N, K, _dev(max_out, torch.float32, (M,), "max_out"),
+                                         None if argmax_out is None else _dev(argmax_out, torch.int32, (M,), "argmax_out")))
+    return max_out, argmax_out
+
+
+def mtmc_linear_cross_entropy_fp8(X8, W8, b, scale_x, scale_w, targets, loss_out=None, lse_out=None, want_lse=False):
+    """mtmc_linear_cross_entropy with float8_e4m3fn operands and per-tensor scales."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    if loss_out is None:
+        loss_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_linear_cross_entropy_fp8(_dev(X8, f8, (M, K), "X8"), _dev(W8, f8, (N, K), "W8"),
+                                                None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                                float(scale_x), float(scale_w), _dev(targets, torch.int64, (M,), "targets"), M, N, K,
+                                                _dev(loss_out, torch.float32, (M,), "loss_out"),
+                                                None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
     return (loss_out, lse_out) if want_lse else loss_out
 
 

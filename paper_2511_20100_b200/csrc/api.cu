@@ -1183,6 +1183,25 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
     return run_row_reduction<EPI_XENT>(X, W, b, targets, M, N, K, lse_out, loss_out, nullptr);
 }
 
+int mtmc_linear_rowmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,
+                           int64_t K, float* max_out, int32_t* argmax_out) {
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
+    int rc = check_common(X8, W8, max_out, M, N, K);
+    if (rc) return rc;
+    if (argmax_out && (reinterpret_cast<uintptr_t>(argmax_out) & 3u)) return fail(MTMC_ERR_INVALID_ARG, "argmax_out must be 4-byte aligned");
+    return run_row_reduction<EPI_ROWMAX>(X8, W8, b, nullptr, M, N, K, max_out, nullptr, argmax_out, true, scale_x * scale_w);
+}
+
+int mtmc_linear_cross_entropy_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                                  const int64_t* targets, int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out) {
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
+    int rc = check_common(X8, W8, loss_out, M, N, K);
+    if (rc) return rc;
+    if (!targets) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(targets) & 7u) return fail(MTMC_ERR_INVALID_ARG, "targets must be 8-byte aligned");
+    return run_row_reduction<EPI_XENT>(X8, W8, b, targets, M, N, K, lse_out, loss_out, nullptr, true, scale_x * scale_w);
+}
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------- allocation-free variant

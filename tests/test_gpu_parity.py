@@ -285,6 +285,29 @@ def test_linear_lse_fp8(M, N, K):
     _assert_close(inputs.to_f64(out), want, TOL["fp32"], "lse fp8 %dx%dx%d" % (M, N, K))
 
 
+@pytest.mark.parametrize("M,N,K", [(5, 8, 64), (200, 1000, 256), (129, 257, 80), (128, 1024, 4096), (600, 1100, 192)])
+def test_linear_rowmax_and_cross_entropy_fp8(M, N, K):
+    fi = inputs.fp8_linear_inputs(M, N, K, seed=7400 + M + N)
+    X8, W8, bf = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    Xd, Wd, bd = fi.X.cuda(), fi.W.cuda(), fi.b.cuda()
+    mx, arg = B.mtmc_linear_rowmax_fp8(Xd, Wd, bd, fi.scale_x, fi.scale_w)
+    want_mx, want_arg = ref.linear_rowmax_fp8(X8, W8, bf, fi.scale_x, fi.scale_w)
+    _assert_close(inputs.to_f64(mx), want_mx, TOL["fp32"], "fp8 rowmax %dx%dx%d" % (M, N, K))
+    z = ref.fused_linear_fp8(X8, W8, bf, fi.scale_x, fi.scale_w, ref.ACT_NONE)
+    a = arg.cpu().numpy().astype(np.int64)
+    assert np.all((a >= 0) & (a < N))
+    assert np.all(np.abs(z[np.arange(M), a] - want_mx) <= 1e-3 + 1e-3 * np.abs(want_mx))       # the named column holds the maximum
+    if N > 1:
+        clear = (want_mx - np.partition(z, -2, axis=1)[:, -2]) > 1e-2
+        assert np.array_equal(a[clear], want_arg[clear])
+    tgt = torch.from_numpy(np.random.default_rng(M + N).integers(0, N, size=M))
+    loss, lse = B.mtmc_linear_cross_entropy_fp8(Xd, Wd, bd, fi.scale_x, fi.scale_w, tgt.cuda(), want_lse=True)
+    B.mtmc_check_status()
+    want_loss, want_lse = ref.linear_cross_entropy_fp8(X8, W8, bf, fi.scale_x, fi.scale_w, tgt.numpy())
+    _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "fp8 cross entropy %dx%dx%d" % (M, N, K))
+    _assert_close(inputs.to_f64(lse), want_lse, TOL["fp32"], "fp8 lse of cross entropy")
+
+
 def test_fused_linear_fp8_exact_small_integers():
     # operands in {-2..2} are exact in E4M3 and every fp32 partial sum is exact: the result must be exact too
     g = torch.Generator().manual_seed(6)
