@@ -124,6 +124,18 @@ __device__ __forceinline__ float gelu_tanh_fast(float z) {
     const float hz = 0.5f * z;
     return fmaf(hz, t, hz);
 }
+// Two values at once with packed fp32 pairs for the polynomial and the final product: half the issue slots.
+__device__ __forceinline__ void gelu_tanh_fast2(float& z0, float& z1) {
+    float a0, a1, u0, u1, h0, h1, t0, t1;
+    mul_f32x2(a0, a1, z0, z1, 0.044715f, 0.044715f);
+    fma_f32x2(a0, a1, a0, a1, z0, z1, 1.0f, 1.0f);                       // 1 + 0.044715 z^2
+    mul_f32x2(u0, u1, z0, z1, 0.7978845608028654f, 0.7978845608028654f);
+    mul_f32x2(u0, u1, u0, u1, a0, a1);
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t0) : "f"(u0));
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t1) : "f"(u1));
+    mul_f32x2(h0, h1, z0, z1, 0.5f, 0.5f);
+    fma_f32x2(z0, z1, h0, h1, t0, t1, h0, h1);
+}
 __device__ __forceinline__ float apply_act(int act, float z) {
     switch (act) {
         case ACT_RELU: return fmaxf(z, 0.0f);
@@ -140,7 +152,10 @@ __device__ __forceinline__ void apply_act_chunk(int act, float (&y)[32]) {
         for (int j = 0; j < 32; ++j) y[j] = fmaxf(y[j], 0.0f);
     } else if (act == ACT_GELU_TANH) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) y[j] = OUT_BF16 ? gelu_tanh_fast(y[j]) : gelu_tanh_f(y[j]);
+        for (int j = 0; j < 32; j += 2) {
+            if (OUT_BF16) gelu_tanh_fast2(y[j], y[j + 1]);
+            else { y[j] = gelu_tanh_f(y[j]); y[j + 1] = gelu_tanh_f(y[j + 1]); }
+        }
     } else if (act == ACT_SILU) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) y[j] = silu_f(y[j]);
@@ -330,7 +345,8 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tmem_ld_wait();                                  // chunk c has landed in r
             float y[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = fmaf(__uint_as_float(r[j]), p.acc_scale, bv[j]);
+            for (int j = 0; j < 32; j += 2)
+                fma_f32x2(y[j], y[j + 1], __uint_as_float(r[j]), __uint_as_float(r[j + 1]), p.acc_scale, p.acc_scale, bv[j], bv[j + 1]);
             if (c + 1 < live) {                              // r and bv are free again: refill them for chunk c + 1
                 tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
                 tile_bias_chunk(p, bias_tile, n_tile0, n0 + 32, bv);
@@ -362,7 +378,14 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
                 }
             }
 #pragma unroll
-            for (int j = 0; j < 32; ++j) y[j] = silu_f(__uint_as_float(g[j])) * __uint_as_float(u[j]);
+            for (int j = 0; j < 32; j += 2) {                       // packed fp32 pairs: half the issue slots of the FP part
+                const float g0 = __uint_as_float(g[j]), g1 = __uint_as_float(g[j + 1]);
+                float t0, t1, d0, d1, s0, s1;
+                mul_f32x2(t0, t1, g0, g1, -1.4426950408889634f, -1.4426950408889634f);
+                add_f32x2(d0, d1, ex2_approx(t0), ex2_approx(t1), 1.0f, 1.0f);
+                mul_f32x2(s0, s1, g0, g1, rcp_approx(d0), rcp_approx(d1));
+                mul_f32x2(y[j], y[j + 1], s0, s1, __uint_as_float(u[j]), __uint_as_float(u[j + 1]));
+            }
             if (c + 1 < live) {
                 tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, g);
                 tmem_ld_32x32b_x32(t_addr + width + (c + 1) * 32, u);
@@ -423,9 +446,12 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tmem_ld_wait();
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                tv[j] = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);
+            for (int j = 0; j < 32; j += 2) {
+                float b0, b1;
+                mul_f32x2(b0, b1, bv[j], bv[j + 1], LOG2E, LOG2E);
+                fma_f32x2(tv[j], tv[j + 1], __uint_as_float(r[j]), __uint_as_float(r[j + 1]), zscale, zscale, b0, b1);
                 m4[j & 3] = fmaxf(m4[j & 3], tv[j]);
+                m4[(j + 1) & 3] = fmaxf(m4[(j + 1) & 3], tv[j + 1]);
             }
             if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);      // r is free again
             if (n0 + 32 > p.N) {      // ragged last chunk: columns past N are zero-filled weight rows, mask them out
@@ -449,7 +475,11 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             const float nm = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
             float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-            for (int j = 0; j < 32; ++j) s4[j & 3] += ex2_approx(tv[j] - nm);
+            for (int j = 0; j < 32; j += 2) {
+                float d0, d1;
+                add_f32x2(d0, d1, tv[j], tv[j + 1], -nm, -nm);
+                add_f32x2(s4[j & 3], s4[(j + 1) & 3], s4[j & 3], s4[(j + 1) & 3], ex2_approx(d0), ex2_approx(d1));
+            }
             sum = sum * ex2_approx(mx - nm) + ((s4[0] + s4[1]) + (s4[2] + s4[3]));
             mx = nm;
         }
