@@ -36,8 +36,11 @@ import torch
 from paper_2511_20100_b200 import inputs
 
 ORDER = ["C1", "C2", "C3", "C4", "C5"]
-# rows of X the CPU reference computes per step and per configuration (bounded sample)
+# rows of X the CPU reference arm computes per step and per configuration (bounded sample: about a second per step)
 REF_ROWS = {"C1": 256, "C2": 64, "C3": 32, "C4": 32, "C5": 16}
+# rows for the cpu_baseline leg of our own arm, run once: C1, C2 and C5 in full, C3 and C4 on a row sample
+# (about 15 s of CPU work on 16 cores); --full-cpu-baseline runs all five in full (about two minutes)
+CPU_BASELINE_ROWS = {"C1": 256, "C2": 4096, "C3": 512, "C4": 512, "C5": 16}
 
 
 def flops(c) -> float:
@@ -209,31 +212,40 @@ def eager_call(pr, dev):
     return z if c["out_dtype"] == "fp32" else z.to(torch.bfloat16)
 
 
-def cpu_baseline_sample():
-    """The oracle timed on a bounded sample: the first REF_ROWS rows of every configuration."""
+def cpu_baseline_sample(rows_by_cfg):
+    """The oracle, as it stands, timed on the first rows_by_cfg[c] rows of X of every configuration.  Returns the
+    TFLOP/s of one step (all five configurations) with the time of a sampled configuration scaled to all its rows,
+    the thread count, the names of the scaled configurations and the per-configuration seconds (scaled)."""
     from oracle import ref
-    t_total, fl_total = 0.0, 0.0
+    step_s, scaled, secs = 0.0, [], {}
     for name in ORDER:
-        t, fl = reference_step_one(ref, name, prepared_reference_inputs(name))
-        t_total += t
-        fl_total += fl
-    return fl_total / t_total / 1e12, ref.get_threads()
+        c = inputs.CONFIGS[name]
+        t, _ = reference_step_one(ref, name, prepared_reference_inputs(name, rows_by_cfg))
+        r = min(rows_by_cfg[name], c["M"])
+        if r < c["M"]:
+            scaled.append("%s %d/%d" % (name, r, c["M"]))
+        secs[name] = t * c["M"] / r
+        step_s += secs[name]
+    fl = sum(flops(inputs.CONFIGS[n]) for n in ORDER)
+    return fl / step_s / 1e12, ref.get_threads(), scaled, secs
 
 
 _ref_cache = {}
 
 
-def prepared_reference_inputs(name):
-    if name not in _ref_cache:
+def prepared_reference_inputs(name, rows_by_cfg=None):
+    rows_by_cfg = rows_by_cfg or REF_ROWS
+    key = (name, rows_by_cfg[name])
+    if key not in _ref_cache:
         c = inputs.CONFIGS[name]
-        r = min(REF_ROWS[name], c["M"])
+        r = min(rows_by_cfg[name], c["M"])
         if c["op"] == "swiglu":
             si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
-            _ref_cache[name] = (inputs.bf16_bits(si.X[:r].contiguous()), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu))
+            _ref_cache[key] = (inputs.bf16_bits(si.X[:r].contiguous()), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu))
         else:
             li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
-            _ref_cache[name] = (inputs.bf16_bits(li.X[:r].contiguous()), inputs.bf16_bits(li.W), inputs.f32(li.b))
-    return _ref_cache[name]
+            _ref_cache[key] = (inputs.bf16_bits(li.X[:r].contiguous()), inputs.bf16_bits(li.W), inputs.f32(li.b))
+    return _ref_cache[key]
 
 
 def reference_step_one(ref, name, arrs):
@@ -250,9 +262,10 @@ def reference_step_one(ref, name, arrs):
     return dt, flops(c) * r / c["M"]
 
 
-def sample_description():
-    return "first rows of X per configuration: " + ", ".join("%s %d/%d" % (n, min(REF_ROWS[n], inputs.CONFIGS[n]["M"]),
-                                                                               inputs.CONFIGS[n]["M"]) for n in ORDER)
+def sample_description(rows_by_cfg=None):
+    rows_by_cfg = rows_by_cfg or REF_ROWS
+    return "first rows of X: " + ", ".join("%s %d/%d" % (n, min(rows_by_cfg[n], inputs.CONFIGS[n]["M"]),
+                                                          inputs.CONFIGS[n]["M"]) for n in ORDER)
 
 
 def run_ours(args, rank, world, local_rank):
@@ -304,27 +317,35 @@ def run_ours(args, rank, world, local_rank):
     # ---- per configuration: the same call back to back, rotating over enough copies of the
     # operands that their total exceeds twice the L2 (so every launch reads its operands from HBM);
     # one event pair around the loop, so launch overhead is amortised as it is inside a step.
+    #   burst     : 8 launches right after `settle_s` of idle (boost clocks, before the power cap bites) -> compared
+    #               with the measured burst peak
+    #   sustained : tensor-bound configurations run back to back for `sustain_s` seconds -> compared with the measured
+    #               sustained peak; the short ones (C1, C5) loop for `loop_ms`
     L2_BYTES = 126e6
     per_cfg_ms, per_cfg_reps, per_cfg_copies, per_cfg_eager, per_cfg_burst, per_cfg_warm = {}, {}, {}, {}, {}, {}
-    extras = [] if (args.no_extras or ORDER != list(inputs.CONFIGS)) else [make_device_problem(n, device) for n in inputs.EXTRA_CONFIGS]
+    per_cfg_kernel, per_cfg_enqueue = {}, {}
+    extras = [make_device_problem(n, device) for n in inputs.EXTRA_CONFIGS] if (args.extras and ORDER == list(inputs.CONFIGS)) else []
     for pr in problems + extras:
         n, c = pr["name"], pr["cfg"]
+        tensor_bound = c["M"] > 128 and n != "C1"
         nbytes = sum(t.numel() * t.element_size() for t in pr["dev"] if t is not None)
         copies = 1 if n == "C1" else max(1, min(4, int(-(-2 * L2_BYTES // nbytes))))
         variants = [pr] + [dict(pr, dev=[None if t is None else t.clone() for t in pr["dev"]]) for _ in range(copies - 1)]
         for v in variants:
             call_device(B, v)
+        per_cfg_kernel[n] = B.mtmc_last_kernel_name()       # the library's own account of what it launched
         torch.cuda.synchronize()
         time.sleep(args.settle_s)      # let the power/clock state left by the previous loop settle: each loop describes its own kernel
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for r in range(8):             # a burst right after the idle: boost clocks, before the power cap bites
+        for r in range(8):
             call_device(B, variants[r % copies])
         e1.record()
         torch.cuda.synchronize()
         per_cfg_burst[n] = e0.elapsed_time(e1) / 8
         est = max(per_cfg_burst[n], 1e-3)
-        reps = int(max(10, min(2000, args.loop_ms / est)))
+        target_ms = args.sustain_s * 1e3 if tensor_bound else args.loop_ms
+        reps = int(max(10, min(20000, target_ms / est)))
         e0.record()
         for r in range(reps):
             call_device(B, variants[r % copies])
@@ -332,6 +353,18 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
         per_cfg_ms[n] = e0.elapsed_time(e1) / reps
         per_cfg_reps[n], per_cfg_copies[n] = reps, copies
+        if not tensor_bound:
+            # launch-latency sized calls: host time to enqueue one call (argument checks, cached tensor maps, launch),
+            # measured on an empty queue in batches short enough never to fill it
+            t_host = 0.0
+            for _ in range(5):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                for r in range(50):
+                    call_device(B, variants[r % copies])
+                t_host += time.perf_counter() - t0
+            torch.cuda.synchronize()
+            per_cfg_enqueue[n] = t_host / 250 * 1e6
         if c["M"] <= 128 and n != "C1" and copies > 1:
             # weight-streaming shapes: also the same call on ONE copy of the operands, i.e. with whatever part of W
             # the 126 MB L2 keeps from the launch before (labelled warm; the headline figure above is the cold one)
@@ -346,7 +379,7 @@ def run_ours(args, rank, world, local_rank):
             for v in variants:
                 eager_call(pr, v["dev"])
             torch.cuda.synchronize()
-            ereps = max(5, reps // 4)
+            ereps = max(5, min(reps // 4, int(300.0 / est)))
             e0.record()
             for r in range(ereps):
                 eager_call(pr, variants[r % copies]["dev"])
@@ -356,62 +389,74 @@ def run_ours(args, rank, world, local_rank):
         del variants
     B.mtmc_check_status()
     clocks = sampler.stop()
-    per_cfg_best = per_cfg_ms
     step_flops = sum(flops(inputs.CONFIGS.get(n) or inputs.EXTRA_CONFIGS[n]) for n in ORDER)
     value = world * step_flops / (ms_per_step * 1e-3) / 1e12
 
-    per_config = {}
-    for n in ORDER + [e["name"] for e in extras]:
-        c = inputs.CONFIGS.get(n) or inputs.EXTRA_CONFIGS[n]
-        ms = per_cfg_ms[n]
-        entry = {"call": c["op"], "M": c["M"], "N": c["N"], "K": c["K"], "ms": round(ms, 5),
-                 "launches_timed": per_cfg_reps[n], "operand_copies_rotated": per_cfg_copies[n],
-                 "tflops": round(flops(c) / (ms * 1e-3) / 1e12, 3), "gbs": round(algorithmic_bytes(c) / (ms * 1e-3) / 1e9, 2)}
-        if n in per_cfg_warm:
-            entry["l2_warm_ms"] = round(per_cfg_warm[n], 5)
-        if c["M"] > 128 and n != "C1":      # tensor-bound shapes: 8 launches after 0.5 s of idle run at boost clocks
-            entry["burst_ms"] = round(per_cfg_burst[n], 5)
-            entry["burst_tflops"] = round(flops(c) / (per_cfg_burst[n] * 1e-3) / 1e12, 3)
-        if n in inputs.EXTRA_CONFIGS:
-            entry["note"] = "further operator of the same family; measured beside the step, not part of it"
-        if n in per_cfg_eager:
-            entry["eager_ms"] = round(per_cfg_eager[n], 5)
-            entry["speedup_vs_eager"] = round(per_cfg_eager[n] / ms, 3)
-        if n == "C5" or (n in inputs.EXTRA_CONFIGS and c["M"] <= 128):     # weight streaming: bound by HBM
-            entry["roofline"] = {"bound": "hbm", "achieved": entry["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                 "frac": round(entry["gbs"] / peaks["hbm_gbs"], 4), "of": peaks["source"],
-                                 "frac_of_nominal_8000": round(entry["gbs"] / 8000.0, 4)}
-        elif c["op"] == "fused_linear_fp8":
-            peak8 = 2.0 * peaks["tflops_sustained"]       # E4M3 peak = measured bf16 peak x the nominal 2:1 ratio
-            entry["roofline"] = {"bound": "tensor", "achieved": entry["tflops"], "peak": peak8, "unit": "TFLOP/s",
-                                 "frac": round(entry["tflops"] / peak8, 4),
-                                 "of": peaks["source"] + " sustained cuBLAS bf16 x 2 (nominal fp8:bf16 ratio)",
-                                 "frac_of_nominal_4500": round(entry["tflops"] / 4500.0, 4)}
-        elif n != "C1":
-            entry["roofline"] = {"bound": "tensor", "achieved": entry["tflops"], "peak": peaks["tflops_sustained"],
-                                 "unit": "TFLOP/s", "frac": round(entry["tflops"] / peaks["tflops_sustained"], 4),
-                                 "of": peaks["source"] + " (sustained cuBLAS bf16)",
-                                 "frac_of_burst": round(entry["tflops"] / peaks["tflops_burst"], 4),
-                                 "burst_frac_of_burst": round(entry.get("burst_tflops", 0.0) / peaks["tflops_burst"], 4),
-                                 "frac_of_nominal_2250": round(entry["tflops"] / 2250.0, 4)}
-        else:
-            entry["note"] = "launch-latency bound parity configuration"
-        per_config[n] = entry
-
-    # dominant kernel of the step: the tiled tcgen05 kernel, on its longest launch (C3, SwiGLU)
-    dom_name = max(ORDER, key=lambda n: per_cfg_ms[n])
-    dom = per_config[dom_name]
-    roofline = dict(dom.get("roofline", {"bound": "tensor", "achieved": dom["tflops"], "peak": peaks["tflops_sustained"],
-                                          "unit": "TFLOP/s", "frac": round(dom["tflops"] / peaks["tflops_sustained"], 4)}))
-    roofline["kernel"] = ("skinny_splitk_kernel" if dom_name == "C5" else "gemm_pair_kernel (tcgen05 cta_group::2)") + " on " + dom_name
-    roofline["peak_source"] = peaks["source"] + (" copy bandwidth" if dom_name == "C5" else " sustained cuBLAS bf16")
-    roofline["traffic"] = None
-    prof = os.path.join(ROOT, "profiles", "traffic.txt")      # DRAM bytes per launch from the committed ncu summaries
+    # DRAM bytes per launch from the committed ncu summaries (a pointer to a capture, not something this run measured)
+    traffic = {}
+    prof = os.path.join(ROOT, "profiles", "traffic.txt")
     if os.path.exists(prof):
         for ln in open(prof):
             tok = ln.split()
-            if len(tok) == 2 and tok[0] == "%s_dram_bytes_per_launch" % dom_name:
-                roofline["traffic"] = int(tok[1])
+            if len(tok) == 2 and tok[0].endswith("_dram_bytes_per_launch"):
+                traffic[tok[0].split("_")[0]] = int(tok[1])
+
+    def describe(n, full):
+        """Per-configuration entry; `full` adds the fields that only the detailed (stderr) record carries."""
+        c = inputs.CONFIGS.get(n) or inputs.EXTRA_CONFIGS[n]
+        ms = per_cfg_ms[n]
+        tf, gb = flops(c) / (ms * 1e-3) / 1e12, algorithmic_bytes(c) / (ms * 1e-3) / 1e9
+        e = {"ms": round(ms, 5), "kernel": per_cfg_kernel[n]}
+        hbm_bound = n == "C5" or (n in inputs.EXTRA_CONFIGS and c["M"] <= 128)
+        if n == "C1":
+            e.update({"tflops": round(tf, 2), "bound": "launch latency"})
+        elif hbm_bound:
+            e.update({"gbs": round(gb, 1), "bound": "hbm", "frac": round(gb / peaks["hbm_gbs"], 4), "frac_of_8000": round(gb / 8000.0, 4)})
+        else:
+            scale = 2.0 if c["op"] == "fused_linear_fp8" else 1.0        # E4M3: measured bf16 peak x the nominal 2:1 ratio
+            btf = flops(c) / (per_cfg_burst[n] * 1e-3) / 1e12
+            e.update({"tflops": round(tf, 1), "bound": "tensor", "burst_ms": round(per_cfg_burst[n], 5),
+                      "frac_burst": round(btf / (scale * peaks["tflops_burst"]), 4),
+                      "frac_sustained": round(tf / (scale * peaks["tflops_sustained"]), 4),
+                      "frac_of_nominal": round(tf / (scale * 2250.0), 4), "loop_s": round(ms * per_cfg_reps[n] * 1e-3, 2)})
+        if n in per_cfg_enqueue:
+            e["host_enqueue_us"] = round(per_cfg_enqueue[n], 2)
+        if n in per_cfg_eager:
+            e["eager_ms"] = round(per_cfg_eager[n], 5)
+        if full:
+            e.update({"call": c["op"], "M": c["M"], "N": c["N"], "K": c["K"], "launches_timed": per_cfg_reps[n],
+                      "operand_copies_rotated": per_cfg_copies[n], "tflops": round(tf, 3), "gbs": round(gb, 2),
+                      "algorithmic_bytes": int(algorithmic_bytes(c)), "flops": flops(c)})
+            if n in per_cfg_warm:
+                e["l2_warm_ms"] = round(per_cfg_warm[n], 5)
+            if n in traffic:
+                e["dram_bytes_per_launch_ncu"] = traffic[n]
+        return e
+
+    per_config = {n: describe(n, False) for n in ORDER}
+
+    # dominant kernel of the step: the one with the longest launch (C3's SwiGLU kernel when all five run)
+    dom_name = max(ORDER, key=lambda n: per_cfg_ms[n])
+    dc = inputs.CONFIGS.get(dom_name) or inputs.EXTRA_CONFIGS[dom_name]
+    if dom_name == "C5" or dc["M"] <= 128:
+        gb = algorithmic_bytes(dc) / (per_cfg_ms[dom_name] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "achieved": round(gb, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": round(gb / peaks["hbm_gbs"], 4), "peak_source": peaks["source"] + " copy bandwidth"}
+    else:
+        # frac compares like with like: the kernel timed alone in a burst after idle against the burst peak; the
+        # seconds-long loop against the sustained peak rides along
+        btf = flops(dc) / (per_cfg_burst[dom_name] * 1e-3) / 1e12
+        stf = flops(dc) / (per_cfg_ms[dom_name] * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "achieved": round(btf, 1), "peak": peaks["tflops_burst"], "unit": "TFLOP/s",
+                    "frac": round(btf / peaks["tflops_burst"], 4),
+                    "peak_source": peaks["source"] + " cuBLAS bf16 burst; 8 launches after %.1f s idle" % args.settle_s,
+                    "sustained": {"achieved": round(stf, 1), "peak": peaks["tflops_sustained"],
+                                  "frac": round(stf / peaks["tflops_sustained"], 4),
+                                  "loop_s": round(per_cfg_ms[dom_name] * per_cfg_reps[dom_name] * 1e-3, 2)},
+                    "frac_of_nominal_2250": round(stf / 2250.0, 4)}
+    roofline["kernel"] = per_cfg_kernel[dom_name] + " on " + dom_name
+    roofline["traffic"] = traffic.get(dom_name)
+    roofline["traffic_source"] = "profiles/traffic.txt (ncu capture of one launch, not this run)"
 
     # ------------------------------------------------------------------ end to end through the host-pointer C ABI
     e2e = None
@@ -452,30 +497,33 @@ def run_ours(args, rank, world, local_rank):
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                "ms_per_step": round(e2e_s / e2e_steps * 1e3, 3),
                "ms_per_step_blocking_calls": round(blocking_s * 1e3, 3),
-               "api": "mtmc_*_host_async + mtmc_host_sync once per step: pinned host buffers in, host results out, "
-                      "all copies inside the timed region"}
+               "api": "mtmc_*_host_async x5 + mtmc_host_sync per step; pinned host buffers, copies inside the timed region"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores = cpu_baseline_sample()
-        cpu = {"value": round(v, 6), "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": sample_description()}
+        rows = {n: inputs.CONFIGS[n]["M"] for n in ORDER} if args.full_cpu_baseline else CPU_BASELINE_ROWS
+        v, cores, scaled, secs = cpu_baseline_sample(rows)
+        cpu = {"value": round(v, 6), "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
+               "sample": "full " + "+".join(n for n in ORDER if not any(x.startswith(n) for x in scaled)) +
+                         ("; first rows of X, time scaled to all rows: " + ", ".join(scaled) if scaled else ""),
+               "extrapolated": bool(scaled), "seconds": {n: round(t, 3) for n, t in secs.items()}}
 
     if rank == 0:
+        if extras or args.details:
+            detail = {"detail": "per-configuration record of the same run (not the bench line)",
+                      "per_config": {n: describe(n, True) for n in ORDER + [e["name"] for e in extras]}}
+            print(json.dumps(detail), file=sys.stderr, flush=True)
         line = {
-            "metric": "TFLOP/s over one pass of the fused-linear hot path (per-config TFLOP/s, GB/s and roofline fractions in per_config)",
+            "metric": "TFLOP/s over one pass of the fused-linear hot path (C1-C5, one call each)",
             "value": round(value, 3), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": round(ms_per_step, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "+".join(ORDER) + " (one call each per step)",
-                       "l2": "inputs larger than L2: a step reads ~1.0 GB of distinct operands (L2 126 MB), every call starts cold; "
-                             "per_config loops rotate operand copies totalling > 2x L2 and start after 0.5 s of idle",
-                       "static_weights": "mtmc_set_static_weights(1): the weight-streaming kernel may start its W loads before "
-                                         "the preceding kernel has finished (about 0.6 us per C5 launch)",
-                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "config": {"workload": "+".join(ORDER), "l2": "inputs > L2: a step reads ~1 GB of distinct operands; per_config loops rotate operand copies > 2x L2",
+                       "static_weights": 1, "parallelism": "replicas only" if world > 1 else "single GPU"},
             "per_config": per_config, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches), "clocks": clocks,
         }
-        print(json.dumps(line), flush=True)
+        print(json.dumps(line, separators=(",", ":")), flush=True)
     if dist is not None:
         dist.destroy_process_group()
 
@@ -499,12 +547,11 @@ def run_reference(args, rank, world):
     value = fl_total / t_total / 1e12
     line = {
         "impl": "reference",
-        "metric": "TFLOP/s over one pass of the fused-linear hot path (per-config TFLOP/s, GB/s and roofline fractions in per_config)",
+        "metric": "TFLOP/s over one pass of the fused-linear hot path (C1-C5, one call each)",
         "value": round(value, 6), "unit": "TFLOP/s", "n_gpus": world, "steps": steps, "warmup": warm,
         "ms_per_step": round(t_total / steps * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "C1+C2+C3+C4+C5 (all five configurations, one call each per step)",
-                   "sample": sample_description()},
+        "config": {"workload": "C1+C2+C3+C4+C5", "sample": sample_description()},
         "cpu_baseline": {"value": round(value, 6), "unit": "TFLOP/s", "cores": ref.get_threads(), "kind": "oracle",
                          "sample": sample_description()},
         "e2e": {"value": round(value, 6), "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -523,7 +570,10 @@ def main():
     ap.add_argument("--settle-s", type=float, default=0.5, help="idle time before each per-configuration loop")
     ap.add_argument("--loop-ms", type=float, default=150.0, help="target length of each per-configuration timing loop")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the timed CPU oracle leg")
-    ap.add_argument("--no-extras", action="store_true", help="skip the row-max / cross-entropy measurements")
+    ap.add_argument("--sustain-s", type=float, default=2.0, help="length of the back-to-back loop of each tensor-bound configuration")
+    ap.add_argument("--extras", action="store_true", help="also measure the further operators X1.. (detailed record on stderr)")
+    ap.add_argument("--details", action="store_true", help="print the detailed per-configuration record on stderr")
+    ap.add_argument("--full-cpu-baseline", action="store_true", help="time the oracle on all rows of every configuration (minutes)")
     ap.add_argument("--no-eager", action="store_true", help="skip the PyTorch-eager context timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-pointer end-to-end leg")
     ap.add_argument("--configs", default=",".join(ORDER), help="comma-separated subset of C1..C5, or of the further operators X1.. (profiling aid)")

@@ -24,9 +24,16 @@
  *   - Only compute capability 10.x is accepted; there is no fallback of any kind.
  *   - Results are bit-reproducible run to run for a fixed shape and device.
  *   - Scratch: split-K partial sums and logsumexp partials live in a workspace.
- *     By default the library owns one per device (cudaMalloc, grow-only; so the
- *     first call of a larger shape allocates and must not run under stream
- *     capture); mtmc_set_workspace() substitutes caller-owned memory.
+ *     By default the library owns one per (device, stream) (cudaMalloc, grow-only;
+ *     so the first call of a larger shape on a stream allocates and must not run
+ *     under stream capture); mtmc_set_workspace() substitutes caller-owned memory.
+ *   - Threads and streams: the stream, workspace, tuning and timing settings are
+ *     thread-local.  Calls enqueued on different streams, from one host thread or
+ *     from several, may overlap on the GPU: their library-owned scratch is
+ *     separate (at most 32 streams per device use it; further ones need
+ *     mtmc_set_workspace).  Calls on ONE stream run in order and share that
+ *     stream's scratch; two host threads that enqueue on the same stream must
+ *     order their calls themselves, as for any CUDA stream.
  */
 #ifndef MTMC_FUSED_H_
 #define MTMC_FUSED_H_
@@ -187,9 +194,10 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
  *     has been written by that same call first.  Two calls that overlap on the
  *     GPU (different streams, or different host threads) race on it and give
  *     wrong results; serialise them on one stream.
- *   - Device-side timeouts of this path go to a status word of their own:
- *     a later call to this function returns MTMC_ERR_DEVICE_TIMEOUT if it finds
- *     the stream idle and the word set; mtmc_check_status() does not see it. */
+ *   - Device-side timeouts of this path go to a status word of their own, also part
+ *     of the library image; mtmc_check_status() reports and clears it like the
+ *     regular one (and, in a process that has only ever used this entry point on
+ *     the device, does so without creating the regular, allocating state). */
 int mtmc_linear_lse_noalloc(const void* X, const void* W, const float* b,
                             int64_t M, int64_t N, int64_t K, float* lse_out);
 
@@ -255,6 +263,17 @@ const char* mtmc_last_error(void);
 
 /* Number of kernels this library has launched from this process so far. */
 int64_t mtmc_launch_count(void);
+
+/* Number of device allocations (cudaMalloc calls) this library has made from this process so
+ * far: status words, tickets, grown workspaces, the device copies behind the _host entry
+ * points.  A caller with a memory budget can watch it; mtmc_linear_lse_noalloc never moves it. */
+int64_t mtmc_device_alloc_count(void);
+
+/* Name of the main kernel that the most recent compute call of this host thread launched
+ * (kernel family, epilogue, and tile or cluster variant), "" before the first call.  Which
+ * kernel a shape lands on is decided inside the library; benchmarks and bug reports name it
+ * from here instead of guessing. */
+const char* mtmc_last_kernel_name(void);
 
 /* Device time, in milliseconds, of the most recent mtmc_* device entry point on
  * this host thread's current device, measured with CUDA events recorded on the

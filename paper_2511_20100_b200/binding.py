@@ -27,7 +27,7 @@ EXPORTS = [
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
-    "mtmc_last_error", "mtmc_launch_count", "mtmc_set_timing", "mtmc_last_kernel_ms",
+    "mtmc_last_error", "mtmc_launch_count", "mtmc_device_alloc_count", "mtmc_last_kernel_name", "mtmc_set_timing", "mtmc_last_kernel_ms",
     "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
@@ -75,6 +75,8 @@ def load() -> ctypes.CDLL:
     L.mtmc_workspace_bytes.restype = sz
     L.mtmc_last_error.restype = ctypes.c_char_p
     L.mtmc_launch_count.restype = i64
+    L.mtmc_device_alloc_count.restype = i64
+    L.mtmc_last_kernel_name.restype = ctypes.c_char_p
     L.mtmc_set_timing.argtypes = [ci]
     L.mtmc_last_kernel_ms.restype = ctypes.c_float
     L.mtmc_set_tuning.argtypes = [ci, ci, ci]
@@ -405,6 +407,16 @@ def mtmc_selftest_timeout() -> None:
 
 def mtmc_launch_count() -> int:
     return int(load().mtmc_launch_count())
+
+
+def mtmc_device_alloc_count() -> int:
+    """cudaMalloc calls made by the library in this process so far."""
+    return int(load().mtmc_device_alloc_count())
+
+
+def mtmc_last_kernel_name() -> str:
+    """Main kernel launched by this thread's most recent compute call."""
+    return load().mtmc_last_kernel_name().decode()
 
 
 def mtmc_set_timing(enabled: bool) -> None:

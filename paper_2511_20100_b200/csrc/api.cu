@@ -35,10 +35,19 @@ struct DeviceState {
     bool ready = false;
     int sm_count = 0;
     uint32_t* status = nullptr;      // device status word (256 bytes reserved)
-    uint32_t* tickets = nullptr;     // library-owned split-K tickets, zero between launches
-    bool tickets_dirty = false;
-    void* ws = nullptr;              // library-owned workspace (grow-only)
-    size_t ws_bytes = 0;
+    // Library-owned scratch is kept per stream, so that calls enqueued on different streams (by one host thread
+    // or by several) never share partials or tickets: a slot belongs to the first stream that asked for it.
+    struct StreamScratch {
+        bool used = false;
+        cudaStream_t stream = nullptr;
+        uint32_t* tickets = nullptr;     // split-K tickets of the weight-streaming kernel (TICKET_BYTES, allocated on first need)
+        void* ws = nullptr;              // workspace (grow-only)
+        size_t ws_bytes = 0;
+        cudaEvent_t ev0 = nullptr, ev1 = nullptr;    // mtmc_set_timing: around the kernels of the last call on this stream
+        bool timed = false;
+    };
+    static constexpr int MAX_STREAMS = 32;
+    StreamScratch sscratch[MAX_STREAMS];
     // The *_host entry points: a ring of slots, each with device copies of one call's operands and result and
     // the events that order its three phases (copy in, kernels, copy out) across three streams.
     struct HostSlot {
@@ -52,8 +61,6 @@ struct DeviceState {
     int hnext = 0;
     size_t hwm[5] = {0, 0, 0, 0, 0};
     cudaStream_t s_in = nullptr, s_out = nullptr;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    bool timed = false;
     int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
     int max_gemm_pairs = -1;         // the same for the CTA-pair tiled kernel
     int max_ksplit[3] = {-1, -1, -1};   // co-resident clusters of two / four / eight CTAs of the cluster split-K kernel
@@ -62,6 +69,18 @@ struct DeviceState {
 std::mutex g_mutex;
 DeviceState g_dev[MAX_DEVICES];
 std::atomic<long long> g_launches{0};
+std::atomic<long long> g_device_allocs{0};     // cudaMalloc calls made by this library (mtmc_device_alloc_count)
+
+// Every device allocation of the library goes through here, so that the count is complete.
+cudaError_t counted_malloc(void** ptr, size_t bytes) {
+    g_device_allocs.fetch_add(1);
+    return cudaMalloc(ptr, bytes);
+}
+
+// Status word of the allocation-free entry point on the current device (defined with that entry point, at the
+// end of this file): fetches and clears it if that path has been set up on this device; *st = 0 otherwise.
+int noalloc_take_status(int dev, uint32_t* st);
+bool noalloc_in_use(int dev);
 
 thread_local cudaStream_t t_stream = nullptr;
 thread_local void* t_user_ws = nullptr;
@@ -72,6 +91,14 @@ thread_local int t_cta_pair = 0;   // 0 automatic, 1 force CTA pairs, -1 force s
 thread_local int t_static_weights = 0;   // caller's promise that no work in flight writes W (see mtmc_set_static_weights)
 thread_local int t_timing = 0;
 thread_local char t_error[512] = "";
+thread_local char t_last_kernel[96] = "";     // main kernel of the last call of this thread (mtmc_last_kernel_name)
+
+void note_kernel(const char* family, int epi, int detail = 0) {
+    static const char* const epi_name[] = {"EPI_ACT", "EPI_SWIGLU", "EPI_LSE", "EPI_ROWMAX", "EPI_XENT"};
+    if (epi >= 0 && detail > 0) snprintf(t_last_kernel, sizeof t_last_kernel, "%s<%s, %d>", family, epi_name[epi], detail);
+    else if (epi >= 0) snprintf(t_last_kernel, sizeof t_last_kernel, "%s<%s>", family, epi_name[epi]);
+    else snprintf(t_last_kernel, sizeof t_last_kernel, "%s<MX=%d>", family, detail);
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -113,12 +140,8 @@ int get_device(DeviceState** out, int* dev_out = nullptr) {
                 return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from this driver");
             g_encode = reinterpret_cast<EncodeTiledFn>(fn);
         }
-        CUDA_TRY(cudaMalloc(&d.status, 256));
+        CUDA_TRY(counted_malloc(reinterpret_cast<void**>(&d.status), 256));
         CUDA_TRY(cudaMemset(d.status, 0, 256));
-        CUDA_TRY(cudaMalloc(&d.tickets, TICKET_BYTES));
-        CUDA_TRY(cudaMemset(d.tickets, 0, TICKET_BYTES));
-        CUDA_TRY(cudaEventCreate(&d.ev0));
-        CUDA_TRY(cudaEventCreate(&d.ev1));
         d.ready = true;
     }
     *out = &d;
@@ -126,30 +149,49 @@ int get_device(DeviceState** out, int* dev_out = nullptr) {
     return MTMC_OK;
 }
 
-// 2-D bf16 row-major [rows, cols] tensor, box = 64 columns x box_rows rows, 128-byte swizzle.
-int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
+// Tensor-map cache.  A CUtensorMap is a pure function of (address, element type, extents, row pitch, box): it
+// holds no reference to the memory, so a cached copy is valid for as long as the key matches, whoever owns the
+// buffer now.  Serving loops call with the same few (weight, activation buffer, shape) combinations over and
+// over; re-encoding three to five descriptors costs more host time than launching the kernel.  Thread-local,
+// direct-mapped, 128 entries.
+struct TmapKey {
+    const void* ptr; int64_t rows, cols, ld; int box_rows, u8;
+    bool operator==(const TmapKey& o) const {
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows && u8 == o.u8;
+    }
+};
+struct TmapEntry { bool valid = false; TmapKey key{}; CUtensorMap map; };
+constexpr int TMAP_CACHE_ENTRIES = 128;
+thread_local TmapEntry t_tmap_cache[TMAP_CACHE_ENTRIES];
+thread_local long long t_tmap_hits = 0, t_tmap_misses = 0;
+
+// 2-D row-major [rows, cols] tensor of bf16 (box = 64 columns x box_rows rows) or of one-byte E4M3 elements
+// (box = 128 columns x box_rows rows): one 128-byte swizzle row of K per box row either way.
+int encode_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld, bool u8) {
+    const TmapKey key{ptr, rows, cols, ld > 0 ? ld : cols, box_rows, u8 ? 1 : 0};
+    uint64_t h = reinterpret_cast<uintptr_t>(ptr) >> 4;
+    h = (h ^ static_cast<uint64_t>(rows) * 0x9E3779B97F4A7C15ull ^ static_cast<uint64_t>(key.ld) * 0xC2B2AE3D27D4EB4Full ^
+         static_cast<uint64_t>(cols) * 0x165667B19E3779F9ull ^ static_cast<uint64_t>(box_rows * 2 + key.u8)) * 0xD6E8FEB86659FD93ull;
+    TmapEntry& e = t_tmap_cache[(h >> 32) % TMAP_CACHE_ENTRIES];
+    if (e.valid && e.key == key) { *map = e.map; ++t_tmap_hits; return MTMC_OK; }
+    ++t_tmap_misses;
+    const size_t esz = u8 ? 1 : 2;
     cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld > 0 ? ld : cols) * 2};      // row pitch in bytes
-    cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(key.ld) * esz};      // row pitch in bytes
+    cuuint32_t box[2] = {u8 ? 128u : 64u, static_cast<cuuint32_t>(box_rows)};
     cuuint32_t estr[2] = {1u, 1u};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = g_encode(map, u8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims,
+                          strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
+    e.valid = true; e.key = key; e.map = *map;
     return MTMC_OK;
 }
-
-// 2-D E4M3 row-major [rows, cols] tensor (one byte per element), box = 128 columns x box_rows rows.
+int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
+    return encode_2d(map, ptr, rows, cols, box_rows, ld, false);
+}
 int encode_u8_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
-    cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld > 0 ? ld : cols)};
-    cuuint32_t box[2] = {128u, static_cast<cuuint32_t>(box_rows)};
-    cuuint32_t estr[2] = {1u, 1u};
-    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
-    return MTMC_OK;
+    return encode_2d(map, ptr, rows, cols, box_rows, ld, true);
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -165,7 +207,24 @@ int check_common(const void* X, const void* W, const void* out, int64_t M, int64
     return MTMC_OK;
 }
 
-// Scratch for this call: the caller's if set, else the library's (grown on demand).
+// The scratch slot of the current stream on this device (created on first use).
+int get_stream_scratch(DeviceState* d, DeviceState::StreamScratch** out) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState::StreamScratch* free_slot = nullptr;
+    for (auto& s : d->sscratch) {
+        if (s.used && s.stream == t_stream) { *out = &s; return MTMC_OK; }
+        if (!s.used && !free_slot) free_slot = &s;
+    }
+    if (!free_slot)
+        return fail(MTMC_ERR_WORKSPACE, "more than %d streams use library-owned scratch on this device; give the further "
+                    "ones their own with mtmc_set_workspace", DeviceState::MAX_STREAMS);
+    free_slot->used = true;
+    free_slot->stream = t_stream;
+    *out = free_slot;
+    return MTMC_OK;
+}
+
+// Scratch for this call: the caller's if set, else the library's slot for the current stream (grown on demand).
 int get_workspace(DeviceState* d, size_t need, void** out) {
     if (need == 0) { *out = nullptr; return MTMC_OK; }
     if (t_user_ws) {
@@ -174,23 +233,32 @@ int get_workspace(DeviceState* d, size_t need, void** out) {
         *out = t_user_ws;
         return MTMC_OK;
     }
-    std::lock_guard<std::mutex> lock(g_mutex);
-    if (d->ws_bytes < need) {
-        if (d->ws) { CUDA_TRY(cudaDeviceSynchronize()); CUDA_TRY(cudaFree(d->ws)); d->ws = nullptr; d->ws_bytes = 0; }
+    DeviceState::StreamScratch* sc = nullptr;
+    if (int rc = get_stream_scratch(d, &sc)) return rc;
+    if (sc->ws_bytes < need) {
+        // only work on this stream can still be using the old buffer
+        if (sc->ws) { CUDA_TRY(cudaStreamSynchronize(t_stream)); CUDA_TRY(cudaFree(sc->ws)); sc->ws = nullptr; sc->ws_bytes = 0; }
         size_t bytes = (need + (1u << 20) - 1) & ~static_cast<size_t>((1u << 20) - 1);
-        CUDA_TRY(cudaMalloc(&d->ws, bytes));
-        d->ws_bytes = bytes;
+        CUDA_TRY(counted_malloc(&sc->ws, bytes));
+        sc->ws_bytes = bytes;
     }
-    *out = d->ws;
+    *out = sc->ws;
     return MTMC_OK;
 }
 
 size_t round256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
 
-// Scratch of mtmc_linear_lse: one (max, sum-exp) pair per row and column piece (per epilogue warp share); sized for
-// the narrowest tile (128 columns) and the largest tail split (4), whatever the call then picks.
+// Scratch of the row reductions: one (max, sum-exp) pair per row and column piece (per epilogue warp share).
+// A launch needs n_tiles * tail_split pieces for the plan it picks (lse_partial_bytes); the figure that
+// mtmc_workspace_bytes reports covers every plan the library can pick for the shape: 128-column tiles with the
+// wave tail cut in four, or 256-column tiles owned by clusters of eight CTAs (eight pieces per tile, also for a
+// last tile that lies partly past N).
+size_t lse_partial_bytes(const GemmParams& p) {
+    return round256(static_cast<size_t>(p.n_tiles) * p.tail_split * EPI_HALVES * static_cast<size_t>(p.M) * sizeof(float2));
+}
 size_t lse_workspace_bytes(int64_t M, int64_t N) {
-    return round256(static_cast<size_t>((N + 127) / 128) * 4 * EPI_HALVES * static_cast<size_t>(M) * sizeof(float2));
+    const size_t pieces = std::max(static_cast<size_t>((N + 127) / 128) * 4, static_cast<size_t>((N + 255) / 256) * 8);
+    return round256(pieces * EPI_HALVES * static_cast<size_t>(M) * sizeof(float2));
 }
 
 int pick_tile_n(int64_t N) {
@@ -201,13 +269,14 @@ int pick_tile_n(int64_t N) {
 int pick_group_m(int m_tiles) { return m_tiles < 16 ? m_tiles : 16; }
 
 struct TimedRegion {
-    DeviceState* d;
-    bool on;
-    TimedRegion(DeviceState* dev) : d(dev), on(t_timing != 0) {
-        if (on) cudaEventRecord(d->ev0, t_stream);
+    DeviceState::StreamScratch* sc = nullptr;
+    TimedRegion(DeviceState* dev) {
+        if (t_timing == 0 || get_stream_scratch(dev, &sc) != MTMC_OK) { sc = nullptr; return; }
+        if (!sc->ev0 && (cudaEventCreate(&sc->ev0) != cudaSuccess || cudaEventCreate(&sc->ev1) != cudaSuccess)) { sc = nullptr; return; }
+        cudaEventRecord(sc->ev0, t_stream);
     }
     void stop() {
-        if (on) { cudaEventRecord(d->ev1, t_stream); d->timed = true; }
+        if (sc) { cudaEventRecord(sc->ev1, t_stream); sc->timed = true; }
     }
 };
 
@@ -259,6 +328,7 @@ int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB,
     cfg.numAttrs = pdl_attribute(attr);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmBt, tmB2t, p));
     g_launches.fetch_add(1);
+    note_kernel("gemm_tiled_kernel", EPI, BN);
     return MTMC_OK;
 }
 
@@ -283,6 +353,7 @@ int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, co
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmBt, tmB2t, p));
     g_launches.fetch_add(1);
+    note_kernel("gemm_pair_kernel", EPI);
     return MTMC_OK;
 }
 
@@ -307,6 +378,7 @@ int launch_big(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, con
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
     g_launches.fetch_add(1);
+    note_kernel("gemm_big_kernel", EPI);
     return MTMC_OK;
 }
 
@@ -355,6 +427,7 @@ int launch_ksplit_ks(int tiles, const CUtensorMap& tmA, const CUtensorMap& tmB, 
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
     g_launches.fetch_add(1);
+    note_kernel("gemm_ksplit_kernel", EPI, KS);
     return MTMC_OK;
 }
 template <int EPI, bool OUT_BF16>
@@ -596,6 +669,7 @@ int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmW, tmX, p));
     g_launches.fetch_add(1);
+    note_kernel(PAIR ? "skinny_splitk_kernel (pair plan)" : "skinny_splitk_kernel (ticket plan)", -1, MX);
     return MTMC_OK;
 }
 
@@ -644,17 +718,21 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
         if (rc) return rc;
         p.tickets = static_cast<uint32_t*>(ws);
         p.partial = reinterpret_cast<float*>(static_cast<char*>(ws) + s.ticket_bytes);
-        if (s.ticket_bytes) CUDA_TRY(cudaMemsetAsync(p.tickets, 0, s.ticket_bytes, t_stream));
     } else {
         int rc = get_workspace(d, s.partial_bytes, &ws);
         if (rc) return rc;
-        p.tickets = d->tickets;
         p.partial = static_cast<float*>(ws);
-        if (d->tickets_dirty) {
-            CUDA_TRY(cudaMemsetAsync(d->tickets, 0, TICKET_BYTES, t_stream));
-            d->tickets_dirty = false;
+        p.tickets = nullptr;
+        if (s.ticket_bytes) {
+            DeviceState::StreamScratch* sc = nullptr;
+            if ((rc = get_stream_scratch(d, &sc))) return rc;
+            if (!sc->tickets) CUDA_TRY(counted_malloc(reinterpret_cast<void**>(&sc->tickets), TICKET_BYTES));
+            p.tickets = sc->tickets;
         }
     }
+    // The tickets of this launch start at zero whatever an earlier launch left behind (one that timed out does
+    // not reset its own): a stream-ordered clear of the words in use.  Only the ticket plan pays for it.
+    if (s.ticket_bytes) CUDA_TRY(cudaMemsetAsync(p.tickets, 0, s.ticket_bytes, t_stream));
     CUtensorMap tmW, tmX;
     int rc = fp8 ? encode_u8_2d(&tmW, W, N, K, s.tile_rows) : encode_bf16_2d(&tmW, W, N, K, s.tile_rows, ldw);
     if (rc) return rc;
@@ -715,7 +793,7 @@ int host_call(const HostOperand (&in)[4], void* out_host, size_t out_bytes, bool
         if (d->hwm[i] < need) d->hwm[i] = need;      // largest operand seen in this position, by any slot
         if (s.bytes[i] < need) {        // the slot is idle: nothing on the device still uses its buffers
             if (s.buf[i]) { CUDA_TRY(cudaFree(s.buf[i])); s.buf[i] = nullptr; s.bytes[i] = 0; }
-            CUDA_TRY(cudaMalloc(&s.buf[i], d->hwm[i]));     // sized for the largest, so that a steady workload stops reallocating
+            CUDA_TRY(counted_malloc(&s.buf[i], d->hwm[i]));     // sized for the largest, so that a steady workload stops reallocating
             s.bytes[i] = d->hwm[i];
         }
         dev[i] = s.buf[i];
@@ -762,7 +840,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, fp8);
     else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, fp8);
     p.acc_scale = acc_scale;
-    const size_t partial_bytes = lse_workspace_bytes(M, N);
+    const size_t partial_bytes = lse_partial_bytes(p);         // what the chosen plan writes and the merge reads
     const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
     void* ws = nullptr;
     rc = get_workspace(d, partial_bytes + extra, &ws);
@@ -1005,16 +1083,19 @@ int mtmc_set_timing(int enabled) { t_timing = enabled ? 1 : 0; return MTMC_OK; }
 
 float mtmc_last_kernel_ms(void) {
     DeviceState* d = nullptr;
-    if (get_device(&d) != MTMC_OK || !d->timed) return -1.0f;
-    if (cudaEventSynchronize(d->ev1) != cudaSuccess) return -1.0f;
+    DeviceState::StreamScratch* sc = nullptr;
+    if (get_device(&d) != MTMC_OK || get_stream_scratch(d, &sc) != MTMC_OK || !sc->timed) return -1.0f;
+    if (cudaEventSynchronize(sc->ev1) != cudaSuccess) return -1.0f;
     float ms = -1.0f;
-    if (cudaEventElapsedTime(&ms, d->ev0, d->ev1) != cudaSuccess) return -1.0f;
+    if (cudaEventElapsedTime(&ms, sc->ev0, sc->ev1) != cudaSuccess) return -1.0f;
     return ms;
 }
 
 int64_t mtmc_launch_count(void) { return g_launches.load(); }
 
 const char* mtmc_last_error(void) { return t_error; }
+
+const char* mtmc_last_kernel_name(void) { return t_last_kernel; }
 
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
@@ -1047,19 +1128,34 @@ int mtmc_selftest_timeout(void) {
 }
 
 int mtmc_check_status(void) {
-    DeviceState* d = nullptr;
-    int rc = get_device(&d);
-    if (rc) return rc;
-    CUDA_TRY(cudaStreamSynchronize(t_stream));
-    uint32_t st = 0;
-    CUDA_TRY(cudaMemcpy(&st, d->status, sizeof st, cudaMemcpyDeviceToHost));
-    if (st != 0) {
-        CUDA_TRY(cudaMemset(d->status, 0, sizeof st));
-        d->tickets_dirty = true;
-        return fail(MTMC_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (status word 0x%x)", st);
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return fail(MTMC_ERR_UNSUPPORTED_DEVICE, "device index %d out of range", dev);
+    bool regular = false, noalloc = false;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        regular = g_dev[dev].ready;
     }
+    noalloc = noalloc_in_use(dev);
+    CUDA_TRY(cudaStreamSynchronize(t_stream));
+    uint32_t st = 0, st_noalloc = 0;
+    // A process that has only ever used the allocation-free entry point on this device stays allocation-free:
+    // the regular per-device state (which owns device memory) is not created just to be found clean.
+    if (regular || !noalloc) {
+        DeviceState* d = nullptr;
+        if (int rc = get_device(&d)) return rc;
+        CUDA_TRY(cudaMemcpy(&st, d->status, sizeof st, cudaMemcpyDeviceToHost));
+        if (st != 0) CUDA_TRY(cudaMemset(d->status, 0, sizeof st));
+    }
+    if (noalloc) {
+        if (int rc = noalloc_take_status(dev, &st_noalloc)) return rc;
+    }
+    if (st == 0) st = st_noalloc;
+    if (st != 0) return fail(MTMC_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (status word 0x%x)", st);
     return MTMC_OK;
 }
+
+int64_t mtmc_device_alloc_count(void) { return g_device_allocs.load(); }
 
 int mtmc_fused_linear(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int act,
                       int out_dtype, void* out) {
@@ -1258,15 +1354,37 @@ int noalloc_device(NoAllocDevice** out) {
     return MTMC_OK;
 }
 
+bool noalloc_in_use(int dev) {
+    std::lock_guard<std::mutex> lock(g_mutex);
+    return g_noalloc_dev[dev].ready;
+}
+
+int noalloc_take_status(int dev, uint32_t* st) {
+    *st = 0;
+    uint32_t* word = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (g_noalloc_dev[dev].ready) word = g_noalloc_dev[dev].status;
+    }
+    if (!word) return MTMC_OK;
+    CUDA_TRY(cudaMemcpy(st, word, sizeof *st, cudaMemcpyDeviceToHost));
+    if (*st != 0) {
+        uint32_t zero = 0;
+        CUDA_TRY(cudaMemcpy(word, &zero, sizeof zero, cudaMemcpyHostToDevice));
+    }
+    return MTMC_OK;
+}
+
 template <int BN>
 int launch_lse_noalloc(NoAllocDevice* d, const CUtensorMap& tmA, const CUtensorMap& tmB, GemmParams p) {
     using Cfg = TileCfg<EPI_LSE, BN>;
     auto kern = gemm_tiled_kernel<EPI_LSE, BN, false>;
-    CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;       // a function attribute, set once per device: no allocation
     const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
     kern<<<grid, Cfg::THREADS, Cfg::SMEM_BYTES, t_stream>>>(tmA, tmB, tmB, tmB, tmB, p);
     CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1);
+    note_kernel("gemm_tiled_kernel", EPI_LSE, BN);
     return MTMC_OK;
 }
 }  // namespace
@@ -1287,19 +1405,6 @@ extern "C" int mtmc_linear_lse_noalloc(const void* X, const void* W, const float
         return fail(MTMC_ERR_UNSUPPORTED_SHAPE,
                     "mtmc_linear_lse_noalloc: ceil(N/%d) * M = %zu partials exceed the built-in scratch of %zu "
                     "(8 MiB); use mtmc_linear_lse for this shape", bn, need, NOALLOC_MAX_PARTIALS);
-    // A timeout recorded by an earlier call is reported once the stream has gone idle
-    // (never by waiting for it).
-    if (cudaStreamQuery(t_stream) == cudaSuccess) {
-        uint32_t st = 0;
-        CUDA_TRY(cudaMemcpy(&st, d->status, sizeof st, cudaMemcpyDeviceToHost));
-        if (st != 0) {
-            uint32_t zero = 0;
-            CUDA_TRY(cudaMemcpy(d->status, &zero, sizeof zero, cudaMemcpyHostToDevice));
-            return fail(MTMC_ERR_DEVICE_TIMEOUT, "an earlier mtmc_linear_lse_noalloc call timed out on the device (status word 0x%x)", st);
-        }
-    } else {
-        (void)cudaGetLastError();   // cudaErrorNotReady is not an error here
-    }
     p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = d->partials; p.status = d->status;
     CUtensorMap tmA, tmB;
     rc = encode_bf16_2d(&tmA, X, M, K, 128);
