@@ -53,6 +53,7 @@ extern "C" {
 #define MTMC_ERR_CUDA 4               /* CUDA runtime / driver error; text in mtmc_last_error() */
 #define MTMC_ERR_DEVICE_TIMEOUT 5     /* a bounded device-side wait expired */
 #define MTMC_ERR_WORKSPACE 6          /* caller-provided workspace too small */
+#define MTMC_ERR_DEVICE_CHECK 7       /* -DMTMC_CHECKS builds only: a device-side index check failed (the access was skipped) */
 
 /* activation ids for mtmc_fused_linear */
 #define MTMC_ACT_NONE 0
@@ -243,8 +244,9 @@ int mtmc_set_stream(void* cuda_stream);
  * workspace.  Thread-local. */
 int mtmc_set_workspace(void* dptr, size_t bytes);
 
-/* Scratch bytes the given operation needs for this shape on the current device
- * (0 if none; (size_t)-1 on invalid arguments). */
+/* Scratch bytes that suffice for the given operation and shape on the current device under this
+ * thread's current tuning, whichever kernel and schedule the library picks (0 if none; (size_t)-1 on
+ * invalid arguments). */
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K);
 
 /* Synchronises the current stream, then returns and clears the sticky device
@@ -295,6 +297,31 @@ float mtmc_last_kernel_ms(void);
  *              reductions and for activation epilogues with a long K, never for SwiGLU
  *              (measured on a par at best) */
 int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
+
+/* Device-side trace, for builds of the library compiled with -DMTMC_TRACE (the default build has none:
+ * mtmc_trace_enabled() returns 0 and mtmc_set_trace() with a buffer fails with MTMC_ERR_INVALID_ARG).
+ * dptr is a zero-filled device buffer of `bytes` bytes, 8-byte aligned, owned by the caller; (NULL, 0)
+ * switches tracing off.  Thread-local.  While set, the CTA-pair kernels and the weight-streaming kernel
+ * write one record of 32 uint64 per CTA (launches of more CTAs than the buffer holds are not traced):
+ * %globaltimer stamps of set-up, first / last load, first / last MMA, first / last epilogue, and cycle
+ * totals of each role's waits (producer on a free stage, MMA issuer on data and on a drained accumulator,
+ * epilogue on an accumulator, stream-K hand-overs); word indices are the TR_* constants of
+ * paper_2511_20100_b200/csrc/ptx.cuh, decoded by `python -m paper_2511_20100_b200.trace`.  Stall figures
+ * quoted for this library come from there.  No counterpart in the paper. */
+int mtmc_trace_enabled(void);
+int mtmc_set_trace(void* dptr, size_t bytes);
+
+/* Work schedule of the CTA-pair kernel with 256 x 256 tiles (thread-local; default 0).
+ *   stream_k : 1 = deal the last full wave of tiles plus the remainder by k-blocks: the flat list of that
+ *              region's (tile, k-block) units is cut into one equal, contiguous share per CTA pair, so that
+ *              all pairs finish together whatever the tile count (needs at least as many tiles as pairs); a
+ *              tile whose k-blocks straddle two shares is finished by whichever of its two holders comes
+ *              second, from fp32 accumulator parts kept in the workspace (bit-reproducible: two addends
+ *              commute); 0 or negative = whole tiles, the last wave's tiles cut into column pieces (the
+ *              default: measured on a par or ahead on this library's benchmark shapes).
+ * The schedule needs workspace (mtmc_workspace_bytes includes it while it is switched on).  It follows the
+ * paper's Tiling and Reordering principles: the same tiles, dealt differently. */
+int mtmc_set_schedule(int stream_k);
 
 /* Static weights (thread-local, default 0 = off).  With enabled != 0 the caller promises, for
  * the calls that follow on this thread, that no work still in flight on the device writes

@@ -13,10 +13,12 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmtmcfused.so")
+# MTMC_LIB_VARIANT=trace loads the build with device-side trace stamps (libmtmcfused_trace.so, see build.py)
+VARIANT = os.environ.get("MTMC_LIB_VARIANT", "")
+LIB_PATH = os.path.join(_HERE, "libmtmcfused%s.so" % ("_" + VARIANT if VARIANT else ""))
 
 OK = 0
-ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_WORKSPACE = 1, 2, 3, 4, 5, 6
+ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_WORKSPACE, ERR_DEVICE_CHECK = 1, 2, 3, 4, 5, 6, 7
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}
 OUT_DTYPE = {"fp32": 0, "bf16": 1}
 OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4}
@@ -28,7 +30,7 @@ EXPORTS = [
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_device_alloc_count", "mtmc_last_kernel_name", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_schedule", "mtmc_trace_enabled", "mtmc_set_trace", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -46,10 +48,10 @@ def load() -> ctypes.CDLL:
     if _lib is not None:
         return _lib
     from . import build as _build
-    if _build.needs_build():
+    if _build.needs_build(VARIANT):
         # missing or older than its sources: compile it in-tree (nvcc); there is no other code path to fall back on
         try:
-            _build.build()
+            _build.build(variant=VARIANT)
         except Exception as e:
             raise RuntimeError("libmtmcfused.so is missing or stale at %s and could not be built (%s); "
                                "there is no fallback path" % (LIB_PATH, e))
@@ -81,6 +83,8 @@ def load() -> ctypes.CDLL:
     L.mtmc_last_kernel_ms.restype = ctypes.c_float
     L.mtmc_set_tuning.argtypes = [ci, ci, ci]
     L.mtmc_set_static_weights.argtypes = [ci]
+    L.mtmc_set_schedule.argtypes = [ci]
+    L.mtmc_set_trace.argtypes = [vp, sz]
     _lib = L
     return L
 
@@ -429,6 +433,23 @@ def mtmc_last_kernel_ms() -> float:
 
 def mtmc_set_tuning(split_k: int = 0, tile_n: int = 0, cta_pair: int = 0) -> None:
     _check(load().mtmc_set_tuning(int(split_k), int(tile_n), int(cta_pair)))
+
+
+def mtmc_trace_enabled() -> bool:
+    return bool(load().mtmc_trace_enabled())
+
+
+def mtmc_set_trace(t: torch.Tensor | None) -> None:
+    """Hands the trace build a zero-filled int64 CUDA tensor (32 words per CTA), or None to stop tracing."""
+    if t is None:
+        _check(load().mtmc_set_trace(None, 0))
+    else:
+        _check(load().mtmc_set_trace(ctypes.c_void_p(t.data_ptr()), t.numel() * t.element_size()))
+
+
+def mtmc_set_schedule(stream_k: int = 0) -> None:
+    """Stream-K schedule of the 256 x 256 pair kernel: 1 wherever legal, -1 never, 0 automatic."""
+    _check(load().mtmc_set_schedule(int(stream_k)))
 
 
 def mtmc_set_static_weights(enabled: bool = True) -> None:

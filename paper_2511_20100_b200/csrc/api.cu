@@ -26,6 +26,9 @@ using namespace mtmc;
 
 constexpr int MAX_DEVICES = 64;
 constexpr size_t TICKET_BYTES = 64 * 1024;   // library-owned split-K tickets: 16384 tiles
+constexpr int SK_MAX_PAIRS = 256;            // stream-K boundaries (pairs of one launch) the flag array covers
+constexpr size_t SK_FLAG_BYTES = SK_MAX_PAIRS * 8 * sizeof(uint32_t);
+constexpr size_t SK_PART_BYTES = 2 * 2 * 4 * 8 * 8 * 32 * sizeof(float4);   // per boundary: 2 sides x 2 ranks x 4 quadrants x 32 KiB
 #ifndef MTMC_SKINNY_MAX_M
 #define MTMC_SKINNY_MAX_M 64
 #endif
@@ -45,6 +48,8 @@ struct DeviceState {
         size_t ws_bytes = 0;
         cudaEvent_t ev0 = nullptr, ev1 = nullptr;    // mtmc_set_timing: around the kernels of the last call on this stream
         bool timed = false;
+        uint32_t* sk_flags = nullptr;    // stream-K flag words (SK_FLAG_BYTES, zeroed once: launches tell themselves apart by epoch)
+        uint32_t sk_epoch = 0;
     };
     static constexpr int MAX_STREAMS = 32;
     StreamScratch sscratch[MAX_STREAMS];
@@ -88,8 +93,11 @@ thread_local size_t t_user_ws_bytes = 0;
 thread_local int t_split_k = 0;
 thread_local int t_tile_n = 0;
 thread_local int t_cta_pair = 0;   // 0 automatic, 1 force CTA pairs, -1 force single CTAs
+thread_local int t_stream_k = 0;   // 0 automatic, 1 stream-K wherever it is legal, -1 never (mtmc_set_schedule)
 thread_local int t_static_weights = 0;   // caller's promise that no work in flight writes W (see mtmc_set_static_weights)
 thread_local int t_timing = 0;
+thread_local unsigned long long* t_trace = nullptr;   // caller's trace buffer (mtmc_set_trace), used by -DMTMC_TRACE builds
+thread_local size_t t_trace_bytes = 0;
 thread_local char t_error[512] = "";
 thread_local char t_last_kernel[96] = "";     // main kernel of the last call of this thread (mtmc_last_kernel_name)
 
@@ -104,6 +112,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
+
+// The trace buffer for a launch of `ctas` CTAs, if the caller gave one that is large enough.
+unsigned long long* trace_for(unsigned ctas) {
+#ifdef MTMC_TRACE
+    if (t_trace && t_trace_bytes >= static_cast<size_t>(ctas) * TRACE_WORDS * sizeof(unsigned long long)) return t_trace;
+#endif
+    (void)ctas;
+    return nullptr;
+}
 
 int fail(int code, const char* fmt, ...) {
     va_list ap;
@@ -351,7 +368,9 @@ int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, co
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmBt, tmB2t, p));
+    GemmParams q = p;
+    q.trace = trace_for(cfg.gridDim.x);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmBt, tmB2t, q));
     g_launches.fetch_add(1);
     note_kernel("gemm_pair_kernel", EPI);
     return MTMC_OK;
@@ -376,7 +395,9 @@ int launch_big(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, con
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
+    GemmParams q = p;
+    q.trace = trace_for(cfg.gridDim.x);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, q));
     g_launches.fetch_add(1);
     note_kernel("gemm_big_kernel", EPI);
     return MTMC_OK;
@@ -580,6 +601,65 @@ void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
     p.tail_split = ks;
 }
 
+// Stream-K schedule of the pair kernel's last waves (see gemm_pair.cuh).  Needs at least one full wave (the
+// region dealt by k-blocks is the last full wave plus the remainder, so a tile has at most two holders).
+// Only on request (mtmc_set_schedule(1)): measured against the default -- whole tiles with the last wave's tiles
+// cut into column pieces -- it is on a par on C2 (3.46 waves: 104.6 against 103.3 us), C3 and C4 and 3 % behind
+// on 8192 x 4096 x 11008 (6.9 waves), because the column pieces already recover most of a partial wave and the
+// k-block shares run 4 % slower per k-block (pairs that run together no longer work on neighbouring tiles).
+bool want_streamk(const GemmParams& p, int clusters) {
+    if (EPI_HALVES != 1 || t_stream_k <= 0 || clusters <= 0 || clusters > SK_MAX_PAIRS) return false;
+    return p.num_tiles >= clusters && p.num_tiles % clusters != 0;
+}
+size_t streamk_bytes(int clusters) { return SK_FLAG_BYTES + static_cast<size_t>(clusters) * SK_PART_BYTES; }
+
+// Switches `p` (a pair-kernel tiling) to the stream-K schedule and points it at its scratch, which starts
+// `offset` bytes into this call's workspace `ws` (flags first with a caller's workspace, cleared per launch;
+// the library's own flags live beside its per-stream scratch and are told apart by epoch instead).
+int attach_streamk(DeviceState* d, GemmParams& p, int clusters, void* ws, size_t offset) {
+    p.sk = 1;
+    p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1;
+    p.sk_first_tile = (p.num_tiles / clusters - 1) * clusters;     // all full waves but the last are dealt round-robin
+    char* base = static_cast<char*>(ws) + offset;
+    if (t_user_ws) {
+        p.sk_flags = reinterpret_cast<uint32_t*>(base);
+        p.sk_partial = reinterpret_cast<float4*>(base + SK_FLAG_BYTES);
+        p.sk_epoch = 1;
+        CUDA_TRY(cudaMemsetAsync(p.sk_flags, 0, SK_FLAG_BYTES, t_stream));
+    } else {
+        DeviceState::StreamScratch* sc = nullptr;
+        if (int rc = get_stream_scratch(d, &sc)) return rc;
+        if (!sc->sk_flags) {
+            CUDA_TRY(counted_malloc(reinterpret_cast<void**>(&sc->sk_flags), SK_FLAG_BYTES));
+            CUDA_TRY(cudaMemsetAsync(sc->sk_flags, 0, SK_FLAG_BYTES, t_stream));
+        }
+        sc->sk_epoch = (sc->sk_epoch % 0x3fffffffu) + 1;        // 1 .. 2^30 - 1: the marker (epoch << 2 | side) is never 0
+        p.sk_flags = sc->sk_flags;
+        p.sk_partial = reinterpret_cast<float4*>(base + SK_FLAG_BYTES);
+        p.sk_epoch = sc->sk_epoch;
+    }
+    return MTMC_OK;
+}
+
+// Tiling for the 256-row pair kernel: the stream-K schedule when it pays, else whole tiles with a split wave
+// tail.  Returns whether stream-K was chosen; the caller then adds streamk_bytes() to its workspace request
+// and calls attach_streamk().
+bool plan_pair(DeviceState* d, GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, bool fp8) {
+    const int clusters = gemm_pairs(d);
+    fill_tiling(p, M, N, K, out_tile_n, clusters, false, 256, fp8);
+    if (want_streamk(p, clusters)) return true;
+    fill_tiling(p, M, N, K, out_tile_n, clusters, true, 256, fp8);
+    return false;
+}
+// The workspace of a pair-kernel call with no other scratch: nothing, or the stream-K region.
+int pair_scratch(DeviceState* d, GemmParams& p, bool sk) {
+    if (!sk) return MTMC_OK;
+    const int clusters = std::min(gemm_pairs(d), p.num_tiles);
+    void* ws = nullptr;
+    if (int rc = get_workspace(d, streamk_bytes(clusters), &ws)) return rc;
+    return attach_streamk(d, p, clusters, ws, 0);
+}
+
 int skinny_cta_of_unit_host(long long u, long long total, int grid) {
     return static_cast<int>(((u + 1) * grid - 1) / total);
 }
@@ -667,7 +747,9 @@ int launch_skinny(const SkinnyPlan& s, const CUtensorMap& tmW, const CUtensorMap
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmW, tmX, p));
+    SkinnyParams q = p;
+    q.trace = trace_for(cfg.gridDim.x);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmW, tmX, q));
     g_launches.fetch_add(1);
     note_kernel(PAIR ? "skinny_splitk_kernel (pair plan)" : "skinny_splitk_kernel (ticket plan)", -1, MX);
     return MTMC_OK;
@@ -704,7 +786,7 @@ int run_skinny(DeviceState* d, const void* X, const void* W, const float* b, con
                int act, int out_dtype, void* out, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0,
                int64_t ldo = 0) {
     SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, fp8 ? 128 : 64);
-    SkinnyParams p;
+    SkinnyParams p{};
     p.acc_scale = acc_scale;
     p.early_w = t_static_weights;
     p.M = static_cast<int>(M); p.N = static_cast<int>(N); p.K = static_cast<int>(K);
@@ -835,16 +917,19 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     const bool pair = !ks && !big && use_pair(d, M, N);
     const int bn = (pair || ks || big) ? 256 : pick_tile_n(N);
     GemmParams p{};
+    bool sk = false;
     if (ks) fill_ksplit(p, M, N, K, 256, ks, fp8);
     else if (big) fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512, fp8);
-    else if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, fp8);
+    else if (pair) sk = plan_pair(d, p, M, N, K, 256, fp8);
     else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, fp8);
     p.acc_scale = acc_scale;
     const size_t partial_bytes = lse_partial_bytes(p);         // what the chosen plan writes and the merge reads
     const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
+    const int sk_clusters = sk ? std::min(gemm_pairs(d), p.num_tiles) : 0;
     void* ws = nullptr;
-    rc = get_workspace(d, partial_bytes + extra, &ws);
+    rc = get_workspace(d, partial_bytes + extra + (sk ? streamk_bytes(sk_clusters) : 0), &ws);
     if (rc) return rc;
+    if (sk && (rc = attach_streamk(d, p, sk_clusters, ws, partial_bytes + extra))) return rc;
     p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
     p.targets = reinterpret_cast<const long long*>(targets);
     p.target_logit = EPI == EPI_XENT ? reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes) : nullptr;
@@ -913,7 +998,8 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     }
     if (use_pair(d, M, N)) {
         GemmParams p{};
-        fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256);
+        const bool sk = plan_pair(d, p, M, N, K, 256, false);
+        if ((rc = pair_scratch(d, p, sk))) return rc;
         p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB, tmBt;
         if ((rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, 128, ldw)) ||
@@ -985,7 +1071,8 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     }
     if (use_pair(d, M, N)) {
         GemmParams p{};
-        fill_tiling(p, M, N, K, 128, gemm_pairs(d), true, 256, fp8);
+        const bool sk = plan_pair(d, p, M, N, K, 128, fp8);
+        if ((rc = pair_scratch(d, p, sk))) return rc;
         p.acc_scale = sg; p.acc_scale2 = su;
         p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
@@ -1077,6 +1164,28 @@ int mtmc_set_tuning(int split_k, int tile_n, int cta_pair) {
     return MTMC_OK;
 }
 
+int mtmc_trace_enabled(void) {
+#ifdef MTMC_TRACE
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int mtmc_set_trace(void* dptr, size_t bytes) {
+    if (dptr != nullptr && !mtmc_trace_enabled())
+        return fail(MTMC_ERR_INVALID_ARG, "this build of the library has no device-side trace (compile with -DMTMC_TRACE)");
+    if (dptr != nullptr && (reinterpret_cast<uintptr_t>(dptr) & 7u)) return fail(MTMC_ERR_INVALID_ARG, "trace buffer must be 8-byte aligned");
+    t_trace = static_cast<unsigned long long*>(dptr);
+    t_trace_bytes = dptr ? bytes : 0;
+    return MTMC_OK;
+}
+
+int mtmc_set_schedule(int stream_k) {
+    t_stream_k = stream_k > 0 ? 1 : (stream_k < 0 ? -1 : 0);
+    return MTMC_OK;
+}
+
 int mtmc_set_static_weights(int enabled) { t_static_weights = enabled ? 1 : 0; return MTMC_OK; }
 
 int mtmc_set_timing(int enabled) { t_timing = enabled ? 1 : 0; return MTMC_OK; }
@@ -1099,21 +1208,26 @@ const char* mtmc_last_kernel_name(void) { return t_last_kernel; }
 
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
+    if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_CROSS_ENTROPY) return static_cast<size_t>(-1);
+    DeviceState* d = nullptr;
+    if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
+    // An upper bound over the kernels the library may pick for the shape under the current tuning: the stream-K
+    // region of the pair kernel wherever CTA pairs are possible (whether or not this shape ends up on that schedule).
+    const bool pairs_possible = gemm_pairs(d) > 0 && t_stream_k > 0 && t_cta_pair >= 0 && t_tile_n != 128 &&
+                                (t_cta_pair > 0 || (M >= 512 && N >= 256));
+    const size_t sk = pairs_possible ? streamk_bytes(gemm_pairs(d)) : 0;
     switch (op) {
         case MTMC_OP_FUSED_LINEAR: {
-            if (!use_skinny(M, N)) return 0;
-            DeviceState* d = nullptr;
-            if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
+            if (!use_skinny(M, N)) return sk;
             // the larger of the bf16 and the E4M3 plan: mtmc_fused_linear_fp8 shares this op id
             SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
             SkinnyPlan s8 = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, 128);
             return std::max(s.ticket_bytes + s.partial_bytes, s8.ticket_bytes + s8.partial_bytes);
         }
-        case MTMC_OP_SWIGLU: return 0;
-        case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N);
-        case MTMC_OP_LINEAR_ROWMAX: return lse_workspace_bytes(M, N);
-        case MTMC_OP_LINEAR_CROSS_ENTROPY: return lse_workspace_bytes(M, N) + round256(static_cast<size_t>(M) * sizeof(float));
-        default: return static_cast<size_t>(-1);
+        case MTMC_OP_SWIGLU: return sk;
+        case MTMC_OP_LINEAR_LSE: return lse_workspace_bytes(M, N) + sk;
+        case MTMC_OP_LINEAR_ROWMAX: return lse_workspace_bytes(M, N) + sk;
+        default: return lse_workspace_bytes(M, N) + round256(static_cast<size_t>(M) * sizeof(float)) + sk;
     }
 }
 
@@ -1151,6 +1265,8 @@ int mtmc_check_status(void) {
         if (int rc = noalloc_take_status(dev, &st_noalloc)) return rc;
     }
     if (st == 0) st = st_noalloc;
+    if ((st & 0xff00u) == STATUS_CHECK_FAILED)
+        return fail(MTMC_ERR_DEVICE_CHECK, "a device-side index check of the -DMTMC_CHECKS build failed (status word 0x%x)", st);
     if (st != 0) return fail(MTMC_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (status word 0x%x)", st);
     return MTMC_OK;
 }
@@ -1218,8 +1334,12 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     const bool pair = use_pair(d, M, N);
     const int bn = pair ? 256 : pick_tile_n(N);
     GemmParams p{};
-    if (pair) fill_tiling(p, M, N, K, 256, gemm_pairs(d), true, 256, true);
-    else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, true);
+    if (pair) {
+        const bool sk = plan_pair(d, p, M, N, K, 256, true);
+        if ((rc = pair_scratch(d, p, sk))) return rc;
+    } else {
+        fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, true);
+    }
     p.acc_scale = scale_x * scale_w;
     p.act = act; p.bias = b; p.residual = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
     CUtensorMap tmA, tmB, tmBt;

@@ -82,8 +82,10 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t rank = cluster_ctarank();            // 0: issues the MMAs, owns the shared barriers
     const int pair_id = static_cast<int>(blockIdx.x >> 1);
     const int num_pairs = static_cast<int>(gridDim.x >> 1);
+    const Trace tr(p.trace);
 
     if (threadIdx.x == 0) {
+        tr.stamp(TR_START_NS);
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(accf_bar, 1);
         mbar_init(acce_bar, 2 * Cfg::WARPS_EPI);         // every epilogue warp of both CTAs
@@ -106,6 +108,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
     pdl_launch_dependents();
     pdl_wait();
+    if (threadIdx.x == 0) tr.stamp(TR_SETUP_NS);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -124,7 +127,10 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const CUtensorMap* mapB = (EPI == EPI_SWIGLU && rank == 1) ? &tmB2 : &tmB;
                 int kx = 0;
                 for (int kb = 0; kb < p.k_blocks; ++kb, kx += p.bk_elems) {
+                    const long long tw = tr.now();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 5u)) { ok = false; break; }
+                    tr.add(TR_PROD_STALL, tr.now() - tw);
+                    tr.stamp_once(TR_PROD_FIRST_NS);
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = full0_base + 8u * s;
                     tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
@@ -133,6 +139,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
+            tr.stamp(TR_PROD_LAST_NS);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -144,11 +151,17 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(256, Cfg::BN) : umma_idesc_bf16(256, Cfg::BN);
             for (int t = pair_id; t < p.num_tiles && ok; t += num_pairs) {
                 // the one accumulator set is free again once every epilogue warp of both CTAs has drained it
+                const long long ta = tr.now();
                 if (!mbar_wait_cluster(acce_bar, acc_ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 8u)) { ok = false; break; }
+                tr.add(TR_MMA_STALL_ACC, tr.now() - ta);
                 acc_ph ^= 1u;
                 tc_fence_after();
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
+                    const long long tw = tr.now();
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 9u)) { ok = false; break; }
+                    tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
+                    tr.add(TR_MMA_KBLOCKS, 1);
+                    tr.stamp_once(TR_MMA_FIRST_NS);
                     tc_fence_after();
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                     const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
@@ -171,6 +184,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 if (ok) umma_commit_pair(accf_bar, 3);           // both halves complete, in both CTAs
             }
+            tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();
     } else {
@@ -199,7 +213,11 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bias_bar);
             }
+            const bool tracer = warp == 2 && lane == 0;      // one writer for the epilogue's trace words
+            const long long tw = tr.now();
             if (!mbar_wait(accf_bar, acc_ph, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 6u)) { ok = false; break; }
+            const long long tb = tr.now();
+            if (tracer) { tr.add(TR_EPI_STALL, tb - tw); tr.add(TR_EPI_ITEMS, 1); tr.stamp_once(TR_EPI_FIRST_NS); }
             acc_ph ^= 1u;
             tc_fence_after();
             // the other warps' parts of the bias copy (an mbarrier, so that this wait is bounded like every other)
@@ -211,6 +229,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(cluster_map_shared(acce_bar, 0));
+            if (tracer) { tr.add(TR_EPI_BUSY, tr.now() - tb); tr.stamp(TR_EPI_END_NS); }
         }
     }
 
@@ -218,6 +237,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // Neither CTA may free its TMEM or leave while the other can still touch its memory or barriers.
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) tr.stamp(TR_END_NS);
     cluster_arrive();
     cluster_wait();
     if (*abort_flag != 0u) {

@@ -10,6 +10,20 @@
 // barrier; tcgen05.commit with a cluster mask frees the stage in both CTAs and publishes
 // the accumulator to both; the epilogue warps of both CTAs arrive on the even CTA's
 // `accumulator empty` barrier.  No TMA load uses cluster multicast.
+//
+// Stream-K schedule for the last waves (GemmParams::sk).  Whole tiles dealt round-robin leave the last wave
+// partly empty: 3.46 waves of tiles cost 4 tile-times.  With this schedule the full waves but one are dealt
+// round-robin as before (pairs that run together work on neighbouring tiles and share operands in L2), and the
+// last full wave plus the remainder -- between one and two tiles per pair -- is dealt by k-blocks: the flat
+// list of that region's (tile, k-block) units is cut into one contiguous, equal share per pair, so all pairs
+// finish together.  A pair's share begins with the END of a tile's K range (the tile's beginning belongs to
+// the pair before) and ends with the BEGINNING of another tile's K range; every tile has at most two holders.
+// The two holders of a shared tile meet without waiting for one another: each epilogue warp that finishes
+// its part either finds its counterpart's part already in global memory and adds it to its accumulator
+// (then runs the ordinary epilogue), or leaves its own part there, marks the flag word and moves on;
+// whoever marks second finishes the tile.  A pair works on its two shared pieces first and on its whole tiles
+// after them, so the hand-overs run under the mainloop of the tiles that follow.  Two fp32 addends commute,
+// so the result does not depend on who finishes.
 #pragma once
 #include "gemm_tiled.cuh"
 
@@ -30,6 +44,125 @@ struct PairCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
 };
+
+// One work item of a pair: a whole tile or tail piece (side == 0), or k-blocks [kb0, kb1) of a tile shared with
+// a neighbouring pair under the stream-K schedule (side 1: the beginning of the tile's K range, 2: its end).
+struct PairWork {
+    int item, kb0, kb1;
+    int side, slot;      // slot: the boundary's index = the lower of the two pairs that share the tile
+};
+
+struct PairWalk {
+    int u, dp_end, step;                   // round-robin part: next item, end, stride
+    int KB, pair_id, sk_first;
+    int tail_tile, tail_kb0;               // stream-K region: the END of a tile's K range that opens this pair's share (tail_kb0 > 0), if any
+    int head_tile, head_kb1;               // ... the BEGINNING of a tile's K range that closes it (head_kb1 < KB), if any
+    int whole, whole_end;                  // ... and the whole tiles in between
+    int phase;                             // 0 round-robin, 1 tail piece, 2 head piece, 3 whole tiles of the share
+    __device__ __forceinline__ PairWalk(const GemmParams& p, int pair, int num_pairs) {
+        KB = p.k_blocks; pair_id = pair; step = num_pairs;
+        u = pair;
+        dp_end = p.sk ? p.sk_first_tile : p.num_items;
+        sk_first = p.sk_first_tile;
+        phase = 0;
+        tail_tile = head_tile = -1; tail_kb0 = head_kb1 = 0; whole = whole_end = 0;
+        if (p.sk) {
+            const long long U = static_cast<long long>(p.num_items - p.sk_first_tile) * KB;
+            const long long su = U * pair / num_pairs, su_end = U * (pair + 1) / num_pairs;
+            const int t0 = static_cast<int>(su / KB), a = static_cast<int>(su - static_cast<long long>(t0) * KB);
+            const int t1 = static_cast<int>((su_end - 1) / KB), b = static_cast<int>(su_end - static_cast<long long>(t1) * KB);
+            whole = t0; whole_end = t1 + 1;
+            if (a > 0) { tail_tile = t0; tail_kb0 = a; whole = t0 + 1; }
+            if (b < KB) { head_tile = t1; head_kb1 = b; whole_end = t1; }
+        }
+    }
+    // Order inside the share: the two pieces of shared tiles first, then the whole tiles.  The piece that closes the
+    // share comes second, not last, so that its hand-over (and, if this pair comes second, the tile's completion)
+    // runs under the mainloop of the whole tiles that follow instead of after the last MMA of the launch.
+    __device__ __forceinline__ bool next(PairWork& w) {
+        if (phase == 0) {
+            if (u < dp_end) { w.item = u; w.kb0 = 0; w.kb1 = KB; w.side = 0; w.slot = 0; u += step; return true; }
+            phase = 1;
+        }
+        if (phase == 1) {
+            phase = 2;
+            if (tail_tile >= 0) { w.item = sk_first + tail_tile; w.kb0 = tail_kb0; w.kb1 = KB; w.side = 2; w.slot = pair_id - 1; return true; }
+        }
+        if (phase == 2) {
+            phase = 3;
+            if (head_tile >= 0) { w.item = sk_first + head_tile; w.kb0 = 0; w.kb1 = head_kb1; w.side = 1; w.slot = pair_id; return true; }
+        }
+        if (whole < whole_end) { w.item = sk_first + whole; w.kb0 = 0; w.kb1 = KB; w.side = 0; w.slot = 0; ++whole; return true; }
+        return false;
+    }
+};
+
+// Stream-K hand-over for one epilogue warp (CTA `rank` of the pair, TMEM lane quadrant q) whose accumulator holds
+// part of a shared tile's K range.  Returns true if this warp has to finish the tile: its accumulator in tensor
+// memory then holds the whole sum.  Returns false if it left its part for the other holder.
+template <int BN>
+__device__ __forceinline__ bool streamk_meet(const GemmParams& p, const PairWork& w, uint32_t t_addr, int rank, int q, int lane) {
+    constexpr int CHUNKS = BN / 32;
+    constexpr size_t WARP_F4 = static_cast<size_t>(CHUNKS) * 8 * 32;           // float4 per warp and part
+    if (!MTMC_CHECK(w.slot >= 0 && w.slot < static_cast<int>(gridDim.x >> 1) - 1 && (w.side == 1 || w.side == 2), p.status, 3u)) return false;
+    uint32_t* flag = p.sk_flags + (static_cast<size_t>(w.slot) * 2 + rank) * 4 + q;
+    const uint32_t mine = (p.sk_epoch << 2) | static_cast<uint32_t>(w.side);
+    const uint32_t theirs = (p.sk_epoch << 2) | static_cast<uint32_t>(3 - w.side);
+    float4* my_part = p.sk_partial + (((static_cast<size_t>(w.slot) * 2 + (w.side - 1)) * 2 + rank) * 4 + q) * WARP_F4;
+    const float4* peer_part = p.sk_partial + (((static_cast<size_t>(w.slot) * 2 + (2 - w.side)) * 2 + rank) * 4 + q) * WARP_F4;
+    uint32_t seen = 0;
+    if (lane == 0) seen = ld_acquire_gpu(flag);
+    seen = __shfl_sync(0xffffffffu, seen, 0);
+    if (seen != theirs) {
+        // the other holder has not been here yet: leave this part (every store instruction of the warp writes 512
+        // contiguous bytes; the reader is the thread at the same place of the other pair, so the layout is private)
+#pragma unroll 1
+        for (int c = 0; c < CHUNKS; ++c) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + c * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int v = 0; v < 8; ++v)
+                __stcg(my_part + (c * 8 + v) * 32 + lane, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                                      __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+        }
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) seen = atom_exch_acq_rel_gpu(flag, mine);
+        seen = __shfl_sync(0xffffffffu, seen, 0);
+        if (seen != theirs) return false;            // marked first: the other holder finishes the tile
+    }
+    __threadfence();                                 // the other part was complete before its flag was set
+    // own part from tensor memory + the other part from L2 (the next chunk's loads in flight meanwhile), back to tensor memory
+    float4 o[8];
+#pragma unroll
+    for (int v = 0; v < 8; ++v) o[v] = __ldcg(peer_part + v * 32 + lane);
+#pragma unroll 1
+    for (int c = 0; c < CHUNKS; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_addr + c * 32, r);
+        float4 nx[8];
+        if (c + 1 < CHUNKS) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) nx[v] = __ldcg(peer_part + ((c + 1) * 8 + v) * 32 + lane);
+        }
+        tmem_ld_wait();
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+            r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + o[v].x);
+            r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + o[v].y);
+            r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + o[v].z);
+            r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + o[v].w);
+        }
+        tmem_st_32x32b_x32(t_addr + c * 32, r);
+        if (c + 1 < CHUNKS) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) o[v] = nx[v];
+        }
+    }
+    tmem_st_wait();
+    return true;
+}
 
 template <int EPI, bool OUT_BF16>
 __global__ void __launch_bounds__(64 + 32 * EPI_WARPS, 1)
@@ -57,8 +190,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t rank = cluster_ctarank();            // 0: issues the MMAs, owns the shared barriers
     const int pair_id = static_cast<int>(blockIdx.x >> 1);
     const int num_pairs = static_cast<int>(gridDim.x >> 1);
+    const Trace tr(p.trace);
 
     if (threadIdx.x == 0) {
+        tr.stamp(TR_START_NS);
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 2 * EPI_WARPS); }   // every epilogue warp of both CTAs
         *abort_flag = 0u;
@@ -79,6 +214,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = *tmem_slot;
     pdl_launch_dependents();     // the next kernel in the stream may begin its own set-up
     pdl_wait();                  // everything before this line touched only shared and tensor memory
+    if (threadIdx.x == 0) tr.stamp(TR_SETUP_NS);
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -87,9 +223,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t ph = 0;
             bool ok = true;
             const uint32_t full0_base = cluster_map_shared(full_bar(0), 0);   // the even CTA's full barriers
-            for (int t = pair_id; t < p.num_items && ok; t += num_pairs) {
+            PairWalk walk(p, pair_id, num_pairs);
+            PairWork w;
+            while (ok && walk.next(w)) {
                 int mb, nb, sub, width;
-                item_coords(p, t, Cfg::OUT_TILE_N, mb, nb, sub, width);
+                item_coords(p, w.item, Cfg::OUT_TILE_N, mb, nb, sub, width);
                 const bool whole = width == Cfg::OUT_TILE_N;
                 const int m0 = mb * Cfg::BM + static_cast<int>(rank) * 128;
                 // This CTA's share of the B operand: SwiGLU -> rank 0 the gate rows, rank 1 the up rows of
@@ -98,19 +236,24 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int n_row0 = nb * Cfg::OUT_TILE_N + sub * width + ((EPI == EPI_SWIGLU) ? 0 : static_cast<int>(rank) * b_rows);
                 const CUtensorMap* mapB = (EPI == EPI_SWIGLU && rank == 1) ? (whole ? &tmB2 : &tmB2t) : (whole ? &tmB : &tmBt);
                 const uint32_t cta_bytes = Cfg::A_BYTES + static_cast<uint32_t>(b_rows) * Cfg::BK * 2;
-                int kx = 0;                                              // K coordinate of the next k-block
-                for (int kb = 0; kb < p.k_blocks; ++kb, kx += p.bk_elems) {
+                int kx = w.kb0 * p.bk_elems;                             // K coordinate of the next k-block
+                for (int kb = w.kb0; kb < w.kb1; ++kb, kx += p.bk_elems) {
+                    const long long tw = tr.now();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 3u)) { ok = false; break; }
+                    tr.add(TR_PROD_STALL, tr.now() - tw);
+                    tr.stamp_once(TR_PROD_FIRST_NS);
                     // loads first, bookkeeping after: the time from "slot free" to "load issued" is on the ring's
                     // critical path (a transaction count may run ahead of its expect_tx within a phase)
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = full0_base + 8u * s;
+                    if (!MTMC_CHECK(a_dst + cta_bytes <= epi_stage_base && (kx & 7) == 0 && m0 >= 0 && n_row0 >= 0, p.status, 4u)) { ok = false; break; }
                     tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
                     tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kx, n_row0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), 2u * cta_bytes);     // both CTAs' bytes
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
+            tr.stamp(TR_PROD_LAST_NS);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -121,17 +264,25 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t acc_ph = 0;
             int it = 0;
             bool ok = true;
-            for (int t = pair_id; t < p.num_items && ok; t += num_pairs, ++it) {
+            PairWalk walk(p, pair_id, num_pairs);
+            PairWork w;
+            for (; ok && walk.next(w); ++it) {
                 const int buf = it & 1;
-                const int width = t < p.n_full ? Cfg::OUT_TILE_N : p.tail_width;
+                const int width = w.item < p.n_full ? Cfg::OUT_TILE_N : p.tail_width;
                 const int mma_n = EPI == EPI_SWIGLU ? 2 * width : width;
                 const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(Cfg::BM, mma_n) : umma_idesc_bf16(Cfg::BM, mma_n);
+                const long long ta = tr.now();
                 if (!mbar_wait_cluster(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 5u)) { ok = false; break; }
+                tr.add(TR_MMA_STALL_ACC, tr.now() - ta);
                 acc_ph ^= 1u << buf;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * Cfg::BN);
-                for (int kb = 0; kb < p.k_blocks; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb) {
+                    const long long tw = tr.now();
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 6u)) { ok = false; break; }
+                    tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
+                    tr.add(TR_MMA_KBLOCKS, 1);
+                    tr.stamp_once(TR_MMA_FIRST_NS);
                     tc_fence_after();
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                     const uint64_t a_desc = umma_smem_desc_sw128(a_src);
@@ -140,17 +291,18 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     if (p.fp8) {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_fp8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            umma_fp8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | k) != 0 ? 1u : 0u);
                     } else {
 #pragma unroll
                         for (int k = 0; k < 4; ++k)
-                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | k) != 0 ? 1u : 0u);
                     }
                     umma_commit_pair(empty_bar(s), 3);           // frees the stage in both CTAs
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit_pair(accf_bar(buf), 3);      // accumulator complete, in both CTAs
             }
+            tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();
     } else {
@@ -162,23 +314,34 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t acc_ph = 0;
         int it = 0;
         bool ok = true;
-        for (int t = pair_id; t < p.num_items && ok; t += num_pairs, ++it) {
+        PairWalk walk(p, pair_id, num_pairs);
+        PairWork w;
+        for (; ok && walk.next(w); ++it) {
             const int buf = it & 1;
             int mb, nb, sub, width;
-            item_coords(p, t, Cfg::OUT_TILE_N, mb, nb, sub, width);
+            item_coords(p, w.item, Cfg::OUT_TILE_N, mb, nb, sub, width);
             const int row = mb * Cfg::BM + static_cast<int>(rank) * 128 + q * 32 + lane;
             const int n_tile0 = nb * Cfg::OUT_TILE_N + sub * width;
+            const bool tracer = warp == 2 && lane == 0;      // one writer for the epilogue's trace words
+            const long long tw = tr.now();
             if (!mbar_wait(accf_bar(buf), (acc_ph >> buf) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 5u)) { ok = false; break; }
+            const long long tb = tr.now();
+            if (tracer) { tr.add(TR_EPI_STALL, tb - tw); tr.add(TR_EPI_ITEMS, 1); tr.stamp_once(TR_EPI_FIRST_NS); }
             acc_ph ^= 1u << buf;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::BN);
             const int chunks = width / 32, split_at = EPI_HALVES == 2 ? (chunks + 1) / 2 : chunks;      // two warps per lane quadrant share the columns
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, half ? split_at : 0, half ? chunks : split_at, width, nb, sub, half,
-                                         vec_ok, smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
+            // part of a shared tile (stream-K): either the whole sum ends up in this accumulator, or the other holder finishes
+            const bool finish = w.side == 0 || streamk_meet<Cfg::BN>(p, w, t_addr, static_cast<int>(rank), q, lane);
+            if (tracer && w.side != 0) tr.add(TR_EPI_HANDOVER, tr.now() - tb);
+            if (finish)
+                epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, half ? split_at : 0, half ? chunks : split_at, width, nb, sub, half,
+                                             vec_ok, smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
             // this CTA's half of the accumulator is drained: tell the MMA issuer in the even CTA
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(cluster_map_shared(acce_bar(buf), 0));
+            if (tracer) { tr.add(TR_EPI_BUSY, tr.now() - tb); tr.stamp(TR_EPI_END_NS); }
         }
     }
 
@@ -186,6 +349,7 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // Neither CTA may free its TMEM or leave while the other can still touch its memory or barriers.
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) tr.stamp(TR_END_NS);
     cluster_arrive();
     cluster_wait();
     if (*abort_flag != 0u) {

@@ -56,6 +56,15 @@ struct GemmParams {
     const long long* targets;   // [M] target column per row (EPI_XENT)
     float* target_logit;        // [M] logit at the target column, written by the one piece that holds it (EPI_XENT)
     uint32_t* status;     // device status word
+    unsigned long long* trace;   // per-CTA trace records (-DMTMC_TRACE builds, mtmc_set_trace), else null
+    // Stream-K schedule of the CTA-pair kernel (gemm_pair.cuh): tiles [0, sk_first_tile) are dealt round-robin; the
+    // (tile, k-block) units of the remaining tiles (between one and two per pair) are cut into one contiguous, equal
+    // share per pair, so a tile whose k-blocks straddle a boundary is finished by two pairs.
+    int sk;               // 1: stream-K schedule (whole tiles only: n_full == num_items == num_tiles)
+    int sk_first_tile;    // a multiple of the number of pairs
+    uint32_t sk_epoch;    // launch counter: flag words of earlier launches never match this launch's markers
+    uint32_t* sk_flags;   // [pairs][2 ranks][4 lane quadrants] one word per (boundary, epilogue warp)
+    float4* sk_partial;   // [pairs][2 sides][2 ranks][4 quadrants][8 chunks][8][32 lanes] fp32 accumulator parts
 };
 
 template <int EPI, int BN>
@@ -328,6 +337,9 @@ template <int EPI, bool OUT_BF16>
 __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int c_begin,
                                               int c_end, int width, int nb, int sub, int half, bool vec_ok, uint8_t* stage,
                                               int lane, const float* bias_tile = nullptr) {
+    // the chunks lie inside the 512 columns of tensor memory and inside the item; the item starts inside the padded output
+    if (!MTMC_CHECK((t_addr & 0xffffu) + static_cast<uint32_t>((EPI == EPI_SWIGLU ? width : 0) + c_end * 32) <= 512u &&
+                    c_begin >= 0 && c_end * 32 <= width && n_tile0 >= 0 && n_tile0 < p.N + 256, p.status, 1u)) return;
     if (EPI == EPI_ACT) {
         // Two chunks in flight: while chunk c is being activated and stored, the TMEM load and the
         // bias fetch of chunk c + 1 are already under way.
@@ -353,6 +365,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             }
             apply_act_chunk<OUT_BF16>(p.act, y);
             if (p.residual != nullptr && row < p.M) add_residual_chunk<OUT_BF16>(p.residual, row, n0, p.N, y, vec_ok);
+            if (!MTMC_CHECK(n0 >= 0 && n0 < p.N && p.ldo >= p.N, p.status, 5u)) continue;
             if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.ldo, y, lane);
             else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, p.ldo, y, false);
         }
@@ -421,7 +434,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             for (int k = 0; k < 4; ++k)
                 if (m4[k] > mx || (m4[k] == mx && a4[k] < arg)) { mx = m4[k]; arg = a4[k]; }
         }
-        if (row < p.M)
+        if (row < p.M && MTMC_CHECK((nb * p.tail_split + sub) * EPI_HALVES + half < p.n_tiles * p.tail_split * EPI_HALVES, p.status, 2u))
             p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] = make_float2(mx, __int_as_float(arg));
     } else {
         // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
@@ -484,7 +497,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             mx = nm;
         }
         // a piece that lies wholly past N (only possible in the last column tile) stays neutral
-        if (row < p.M)
+        if (row < p.M && MTMC_CHECK((nb * p.tail_split + sub) * EPI_HALVES + half < p.n_tiles * p.tail_split * EPI_HALVES, p.status, 2u))
             p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] =
                 make_float2(mx * 0.6931471805599453f, sum);
         if (EPI == EPI_XENT && found) p.target_logit[row] = tz;

@@ -16,6 +16,16 @@ namespace mtmc {
 constexpr uint32_t STATUS_TIMEOUT_PRODUCER = 0x100u;
 constexpr uint32_t STATUS_TIMEOUT_MMA = 0x200u;
 constexpr uint32_t STATUS_TIMEOUT_EPILOGUE = 0x300u;
+constexpr uint32_t STATUS_CHECK_FAILED = 0x400u;     // -DMTMC_CHECKS builds: an index check failed (low byte: which)
+
+// Index checks of -DMTMC_CHECKS builds (compute-sanitizer's stand-in where that tool cannot run): a failed check
+// records STATUS_CHECK_FAILED | code in the status word and yields false, and the caller skips the access --
+// nothing traps or faults.  In a regular build the condition is not evaluated and the value is true.
+#ifdef MTMC_CHECKS
+#define MTMC_CHECK(cond, status_ptr, code) ((cond) ? true : (atomicCAS((status_ptr), 0u, mtmc::STATUS_CHECK_FAILED | (code)), false))
+#else
+#define MTMC_CHECK(cond, status_ptr, code) true
+#endif
 
 // About one second at the clocks this part runs at; any legitimate wait is
 // microseconds to a few milliseconds.
@@ -363,6 +373,61 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
 // concerned, the next kernel may be scheduled.  Without the attribute both are no-ops.
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------- device-side trace (-DMTMC_TRACE builds only)
+// One record of TRACE_WORDS 64-bit words per CTA in a buffer the caller hands in with mtmc_set_trace(); every
+// word has one writer.  Time stamps are %globaltimer nanoseconds (comparable across SMs), stall and busy
+// totals are clock64 cycles.  In a regular build every member is empty and the calls vanish.
+constexpr int TRACE_WORDS = 32;
+enum {
+    TR_START_NS = 0,        // kernel entry
+    TR_SETUP_NS = 1,        // set-up done, preceding kernel finished (after griddepcontrol.wait)
+    TR_PROD_FIRST_NS = 2,   // producer: first load issued
+    TR_PROD_LAST_NS = 3,    // producer: last load issued
+    TR_PROD_STALL = 4,      // producer: cycles waiting for a free ring stage
+    TR_MMA_FIRST_NS = 5,    // MMA issuer: first MMA issued
+    TR_MMA_LAST_NS = 6,     // MMA issuer: last accumulator committed
+    TR_MMA_STALL_DATA = 7,  // MMA issuer: cycles waiting for a full ring stage
+    TR_MMA_STALL_ACC = 8,   // MMA issuer: cycles waiting for a drained accumulator
+    TR_MMA_KBLOCKS = 9,     // MMA issuer: k-blocks multiplied
+    TR_EPI_FIRST_NS = 10,   // first epilogue warp: first accumulator ready
+    TR_EPI_END_NS = 11,     // first epilogue warp: last item finished
+    TR_EPI_STALL = 12,      // first epilogue warp: cycles waiting for accumulators
+    TR_EPI_BUSY = 13,       // first epilogue warp: cycles inside epilogues
+    TR_EPI_ITEMS = 14,      // first epilogue warp: items
+    TR_EPI_HANDOVER = 15,   // first epilogue warp: cycles inside stream-K / split-K hand-overs
+    TR_END_NS = 16,         // teardown reached
+};
+struct Trace {
+#ifdef MTMC_TRACE
+    unsigned long long* rec;
+    __device__ __forceinline__ explicit Trace(unsigned long long* base) : rec(base ? base + static_cast<size_t>(blockIdx.x) * TRACE_WORDS : nullptr) {}
+    __device__ __forceinline__ void stamp(int i) const {
+        if (rec) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); rec[i] = t; }
+    }
+    __device__ __forceinline__ void stamp_once(int i) const { if (rec && rec[i] == 0ull) stamp(i); }
+    __device__ __forceinline__ void add(int i, long long v) const { if (rec) rec[i] += static_cast<unsigned long long>(v); }
+    __device__ __forceinline__ long long now() const { return rec ? clock64() : 0ll; }
+#else
+    __device__ __forceinline__ explicit Trace(unsigned long long*) {}
+    __device__ __forceinline__ void stamp(int) const {}
+    __device__ __forceinline__ void stamp_once(int) const {}
+    __device__ __forceinline__ void add(int, long long) const {}
+    __device__ __forceinline__ long long now() const { return 0ll; }
+#endif
+};
+
+// ----------------------------------------------------------------------------- global flags between CTAs
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t atom_exch_acq_rel_gpu(uint32_t* p, uint32_t v) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.gpu.global.exch.b32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 
 // ----------------------------------------------------------------------------- misc
 __device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t nthreads) {

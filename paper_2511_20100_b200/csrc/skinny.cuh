@@ -49,6 +49,7 @@ struct SkinnyParams {
     float* partial;          // [n_tiles][max_slots][MX][128] fp32
     uint32_t* tickets;       // [n_tiles], zero between launches
     uint32_t* status;
+    unsigned long long* trace;   // per-CTA trace records (-DMTMC_TRACE builds, mtmc_set_trace), else null
 };
 
 template <int MX_>
@@ -153,6 +154,8 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int KB = p.k_blocks;
+    const Trace tr(p.trace);
+    if (threadIdx.x == 0) tr.stamp(TR_START_NS);
     // This CTA's share of the unit list.
     int first_tile, first_kb, n_units;
     uint32_t crank = 0;
@@ -198,7 +201,10 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 const bool begun = !early && idx < pre;        // W already on its way, bytes already announced
                 const uint32_t dst = base + s * stage_bytes;
                 if (!begun) {
+                    const long long tw = tr.now();
                     if (!early && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 2u)) return;
+                    tr.add(TR_PROD_STALL, tr.now() - tw);
+                    tr.stamp_once(TR_PROD_FIRST_NS);
                     mbar_expect_tx(full_bar(s), nkb * (w_bytes + Cfg::X_BYTES));
                     for (int i = 0; i < nkb; ++i)
                         tma_load_2d_hint(dst + i * w_bytes, &tmW, full_bar(s), (kb + i) * BKE, tile * R, pol_stream);
@@ -215,6 +221,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             ++tile;
             kb = 0;
         }
+        if (!early) tr.stamp(TR_PROD_LAST_NS);
     };
 
     // Set-up.  Warp 0 initialises the barriers and goes straight on to issue loads; it only
@@ -238,6 +245,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         if (lane == 0 && p.early_w) produce(true);
         pdl_launch_dependents();
         pdl_wait();                          // before the first load of anything a preceding kernel may have written
+        if (lane == 0) tr.stamp(TR_SETUP_NS);
     } else {
         if (warp == 1) {
             tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
@@ -275,7 +283,11 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 uint32_t step = 0;                                // MMA count within this segment
                 while (seg > 0) {
                     const int nkb = min(KPS, seg);
+                    const long long tw = tr.now();
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 4u)) { ok = false; break; }
+                    tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
+                    tr.add(TR_MMA_KBLOCKS, nkb);
+                    tr.stamp_once(TR_MMA_FIRST_NS);
                     tc_fence_after();
                     const uint32_t src = base + s * stage_bytes;
                     for (int i = 0; i < nkb; ++i) {
@@ -296,6 +308,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                 kb = 0;
                 ++seg_idx;
             }
+            tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();
     } else {
@@ -317,6 +330,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
 #pragma unroll
             for (int m = 0; m < MX; ++m) acc[m] = 0.0f;
             if (n_units > 0) ok = mbar_wait(accf_bar(0), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 3u);
+            if (warp == 2 && lane == 0) tr.stamp(TR_EPI_FIRST_NS);
             if (ok && n_units > 0) {
                 tc_fence_after();
                 skinny_sum_ways<MX, Cfg::WAYS>(tmem_base + lane_base, min(Cfg::WAYS, n_units * (Cfg::BK / 16)), acc);
@@ -423,8 +437,10 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         }
     }
 
+    if (warp == 2 && lane == 0) tr.stamp(TR_EPI_END_NS);
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) tr.stamp(TR_END_NS);
     if (PAIR) {
         // Neither CTA may leave while its peer can still write into (or arrive on) its shared
         // memory.  The epilogue warps consumed the set-up phase already; the others do it here.

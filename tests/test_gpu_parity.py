@@ -717,6 +717,103 @@ def test_calls_on_two_streams_keep_their_scratch_apart():
             _assert_close(inputs.to_f64(o), want, TOL["fp32"], "stream %d" % i)
 
 
+# ------------------------------------------------------------------ stream-K schedule of the 256 x 256 pair kernel
+# Forced by the schedule hook on problems with at least as many tiles as CTA pairs (81 to 100 tiles on 74 pairs):
+# shares that begin and end inside tiles, k-block counts that do not divide, ragged rows / columns / K.
+STREAMK = [(2304, 2304, 328), (2304, 2400, 4096), (2500, 2200, 72), (2304, 2304, 64)]
+
+
+def _streamk(fn):
+    B.mtmc_set_tuning(cta_pair=1)
+    B.mtmc_set_schedule(1)
+    try:
+        return fn()
+    finally:
+        B.mtmc_set_schedule(0)
+        B.mtmc_set_tuning()
+
+
+@pytest.mark.parametrize("M,N,K", STREAMK)
+@pytest.mark.parametrize("act,odt", [("gelu_tanh", "bf16"), ("none", "fp32")])
+def test_stream_k_fused_linear(M, N, K, act, odt):
+    li = inputs.linear_inputs(M, N, K, seed=8600 + M + N + K)
+    want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), B.ACT[act])
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+
+    def run():
+        B.mtmc_fused_linear(Xd, Wd, bd, act, odt, out=out)
+        assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+        B.mtmc_check_status()
+        return [B.mtmc_fused_linear(Xd, Wd, bd, act, odt) for _ in range(4)]
+    again = _streamk(run)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    _assert_close(inputs.to_f64(out), want, TOL[odt], "stream-K %dx%dx%d %s" % (M, N, K, odt))
+    for o in again:                    # whoever of a shared tile's two holders finishes it, the bits are the same
+        assert torch.equal(o, out)
+
+
+@pytest.mark.parametrize("M,N,K", [(2304, 1160, 328), (2304, 2400, 1096)])
+def test_stream_k_other_epilogues(M, N, K):
+    li = inputs.linear_inputs(M, N, K, seed=8700 + M + N)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    tgt = torch.from_numpy(np.random.default_rng(M + N).integers(0, N, size=M))
+    si = inputs.swiglu_inputs(M, N, K, seed=8710 + M)
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=8720 + M)
+    R = torch.randn(M, N, generator=torch.Generator().manual_seed(M + N)).bfloat16()
+
+    def run():
+        r = {}
+        r["lse"] = B.mtmc_linear_lse(Xd, Wd, bd)
+        r["rowmax"] = B.mtmc_linear_rowmax(Xd, Wd, bd)
+        r["xent"] = B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt.cuda())
+        r["swiglu"] = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+        r["res"] = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "silu", "bf16")
+        r["fp8"] = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "gelu_tanh", "bf16")
+        assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+        B.mtmc_check_status()
+        return r
+    r = _streamk(run)
+    _assert_close(inputs.to_f64(r["lse"]), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "stream-K lse")
+    _check_rowmax(li, r["rowmax"][0], r["rowmax"][1], "stream-K rowmax")
+    want_loss, _ = ref.linear_cross_entropy(Xb, Wb, bf, tgt.numpy())
+    _assert_close(inputs.to_f64(r["xent"]), want_loss, TOL["fp32"], "stream-K cross entropy")
+    _assert_close(inputs.to_f64(r["swiglu"]), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                  TOL["bf16"], "stream-K swiglu")
+    _assert_close(inputs.to_f64(r["res"]), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_SILU), TOL["bf16"],
+                  "stream-K residual")
+    want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(r["fp8"]), want8, TOL["bf16"], "stream-K fp8")
+
+
+def test_stream_k_with_caller_workspace():
+    """The accumulator parts and flag words in a caller's workspace of exactly mtmc_workspace_bytes, canaries around it."""
+    M, N, K = 2304, 2304, 328
+    li = inputs.linear_inputs(M, N, K, seed=8800)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+
+    def run():
+        need = B.mtmc_workspace_bytes("linear_lse", M, N, K)
+        assert need >= B.mtmc_workspace_bytes("fused_linear", M, N, K) > 0
+        guard = torch.full((need + 8192,), 0x5A, dtype=torch.uint8, device="cuda")
+        off = (-guard.data_ptr()) % 256 + 3840
+        B.mtmc_set_workspace(guard[off:off + need])
+        try:
+            out = B.mtmc_fused_linear(Xd, Wd, bd, "relu", "fp32")
+            lse = B.mtmc_linear_lse(Xd, Wd, bd)
+            B.mtmc_check_status()
+        finally:
+            B.mtmc_set_workspace(None)
+        assert bool((guard[:off] == 0x5A).all()) and bool((guard[off + need:] == 0x5A).all())
+        return out, lse
+    out, lse = _streamk(run)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, ref.ACT_RELU), TOL["fp32"], "stream-K, caller workspace")
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "stream-K lse, caller workspace")
+
+
 # ------------------------------------------------------------------ skinny / split-K path
 @pytest.mark.parametrize("M,N,K", [
     (16, 512, 1024), (1, 128, 64), (5, 300, 2048), (16, 136, 8192), (9, 1032, 392),   # few rows: ticketed split-K
