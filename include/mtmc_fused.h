@@ -105,6 +105,19 @@ int mtmc_fused_linear_residual(const void* X, const void* W, const float* b, con
 int mtmc_fused_linear_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b,
                               int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out, int64_t ldo);
 
+/* The other operators on row-major views, with the same rules (ldx, ldw... >= K and multiples of 8; ldo >= N,
+ * any value): mtmc_swiglu with X, Wg, Wu and out as column slices of wider matrices (the gate and up projections
+ * stored side by side in one fused weight, the output written into a concatenated buffer), and the three row
+ * reductions with X and W as views (their outputs are dense vectors).  Same kernels, same bits as the dense calls. */
+int mtmc_swiglu_strided(const void* X, int64_t ldx, const void* Wg, int64_t ldwg, const void* Wu, int64_t ldwu,
+                        int64_t M, int64_t N, int64_t K, void* out, int64_t ldo);
+int mtmc_linear_lse_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b,
+                            int64_t M, int64_t N, int64_t K, float* lse_out);
+int mtmc_linear_rowmax_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b,
+                               int64_t M, int64_t N, int64_t K, float* max_out, int32_t* argmax_out);
+int mtmc_linear_cross_entropy_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, const int64_t* targets,
+                                      int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out);
+
 /* The same layer with 8-bit floating-point operands:
  *   out[m][n] = act( scale_x * scale_w * sum_k X8[m][k] W8[n][k] + b[n] ).
  * X8 [M,K] and W8 [N,K] hold E4M3 values (1 sign, 4 exponent bits with bias 7, 3 mantissa

@@ -30,7 +30,8 @@ EXPORTS = [
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_device_alloc_count", "mtmc_last_kernel_name", "mtmc_set_timing", "mtmc_last_kernel_ms",
-    "mtmc_fused_linear_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_schedule", "mtmc_trace_enabled", "mtmc_set_trace", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
+    "mtmc_fused_linear_strided", "mtmc_swiglu_strided", "mtmc_linear_lse_strided", "mtmc_linear_rowmax_strided",
+    "mtmc_linear_cross_entropy_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_schedule", "mtmc_trace_enabled", "mtmc_set_trace", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
 
 _lib = None
@@ -62,6 +63,10 @@ def load() -> ctypes.CDLL:
     L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, i64]
+    L.mtmc_swiglu_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, vp, i64]
+    L.mtmc_linear_lse_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, vp]
+    L.mtmc_linear_rowmax_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, vp, vp]
+    L.mtmc_linear_cross_entropy_strided.argtypes = [vp, i64, vp, i64, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_swiglu_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     L.mtmc_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
     L.mtmc_linear_rowmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
@@ -166,6 +171,57 @@ def mtmc_fused_linear_strided(X, W, b, act="none", out_dtype="bf16", out=None):
     _check(load().mtmc_fused_linear_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"),
                                             M, N, K, ACT[act], OUT_DTYPE[out_dtype], op, ldo))
     return out
+
+
+def mtmc_swiglu_strided(X, Wg, Wu, out=None):
+    """mtmc_swiglu on views: X [M,K], Wg / Wu [N,K] and out [M,N] may be column slices of wider row-major tensors."""
+    M, K = X.shape
+    N = Wg.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (gp, ldg), (up, ldu), (op, ldo) = (_view2d(X, torch.bfloat16, (M, K), "X"), _view2d(Wg, torch.bfloat16, (N, K), "Wg"),
+                                                  _view2d(Wu, torch.bfloat16, (N, K), "Wu"), _view2d(out, torch.bfloat16, (M, N), "out"))
+    _check(load().mtmc_swiglu_strided(xp, ldx, gp, ldg, up, ldu, M, N, K, op, ldo))
+    return out
+
+
+def mtmc_linear_lse_strided(X, W, b, lse_out=None):
+    """mtmc_linear_lse with X [M,K] and W [N,K] as views (unit column stride, any row pitch that is a multiple of 8)."""
+    M, K = X.shape
+    N = W.shape[0]
+    if lse_out is None:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (wp, ldw) = _view2d(X, torch.bfloat16, (M, K), "X"), _view2d(W, torch.bfloat16, (N, K), "W")
+    _check(load().mtmc_linear_lse_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"), M, N, K,
+                                          _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
+
+
+def mtmc_linear_rowmax_strided(X, W, b):
+    """mtmc_linear_rowmax with X and W as views; returns (max fp32 [M], argmax int32 [M])."""
+    M, K = X.shape
+    N = W.shape[0]
+    mx = torch.empty((M,), dtype=torch.float32, device=X.device)
+    arg = torch.empty((M,), dtype=torch.int32, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (wp, ldw) = _view2d(X, torch.bfloat16, (M, K), "X"), _view2d(W, torch.bfloat16, (N, K), "W")
+    _check(load().mtmc_linear_rowmax_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"), M, N, K,
+                                             mx.data_ptr(), arg.data_ptr()))
+    return mx, arg
+
+
+def mtmc_linear_cross_entropy_strided(X, W, b, targets):
+    """mtmc_linear_cross_entropy with X and W as views; returns the loss, fp32 [M]."""
+    M, K = X.shape
+    N = W.shape[0]
+    loss = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (wp, ldw) = _view2d(X, torch.bfloat16, (M, K), "X"), _view2d(W, torch.bfloat16, (N, K), "W")
+    _check(load().mtmc_linear_cross_entropy_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                                    _dev(targets, torch.int64, (M,), "targets"), M, N, K, loss.data_ptr(), None))
+    return loss
 
 
 def mtmc_fused_linear_fp8(X8, W8, b, scale_x, scale_w, act="none", out_dtype="bf16", out=None):

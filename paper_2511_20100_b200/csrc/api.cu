@@ -27,8 +27,8 @@ using namespace mtmc;
 constexpr int MAX_DEVICES = 64;
 constexpr size_t TICKET_BYTES = 64 * 1024;   // library-owned split-K tickets: 16384 tiles
 constexpr int SK_MAX_PAIRS = 256;            // stream-K boundaries (pairs of one launch) the flag array covers
-constexpr size_t SK_FLAG_BYTES = SK_MAX_PAIRS * 8 * sizeof(uint32_t);
-constexpr size_t SK_PART_BYTES = 2 * 2 * 4 * 8 * 8 * 32 * sizeof(float4);   // per boundary: 2 sides x 2 ranks x 4 quadrants x 32 KiB
+constexpr size_t SK_FLAG_BYTES = 2 * SK_MAX_PAIRS * 8 * sizeof(uint32_t);    // one ticket word per (region tile, epilogue warp): fewer than two tiles per pair
+constexpr size_t SK_PART_BYTES = 2 * 2 * 4 * 8 * 8 * 32 * sizeof(float4);   // per pair: 2 parts x 2 ranks x 4 quadrants x 32 KiB
 #ifndef MTMC_SKINNY_MAX_M
 #define MTMC_SKINNY_MAX_M 64
 #endif
@@ -355,7 +355,7 @@ int launch_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, co
     using Cfg = PairCfg<EPI>;
     auto kern = gemm_pair_kernel<EPI, OUT_BF16>;
     if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
-    const int pairs = p.num_items < clusters ? p.num_items : clusters;
+    const int pairs = (p.sk || p.num_items >= clusters) ? clusters : p.num_items;      // stream-K: every pair takes a share
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
     cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
@@ -601,15 +601,21 @@ void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
     p.tail_split = ks;
 }
 
-// Stream-K schedule of the pair kernel's last waves (see gemm_pair.cuh).  Needs at least one full wave (the
-// region dealt by k-blocks is the last full wave plus the remainder, so a tile has at most two holders).
-// Only on request (mtmc_set_schedule(1)): measured against the default -- whole tiles with the last wave's tiles
-// cut into column pieces -- it is on a par on C2 (3.46 waves: 104.6 against 103.3 us), C3 and C4 and 3 % behind
-// on 8192 x 4096 x 11008 (6.9 waves), because the column pieces already recover most of a partial wave and the
-// k-block shares run 4 % slower per k-block (pairs that run together no longer work on neighbouring tiles).
+// Stream-K schedule of the pair kernel (see gemm_pair.cuh): the last full wave plus the remainder (everything, when
+// there is less than a wave) is dealt by k-blocks, one equal share per pair.  Needs at least one k-block per pair
+// in that region (the holders of a tile are then consecutive pairs).
+// Only on request (mtmc_set_schedule(1)).  Measured against the default -- whole tiles with the last wave's tiles
+// cut into column pieces, and cluster split-K below half a wave -- it is on a par on C2 (3.46 waves: 104.6 against
+// 103.3 us), C3 and C4, 3 % behind on 8192 x 4096 x 11008 (6.9 waves), a few per cent ahead at 1.3 waves
+// (768 x 8192 x 8192: 108.7 against 113.3 us) and well behind below one wave (128 x 8192 x 8192: 59 against 35 us
+// for cluster split-K): the column pieces already recover most of a partial wave, a share runs 4-6 % slower per
+// k-block than whole tiles walked side by side, and a hand-over costs its last holder a serial read of the other
+// holders' parts (5 us for a writer, up to 20 us for the reader of two parts, exposed when the share has no whole
+// tile to hide it under).
 bool want_streamk(const GemmParams& p, int clusters) {
     if (EPI_HALVES != 1 || t_stream_k <= 0 || clusters <= 0 || clusters > SK_MAX_PAIRS) return false;
-    return p.num_tiles >= clusters && p.num_tiles % clusters != 0;
+    const int region = p.num_tiles - std::max(0, p.num_tiles / clusters - 1) * clusters;
+    return p.num_tiles % clusters != 0 && static_cast<long long>(region) * p.k_blocks >= clusters;
 }
 size_t streamk_bytes(int clusters) { return SK_FLAG_BYTES + static_cast<size_t>(clusters) * SK_PART_BYTES; }
 
@@ -619,7 +625,7 @@ size_t streamk_bytes(int clusters) { return SK_FLAG_BYTES + static_cast<size_t>(
 int attach_streamk(DeviceState* d, GemmParams& p, int clusters, void* ws, size_t offset) {
     p.sk = 1;
     p.n_full = p.num_tiles; p.num_items = p.num_tiles; p.tail_split = 1;
-    p.sk_first_tile = (p.num_tiles / clusters - 1) * clusters;     // all full waves but the last are dealt round-robin
+    p.sk_first_tile = std::max(0, p.num_tiles / clusters - 1) * clusters;     // all full waves but the last are dealt round-robin
     char* base = static_cast<char*>(ws) + offset;
     if (t_user_ws) {
         p.sk_flags = reinterpret_cast<uint32_t*>(base);
@@ -633,7 +639,7 @@ int attach_streamk(DeviceState* d, GemmParams& p, int clusters, void* ws, size_t
             CUDA_TRY(counted_malloc(reinterpret_cast<void**>(&sc->sk_flags), SK_FLAG_BYTES));
             CUDA_TRY(cudaMemsetAsync(sc->sk_flags, 0, SK_FLAG_BYTES, t_stream));
         }
-        sc->sk_epoch = (sc->sk_epoch % 0x3fffffffu) + 1;        // 1 .. 2^30 - 1: the marker (epoch << 2 | side) is never 0
+        sc->sk_epoch = (sc->sk_epoch % 0xfffffeu) + 1;          // 1 .. 2^24 - 2: fits the ticket word's upper 24 bits, never 0
         p.sk_flags = sc->sk_flags;
         p.sk_partial = reinterpret_cast<float4*>(base + SK_FLAG_BYTES);
         p.sk_epoch = sc->sk_epoch;
@@ -654,7 +660,7 @@ bool plan_pair(DeviceState* d, GemmParams& p, int64_t M, int64_t N, int64_t K, i
 // The workspace of a pair-kernel call with no other scratch: nothing, or the stream-K region.
 int pair_scratch(DeviceState* d, GemmParams& p, bool sk) {
     if (!sk) return MTMC_OK;
-    const int clusters = std::min(gemm_pairs(d), p.num_tiles);
+    const int clusters = gemm_pairs(d);
     void* ws = nullptr;
     if (int rc = get_workspace(d, streamk_bytes(clusters), &ws)) return rc;
     return attach_streamk(d, p, clusters, ws, 0);
@@ -906,7 +912,7 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 //   EPI_XENT   : out_b = loss, out_a = lse (may be null); the target logits sit behind the partials
 template <int EPI>
 int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
-                      float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f) {
+                      float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0) {
     auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
     if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
     DeviceState* d = nullptr;
@@ -925,7 +931,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     p.acc_scale = acc_scale;
     const size_t partial_bytes = lse_partial_bytes(p);         // what the chosen plan writes and the merge reads
     const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
-    const int sk_clusters = sk ? std::min(gemm_pairs(d), p.num_tiles) : 0;
+    const int sk_clusters = sk ? gemm_pairs(d) : 0;
     void* ws = nullptr;
     rc = get_workspace(d, partial_bytes + extra + (sk ? streamk_bytes(sk_clusters) : 0), &ws);
     if (rc) return rc;
@@ -936,8 +942,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
     if (EPI == EPI_XENT) CUDA_TRY(cudaMemsetAsync(p.target_logit, 0xFF, static_cast<size_t>(M) * sizeof(float), t_stream));
     CUtensorMap tmA, tmB, tmBt;
-    if ((rc = encode(&tmA, X, M, K, big ? 256 : 128, 0)) || (rc = encode(&tmB, W, N, K, (pair || big) ? 128 : bn, 0)) ||
-        (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width, 0)))
+    if ((rc = encode(&tmA, X, M, K, big ? 256 : 128, ldx)) || (rc = encode(&tmB, W, N, K, (pair || big) ? 128 : bn, ldw)) ||
+        (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width, ldw)))
         return rc;
     TimedRegion tr(d);
     if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
@@ -1034,7 +1040,8 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     return rc;
 }
 // out = silu(sg * X.Wg^T) * (su * X.Wu^T): bf16 operands (sg = su = 1) or E4M3 operands with the scale products.
-int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out, bool fp8, float sg, float su) {
+int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out, bool fp8, float sg, float su,
+                int64_t ldx = 0, int64_t ldwg = 0, int64_t ldwu = 0, int64_t ldo = 0) {
     auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
     int rc = check_common(X, Wg, out, M, N, K);
     if (rc) return rc;
@@ -1047,10 +1054,10 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         GemmParams p{};
         fill_ksplit(p, M, N, K, 128, ks, fp8);
         p.acc_scale = sg; p.acc_scale2 = su;
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU;
-        if ((rc = encode(&tmA, X, M, K, 128, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) ||
-            (rc = encode(&tmU, Wu, N, K, 128, 0)))
+        if ((rc = encode(&tmA, X, M, K, 128, ldx)) || (rc = encode(&tmG, Wg, N, K, 128, ldwg)) ||
+            (rc = encode(&tmU, Wu, N, K, 128, ldwu)))
             return rc;
         TimedRegion tr(d);
         rc = launch_ksplit<EPI_SWIGLU, true>(ks, tmA, tmG, tmU, p);
@@ -1061,9 +1068,9 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         GemmParams p{};
         fill_tiling(p, M, N, K, 128, gemm_pairs(d), false, 512, fp8);
         p.acc_scale = sg; p.acc_scale2 = su;
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU;
-        if ((rc = encode(&tmA, X, M, K, 256, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) || (rc = encode(&tmU, Wu, N, K, 128, 0))) return rc;
+        if ((rc = encode(&tmA, X, M, K, 256, ldx)) || (rc = encode(&tmG, Wg, N, K, 128, ldwg)) || (rc = encode(&tmU, Wu, N, K, 128, ldwu))) return rc;
         TimedRegion tr(d);
         rc = launch_big<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, p);
         tr.stop();
@@ -1074,11 +1081,11 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         const bool sk = plan_pair(d, p, M, N, K, 128, fp8);
         if ((rc = pair_scratch(d, p, sk))) return rc;
         p.acc_scale = sg; p.acc_scale2 = su;
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-        if ((rc = encode(&tmA, X, M, K, 128, 0)) || (rc = encode(&tmG, Wg, N, K, 128, 0)) ||
-            (rc = encode(&tmU, Wu, N, K, 128, 0)) || (rc = encode(&tmGt, Wg, N, K, p.tail_width, 0)) ||
-            (rc = encode(&tmUt, Wu, N, K, p.tail_width, 0)))
+        if ((rc = encode(&tmA, X, M, K, 128, ldx)) || (rc = encode(&tmG, Wg, N, K, 128, ldwg)) ||
+            (rc = encode(&tmU, Wu, N, K, 128, ldwu)) || (rc = encode(&tmGt, Wg, N, K, p.tail_width, ldwg)) ||
+            (rc = encode(&tmUt, Wu, N, K, p.tail_width, ldwu)))
             return rc;
         TimedRegion tr(d);
         rc = launch_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmG, tmU, tmGt, tmUt, p);
@@ -1088,17 +1095,17 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     GemmParams p{};
     fill_tiling(p, M, N, K, 128, d->sm_count, true, 128, fp8);   // 128 output columns = 128 gate + 128 up accumulator columns
     p.acc_scale = sg; p.acc_scale2 = su;
-        p.act = ACT_NONE; p.bias = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
+        p.act = ACT_NONE; p.bias = nullptr; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
     CUtensorMap tmA, tmG, tmU, tmGt, tmUt;
-    rc = encode(&tmA, X, M, K, 128, 0);
+    rc = encode(&tmA, X, M, K, 128, ldx);
     if (rc) return rc;
-    rc = encode(&tmG, Wg, N, K, 128, 0);
+    rc = encode(&tmG, Wg, N, K, 128, ldwg);
     if (rc) return rc;
-    rc = encode(&tmU, Wu, N, K, 128, 0);
+    rc = encode(&tmU, Wu, N, K, 128, ldwu);
     if (rc) return rc;
-    rc = encode(&tmGt, Wg, N, K, p.tail_width, 0);
+    rc = encode(&tmGt, Wg, N, K, p.tail_width, ldwg);
     if (rc) return rc;
-    rc = encode(&tmUt, Wu, N, K, p.tail_width, 0);
+    rc = encode(&tmUt, Wu, N, K, p.tail_width, ldwu);
     if (rc) return rc;
     TimedRegion tr(d);
     rc = launch_tiled<EPI_SWIGLU, 256, true>(d, tmA, tmG, tmU, tmGt, tmUt, p);
@@ -1362,6 +1369,15 @@ int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
     return swiglu_impl(X, Wg, Wu, M, N, K, out, false, 1.0f, 1.0f);
 }
 
+int mtmc_swiglu_strided(const void* X, int64_t ldx, const void* Wg, int64_t ldwg, const void* Wu, int64_t ldwu, int64_t M, int64_t N,
+                        int64_t K, void* out, int64_t ldo) {
+    if (ldx < K || ldwg < K || ldwu < K || ldo < N) return fail(MTMC_ERR_INVALID_ARG, "row pitches must cover the rows (ldx, ldwg, ldwu >= K, ldo >= N)");
+    if (ldx % 8 != 0 || ldwg % 8 != 0 || ldwu % 8 != 0)
+        return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "ldx, ldwg and ldwu must be multiples of 8 elements (16-byte rows for TMA)");
+    if (ldx >= (1ll << 31) || ldwg >= (1ll << 31) || ldwu >= (1ll << 31) || ldo >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "row pitches must be below 2^31");
+    return swiglu_impl(X, Wg, Wu, M, N, K, out, false, 1.0f, 1.0f, ldx, ldwg, ldwu, ldo);
+}
+
 int mtmc_swiglu_fp8(const void* X8, const void* Wg8, const void* Wu8, float scale_x, float scale_g, float scale_u,
                     int64_t M, int64_t N, int64_t K, void* out) {
     if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
@@ -1372,6 +1388,39 @@ int mtmc_linear_lse(const void* X, const void* W, const float* b, int64_t M, int
     int rc = check_common(X, W, lse_out, M, N, K);
     if (rc) return rc;
     return run_row_reduction<EPI_LSE>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr);
+}
+
+namespace {
+int check_row_pitches(int64_t ldx, int64_t ldw, int64_t K) {
+    if (ldx < K || ldw < K) return fail(MTMC_ERR_INVALID_ARG, "row pitches must cover the rows (ldx, ldw >= K)");
+    if (ldx % 8 != 0 || ldw % 8 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "ldx and ldw must be multiples of 8 elements (16-byte rows for TMA)");
+    if (ldx >= (1ll << 31) || ldw >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "row pitches must be below 2^31");
+    return MTMC_OK;
+}
+}  // namespace
+
+int mtmc_linear_lse_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, int64_t M, int64_t N, int64_t K,
+                            float* lse_out) {
+    int rc = check_common(X, W, lse_out, M, N, K);
+    if (rc || (rc = check_row_pitches(ldx, ldw, K))) return rc;
+    return run_row_reduction<EPI_LSE>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr, false, 1.0f, ldx, ldw);
+}
+
+int mtmc_linear_rowmax_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, int64_t M, int64_t N, int64_t K,
+                               float* max_out, int32_t* argmax_out) {
+    int rc = check_common(X, W, max_out, M, N, K);
+    if (rc || (rc = check_row_pitches(ldx, ldw, K))) return rc;
+    if (argmax_out && (reinterpret_cast<uintptr_t>(argmax_out) & 3u)) return fail(MTMC_ERR_INVALID_ARG, "argmax_out must be 4-byte aligned");
+    return run_row_reduction<EPI_ROWMAX>(X, W, b, nullptr, M, N, K, max_out, nullptr, argmax_out, false, 1.0f, ldx, ldw);
+}
+
+int mtmc_linear_cross_entropy_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, const int64_t* targets,
+                                      int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out) {
+    int rc = check_common(X, W, loss_out, M, N, K);
+    if (rc || (rc = check_row_pitches(ldx, ldw, K))) return rc;
+    if (!targets) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (reinterpret_cast<uintptr_t>(targets) & 7u) return fail(MTMC_ERR_INVALID_ARG, "targets must be 8-byte aligned");
+    return run_row_reduction<EPI_XENT>(X, W, b, targets, M, N, K, lse_out, loss_out, nullptr, false, 1.0f, ldx, ldw);
 }
 
 int mtmc_linear_lse_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,

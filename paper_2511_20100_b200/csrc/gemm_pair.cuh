@@ -11,19 +11,18 @@
 // the accumulator to both; the epilogue warps of both CTAs arrive on the even CTA's
 // `accumulator empty` barrier.  No TMA load uses cluster multicast.
 //
-// Stream-K schedule for the last waves (GemmParams::sk).  Whole tiles dealt round-robin leave the last wave
-// partly empty: 3.46 waves of tiles cost 4 tile-times.  With this schedule the full waves but one are dealt
-// round-robin as before (pairs that run together work on neighbouring tiles and share operands in L2), and the
-// last full wave plus the remainder -- between one and two tiles per pair -- is dealt by k-blocks: the flat
-// list of that region's (tile, k-block) units is cut into one contiguous, equal share per pair, so all pairs
-// finish together.  A pair's share begins with the END of a tile's K range (the tile's beginning belongs to
-// the pair before) and ends with the BEGINNING of another tile's K range; every tile has at most two holders.
-// The two holders of a shared tile meet without waiting for one another: each epilogue warp that finishes
-// its part either finds its counterpart's part already in global memory and adds it to its accumulator
-// (then runs the ordinary epilogue), or leaves its own part there, marks the flag word and moves on;
-// whoever marks second finishes the tile.  A pair works on its two shared pieces first and on its whole tiles
-// after them, so the hand-overs run under the mainloop of the tiles that follow.  Two fp32 addends commute,
-// so the result does not depend on who finishes.
+// Stream-K schedule (GemmParams::sk).  Whole tiles dealt round-robin leave the last wave partly empty (3.46
+// waves of tiles cost 4 tile-times) and a problem of fewer tiles than pairs leaves pairs idle while the others
+// walk all of K.  With this schedule the full waves but one are dealt round-robin as before (pairs that run
+// together work on neighbouring tiles and share operands in L2), and the rest -- the last full wave plus the
+// remainder, or everything when there is less than a wave -- is dealt by k-blocks: the flat list of that region's
+// (tile, k-block) units is cut into one contiguous, equal share per pair, so all pairs stream the same number of
+// operand bytes and finish together.  A tile whose k-blocks straddle shares has several holders (consecutive
+// pairs).  They meet without waiting for one another: each epilogue warp that finishes its part either finds
+// all other holders' parts already in global memory, adds them to its accumulator in holder order and runs the
+// ordinary epilogue, or leaves its own part there, counts itself in on the tile's ticket word and moves on.  A
+// pair works on its pieces of shared tiles first and on its whole tiles after them, so the hand-overs run under
+// the mainloop of the tiles that follow.
 #pragma once
 #include "gemm_tiled.cuh"
 
@@ -45,77 +44,105 @@ struct PairCfg {
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
 };
 
-// One work item of a pair: a whole tile or tail piece (side == 0), or k-blocks [kb0, kb1) of a tile shared with
-// a neighbouring pair under the stream-K schedule (side 1: the beginning of the tile's K range, 2: its end).
+// One work item of a pair: a whole tile or tail piece (part < 0), or k-blocks [kb0, kb1) of a tile that this pair
+// shares with its neighbours under the stream-K schedule (part 0 or 1: which of the pair's two part buffers).
 struct PairWork {
     int item, kb0, kb1;
-    int side, slot;      // slot: the boundary's index = the lower of the two pairs that share the tile
+    int part;
 };
+
+// Owner of unit x when `total` units are cut into `pairs` contiguous shares [total*p/pairs, total*(p+1)/pairs).
+__device__ __forceinline__ int streamk_owner(long long x, long long total, int pairs) {
+    return static_cast<int>(((x + 1) * pairs - 1) / total);
+}
 
 struct PairWalk {
     int u, dp_end, step;                   // round-robin part: next item, end, stride
-    int KB, pair_id, sk_first;
-    int tail_tile, tail_kb0;               // stream-K region: the END of a tile's K range that opens this pair's share (tail_kb0 > 0), if any
-    int head_tile, head_kb1;               // ... the BEGINNING of a tile's K range that closes it (head_kb1 < KB), if any
-    int whole, whole_end;                  // ... and the whole tiles in between
-    int phase;                             // 0 round-robin, 1 tail piece, 2 head piece, 3 whole tiles of the share
+    int KB, sk_first;
+    int t0, a, t1, b;                      // stream-K share: from k-block a of region tile t0 to k-block b (exclusive) of region tile t1
+    int whole, whole_end;                  // whole tiles of the share still to hand out
+    int phase;                             // 0 round-robin, 1 first piece, 2 last piece, 3 whole tiles
+    bool sk;
     __device__ __forceinline__ PairWalk(const GemmParams& p, int pair, int num_pairs) {
-        KB = p.k_blocks; pair_id = pair; step = num_pairs;
+        KB = p.k_blocks; step = num_pairs; sk = p.sk != 0;
         u = pair;
-        dp_end = p.sk ? p.sk_first_tile : p.num_items;
+        dp_end = sk ? p.sk_first_tile : p.num_items;
         sk_first = p.sk_first_tile;
         phase = 0;
-        tail_tile = head_tile = -1; tail_kb0 = head_kb1 = 0; whole = whole_end = 0;
-        if (p.sk) {
+        t0 = t1 = a = b = 0; whole = whole_end = 0;
+        if (sk) {
             const long long U = static_cast<long long>(p.num_items - p.sk_first_tile) * KB;
             const long long su = U * pair / num_pairs, su_end = U * (pair + 1) / num_pairs;
-            const int t0 = static_cast<int>(su / KB), a = static_cast<int>(su - static_cast<long long>(t0) * KB);
-            const int t1 = static_cast<int>((su_end - 1) / KB), b = static_cast<int>(su_end - static_cast<long long>(t1) * KB);
-            whole = t0; whole_end = t1 + 1;
-            if (a > 0) { tail_tile = t0; tail_kb0 = a; whole = t0 + 1; }
-            if (b < KB) { head_tile = t1; head_kb1 = b; whole_end = t1; }
+            if (su_end > su) {
+                t0 = static_cast<int>(su / KB); a = static_cast<int>(su - static_cast<long long>(t0) * KB);
+                t1 = static_cast<int>((su_end - 1) / KB); b = static_cast<int>(su_end - static_cast<long long>(t1) * KB);
+                whole = a > 0 ? t0 + 1 : t0;
+                whole_end = b < KB ? t1 : t1 + 1;
+            } else {
+                phase = 4;                 // more pairs than k-blocks: nothing for this one
+                sk = false; dp_end = 0;
+            }
         }
     }
-    // Order inside the share: the two pieces of shared tiles first, then the whole tiles.  The piece that closes the
-    // share comes second, not last, so that its hand-over (and, if this pair comes second, the tile's completion)
-    // runs under the mainloop of the whole tiles that follow instead of after the last MMA of the launch.
+    // Order inside the share: its pieces of shared tiles first, then its whole tiles, so that the hand-overs (and,
+    // where this pair is the last holder to arrive, the tile's completion) run under the mainloop of what follows
+    // instead of after the last MMA of the launch.
     __device__ __forceinline__ bool next(PairWork& w) {
         if (phase == 0) {
-            if (u < dp_end) { w.item = u; w.kb0 = 0; w.kb1 = KB; w.side = 0; w.slot = 0; u += step; return true; }
-            phase = 1;
+            if (u < dp_end) { w.item = u; w.kb0 = 0; w.kb1 = KB; w.part = -1; u += step; return true; }
+            phase = sk ? 1 : 4;
         }
         if (phase == 1) {
             phase = 2;
-            if (tail_tile >= 0) { w.item = sk_first + tail_tile; w.kb0 = tail_kb0; w.kb1 = KB; w.side = 2; w.slot = pair_id - 1; return true; }
+            if (a > 0 || (t0 == t1 && b < KB)) {      // the share begins inside tile t0 (or lies inside it altogether)
+                w.item = sk_first + t0; w.kb0 = a; w.kb1 = t0 == t1 ? b : KB; w.part = 0;
+                return true;
+            }
         }
         if (phase == 2) {
             phase = 3;
-            if (head_tile >= 0) { w.item = sk_first + head_tile; w.kb0 = 0; w.kb1 = head_kb1; w.side = 1; w.slot = pair_id; return true; }
+            if (t1 > t0 && b < KB) { w.item = sk_first + t1; w.kb0 = 0; w.kb1 = b; w.part = 1; return true; }
         }
-        if (whole < whole_end) { w.item = sk_first + whole; w.kb0 = 0; w.kb1 = KB; w.side = 0; w.slot = 0; ++whole; return true; }
+        if (phase == 3 && whole < whole_end) { w.item = sk_first + whole; w.kb0 = 0; w.kb1 = KB; w.part = -1; ++whole; return true; }
         return false;
     }
 };
 
 // Stream-K hand-over for one epilogue warp (CTA `rank` of the pair, TMEM lane quadrant q) whose accumulator holds
-// part of a shared tile's K range.  Returns true if this warp has to finish the tile: its accumulator in tensor
-// memory then holds the whole sum.  Returns false if it left its part for the other holder.
+// the sum over part of a shared tile's K range.  The holders of a tile are the consecutive pairs whose shares
+// meet its k-blocks.  Nobody waits: a warp that finds all other holders' parts in global memory adds them to its
+// accumulator, in holder order, and returns true (its accumulator in tensor memory then holds the whole sum and the
+// ordinary epilogue follows); otherwise it leaves its own part, counts itself in and returns false.  The sum is
+// always formed in holder order, so the bits do not depend on who arrives last.
 template <int BN>
-__device__ __forceinline__ bool streamk_meet(const GemmParams& p, const PairWork& w, uint32_t t_addr, int rank, int q, int lane) {
+__device__ __forceinline__ bool streamk_meet(const GemmParams& p, const PairWork& w, uint32_t t_addr, int pair_id, int num_pairs,
+                                             int rank, int q, int lane) {
     constexpr int CHUNKS = BN / 32;
     constexpr size_t WARP_F4 = static_cast<size_t>(CHUNKS) * 8 * 32;           // float4 per warp and part
-    if (!MTMC_CHECK(w.slot >= 0 && w.slot < static_cast<int>(gridDim.x >> 1) - 1 && (w.side == 1 || w.side == 2), p.status, 3u)) return false;
-    uint32_t* flag = p.sk_flags + (static_cast<size_t>(w.slot) * 2 + rank) * 4 + q;
-    const uint32_t mine = (p.sk_epoch << 2) | static_cast<uint32_t>(w.side);
-    const uint32_t theirs = (p.sk_epoch << 2) | static_cast<uint32_t>(3 - w.side);
-    float4* my_part = p.sk_partial + (((static_cast<size_t>(w.slot) * 2 + (w.side - 1)) * 2 + rank) * 4 + q) * WARP_F4;
-    const float4* peer_part = p.sk_partial + (((static_cast<size_t>(w.slot) * 2 + (2 - w.side)) * 2 + rank) * 4 + q) * WARP_F4;
+    const int KB = p.k_blocks;
+    const int tt = w.item - p.sk_first_tile;                                   // tile index inside the stream-K region
+    const long long U = static_cast<long long>(p.num_items - p.sk_first_tile) * KB;
+    const int h_first = streamk_owner(static_cast<long long>(tt) * KB, U, num_pairs);
+    const int h_last = streamk_owner(static_cast<long long>(tt + 1) * KB - 1, U, num_pairs);
+    const uint32_t holders = static_cast<uint32_t>(h_last - h_first + 1);
+    if (!MTMC_CHECK(tt >= 0 && h_first <= pair_id && pair_id <= h_last && holders >= 2u && holders < 256u && (w.part == 0 || w.part == 1),
+                    p.status, 3u))
+        return false;
+    auto part_of = [&](int holder, int which) {
+        return p.sk_partial + (((static_cast<size_t>(holder) * 2 + which) * 2 + rank) * 4 + q) * WARP_F4;
+    };
+    // which of its two part buffers a holder uses for this tile: 0 if its share begins in this tile, else 1
+    auto which_of = [&](int holder) { return static_cast<int>((U * holder / num_pairs) / KB) == tt ? 0 : 1; };
+    uint32_t* ticket = p.sk_flags + (static_cast<size_t>(tt) * 2 + rank) * 4 + q;
+    // ticket word: launch epoch in the upper 24 bits (a word left by an earlier launch counts as zero), arrivals below
     uint32_t seen = 0;
-    if (lane == 0) seen = ld_acquire_gpu(flag);
+    if (lane == 0) seen = ld_acquire_gpu(ticket);
     seen = __shfl_sync(0xffffffffu, seen, 0);
-    if (seen != theirs) {
-        // the other holder has not been here yet: leave this part (every store instruction of the warp writes 512
-        // contiguous bytes; the reader is the thread at the same place of the other pair, so the layout is private)
+    uint32_t arrived = (seen >> 8) == p.sk_epoch ? (seen & 0xffu) : 0u;
+    if (arrived + 1u < holders) {
+        // not everybody else has been here: leave this part (every store instruction of the warp writes 512
+        // contiguous bytes; the reader is the thread at the same place of another pair, so the layout is private)
+        float4* mine = part_of(pair_id, w.part);
 #pragma unroll 1
         for (int c = 0; c < CHUNKS; ++c) {
             uint32_t r[32];
@@ -123,42 +150,54 @@ __device__ __forceinline__ bool streamk_meet(const GemmParams& p, const PairWork
             tmem_ld_wait();
 #pragma unroll
             for (int v = 0; v < 8; ++v)
-                __stcg(my_part + (c * 8 + v) * 32 + lane, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                                      __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
+                __stcg(mine + (c * 8 + v) * 32 + lane, make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                                   __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3])));
         }
         __threadfence();
         __syncwarp();
-        if (lane == 0) seen = atom_exch_acq_rel_gpu(flag, mine);
+        if (lane == 0) {
+            uint32_t old = seen, now;
+            for (;;) {                                       // arrivals + 1 under this launch's epoch (a handful of contenders at most)
+                now = (old >> 8) == p.sk_epoch ? old + 1u : ((p.sk_epoch << 8) | 1u);
+                const uint32_t prev = atomicCAS(ticket, old, now);
+                if (prev == old) break;
+                old = prev;
+            }
+            seen = now;
+        }
         seen = __shfl_sync(0xffffffffu, seen, 0);
-        if (seen != theirs) return false;            // marked first: the other holder finishes the tile
+        arrived = seen & 0xffu;
+        if (arrived < holders) return false;                 // somebody is still to come: the last one finishes the tile
     }
-    __threadfence();                                 // the other part was complete before its flag was set
-    // own part from tensor memory + the other part from L2 (the next chunk's loads in flight meanwhile), back to tensor memory
-    float4 o[8];
-#pragma unroll
-    for (int v = 0; v < 8; ++v) o[v] = __ldcg(peer_part + v * 32 + lane);
+    __threadfence();                                         // the other parts were complete before their holders counted themselves in
+    // The sum in holder order, chunk by chunk: the other holders' parts from L2 (all loads of a chunk in flight
+    // together), this pair's own from tensor memory at its place in the order; back to tensor memory.
 #pragma unroll 1
     for (int c = 0; c < CHUNKS; ++c) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_addr + c * 32, r);
-        float4 nx[8];
-        if (c + 1 < CHUNKS) {
+        float acc[32];
 #pragma unroll
-            for (int v = 0; v < 8; ++v) nx[v] = __ldcg(peer_part + ((c + 1) * 8 + v) * 32 + lane);
-        }
-        tmem_ld_wait();
+        for (int j = 0; j < 32; ++j) acc[j] = 0.0f;          // 0 + x == x: the sum below is part(first) + part(next) + ...
+        for (int h = h_first; h <= h_last; ++h) {
+            if (h == pair_id) {
+                tmem_ld_wait();
 #pragma unroll
-        for (int v = 0; v < 8; ++v) {
-            r[4 * v] = __float_as_uint(__uint_as_float(r[4 * v]) + o[v].x);
-            r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + o[v].y);
-            r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + o[v].z);
-            r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + o[v].w);
+                for (int j = 0; j < 32; ++j) acc[j] += __uint_as_float(r[j]);
+            } else {
+                const float4* src = part_of(h, which_of(h)) + c * 8 * 32 + lane;
+                float4 o[8];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) o[v] = __ldcg(src + v * 32);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    acc[4 * v] += o[v].x; acc[4 * v + 1] += o[v].y; acc[4 * v + 2] += o[v].z; acc[4 * v + 3] += o[v].w;
+                }
+            }
         }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(acc[j]);
         tmem_st_32x32b_x32(t_addr + c * 32, r);
-        if (c + 1 < CHUNKS) {
-#pragma unroll
-            for (int v = 0; v < 8; ++v) o[v] = nx[v];
-        }
     }
     tmem_st_wait();
     return true;
@@ -332,8 +371,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint32_t t_addr = tmem_base + lane_base + static_cast<uint32_t>(buf * Cfg::BN);
             const int chunks = width / 32, split_at = EPI_HALVES == 2 ? (chunks + 1) / 2 : chunks;      // two warps per lane quadrant share the columns
             // part of a shared tile (stream-K): either the whole sum ends up in this accumulator, or the other holder finishes
-            const bool finish = w.side == 0 || streamk_meet<Cfg::BN>(p, w, t_addr, static_cast<int>(rank), q, lane);
-            if (tracer && w.side != 0) tr.add(TR_EPI_HANDOVER, tr.now() - tb);
+            const bool finish = w.part < 0 || streamk_meet<Cfg::BN>(p, w, t_addr, pair_id, num_pairs, static_cast<int>(rank), q, lane);
+            if (tracer && w.part >= 0) tr.add(TR_EPI_HANDOVER, tr.now() - tb);
             if (finish)
                 epilogue_item<EPI, OUT_BF16>(p, t_addr, row, n_tile0, half ? split_at : 0, half ? chunks : split_at, width, nb, sub, half,
                                              vec_ok, smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);

@@ -58,13 +58,13 @@ struct GemmParams {
     uint32_t* status;     // device status word
     unsigned long long* trace;   // per-CTA trace records (-DMTMC_TRACE builds, mtmc_set_trace), else null
     // Stream-K schedule of the CTA-pair kernel (gemm_pair.cuh): tiles [0, sk_first_tile) are dealt round-robin; the
-    // (tile, k-block) units of the remaining tiles (between one and two per pair) are cut into one contiguous, equal
-    // share per pair, so a tile whose k-blocks straddle a boundary is finished by two pairs.
+    // (tile, k-block) units of the remaining tiles (fewer than two per pair) are cut into one contiguous, equal
+    // share per pair, so a tile whose k-blocks straddle shares is finished by the last of its holders to arrive.
     int sk;               // 1: stream-K schedule (whole tiles only: n_full == num_items == num_tiles)
     int sk_first_tile;    // a multiple of the number of pairs
-    uint32_t sk_epoch;    // launch counter: flag words of earlier launches never match this launch's markers
-    uint32_t* sk_flags;   // [pairs][2 ranks][4 lane quadrants] one word per (boundary, epilogue warp)
-    float4* sk_partial;   // [pairs][2 sides][2 ranks][4 quadrants][8 chunks][8][32 lanes] fp32 accumulator parts
+    uint32_t sk_epoch;    // launch counter (24 bits): ticket words left by earlier launches read as zero arrivals
+    uint32_t* sk_flags;   // [region tiles][2 ranks][4 lane quadrants] one ticket word per (shared tile, epilogue warp)
+    float4* sk_partial;   // [pairs][2 parts][2 ranks][4 quadrants][8 chunks][8][32 lanes] fp32 accumulator parts
 };
 
 template <int EPI, int BN>

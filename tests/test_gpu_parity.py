@@ -184,6 +184,45 @@ def test_fused_linear_strided_views(M, N, K, padx, padw, pado, act, odt):
     assert torch.equal(dense, Ov.contiguous())              # the same kernels on the same values
 
 
+@pytest.mark.parametrize("M,N,K,padx,padw,pado", [(100, 72, 136, 8, 24, 3), (300, 520, 328, 16, 8, 8), (128, 1024, 4096, 64, 64, 1024),
+                                                  (1100, 1300, 1024, 8, 16, 4)])
+def test_other_operators_on_strided_views(M, N, K, padx, padw, pado):
+    """SwiGLU and the three row reductions on column slices of wider matrices (single-CTA, cluster split-K and
+    CTA-pair kernels): the same bits as the dense calls, within tolerance of the oracle, neighbours untouched."""
+    si = inputs.swiglu_inputs(M, N, K, seed=9050 + M + N)
+    li = inputs.linear_inputs(M, N, K, seed=9060 + M + N)
+    tgt = torch.from_numpy(np.random.default_rng(M + N).integers(0, N, size=M)).cuda()
+    Xw = torch.full((M, K + padx), 3.0, dtype=torch.bfloat16, device="cuda")
+    GU = torch.full((N, 2 * K + padw), -2.0, dtype=torch.bfloat16, device="cuda")       # gate and up side by side in one matrix
+    Ow = torch.full((M, N + pado), 7.0, dtype=torch.bfloat16, device="cuda")
+    offx, offo = (8 if padx >= 16 else 0), (8 if pado >= 16 else 0)
+    Xv, Gv, Uv, Ov = Xw[:, offx:offx + K], GU[:, :K], GU[:, K:2 * K], Ow[:, offo:offo + N]
+    Xv.copy_(si.X.cuda()); Gv.copy_(si.Wg.cuda()); Uv.copy_(si.Wu.cuda())
+    B.mtmc_swiglu_strided(Xv, Gv, Uv, out=Ov)
+    B.mtmc_check_status()
+    want = ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu))
+    _assert_close(inputs.to_f64(Ov.contiguous()), want, TOL["bf16"], "strided swiglu %dx%dx%d" % (M, N, K))
+    assert bool((Ow[:, :offo] == 7.0).all()) and bool((Ow[:, offo + N:] == 7.0).all())
+    assert torch.equal(B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda()), Ov.contiguous())
+    # the row reductions: X as above, W as the left half of the wide matrix
+    Xv.copy_(li.X.cuda()); Gv.copy_(li.W.cuda())
+    bd = li.b.cuda()
+    lse = B.mtmc_linear_lse_strided(Xv, Gv, bd)
+    mx, arg = B.mtmc_linear_rowmax_strided(Xv, Gv, bd)
+    loss = B.mtmc_linear_cross_entropy_strided(Xv, Gv, bd, tgt)
+    B.mtmc_check_status()
+    Xd, Wd = li.X.cuda(), li.W.cuda()
+    assert torch.equal(lse, B.mtmc_linear_lse(Xd, Wd, bd))
+    dmx, darg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+    assert torch.equal(mx, dmx) and torch.equal(arg, darg)
+    assert torch.equal(loss, B.mtmc_linear_cross_entropy(Xd, Wd, bd, tgt))
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "strided lse")
+    _check_rowmax(li, mx, arg, "strided rowmax")
+    want_loss, _ = ref.linear_cross_entropy(Xb, Wb, bf, tgt.cpu().numpy())
+    _assert_close(inputs.to_f64(loss), want_loss, TOL["fp32"], "strided cross entropy")
+
+
 def test_large_tile_pair_kernel_chosen_for_long_k():
     """From 96 k-blocks on the 512 x 256 tiles are the default for M >= 512, N >= 256: bf16, residual and FP8 forms."""
     M, N, K = 600, 520, 6144
@@ -718,9 +757,13 @@ def test_calls_on_two_streams_keep_their_scratch_apart():
 
 
 # ------------------------------------------------------------------ stream-K schedule of the 256 x 256 pair kernel
-# Forced by the schedule hook on problems with at least as many tiles as CTA pairs (81 to 100 tiles on 74 pairs):
-# shares that begin and end inside tiles, k-block counts that do not divide, ragged rows / columns / K.
-STREAMK = [(2304, 2304, 328), (2304, 2400, 4096), (2500, 2200, 72), (2304, 2304, 64)]
+# Forced by the schedule hook: problems with somewhat more tiles than CTA pairs (81 to 100 tiles on 74 pairs: the last
+# full wave and the remainder are dealt by k-blocks, two holders per shared tile) and with fewer tiles than pairs
+# (everything is dealt by k-blocks); shares that begin and end inside tiles, k-block counts that do not divide,
+# ragged rows / columns / K.
+STREAMK = [(2304, 2304, 328), (2304, 2400, 4096), (2500, 2200, 72), (2304, 2304, 64),
+           # fewer tiles than pairs: every tile has several holders (up to five), some pairs' shares lie inside one tile
+           (300, 2304, 4096), (128, 8192, 2048), (520, 1000, 1096), (300, 520, 72)]
 
 
 def _streamk(fn):
