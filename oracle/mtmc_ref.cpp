@@ -18,6 +18,10 @@
 //   FP8 linear   :  Y[m][n] = act( sx*sw * sum_k Xq[m][k] Wq[n][k] + b[n] ),  Xq, Wq 8-bit floats
 //                   (E4M3: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities),
 //                   sx, sw per-tensor scales: the lower-precision variant of the same layer
+//   MXFP8 linear :  the same with block scales instead of per-tensor ones (the microscaling format MXFP8):
+//                   z[m][n] = sum_k (2^(SX[m][k/32]-127) Xq[m][k]) (2^(SW[n][k/32]-127) Wq[n][k]) + b[n],
+//                   Xq, Wq E4M3, SX [M,K/32] and SW [N,K/32] one biased power-of-two exponent (UE8M0) per
+//                   32 consecutive elements of K; also as SwiGLU gate and as row logsumexp
 //   SwiGLU       :  out[m][n] = silu(g[m][n]) * u[m][n],  g = X.Wg^T, u = X.Wu^T (no bias)
 //   row LSE      :  lse[m] = log( sum_n exp(z[m][n]) ), computed two-pass (max, then sum)
 //   row max      :  mx[m] = max_n z[m][n], arg[m] = the lowest n attaining it
@@ -70,6 +74,21 @@ double e4m3_to_double(uint8_t bits) {
     else if (e == 0) v = std::ldexp(static_cast<double>(m) / 8.0, -6);
     else v = std::ldexp(1.0 + static_cast<double>(m) / 8.0, e - 7);
     return sign ? -v : v;
+}
+
+// UE8M0 scale byte -> double, exactly: an unsigned biased exponent, 2^(e - 127); 255 is NaN.
+double e8m0_to_double(uint8_t e) {
+    if (e == 255) return std::numeric_limits<double>::quiet_NaN();
+    return std::ldexp(1.0, static_cast<int>(e) - 127);
+}
+
+// One block-scaled dot product: every element is decoded and multiplied by its block's scale first (exact in
+// double: an E4M3 value times a power of two), then the products are summed in ascending k.
+double dot_row_mx(const uint8_t* x, const uint8_t* sx, const uint8_t* w, const uint8_t* sw, int64_t K) {
+    double acc = 0.0;
+    for (int64_t k = 0; k < K; ++k)
+        acc += (e8m0_to_double(sx[k / 32]) * e4m3_to_double(x[k])) * (e8m0_to_double(sw[k / 32]) * e4m3_to_double(w[k]));
+    return acc;
 }
 
 // One pre-activation value: ascending k, one double accumulator, bias added last.
@@ -389,6 +408,53 @@ int mtmc_ref_linear_cross_entropy_fp8(const uint8_t* X, const uint8_t* W, const 
 
 // logsumexp of a plain vector of doubles (pins: closed forms, shift law).
 double mtmc_ref_lse_vector(const double* z, int64_t N) { return lse_of_row(z, N); }
+
+// Scalar decode of one UE8M0 scale byte (for the pins).
+double mtmc_ref_e8m0(uint8_t e) { return e8m0_to_double(e); }
+
+// Y = act(z + b) with block-scaled E4M3 operands: X [M,K], SX [M,K/32], W [N,K], SW [N,K/32]; K % 32 == 0.
+int mtmc_ref_fused_linear_mxfp8(const uint8_t* X, const uint8_t* SX, const uint8_t* W, const uint8_t* SW, const float* b,
+                                int64_t M, int64_t N, int64_t K, int act, double* out) {
+    if (!X || !SX || !W || !SW || !out || M <= 0 || N <= 0 || K <= 0 || K % 32 != 0 || act < 0 || act > 3) return 1;
+    const int64_t KB = K / 32;
+    parallel_for(M, [=](int64_t m) {
+        for (int64_t n = 0; n < N; ++n) {
+            double z = dot_row_mx(X + m * K, SX + m * KB, W + n * K, SW + n * KB, K);
+            if (b) z += static_cast<double>(b[n]);
+            out[m * N + n] = act_apply(act, z);
+        }
+    });
+    return 0;
+}
+
+// out = silu(z_gate) * z_up with block-scaled E4M3 operands; gate and up weights with their own scales.
+int mtmc_ref_swiglu_mxfp8(const uint8_t* X, const uint8_t* SX, const uint8_t* Wg, const uint8_t* SG, const uint8_t* Wu, const uint8_t* SU,
+                          int64_t M, int64_t N, int64_t K, double* out) {
+    if (!X || !SX || !Wg || !SG || !Wu || !SU || !out || M <= 0 || N <= 0 || K <= 0 || K % 32 != 0) return 1;
+    const int64_t KB = K / 32;
+    parallel_for(M, [=](int64_t m) {
+        for (int64_t n = 0; n < N; ++n) {
+            const double g = dot_row_mx(X + m * K, SX + m * KB, Wg + n * K, SG + n * KB, K);
+            const double u = dot_row_mx(X + m * K, SX + m * KB, Wu + n * K, SU + n * KB, K);
+            out[m * N + n] = act_apply(3, g) * u;
+        }
+    });
+    return 0;
+}
+
+// lse[m] = log sum_n exp(z[m][n] + b[n]) with block-scaled E4M3 operands (two passes, as for bf16).
+int mtmc_ref_linear_lse_mxfp8(const uint8_t* X, const uint8_t* SX, const uint8_t* W, const uint8_t* SW, const float* b,
+                              int64_t M, int64_t N, int64_t K, double* lse) {
+    if (!X || !SX || !W || !SW || !lse || M <= 0 || N <= 0 || K <= 0 || K % 32 != 0) return 1;
+    const int64_t KB = K / 32;
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n)
+            z[n] = dot_row_mx(X + m * K, SX + m * KB, W + n * K, SW + n * KB, K) + (b ? static_cast<double>(b[n]) : 0.0);
+        lse[m] = lse_of_row(z.data(), N);
+    });
+    return 0;
+}
 
 // Element-wise comparator.  got/ref are double (the caller widens the GPU result
 // exactly).  An element passes when |got-ref| <= atol + rtol*|ref| and both are

@@ -51,6 +51,11 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_linear_lse_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
         L.mtmc_ref_linear_rowmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp, vp]
         L.mtmc_ref_linear_cross_entropy_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, i64, i64, i64, vp, vp]
+        L.mtmc_ref_e8m0.argtypes = [ctypes.c_uint8]
+        L.mtmc_ref_e8m0.restype = dbl
+        L.mtmc_ref_fused_linear_mxfp8.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, ci, vp]
+        L.mtmc_ref_swiglu_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+        L.mtmc_ref_linear_lse_mxfp8.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_fused_linear_points.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, i64, vp]
         L.mtmc_ref_swiglu.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_swiglu_points.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, vp]
@@ -150,6 +155,54 @@ def fused_linear_fp8(X, W, b, scale_x: float, scale_w: float, act_kind: int) -> 
     _check(lib().mtmc_ref_fused_linear_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
                                            int(act_kind), out.ctypes.data), "mtmc_ref_fused_linear_fp8")
     return out
+
+
+def e8m0(byte: int) -> float:
+    """UE8M0 scale byte -> its value, 2^(byte - 127) (255: NaN)."""
+    return float(lib().mtmc_ref_e8m0(int(byte) & 0xFF))
+
+
+def _scales(a, shape) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    if a.dtype != np.uint8 or tuple(a.shape) != tuple(shape):
+        raise TypeError("block scales must be a uint8 array of shape %r" % (shape,))
+    return a
+
+
+def fused_linear_mxfp8(X, SX, W, SW, b, act_kind: int) -> np.ndarray:
+    """act(z + b) with block-scaled E4M3 operands: X [M,K], W [N,K] bit patterns, SX [M,K/32], SW [N,K/32] UE8M0 bytes."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    SX, SW = _scales(SX, (M, K // 32)), _scales(SW, (N, K // 32))
+    bk, bp = _bias(b, N)
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_fused_linear_mxfp8(X.ctypes.data, SX.ctypes.data, W.ctypes.data, SW.ctypes.data, bp, M, N, K,
+                                             int(act_kind), out.ctypes.data), "mtmc_ref_fused_linear_mxfp8")
+    return out
+
+
+def swiglu_mxfp8(X, SX, Wg, SG, Wu, SU) -> np.ndarray:
+    M, K = X.shape
+    N = Wg.shape[0]
+    X, Wg, Wu = _fp8(X, (M, K)), _fp8(Wg, (N, K)), _fp8(Wu, (N, K))
+    SX, SG, SU = _scales(SX, (M, K // 32)), _scales(SG, (N, K // 32)), _scales(SU, (N, K // 32))
+    out = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_swiglu_mxfp8(X.ctypes.data, SX.ctypes.data, Wg.ctypes.data, SG.ctypes.data, Wu.ctypes.data, SU.ctypes.data,
+                                       M, N, K, out.ctypes.data), "mtmc_ref_swiglu_mxfp8")
+    return out
+
+
+def linear_lse_mxfp8(X, SX, W, SW, b) -> np.ndarray:
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    SX, SW = _scales(SX, (M, K // 32)), _scales(SW, (N, K // 32))
+    bk, bp = _bias(b, N)
+    lse = np.empty(M, dtype=np.float64)
+    _check(lib().mtmc_ref_linear_lse_mxfp8(X.ctypes.data, SX.ctypes.data, W.ctypes.data, SW.ctypes.data, bp, M, N, K, lse.ctypes.data),
+           "mtmc_ref_linear_lse_mxfp8")
+    return lse
 
 
 def fused_linear_fp8_points(X, W, b, scale_x: float, scale_w: float, act_kind: int, rows, cols) -> np.ndarray:

@@ -120,6 +120,46 @@ def fp8_swiglu_inputs(M: int, N: int, K: int, seed: int):
     return out[0][0], out[1][0], out[2][0], out[0][1], out[1][1], out[2][1]
 
 
+def mx_quantize(t: torch.Tensor):
+    """Block-scaled E4M3 (MXFP8) quantisation of a 2-D fp32/bf16 tensor [R, K], K % 32 == 0: per row and block of
+    32 consecutive columns a shared power-of-two scale 2^e with e = floor(log2(max |block|)) - 8 (8 = the exponent
+    of the largest E4M3 binade, as in the OCP microscaling recipe; an all-zero block takes e = 0), elements
+    rounded to E4M3 after division by the scale (saturating at 448).  Returns (float8_e4m3fn [R,K], uint8
+    scales [R,K/32] holding e + 127)."""
+    R, K = t.shape
+    assert K % 32 == 0
+    blocks = t.float().reshape(R, K // 32, 32)
+    amax = blocks.abs().amax(dim=-1)
+    e = torch.where(amax > 0, torch.floor(torch.log2(amax.clamp_min(1e-38))) - 8.0, torch.zeros_like(amax)).clamp(-127.0, 127.0)
+    scaled = (blocks / torch.exp2(e).unsqueeze(-1)).clamp(-448.0, 448.0)
+    return scaled.reshape(R, K).to(torch.float8_e4m3fn), (e + 127.0).to(torch.uint8)
+
+
+@dataclass
+class MxLinearInputs:
+    X: torch.Tensor            # [M, K] float8_e4m3fn, CPU
+    SX: torch.Tensor           # [M, K/32] uint8 (UE8M0), CPU
+    W: torch.Tensor            # [N, K] float8_e4m3fn
+    SW: torch.Tensor           # [N, K/32] uint8
+    b: torch.Tensor | None     # [N] fp32
+
+
+def mx_linear_inputs(M: int, N: int, K: int, seed: int, bias: bool = True, spread: float = 0.0) -> MxLinearInputs:
+    """The bf16 recipe's draws quantised to MXFP8.  spread > 0 multiplies every 32-block of X and of W by its own
+    seeded power of two in [2^-spread, 2^spread] first, so that neighbouring blocks carry very different scales."""
+    li = linear_inputs(M, N, K, seed, bias)
+    X, W = li.X.float(), li.W.float()
+    if spread > 0:
+        g = _gen(seed + 77)
+        ex = torch.randint(-int(spread), int(spread) + 1, (M, K // 32), generator=g).float()
+        ew = torch.randint(-int(spread), int(spread) + 1, (N, K // 32), generator=g).float()
+        X = (X.reshape(M, K // 32, 32) * torch.exp2(ex).unsqueeze(-1)).reshape(M, K)
+        W = (W.reshape(N, K // 32, 32) * torch.exp2(ew).unsqueeze(-1)).reshape(N, K)
+    X8, SX = mx_quantize(X)
+    W8, SW = mx_quantize(W)
+    return MxLinearInputs(X8, SX, W8, SW, li.b)
+
+
 def fp8_bits(t: torch.Tensor) -> np.ndarray:
     """float8_e4m3fn tensor (CPU) -> uint8 numpy array of the raw bit patterns."""
     assert t.dtype == torch.float8_e4m3fn

@@ -282,6 +282,84 @@ def _closed_forms():
     return rows
 
 
+def test_e8m0_decode_every_code():
+    # the scale byte is a biased exponent: 127 = 1, 0 = 2^-127, 254 = 2^127, 255 = NaN
+    assert ref.e8m0(127) == 1.0 and ref.e8m0(128) == 2.0 and ref.e8m0(126) == 0.5
+    assert ref.e8m0(0) == 2.0 ** -127 and ref.e8m0(254) == 2.0 ** 127 and math.isnan(ref.e8m0(255))
+    for e in range(255):
+        assert ref.e8m0(e) == math.ldexp(1.0, e - 127), e
+        if e:
+            assert ref.e8m0(e) == 2.0 * ref.e8m0(e - 1)
+
+
+def _mx_dequant(X8, SX):
+    """fp64 torch tensor of the block-scaled values (every element times its block's power of two)."""
+    scale = torch.exp2(SX.to(torch.float64) - 127.0).repeat_interleave(32, dim=1)
+    return X8.to(torch.float64) * scale
+
+
+def test_mxfp8_linear_pins():
+    mi = inputs.mx_linear_inputs(6, 11, 128, seed=81, spread=5)          # neighbouring blocks with very different scales
+    X8, W8, b = inputs.fp8_bits(mi.X), inputs.fp8_bits(mi.W), inputs.f32(mi.b)
+    SX, SW = mi.SX.numpy(), mi.SW.numpy()
+    assert len(np.unique(SX)) > 4 and len(np.unique(SW)) > 4
+    got = ref.fused_linear_mxfp8(X8, SX, W8, SW, b, ref.ACT_NONE)
+    # library pin: dequantise in torch fp64, then a plain matmul
+    want = _mx_dequant(mi.X, mi.SX) @ _mx_dequant(mi.W, mi.SW).T + mi.b.double()
+    np.testing.assert_allclose(got, want.numpy(), rtol=1e-13, atol=1e-13)
+    # exact brute force with rationals: element = integer / 512, scale = 2^(byte - 127)
+    raw = ref.fused_linear_mxfp8(X8, SX, W8, SW, None, ref.ACT_NONE)
+    xi = (mi.X.to(torch.float64) * 512).numpy().astype(np.int64)
+    wi = (mi.W.to(torch.float64) * 512).numpy().astype(np.int64)
+    for m in range(3):
+        for n in range(4):
+            acc = Fraction(0)
+            for k in range(128):
+                acc += Fraction(int(xi[m, k]), 512) * Fraction(2) ** (int(SX[m, k // 32]) - 127) * \
+                       Fraction(int(wi[n, k]), 512) * Fraction(2) ** (int(SW[n, k // 32]) - 127)
+            assert abs(raw[m, n] - float(acc)) <= 1e-13 * max(1.0, abs(float(acc)))
+    # equal block scales reduce to the per-tensor form, bit for bit (powers of two are exact per-tensor scales)
+    SXc, SWc = np.full_like(SX, 121), np.full_like(SW, 130)
+    same = ref.fused_linear_mxfp8(X8, SXc, W8, SWc, b, ref.ACT_SILU)
+    per_tensor = ref.fused_linear_fp8(X8, W8, b, 2.0 ** (121 - 127), 2.0 ** (130 - 127), ref.ACT_SILU)
+    assert np.array_equal(same, per_tensor)
+    # one more on every X scale doubles z; the contribution of a block depends on its own scales only
+    doubled = ref.fused_linear_mxfp8(X8, SX + 1, W8, SW, None, ref.ACT_NONE)
+    np.testing.assert_allclose(doubled, 2.0 * raw, rtol=1e-15, atol=0)
+    parts = np.zeros_like(raw)
+    for blk in range(4):
+        ks = slice(32 * blk, 32 * blk + 32)
+        parts += ref.fused_linear_mxfp8(np.ascontiguousarray(X8[:, ks]), np.ascontiguousarray(SX[:, blk:blk + 1]),
+                                        np.ascontiguousarray(W8[:, ks]), np.ascontiguousarray(SW[:, blk:blk + 1]), None, ref.ACT_NONE)
+    np.testing.assert_allclose(parts, raw, rtol=1e-13, atol=1e-13)
+    # swapping the scales of two blocks of one row changes that row only, and not into the same value
+    SX2 = SX.copy()
+    SX2[0, 0], SX2[0, 1] = SX[0, 1] + 3, SX[0, 0]
+    swapped = ref.fused_linear_mxfp8(X8, SX2, W8, SW, None, ref.ACT_NONE)
+    assert np.array_equal(swapped[1:], raw[1:]) and not np.allclose(swapped[0], raw[0])
+
+
+def test_mxfp8_swiglu_and_lse_pins():
+    mi = inputs.mx_linear_inputs(5, 9, 96, seed=82, spread=4)
+    up = inputs.mx_linear_inputs(5, 9, 96, seed=83, spread=4)
+    X8, SX = inputs.fp8_bits(mi.X), mi.SX.numpy()
+    G8, SG, U8, SU = inputs.fp8_bits(mi.W), mi.SW.numpy(), inputs.fp8_bits(up.W), up.SW.numpy()
+    got = ref.swiglu_mxfp8(X8, SX, G8, SG, U8, SU)
+    g = ref.fused_linear_mxfp8(X8, SX, G8, SG, None, ref.ACT_SILU)          # product of the two pinned layers
+    u = ref.fused_linear_mxfp8(X8, SX, U8, SU, None, ref.ACT_NONE)
+    np.testing.assert_allclose(got, g * u, rtol=1e-14, atol=0)
+    xd = _mx_dequant(mi.X, mi.SX)
+    want = torch.nn.functional.silu(xd @ _mx_dequant(mi.W, mi.SW).T) * (xd @ _mx_dequant(up.W, up.SW).T)
+    np.testing.assert_allclose(got, want.numpy(), rtol=1e-12, atol=1e-13)
+    assert np.all(ref.swiglu_mxfp8(X8, SX, np.zeros_like(G8), SG, U8, SU) == 0)
+    b = inputs.f32(mi.b)
+    lse = ref.linear_lse_mxfp8(X8, SX, G8, SG, b)
+    z = xd @ _mx_dequant(mi.W, mi.SW).T + mi.b.double()
+    np.testing.assert_allclose(lse, torch.logsumexp(z, dim=-1).numpy(), rtol=1e-13, atol=1e-13)
+    shifted = ref.linear_lse_mxfp8(X8, SX, G8, SG, b + np.float32(2.0))
+    np.testing.assert_allclose(shifted - lse, 2.0, rtol=0, atol=1e-6)       # b + 2 is rounded to fp32 before it is used
+
+
 def test_activation_closed_forms():
     ids = {"relu": ref.ACT_RELU, "gelu_tanh": ref.ACT_GELU_TANH, "silu": ref.ACT_SILU}
     seen = 0
