@@ -71,6 +71,9 @@ extern "C" {
 #define MTMC_OP_LINEAR_LSE 2
 #define MTMC_OP_LINEAR_ROWMAX 3
 #define MTMC_OP_LINEAR_CROSS_ENTROPY 4
+#define MTMC_OP_FUSED_LINEAR_MXFP8 5
+#define MTMC_OP_SWIGLU_MXFP8 6
+#define MTMC_OP_LINEAR_LSE_MXFP8 7
 
 /* out[m][n] = act( sum_k X[m][k] W[n][k] + b[n] ).
  * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
@@ -147,6 +150,26 @@ int mtmc_linear_rowmax_fp8(const void* X8, const void* W8, const float* b, float
                            int64_t M, int64_t N, int64_t K, float* max_out, int32_t* argmax_out);
 int mtmc_linear_cross_entropy_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
                                   const int64_t* targets, int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out);
+
+/* Block-scaled 8-bit operands (the MXFP8 format of the OCP microscaling specification): E4M3 elements with one
+ * power-of-two scale per 32 consecutive elements of K.  X8 [M,K] and W8 [N,K] hold the elements (one byte each,
+ * dense row-major); SX [M, K/32] and SW [N, K/32] hold the scales, one byte each, dense row-major, in UE8M0
+ * (a biased exponent: the scale is 2^(byte - 127); 255 is not a number and out of contract):
+ *   z[m][n] = sum_k ( 2^(SX[m][k/32] - 127) X8[m][k] ) ( 2^(SW[n][k/32] - 127) W8[n][k] )
+ *   mtmc_fused_linear_mxfp8 : out = act(z + b), fp32 or bf16
+ *   mtmc_swiglu_mxfp8       : out = silu(z_gate) * z_up, bf16; gate and up weights with their own scales
+ *   mtmc_linear_lse_mxfp8   : lse_out[m] = log sum_n exp(z[m][n] + b[n]), fp32
+ * The scales differ from k-block to k-block, so they are applied inside the contraction, by the tensor cores
+ * (tcgen05.mma kind::mxf8f6f4.block_scale with the scales in tensor memory); accumulation is fp32 and the
+ * epilogues are those of the bf16 forms.  K % 32 == 0.  All shapes run on single-CTA tiles of 128 x 128.
+ * Workspace: the scales re-arranged for the kernel, mtmc_workspace_bytes(MTMC_OP_..._MXFP8, M, N, K).
+ * The paper's operators are bf16/fp16/fp32; these are the block-scaled low-precision forms of the same fused epilogues. */
+int mtmc_fused_linear_mxfp8(const void* X8, const void* SX, const void* W8, const void* SW, const float* b,
+                            int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);
+int mtmc_swiglu_mxfp8(const void* X8, const void* SX, const void* Wg8, const void* SG, const void* Wu8, const void* SU,
+                      int64_t M, int64_t N, int64_t K, void* out);
+int mtmc_linear_lse_mxfp8(const void* X8, const void* SX, const void* W8, const void* SW, const float* b,
+                          int64_t M, int64_t N, int64_t K, float* lse_out);
 
 /* out[m][n] = silu(sum_k X[m][k] Wg[n][k]) * (sum_k X[m][k] Wu[n][k]);  no bias;
  * out bf16 [M,N].  (Gated MLP up-projection: two GEMMs sharing X plus the gate

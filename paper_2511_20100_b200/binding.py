@@ -21,7 +21,8 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_WORKSPACE, ERR_DEVICE_CHECK = 1, 2, 3, 4, 5, 6, 7
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}
 OUT_DTYPE = {"fp32": 0, "bf16": 1}
-OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4}
+OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4,
+      "fused_linear_mxfp8": 5, "swiglu_mxfp8": 6, "linear_lse_mxfp8": 7}
 
 EXPORTS = [
     "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_fused_linear_fp8", "mtmc_swiglu", "mtmc_linear_lse",
@@ -30,6 +31,7 @@ EXPORTS = [
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
     "mtmc_last_error", "mtmc_launch_count", "mtmc_device_alloc_count", "mtmc_last_kernel_name", "mtmc_set_timing", "mtmc_last_kernel_ms",
+    "mtmc_fused_linear_mxfp8", "mtmc_swiglu_mxfp8", "mtmc_linear_lse_mxfp8",
     "mtmc_fused_linear_strided", "mtmc_swiglu_strided", "mtmc_linear_lse_strided", "mtmc_linear_rowmax_strided",
     "mtmc_linear_cross_entropy_strided", "mtmc_swiglu_fp8", "mtmc_linear_lse_fp8", "mtmc_linear_rowmax_fp8", "mtmc_linear_cross_entropy_fp8", "mtmc_set_tuning", "mtmc_set_schedule", "mtmc_trace_enabled", "mtmc_set_trace", "mtmc_set_static_weights", "mtmc_version", "mtmc_selftest_timeout",
 ]
@@ -63,6 +65,9 @@ def load() -> ctypes.CDLL:
     L.mtmc_fused_linear_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_residual.argtypes = [vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
     L.mtmc_fused_linear_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, ci, vp, i64]
+    L.mtmc_fused_linear_mxfp8.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, ci, ci, vp]
+    L.mtmc_swiglu_mxfp8.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp]
+    L.mtmc_linear_lse_mxfp8.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_swiglu_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, vp, i64]
     L.mtmc_linear_lse_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, vp]
     L.mtmc_linear_rowmax_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, vp, vp]
@@ -171,6 +176,50 @@ def mtmc_fused_linear_strided(X, W, b, act="none", out_dtype="bf16", out=None):
     _check(load().mtmc_fused_linear_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"),
                                             M, N, K, ACT[act], OUT_DTYPE[out_dtype], op, ldo))
     return out
+
+
+def mtmc_fused_linear_mxfp8(X8, SX, W8, SW, b, act="none", out_dtype="bf16", out=None):
+    """out = act(z + b) with block-scaled operands: X8 [M,K], W8 [N,K] float8_e4m3fn; SX [M,K/32], SW [N,K/32] uint8 (UE8M0)."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if out is None:
+        out = torch.empty((M, N), dtype=odt, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_fused_linear_mxfp8(_dev(X8, f8, (M, K), "X8"), _dev(SX, torch.uint8, (M, K // 32), "SX"),
+                                          _dev(W8, f8, (N, K), "W8"), _dev(SW, torch.uint8, (N, K // 32), "SW"),
+                                          None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                          M, N, K, ACT[act], OUT_DTYPE[out_dtype], _dev(out, odt, (M, N), "out")))
+    return out
+
+
+def mtmc_swiglu_mxfp8(X8, SX, Wg8, SG, Wu8, SU, out=None):
+    """out = silu(z_gate) * z_up with block-scaled float8_e4m3fn operands and UE8M0 scales, bf16 [M,N]."""
+    M, K = X8.shape
+    N = Wg8.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.bfloat16, device=X8.device)
+    _use_current_stream(X8.device)
+    f8, u8 = torch.float8_e4m3fn, torch.uint8
+    _check(load().mtmc_swiglu_mxfp8(_dev(X8, f8, (M, K), "X8"), _dev(SX, u8, (M, K // 32), "SX"), _dev(Wg8, f8, (N, K), "Wg8"),
+                                    _dev(SG, u8, (N, K // 32), "SG"), _dev(Wu8, f8, (N, K), "Wu8"), _dev(SU, u8, (N, K // 32), "SU"),
+                                    M, N, K, _dev(out, torch.bfloat16, (M, N), "out")))
+    return out
+
+
+def mtmc_linear_lse_mxfp8(X8, SX, W8, SW, b, lse_out=None):
+    """lse_out[m] = logsumexp_n(z[m] + b) with block-scaled float8_e4m3fn operands and UE8M0 scales, fp32 [M]."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    if lse_out is None:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    _use_current_stream(X8.device)
+    f8, u8 = torch.float8_e4m3fn, torch.uint8
+    _check(load().mtmc_linear_lse_mxfp8(_dev(X8, f8, (M, K), "X8"), _dev(SX, u8, (M, K // 32), "SX"), _dev(W8, f8, (N, K), "W8"),
+                                        _dev(SW, u8, (N, K // 32), "SW"), None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                        M, N, K, _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return lse_out
 
 
 def mtmc_swiglu_strided(X, Wg, Wu, out=None):

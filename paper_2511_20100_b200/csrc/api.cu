@@ -19,6 +19,7 @@
 #include "gemm_ksplit.cuh"
 #include "gemm_big.cuh"
 #include "skinny.cuh"
+#include "gemm_mx.cuh"
 
 namespace {
 
@@ -1144,6 +1145,92 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
     });
 }
 
+// ---------------------------------------------------------------------------- block-scaled E4M3 (MXFP8)
+struct MxPlan { size_t sfa_bytes, sfb_bytes; };
+MxPlan plan_mx(int64_t M, int64_t N, int64_t K, int out_tile_n) {
+    const size_t stages = static_cast<size_t>((K + 127) / 128);
+    return MxPlan{round256(stages * static_cast<size_t>((M + 127) / 128) * 512), round256(stages * static_cast<size_t>((N + out_tile_n - 1) / out_tile_n) * 512)};
+}
+
+int check_mx(const void* X8, const void* SX, const void* W8, const void* SW, const void* out, int64_t M, int64_t N, int64_t K) {
+    if (!X8 || !SX || !W8 || !SW || !out) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (M <= 0 || N <= 0 || K <= 0) return fail(MTMC_ERR_INVALID_ARG, "M, N, K must be positive");
+    if (M >= (1ll << 31) || N >= (1ll << 31) || K >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "dimensions must be below 2^31");
+    if (K % 32 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 32, the scale block of the MX formats", (long long)K);
+    if (!aligned16(X8) || !aligned16(W8) || !aligned16(out)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    return MTMC_OK;
+}
+
+template <int EPI, bool OUT_BF16>
+int launch_mx(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const uint8_t* sfa,
+              const uint8_t* sfb, const GemmParams& p) {
+    using Cfg = MxCfg<EPI>;
+    auto kern = gemm_mx_kernel<EPI, OUT_BF16>;
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
+    const int grid = p.num_tiles < d->sm_count ? p.num_tiles : d->sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid), 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[1];
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_attribute(attr);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, sfa, sfb, p));
+    g_launches.fetch_add(1);
+    note_kernel("gemm_mx_kernel", EPI);
+    return MTMC_OK;
+}
+
+// Scales into the kernel's block layout (two small launches), then the tiled kernel.  EPI_ACT: out / act / out_dtype;
+// EPI_SWIGLU: W = gate, W2 = up with their scales; EPI_LSE: lse_out.
+template <int EPI>
+int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const void* W28, const void* SW2, const float* b,
+           int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out, float* lse_out) {
+    DeviceState* d = nullptr;
+    int rc = get_device(&d);
+    if (rc) return rc;
+    constexpr int OUT_TILE_N = MxCfg<EPI>::OUT_TILE_N;
+    GemmParams p{};
+    fill_tiling(p, M, N, K, OUT_TILE_N, d->sm_count, false, 128, true);
+    p.fp8 = 0;                         // the epilogues see plain fp32 accumulators: the scales are applied inside the MMAs
+    const MxPlan mp = plan_mx(M, N, K, OUT_TILE_N);
+    const size_t lse_bytes = EPI == EPI_LSE ? lse_partial_bytes(p) : 0;
+    void* ws = nullptr;
+    if ((rc = get_workspace(d, mp.sfa_bytes + mp.sfb_bytes + lse_bytes, &ws))) return rc;
+    uint8_t* sfa = static_cast<uint8_t*>(ws);
+    uint8_t* sfb = sfa + mp.sfa_bytes;
+    p.act = act; p.bias = b; p.out = out; p.status = d->status;
+    p.lse_partial = EPI == EPI_LSE ? reinterpret_cast<float2*>(sfb + mp.sfb_bytes) : nullptr;
+    CUtensorMap tmA, tmB, tmB2;
+    if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, OUT_TILE_N)) ||
+        (rc = encode_u8_2d(&tmB2, EPI == EPI_SWIGLU ? W28 : W8, N, K, OUT_TILE_N)))
+        return rc;
+    const int kb32 = static_cast<int>(K / 32);
+    TimedRegion tr(d);
+    {
+        const long long total_a = static_cast<long long>(p.k_blocks) * p.m_tiles * 512, total_b = static_cast<long long>(p.k_blocks) * p.n_tiles * 512;
+        const unsigned ga = static_cast<unsigned>(std::min<long long>((total_a + 255) / 256, 4096)), gb = static_cast<unsigned>(std::min<long long>((total_b + 255) / 256, 4096));
+        mx_retile_scales_kernel<<<ga, 256, 0, t_stream>>>(static_cast<const uint8_t*>(SX), nullptr, static_cast<int>(M), kb32, p.m_tiles, p.k_blocks, 128, sfa);
+        mx_retile_scales_kernel<<<gb, 256, 0, t_stream>>>(static_cast<const uint8_t*>(SW), EPI == EPI_SWIGLU ? static_cast<const uint8_t*>(SW2) : nullptr,
+                                                          static_cast<int>(N), kb32, p.n_tiles, p.k_blocks, EPI == EPI_SWIGLU ? 64 : 128, sfb);
+        CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(2);
+    }
+    if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx<EPI_ACT, true>(d, tmA, tmB, tmB2, sfa, sfb, p) : launch_mx<EPI_ACT, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
+    else if (EPI == EPI_SWIGLU) rc = launch_mx<EPI_SWIGLU, true>(d, tmA, tmB, tmB2, sfa, sfb, p);
+    else rc = launch_mx<EPI_LSE, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
+    tr.stop();
+    if (rc) return rc;
+    if (EPI == EPI_LSE) {
+        lse_merge_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
+                                                                                  p.n_full, p.tail_split, lse_out, nullptr, nullptr);
+        CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    return MTMC_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1215,7 +1302,12 @@ const char* mtmc_last_kernel_name(void) { return t_last_kernel; }
 
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
-    if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_CROSS_ENTROPY) return static_cast<size_t>(-1);
+    if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_LSE_MXFP8) return static_cast<size_t>(-1);
+    if (op >= MTMC_OP_FUSED_LINEAR_MXFP8) {      // the re-arranged scales (+ the logsumexp partials of 128-column tiles)
+        const MxPlan mp = plan_mx(M, N, K, op == MTMC_OP_SWIGLU_MXFP8 ? 64 : 128);
+        const size_t lse = op == MTMC_OP_LINEAR_LSE_MXFP8 ? round256(static_cast<size_t>((N + 127) / 128) * EPI_HALVES * static_cast<size_t>(M) * sizeof(float2)) : 0;
+        return mp.sfa_bytes + mp.sfb_bytes + lse;
+    }
     DeviceState* d = nullptr;
     if (get_device(&d) != MTMC_OK) return static_cast<size_t>(-1);
     // An upper bound over the kernels the library may pick for the shape under the current tuning: the stream-K
@@ -1363,6 +1455,33 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
                  : launch_tiled<EPI_ACT, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
     tr.stop();
     return rc;
+}
+
+int mtmc_fused_linear_mxfp8(const void* X8, const void* SX, const void* W8, const void* SW, const float* b, int64_t M, int64_t N, int64_t K,
+                            int act, int out_dtype, void* out) {
+    int rc = check_mx(X8, SX, W8, SW, out, M, N, K);
+    if (rc) return rc;
+    if (act < 0 || act > 3) return fail(MTMC_ERR_INVALID_ARG, "unknown activation id %d", act);
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    return run_mx<EPI_ACT>(X8, SX, W8, SW, nullptr, nullptr, b, M, N, K, act, out_dtype, out, nullptr);
+}
+
+int mtmc_swiglu_mxfp8(const void* X8, const void* SX, const void* Wg8, const void* SG, const void* Wu8, const void* SU, int64_t M, int64_t N,
+                      int64_t K, void* out) {
+    int rc = check_mx(X8, SX, Wg8, SG, out, M, N, K);
+    if (rc) return rc;
+    if (!Wu8 || !SU) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
+    if (!aligned16(Wu8)) return fail(MTMC_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+    return run_mx<EPI_SWIGLU>(X8, SX, Wg8, SG, Wu8, SU, nullptr, M, N, K, ACT_NONE, MTMC_OUT_BF16, out, nullptr);
+}
+
+int mtmc_linear_lse_mxfp8(const void* X8, const void* SX, const void* W8, const void* SW, const float* b, int64_t M, int64_t N, int64_t K,
+                          float* lse_out) {
+    int rc = check_mx(X8, SX, W8, SW, lse_out, M, N, K);
+    if (rc) return rc;
+    if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
+    return run_mx<EPI_LSE>(X8, SX, W8, SW, nullptr, nullptr, b, M, N, K, ACT_NONE, MTMC_OUT_FP32, nullptr, lse_out);
 }
 
 int mtmc_swiglu(const void* X, const void* Wg, const void* Wu, int64_t M, int64_t N, int64_t K, void* out) {

@@ -347,6 +347,97 @@ def test_linear_rowmax_and_cross_entropy_fp8(M, N, K):
     _assert_close(inputs.to_f64(lse), want_lse, TOL["fp32"], "fp8 lse of cross entropy")
 
 
+# ------------------------------------------------------------------ block-scaled E4M3 (MXFP8)
+def _mx_dev(mi):
+    return mi.X.cuda(), mi.SX.cuda(), mi.W.cuda(), mi.SW.cuda(), None if mi.b is None else mi.b.cuda()
+
+
+def _mx_np(mi):
+    return inputs.fp8_bits(mi.X), mi.SX.numpy(), inputs.fp8_bits(mi.W), mi.SW.numpy(), inputs.f32(mi.b)
+
+
+@pytest.mark.parametrize("vary", ["none", "x_rows", "w_rows", "x_kblocks", "w_kblocks", "all"])
+def test_mxfp8_scale_placement_exact(vary):
+    """Integer-valued elements and power-of-two scales: every product and fp32 partial sum is exact, so the result
+    must equal the oracle bit for bit.  Each case lets the scales vary along one axis only (rows of X, rows of W,
+    k-blocks of X, k-blocks of W), so that a scale read from the wrong row, quadrant or k-block fails its own case."""
+    M, N, K = 256, 384, 512
+    g = torch.Generator().manual_seed(60)
+    X = torch.randint(-2, 3, (M, K), generator=g).float().to(torch.float8_e4m3fn)
+    W = torch.randint(-2, 3, (N, K), generator=g).float().to(torch.float8_e4m3fn)
+    SX = torch.full((M, K // 32), 127, dtype=torch.uint8)
+    SW = torch.full((N, K // 32), 127, dtype=torch.uint8)
+    if vary in ("x_rows", "all"):
+        SX += (torch.arange(M) % 7).to(torch.uint8)[:, None]
+    if vary in ("w_rows", "all"):
+        SW += (torch.arange(N) % 5).to(torch.uint8)[:, None]
+    if vary in ("x_kblocks", "all"):
+        SX -= (torch.arange(K // 32) % 6).to(torch.uint8)[None, :]
+    if vary in ("w_kblocks", "all"):
+        SW -= (torch.arange(K // 32) % 4).to(torch.uint8)[None, :]
+    out = B.mtmc_fused_linear_mxfp8(X.cuda(), SX.cuda(), W.cuda(), SW.cuda(), None, "none", "fp32")
+    B.mtmc_check_status()
+    assert "gemm_mx_kernel" in B.mtmc_last_kernel_name()
+    want = ref.fused_linear_mxfp8(inputs.fp8_bits(X), SX.numpy(), inputs.fp8_bits(W), SW.numpy(), None, ref.ACT_NONE)
+    got = inputs.to_f64(out)
+    bad = np.argwhere(got != want)
+    assert len(bad) == 0, "%s: %d mismatches, first at %r: got %r want %r" % (vary, len(bad), tuple(bad[0]), got[tuple(bad[0])], want[tuple(bad[0])])
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 32), (17, 8, 128), (100, 72, 160), (129, 257, 288), (300, 520, 416), (600, 1000, 672),
+                                   (1024, 2048, 1024)])
+@pytest.mark.parametrize("act,odt", [("none", "fp32"), ("gelu_tanh", "bf16"), ("relu", "fp32")])
+def test_fused_linear_mxfp8(M, N, K, act, odt):
+    """Seeded N(0,1) draws with block magnitudes spread over 2^-6 .. 2^6, quantised to MXFP8; ragged M, N and K (K not a
+    multiple of the 128-element ring stage)."""
+    mi = inputs.mx_linear_inputs(M, N, K, seed=7500 + M + N, spread=6)
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    Xd, SXd, Wd, SWd, bd = _mx_dev(mi)
+    B.mtmc_fused_linear_mxfp8(Xd, SXd, Wd, SWd, bd, act, odt, out=out)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    X8, SX, W8, SW, b = _mx_np(mi)
+    _assert_close(inputs.to_f64(out), ref.fused_linear_mxfp8(X8, SX, W8, SW, b, B.ACT[act]), TOL[odt], "mxfp8 %dx%dx%d %s %s" % (M, N, K, act, odt))
+    assert torch.equal(B.mtmc_fused_linear_mxfp8(Xd, SXd, Wd, SWd, bd, act, odt), out)
+
+
+@pytest.mark.parametrize("M,N,K", [(5, 8, 64), (100, 72, 160), (300, 392, 288), (600, 1000, 672)])
+def test_swiglu_and_lse_mxfp8(M, N, K):
+    mi = inputs.mx_linear_inputs(M, N, K, seed=7600 + M + N, spread=4)
+    up = inputs.mx_linear_inputs(M, N, K, seed=7650 + M + N, spread=4)
+    Xd, SXd, Gd, SGd, bd = _mx_dev(mi)
+    buf, out = _guarded((M, N), torch.bfloat16)
+    B.mtmc_swiglu_mxfp8(Xd, SXd, Gd, SGd, up.W.cuda(), up.SW.cuda(), out=out)
+    lse = B.mtmc_linear_lse_mxfp8(Xd, SXd, Gd, SGd, bd)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    X8, SX, G8, SG, b = _mx_np(mi)
+    want = ref.swiglu_mxfp8(X8, SX, G8, SG, inputs.fp8_bits(up.W), up.SW.numpy())
+    _assert_close(inputs.to_f64(out), want, TOL["bf16"], "mxfp8 swiglu %dx%dx%d" % (M, N, K))
+    _assert_close(inputs.to_f64(lse), ref.linear_lse_mxfp8(X8, SX, G8, SG, b), TOL["fp32"], "mxfp8 lse %dx%dx%d" % (M, N, K))
+
+
+def test_mxfp8_with_caller_workspace_and_full_size_sample():
+    """4096^3 in a caller workspace of exactly mtmc_workspace_bytes; the first and last rows against the oracle."""
+    M = N = K = 4096
+    mi = inputs.mx_linear_inputs(M, N, K, seed=1, spread=3)
+    need = B.mtmc_workspace_bytes("fused_linear_mxfp8", M, N, K)
+    guard = torch.full((need + 8192,), 0x5A, dtype=torch.uint8, device="cuda")
+    off = (-guard.data_ptr()) % 256 + 3840
+    B.mtmc_set_workspace(guard[off:off + need])
+    try:
+        out = B.mtmc_fused_linear_mxfp8(*_mx_dev(mi), "gelu_tanh", "bf16")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_workspace(None)
+    assert bool((guard[:off] == 0x5A).all()) and bool((guard[off + need:] == 0x5A).all())
+    rows = np.array([0, 1, 127, 128, 2047, 4095])
+    X8, SX, W8, SW, b = _mx_np(mi)
+    want = ref.fused_linear_mxfp8(np.ascontiguousarray(X8[rows]), np.ascontiguousarray(SX[rows]), W8, SW, b, ref.ACT_GELU_TANH)
+    _assert_close(inputs.to_f64(out[torch.from_numpy(rows).cuda()]), want, TOL["bf16"], "mxfp8 4096^3 sampled rows")
+    assert bool(torch.isfinite(out.float()).all())
+
+
 def test_fused_linear_fp8_exact_small_integers():
     # operands in {-2..2} are exact in E4M3 and every fp32 partial sum is exact: the result must be exact too
     g = torch.Generator().manual_seed(6)
