@@ -55,6 +55,8 @@ def algorithmic_bytes(c) -> float:
         return 2.0 * (M * K + 2 * N * K) + 2.0 * M * N
     if c["op"] == "fused_linear_fp8":
         return 1.0 * (M * K + N * K) + 4.0 * N + 2.0 * M * N
+    if c["op"] == "fused_linear_mxfp8":
+        return (1.0 + 1.0 / 32) * (M * K + N * K) + 4.0 * N + 2.0 * M * N
     if c["op"] in ("linear_lse", "linear_rowmax", "linear_cross_entropy"):
         extra = {"linear_lse": 0.0, "linear_rowmax": 4.0 * M, "linear_cross_entropy": 8.0 * M}[c["op"]]
         return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M + extra
@@ -144,6 +146,11 @@ def make_device_problem(name, device):
         dev = [fi.X.to(device), fi.W.to(device), fi.b.to(device)]
         out = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=device)
         return {"name": name, "cfg": c, "host": [], "dev": dev, "out": out, "scales": (fi.scale_x, fi.scale_w)}
+    if c["op"] == "fused_linear_mxfp8":
+        mi = inputs.mx_linear_inputs(c["M"], c["N"], c["K"], c["seed"], spread=3)
+        dev = [mi.X.to(device), mi.SX.to(device), mi.W.to(device), mi.SW.to(device), mi.b.to(device)]
+        out = torch.empty((c["M"], c["N"]), dtype=torch.bfloat16, device=device)
+        return {"name": name, "cfg": c, "host": [], "dev": dev, "out": out}
     if c["op"] == "swiglu":
         si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
         host = [si.X, si.Wg, si.Wu]
@@ -177,6 +184,8 @@ def call_device(B, pr):
         B.mtmc_fused_linear_residual(d[0], d[1], d[2], d[3], c["act"], c["out_dtype"], out=pr["out"])
     elif c["op"] == "fused_linear_fp8":
         B.mtmc_fused_linear_fp8(d[0], d[1], d[2], pr["scales"][0], pr["scales"][1], c["act"], c["out_dtype"], out=pr["out"])
+    elif c["op"] == "fused_linear_mxfp8":
+        B.mtmc_fused_linear_mxfp8(d[0], d[1], d[2], d[3], d[4], c["act"], c["out_dtype"], out=pr["out"])
     else:
         B.mtmc_fused_linear(d[0], d[1], d[2], c["act"], c["out_dtype"], out=pr["out"])
 
@@ -374,7 +383,7 @@ def run_ours(args, rank, world, local_rank):
             e1.record()
             torch.cuda.synchronize()
             per_cfg_warm[n] = e0.elapsed_time(e1) / reps
-        if not args.no_eager and c["op"] != "fused_linear_fp8":
+        if not args.no_eager and c["op"] not in ("fused_linear_fp8", "fused_linear_mxfp8"):
             # context: the unfused torch sequence (cuBLAS GEMM + elementwise kernels), same rotation
             for v in variants:
                 eager_call(pr, v["dev"])
@@ -413,7 +422,7 @@ def run_ours(args, rank, world, local_rank):
         elif hbm_bound:
             e.update({"gbs": round(gb, 1), "bound": "hbm", "frac": round(gb / peaks["hbm_gbs"], 4), "frac_of_8000": round(gb / 8000.0, 4)})
         else:
-            scale = 2.0 if c["op"] == "fused_linear_fp8" else 1.0        # E4M3: measured bf16 peak x the nominal 2:1 ratio
+            scale = 2.0 if c["op"] in ("fused_linear_fp8", "fused_linear_mxfp8") else 1.0        # E4M3: measured bf16 peak x the nominal 2:1 ratio
             btf = flops(c) / (per_cfg_burst[n] * 1e-3) / 1e12
             e.update({"tflops": round(tf, 1), "bound": "tensor", "burst_ms": round(per_cfg_burst[n], 5),
                       "frac_burst": round(btf / (scale * peaks["tflops_burst"]), 4),
