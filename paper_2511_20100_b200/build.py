@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libmtmcfused.so")
 SOURCES = ["api.cu"]
-HEADERS = ["ptx.cuh", "gemm_tiled.cuh", "gemm_pair.cuh", "gemm_ksplit.cuh", "gemm_big.cuh", "skinny.cuh", "gemm_mx.cuh"]
+HEADERS = ["ptx.cuh", "gemm_tiled.cuh", "gemm_pair.cuh", "gemm_ksplit.cuh", "gemm_big.cuh", "skinny.cuh", "gemm_mx.cuh", "gemm_mx_pair.cuh"]
 
 
 def _nvcc() -> str:

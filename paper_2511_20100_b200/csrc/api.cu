@@ -20,6 +20,7 @@
 #include "gemm_big.cuh"
 #include "skinny.cuh"
 #include "gemm_mx.cuh"
+#include "gemm_mx_pair.cuh"
 
 namespace {
 
@@ -186,7 +187,7 @@ thread_local long long t_tmap_hits = 0, t_tmap_misses = 0;
 // 2-D row-major [rows, cols] tensor of bf16 (box = 64 columns x box_rows rows) or of one-byte E4M3 elements
 // (box = 128 columns x box_rows rows): one 128-byte swizzle row of K per box row either way.
 int encode_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld, bool u8) {
-    const TmapKey key{ptr, rows, cols, ld > 0 ? ld : cols, box_rows, u8 ? 1 : 0};
+    const TmapKey key{ptr, rows, cols, ld > 0 ? ld : cols, box_rows, u8 ? 1 : 0};      // (kind 2: the plain byte maps of encode_bytes_2d)
     uint64_t h = reinterpret_cast<uintptr_t>(ptr) >> 4;
     h = (h ^ static_cast<uint64_t>(rows) * 0x9E3779B97F4A7C15ull ^ static_cast<uint64_t>(key.ld) * 0xC2B2AE3D27D4EB4Full ^
          static_cast<uint64_t>(cols) * 0x165667B19E3779F9ull ^ static_cast<uint64_t>(box_rows * 2 + key.u8)) * 0xD6E8FEB86659FD93ull;
@@ -203,6 +204,17 @@ int encode_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int
                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
     e.valid = true; e.key = key; e.map = *map;
+    return MTMC_OK;
+}
+// Plain (unswizzled) byte tensor of 256-byte rows, box = 256 bytes x box_rows: the re-arranged MXFP8 scale blocks.
+int encode_bytes_2d(CUtensorMap* map, const void* ptr, int64_t rows, int box_rows) {
+    cuuint64_t dims[2] = {256u, static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {256u};
+    cuuint32_t box[2] = {256u, static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = g_encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MTMC_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", static_cast<int>(r));
     return MTMC_OK;
 }
 int encode_bf16_2d(CUtensorMap* map, const void* ptr, int64_t rows, int64_t cols, int box_rows, int64_t ld = 0) {
@@ -447,7 +459,9 @@ int launch_ksplit_ks(int tiles, const CUtensorMap& tmA, const CUtensorMap& tmB, 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, p));
+    GemmParams q = p;
+    q.trace = trace_for(cfg.gridDim.x);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, q));
     g_launches.fetch_add(1);
     note_kernel("gemm_ksplit_kernel", EPI, KS);
     return MTMC_OK;
@@ -1146,10 +1160,27 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 }
 
 // ---------------------------------------------------------------------------- block-scaled E4M3 (MXFP8)
-struct MxPlan { size_t sfa_bytes, sfb_bytes; };
-MxPlan plan_mx(int64_t M, int64_t N, int64_t K, int out_tile_n) {
+struct MxPlan { bool pair; int out_tile_n; int m_blocks, n_blocks, w_atoms, w_rows_per_block; size_t sfa_bytes, sfb_bytes; };
+// Large problems go to CTA pairs with 256 x 224 tiles (not SwiGLU, whose 112-column tile would not be a whole
+// number of epilogue chunks); everything else to single-CTA tiles of 128 x 128 (SwiGLU: 128 x 64).
+MxPlan plan_mx(DeviceState* d, int epi, int64_t M, int64_t N, int64_t K) {
+    MxPlan mp{};
     const size_t stages = static_cast<size_t>((K + 127) / 128);
-    return MxPlan{round256(stages * static_cast<size_t>((M + 127) / 128) * 512), round256(stages * static_cast<size_t>((N + out_tile_n - 1) / out_tile_n) * 512)};
+    mp.pair = epi != EPI_SWIGLU && d != nullptr && t_cta_pair >= 0 && gemm_pairs(d) > 0 && (t_cta_pair > 0 || (M >= 512 && N >= 224));
+    if (mp.pair) {
+        mp.out_tile_n = 224;
+        mp.m_blocks = 2 * static_cast<int>((M + 255) / 256);          // one 128-row block of X scales per CTA of a pair
+        mp.n_blocks = static_cast<int>((N + 223) / 224);
+        mp.w_atoms = 2; mp.w_rows_per_block = 224;
+    } else {
+        mp.out_tile_n = epi == EPI_SWIGLU ? 64 : 128;
+        mp.m_blocks = static_cast<int>((M + 127) / 128);
+        mp.n_blocks = static_cast<int>((N + mp.out_tile_n - 1) / mp.out_tile_n);
+        mp.w_atoms = 1; mp.w_rows_per_block = epi == EPI_SWIGLU ? 64 : 128;
+    }
+    mp.sfa_bytes = round256(stages * mp.m_blocks * 512);
+    mp.sfb_bytes = round256(stages * mp.n_blocks * mp.w_atoms * 512);
+    return mp;
 }
 
 int check_mx(const void* X8, const void* SX, const void* W8, const void* SW, const void* out, int64_t M, int64_t N, int64_t K) {
@@ -1182,7 +1213,32 @@ int launch_mx(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, co
     return MTMC_OK;
 }
 
-// Scales into the kernel's block layout (two small launches), then the tiled kernel.  EPI_ACT: out / act / out_dtype;
+template <int EPI, bool OUT_BF16>
+int launch_mx_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const CUtensorMap& tmSFA,
+                   const CUtensorMap& tmSFB, const GemmParams& p) {
+    using Cfg = MxPairCfg<EPI>;
+    auto kern = gemm_mx_pair_kernel<EPI, OUT_BF16>;
+    if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
+    const int pairs = p.num_tiles < clusters ? p.num_tiles : clusters;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2u * static_cast<unsigned>(pairs), 1, 1);
+    cfg.blockDim = dim3(Cfg::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1 + pdl_attribute(attr + 1);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmSFA, tmSFB, p));
+    g_launches.fetch_add(1);
+    note_kernel("gemm_mx_pair_kernel", EPI);
+    return MTMC_OK;
+}
+
+// Scales into the kernels' block layout (two small launches), then the tiled kernel.  EPI_ACT: out / act / out_dtype;
 // EPI_SWIGLU: W = gate, W2 = up with their scales; EPI_LSE: lse_out.
 template <int EPI>
 int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const void* W28, const void* SW2, const float* b,
@@ -1190,11 +1246,11 @@ int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    constexpr int OUT_TILE_N = MxCfg<EPI>::OUT_TILE_N;
+    const MxPlan mp = plan_mx(d, EPI, M, N, K);
     GemmParams p{};
-    fill_tiling(p, M, N, K, OUT_TILE_N, d->sm_count, false, 128, true);
+    if (mp.pair) fill_tiling(p, M, N, K, mp.out_tile_n, gemm_pairs(d), false, 256, true);
+    else fill_tiling(p, M, N, K, mp.out_tile_n, d->sm_count, false, 128, true);
     p.fp8 = 0;                         // the epilogues see plain fp32 accumulators: the scales are applied inside the MMAs
-    const MxPlan mp = plan_mx(M, N, K, OUT_TILE_N);
     const size_t lse_bytes = EPI == EPI_LSE ? lse_partial_bytes(p) : 0;
     void* ws = nullptr;
     if ((rc = get_workspace(d, mp.sfa_bytes + mp.sfb_bytes + lse_bytes, &ws))) return rc;
@@ -1203,21 +1259,32 @@ int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const
     p.act = act; p.bias = b; p.out = out; p.status = d->status;
     p.lse_partial = EPI == EPI_LSE ? reinterpret_cast<float2*>(sfb + mp.sfb_bytes) : nullptr;
     CUtensorMap tmA, tmB, tmB2;
-    if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, OUT_TILE_N)) ||
-        (rc = encode_u8_2d(&tmB2, EPI == EPI_SWIGLU ? W28 : W8, N, K, OUT_TILE_N)))
+    const int w_box = mp.pair ? 112 : mp.out_tile_n;
+    if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, w_box)) ||
+        (rc = encode_u8_2d(&tmB2, EPI == EPI_SWIGLU ? W28 : W8, N, K, w_box)))
         return rc;
     const int kb32 = static_cast<int>(K / 32);
     TimedRegion tr(d);
     {
-        const long long total_a = static_cast<long long>(p.k_blocks) * p.m_tiles * 512, total_b = static_cast<long long>(p.k_blocks) * p.n_tiles * 512;
+        const long long total_a = static_cast<long long>(p.k_blocks) * mp.m_blocks * 512, total_b = static_cast<long long>(p.k_blocks) * mp.n_blocks * mp.w_atoms * 512;
         const unsigned ga = static_cast<unsigned>(std::min<long long>((total_a + 255) / 256, 4096)), gb = static_cast<unsigned>(std::min<long long>((total_b + 255) / 256, 4096));
-        mx_retile_scales_kernel<<<ga, 256, 0, t_stream>>>(static_cast<const uint8_t*>(SX), nullptr, static_cast<int>(M), kb32, p.m_tiles, p.k_blocks, 128, sfa);
+        mx_retile_scales_kernel<<<ga, 256, 0, t_stream>>>(static_cast<const uint8_t*>(SX), nullptr, static_cast<int>(M), kb32, mp.m_blocks, p.k_blocks, 128, 1, sfa);
         mx_retile_scales_kernel<<<gb, 256, 0, t_stream>>>(static_cast<const uint8_t*>(SW), EPI == EPI_SWIGLU ? static_cast<const uint8_t*>(SW2) : nullptr,
-                                                          static_cast<int>(N), kb32, p.n_tiles, p.k_blocks, EPI == EPI_SWIGLU ? 64 : 128, sfb);
+                                                          static_cast<int>(N), kb32, mp.n_blocks, p.k_blocks, mp.w_rows_per_block, mp.w_atoms, sfb);
         CUDA_TRY(cudaGetLastError());
         g_launches.fetch_add(2);
     }
-    if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx<EPI_ACT, true>(d, tmA, tmB, tmB2, sfa, sfb, p) : launch_mx<EPI_ACT, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
+    if (mp.pair) {
+        if constexpr (EPI != EPI_SWIGLU) {
+            CUtensorMap tmSFA, tmSFB;
+            if ((rc = encode_bytes_2d(&tmSFA, sfa, static_cast<int64_t>(p.k_blocks) * mp.m_blocks * 2, 2)) ||
+                (rc = encode_bytes_2d(&tmSFB, sfb, static_cast<int64_t>(p.k_blocks) * mp.n_blocks * 4, 4)))
+                return rc;
+            if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p)
+                                                               : launch_mx_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
+            else rc = launch_mx_pair<EPI_LSE, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
+        }
+    } else if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx<EPI_ACT, true>(d, tmA, tmB, tmB2, sfa, sfb, p) : launch_mx<EPI_ACT, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
     else if (EPI == EPI_SWIGLU) rc = launch_mx<EPI_SWIGLU, true>(d, tmA, tmB, tmB2, sfa, sfb, p);
     else rc = launch_mx<EPI_LSE, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
     tr.stop();
@@ -1303,8 +1370,10 @@ const char* mtmc_last_kernel_name(void) { return t_last_kernel; }
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
     if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_LSE_MXFP8) return static_cast<size_t>(-1);
-    if (op >= MTMC_OP_FUSED_LINEAR_MXFP8) {      // the re-arranged scales (+ the logsumexp partials of 128-column tiles)
-        const MxPlan mp = plan_mx(M, N, K, op == MTMC_OP_SWIGLU_MXFP8 ? 64 : 128);
+    if (op >= MTMC_OP_FUSED_LINEAR_MXFP8) {      // the re-arranged scales (+ the logsumexp partials of 128-column tiles, the most pieces)
+        DeviceState* dm = nullptr;
+        if (get_device(&dm) != MTMC_OK) return static_cast<size_t>(-1);
+        const MxPlan mp = plan_mx(dm, op == MTMC_OP_SWIGLU_MXFP8 ? EPI_SWIGLU : (op == MTMC_OP_LINEAR_LSE_MXFP8 ? EPI_LSE : EPI_ACT), M, N, K);
         const size_t lse = op == MTMC_OP_LINEAR_LSE_MXFP8 ? round256(static_cast<size_t>((N + 127) / 128) * EPI_HALVES * static_cast<size_t>(M) * sizeof(float2)) : 0;
         return mp.sfa_bytes + mp.sfb_bytes + lse;
     }

@@ -72,8 +72,10 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();
     const int tile = static_cast<int>(blockIdx.x) / KS;
+    const Trace tr(p.trace);
 
     if (threadIdx.x == 0) {
+        tr.stamp(TR_START_NS);
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(accf_bar, 1);
         mbar_init(ready_bar, KS - 1);             // one arrival per peer CTA
@@ -97,6 +99,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
     pdl_launch_dependents();
     pdl_wait();
+    if (threadIdx.x == 0) tr.stamp(TR_SETUP_NS);
 
     int mb, nb;
     tile_coords(p, tile, mb, nb);
@@ -113,7 +116,10 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             constexpr uint32_t b_rows_bytes = static_cast<uint32_t>(Cfg::OUT_TILE_N) * Tile::BK * 2;
             constexpr uint32_t tx = Tile::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes;
             for (int kb = kb0; kb < kb1; ++kb) {
+                const long long tw = tr.now();
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 7u)) break;
+                tr.add(TR_PROD_STALL, tr.now() - tw);
+                tr.stamp_once(TR_PROD_FIRST_NS);
                 const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                 const uint32_t b_dst = a_dst + Tile::A_BYTES;
                 mbar_expect_tx(full_bar(s), tx);
@@ -122,6 +128,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), kb * p.bk_elems, n0);
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
+            tr.stamp(TR_PROD_LAST_NS);
         }
         __syncwarp();
     } else if (warp == 1) {
@@ -132,7 +139,11 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             bool ok = true;
             const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(128, Cfg::BN) : umma_idesc_bf16(128, Cfg::BN);
             for (int kb = kb0; kb < kb1; ++kb) {
+                const long long tw = tr.now();
                 if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 7u)) { ok = false; break; }
+                tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
+                tr.add(TR_MMA_KBLOCKS, 1);
+                tr.stamp_once(TR_MMA_FIRST_NS);
                 tc_fence_after();
                 const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                 const uint64_t a_desc = umma_smem_desc_sw128(a_src);
@@ -150,6 +161,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
             if (ok) umma_commit(accf_bar);           // my part of the sum is complete and my ring is idle
+            tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();
     } else {
@@ -157,12 +169,14 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t t_addr = tmem_base + lane_base;
-        const int sw = lane & 7;                     // the eight 16-byte pieces of a row sit at piece ^ (row & 7)
         const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);
         // Accumulator chunk held at place `loc` of the receive buffer of CTA `owner`: output chunk
         // owner * OWN_OC + loc % OWN_OC of the gate / only half (loc < OWN_OC) or of the up half.
         auto acc_chunk = [&](int owner, int loc) { return (loc / Cfg::OWN_OC) * Cfg::OC + owner * Cfg::OWN_OC + loc % Cfg::OWN_OC; };
+        const bool tracer = warp == 2 && lane == 0;
         bool ok = mbar_wait(accf_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 7u);
+        const long long tb = tr.now();
+        if (tracer) { tr.stamp(TR_EPI_FIRST_NS); tr.add(TR_EPI_ITEMS, 1); }
         if (ok) {
             tc_fence_after();
             // my ring is idle (every MMA that read it has completed): the peers may write their partials into it
@@ -170,26 +184,35 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             ok = mbar_wait_cluster(ready_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 8u);
         }
         if (ok) {
+            // Everything this warp owes its peers goes out first (the TMEM load of the next chunk in flight while one
+            // chunk is stored), then ONE fence orders all of it, then the peers are told: a fence per peer would
+            // cost a round trip through the cluster each.
+            constexpr int SENDS = (KS - 1) * Cfg::OWN_AC;
+            auto chunk_of = [&](int idx) { return acc_chunk((static_cast<int>(rank) + 1 + idx / Cfg::OWN_AC) % KS, idx % Cfg::OWN_AC); };
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_addr + chunk_of(0) * 32, r);
 #pragma unroll 1
-            for (int i = 1; i < KS; ++i) {
-                const int peer = (static_cast<int>(rank) + i) % KS;
+            for (int idx = 0; idx < SENDS; ++idx) {
+                const int peer = (static_cast<int>(rank) + 1 + idx / Cfg::OWN_AC) % KS;
+                const int loc = idx % Cfg::OWN_AC;
                 const int sidx = static_cast<int>(rank) < peer ? static_cast<int>(rank) : static_cast<int>(rank) - 1;   // my place among the peer's senders
-                const uint32_t peer_ring = cluster_map_shared(base, peer);
-#pragma unroll 1
-                for (int loc = 0; loc < Cfg::OWN_AC; ++loc) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(t_addr + acc_chunk(peer, loc) * 32, r);
-                    tmem_ld_wait();
-                    const uint32_t dst = peer_ring + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 128);
+                tmem_ld_wait();
+                float v[32];
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        st_shared_cluster_v4(dst + ((v ^ sw) << 4), __uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                             __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
-                }
-                fence_acq_rel_cluster();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_remote(cluster_map_shared(recv_bar, peer));
+                for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
+                if (idx + 1 < SENDS) tmem_ld_32x32b_x32(t_addr + chunk_of(idx + 1) * 32, r);
+                // the reader is the thread at the same place (quadrant, lane) of the peer, so the layout inside the 4 KiB
+                // block is private to the two: each store instruction of the warp writes 512 contiguous bytes, which
+                // the cluster network moves in a few large packets instead of 32 small ones
+                const uint32_t dst = cluster_map_shared(base, peer) +
+                                     static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 16);
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    st_shared_cluster_v4(dst + g * 512, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
             }
+            fence_acq_rel_cluster();
+            __syncwarp();
+            if (lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(recv_bar, lane));
             ok = mbar_wait_cluster(recv_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 9u);
         }
         if (ok) {
@@ -208,10 +231,10 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                         for (int j = 0; j < 32; ++j) acc[j] = (s == 0) ? __uint_as_float(r[j]) : acc[j] + __uint_as_float(r[j]);
                     } else {
                         const int sidx = s < static_cast<int>(rank) ? s : s - 1;
-                        const uint32_t src = base + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 128);
+                        const uint32_t src = base + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 16);
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
-                            const float4 t = ld_shared_v4(src + ((g ^ sw) << 4));
+                            const float4 t = ld_shared_v4(src + g * 512);
                             acc[4 * g] = (s == 0) ? t.x : acc[4 * g] + t.x;
                             acc[4 * g + 1] = (s == 0) ? t.y : acc[4 * g + 1] + t.y;
                             acc[4 * g + 2] = (s == 0) ? t.z : acc[4 * g + 2] + t.z;
@@ -224,17 +247,20 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 tmem_st_32x32b_x32(t_addr + a * 32, r);
             }
             tmem_st_wait();
+            if (tracer) tr.add(TR_EPI_HANDOVER, tr.now() - tb);        // reduce-scatter through distributed shared memory
             const int row = mb * 128 + q * 32 + lane;
             epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, static_cast<int>(rank) * Cfg::OWN_OC,
                                          (static_cast<int>(rank) + 1) * Cfg::OWN_OC, Cfg::OUT_TILE_N, nb, static_cast<int>(rank), 0, vec_ok,
                                          smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
         }
+        if (tracer) { tr.add(TR_EPI_BUSY, tr.now() - tb); tr.stamp(TR_EPI_END_NS); }
     }
 
     // ---------------------------------------------------------------------- teardown
     // No CTA frees its TMEM or leaves while a peer can still write into its ring or arrive on its barriers.
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) tr.stamp(TR_END_NS);
     cluster_arrive();
     cluster_wait();
     if (*abort_flag != 0u) {

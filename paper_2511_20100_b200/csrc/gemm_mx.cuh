@@ -74,26 +74,31 @@ __device__ __forceinline__ void umma_mxf8(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
-// Re-arranges row-major scales S [rows, kb32] (one byte per row and 32 elements of K) into the blocks the kernel
-// copies: out[(stage * row_blocks + block) * 512 + 16 r0 + 4 r1 + j] = S[first_row(block) + 32 r1 + r0][4 stage + j],
-// with the neutral scale 127 (2^0) outside the matrix.  A block holds `rows_per_half` rows of S (128, or 64 for
-// SwiGLU) in its first half and, if S2 is given, the same rows of S2 in its second half (gate rows, then up rows:
-// the order of the accumulator columns).
+// Re-arranges row-major scales S [rows, kb32] (one byte per row and 32 elements of K) into the blocks the kernels
+// copy.  Output: [stage][block][atom] x 512 bytes, an atom holding 128 rows x 4 k-blocks with row r0 + 32 r1, k-block
+// j at byte 16 r0 + 4 r1 + j; the neutral scale 127 (2^0) wherever the block has no row of S or K has ended.
+//   S2 == null : block b holds rows [b * rows_per_block, (b + 1) * rows_per_block) of S in its first rows_per_block
+//                rows (128 of one atom, or 224 of two atoms for the 224-column tiles of the CTA-pair kernel);
+//   S2 != null : SwiGLU; rows_per_block rows of S (gate) followed by the same rows of S2 (up), the order of the
+//                accumulator columns.
 __global__ void mx_retile_scales_kernel(const uint8_t* __restrict__ S, const uint8_t* __restrict__ S2, int rows, int kb32,
-                                        int row_blocks, int stages, int rows_per_half, uint8_t* __restrict__ out) {
-    const long long total = static_cast<long long>(stages) * row_blocks * 512;
+                                        int blocks, int stages, int rows_per_block, int atoms, uint8_t* __restrict__ out) {
+    const long long total = static_cast<long long>(stages) * blocks * atoms * 512;
     for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total; i += static_cast<long long>(gridDim.x) * blockDim.x) {
         const int within = static_cast<int>(i & 511);
-        const long long blk = i >> 9;
-        const int block = static_cast<int>(blk % row_blocks), stage = static_cast<int>(blk / row_blocks);
+        const long long at = i >> 9;
+        const int atom = static_cast<int>(at % atoms);
+        const long long blk = at / atoms;
+        const int block = static_cast<int>(blk % blocks), stage = static_cast<int>(blk / blocks);
         const int r0 = within >> 4, r1 = (within >> 2) & 3, j = within & 3;
-        const int r = r0 + 32 * r1;                                   // row inside the 128-row block
+        const int r = atom * 128 + r0 + 32 * r1;                      // row inside the block
         const uint8_t* src = S;
         int row;
-        if (S2 != nullptr) { src = r < rows_per_half ? S : S2; row = block * rows_per_half + (r % rows_per_half); }
-        else row = block * 128 + r;
+        bool valid;
+        if (S2 != nullptr) { src = r < rows_per_block ? S : S2; valid = r < 2 * rows_per_block; row = block * rows_per_block + (r % rows_per_block); }
+        else { valid = r < rows_per_block; row = block * rows_per_block + r; }
         const int kb = stage * 4 + j;
-        out[i] = (row < rows && kb < kb32) ? src[static_cast<size_t>(row) * kb32 + kb] : static_cast<uint8_t>(127);
+        out[i] = (valid && row < rows && kb < kb32) ? src[static_cast<size_t>(row) * kb32 + kb] : static_cast<uint8_t>(127);
     }
 }
 

@@ -32,6 +32,20 @@ def test_library_builds_loads_and_exports_every_declared_symbol():
     assert lib.mtmc_version() >= 100
 
 
+def test_debug_build_variants_compile_and_say_what_they_are():
+    """The trace build (-DMTMC_TRACE) and the index-check build (-DMTMC_CHECKS) compile for sm_100a and export the same
+    symbols; only the trace build reports tracing as available."""
+    plain = ctypes.CDLL(build.build())
+    plain.mtmc_trace_enabled.restype = ctypes.c_int
+    assert plain.mtmc_trace_enabled() == 0
+    for variant in ("trace", "checks"):
+        lib = ctypes.CDLL(build.build(variant=variant))
+        for name in declared_symbols():
+            assert hasattr(lib, name), "%s build: missing export %s" % (variant, name)
+        lib.mtmc_trace_enabled.restype = ctypes.c_int
+        assert lib.mtmc_trace_enabled() == (1 if variant == "trace" else 0)
+
+
 def test_binding_covers_the_header():
     assert sorted(binding.EXPORTS) == declared_symbols()
     for name in binding.EXPORTS:

@@ -356,12 +356,13 @@ def _mx_np(mi):
     return inputs.fp8_bits(mi.X), mi.SX.numpy(), inputs.fp8_bits(mi.W), mi.SW.numpy(), inputs.f32(mi.b)
 
 
+@pytest.mark.parametrize("kernel", ["single-CTA tiles", "CTA pairs"])
 @pytest.mark.parametrize("vary", ["none", "x_rows", "w_rows", "x_kblocks", "w_kblocks", "all"])
-def test_mxfp8_scale_placement_exact(vary):
+def test_mxfp8_scale_placement_exact(vary, kernel):
     """Integer-valued elements and power-of-two scales: every product and fp32 partial sum is exact, so the result
     must equal the oracle bit for bit.  Each case lets the scales vary along one axis only (rows of X, rows of W,
     k-blocks of X, k-blocks of W), so that a scale read from the wrong row, quadrant or k-block fails its own case."""
-    M, N, K = 256, 384, 512
+    M, N, K = (256, 384, 512) if kernel == "single-CTA tiles" else (600, 700, 512)     # pairs: 256 x 224 tiles, ragged in M and N
     g = torch.Generator().manual_seed(60)
     X = torch.randint(-2, 3, (M, K), generator=g).float().to(torch.float8_e4m3fn)
     W = torch.randint(-2, 3, (N, K), generator=g).float().to(torch.float8_e4m3fn)
@@ -375,13 +376,18 @@ def test_mxfp8_scale_placement_exact(vary):
         SX -= (torch.arange(K // 32) % 6).to(torch.uint8)[None, :]
     if vary in ("w_kblocks", "all"):
         SW -= (torch.arange(K // 32) % 4).to(torch.uint8)[None, :]
-    out = B.mtmc_fused_linear_mxfp8(X.cuda(), SX.cuda(), W.cuda(), SW.cuda(), None, "none", "fp32")
-    B.mtmc_check_status()
-    assert "gemm_mx_kernel" in B.mtmc_last_kernel_name()
+    B.mtmc_set_tuning(cta_pair=-1 if kernel == "single-CTA tiles" else 1)
+    try:
+        out = B.mtmc_fused_linear_mxfp8(X.cuda(), SX.cuda(), W.cuda(), SW.cuda(), None, "none", "fp32")
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_tuning()
+    assert ("gemm_mx_kernel" if kernel == "single-CTA tiles" else "gemm_mx_pair_kernel") in B.mtmc_last_kernel_name()
     want = ref.fused_linear_mxfp8(inputs.fp8_bits(X), SX.numpy(), inputs.fp8_bits(W), SW.numpy(), None, ref.ACT_NONE)
     got = inputs.to_f64(out)
     bad = np.argwhere(got != want)
-    assert len(bad) == 0, "%s: %d mismatches, first at %r: got %r want %r" % (vary, len(bad), tuple(bad[0]), got[tuple(bad[0])], want[tuple(bad[0])])
+    assert len(bad) == 0, "%s, %s: %d mismatches, first at %r: got %r want %r; mismatching rows %r.., columns %r.." % (
+        vary, kernel, len(bad), tuple(bad[0]), got[tuple(bad[0])], want[tuple(bad[0])], sorted(set(bad[:, 0]))[:8], sorted(set(bad[:, 1]))[:8])
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (17, 8, 128), (100, 72, 160), (129, 257, 288), (300, 520, 416), (600, 1000, 672),
