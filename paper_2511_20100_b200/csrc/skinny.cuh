@@ -63,7 +63,7 @@ struct SkinnyCfg {
     static constexpr int WAYS = MX == 64 ? 4 : 8;         // independent accumulators
     static constexpr int ACC_COLS = WAYS * MX;            // TMEM columns per accumulator set (128 / 256 / 256)
     static constexpr int TMEM_COLS = 2 * ACC_COLS;        // two sets: MMA on one, epilogue on the other
-    static constexpr int NUM_BARRIERS = 2 * MAX_STAGES + 5;   // ring, accumulator sets, pair reduction
+    static constexpr int NUM_BARRIERS = 2 * MAX_STAGES + 6;   // ring, accumulator sets, pair reduction, store staging
     static constexpr int REDUCE_BYTES = MX * LANES * 4;       // the peer CTA's partial (PAIR mode)
     // One CTA per SM with the whole shared memory: splitting an SM between the running kernel and the next
     // launch (two CTAs of 111 KiB, dependents released after the last load) was measured slower, 28.7-29.2 us
@@ -107,17 +107,71 @@ __device__ __forceinline__ int skinny_cta_of_unit(long long u, long long total, 
     return static_cast<int>(((u + 1) * grid - 1) / total);
 }
 
-// out[m][n] = y (+ R[m][n]), rounded once to the output type.
-template <bool OUT_BF16>
-__device__ __forceinline__ void skinny_store(const SkinnyParams& p, int m, int n, float y) {
-    const size_t idx = static_cast<size_t>(m) * p.ldo + n;
-    if (OUT_BF16) {
-        if (p.residual) y += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.residual)[idx]);
-        reinterpret_cast<__nv_bfloat16*>(p.out)[idx] = __float2bfloat16_rn(y);
-    } else {
-        if (p.residual) y += reinterpret_cast<const float*>(p.residual)[idx];
-        reinterpret_cast<float*>(p.out)[idx] = y;
+// Stores of one band.  The accumulator leaves the MMA transposed (a thread owns one output column n and all rows m),
+// so a direct store would write one 2-byte element per thread and instruction.  Instead every thread parks its
+// activated values in shared memory as stage[m][column in band] (fp32), the four epilogue warps meet on a
+// bounded barrier, and then the 128 threads write the band row by row with 128-bit stores (eight bf16 or four
+// fp32 per thread and instruction; the residual, if any, is read the same way and added here).  `stage` is the
+// pair-reduction buffer, free again by now.  Returns false if the wait gave up.
+template <bool OUT_BF16, int MX>
+__device__ __forceinline__ bool skinny_store_band(const SkinnyParams& p, float* stage, uint32_t stage_bar, uint32_t& stage_phase,
+                                                  volatile uint32_t* abort_flag, int nl, int epi_tid, int lane, int n_band0, int band_rows,
+                                                  bool row_ok, const float (&y)[MX]) {
+    if (row_ok) {
+#pragma unroll
+        for (int m = 0; m < MX; ++m) stage[m * 128 + nl] = y[m];
     }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(stage_bar);
+    if (!mbar_wait(stage_bar, stage_phase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 0xFu)) return false;
+    stage_phase ^= 1u;
+    constexpr int VEC = OUT_BF16 ? 8 : 4;                    // elements per 128-bit store
+    constexpr int SEGS = 128 / VEC;
+    const bool vec_ok = p.ldo % VEC == 0;                    // 16-byte aligned rows of out (and of the residual)
+    const int cols = min(band_rows, p.N - n_band0);          // columns of this band inside the output
+    for (int idx = epi_tid; idx < p.M * SEGS; idx += 128) {
+        const int m = idx / SEGS, c0 = (idx - m * SEGS) * VEC;
+        if (c0 >= cols) continue;
+        const float* src = stage + m * 128 + c0;
+        const size_t off = static_cast<size_t>(m) * p.ldo + n_band0 + c0;
+        float v[VEC];
+#pragma unroll
+        for (int j = 0; j < VEC; j += 4) {
+            const float4 t = *reinterpret_cast<const float4*>(src + j);
+            v[j] = t.x; v[j + 1] = t.y; v[j + 2] = t.z; v[j + 3] = t.w;
+        }
+        if (vec_ok && c0 + VEC <= cols) {
+            if (OUT_BF16) {
+                if (p.residual) {
+                    const uint4 r = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(p.residual) + off);
+                    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) { v[2 * h] += __uint_as_float(w[h] << 16); v[2 * h + 1] += __uint_as_float(w[h] & 0xffff0000u); }
+                }
+                uint4 q;
+                q.x = pack_bf16x2(v[0], v[1]); q.y = pack_bf16x2(v[2], v[3]); q.z = pack_bf16x2(v[4 % VEC], v[5 % VEC]); q.w = pack_bf16x2(v[6 % VEC], v[7 % VEC]);
+                *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.out) + off) = q;
+            } else {
+                if (p.residual) {
+                    const float4 r = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p.residual) + off);
+                    v[0] += r.x; v[1] += r.y; v[2] += r.z; v[3] += r.w;
+                }
+                *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.out) + off) = make_float4(v[0], v[1], v[2], v[3]);
+            }
+        } else {
+            for (int j = 0; j < VEC && c0 + j < cols; ++j) {
+                float t = v[j];
+                if (OUT_BF16) {
+                    if (p.residual) t += __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p.residual)[off + j]);
+                    reinterpret_cast<__nv_bfloat16*>(p.out)[off + j] = __float2bfloat16_rn(t);
+                } else {
+                    if (p.residual) t += reinterpret_cast<const float*>(p.residual)[off + j];
+                    reinterpret_cast<float*>(p.out)[off + j] = t;
+                }
+            }
+        }
+    }
+    return true;
 }
 
 // FP8: E4M3 operands (128 per 128-byte row, K = 32 per MMA) instead of bf16 (64 per row, K = 16);
@@ -146,6 +200,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
     auto accf_bar = [&](int b) { return bar_base + 8u * (2 * MAXS + b); };
     auto acce_bar = [&](int b) { return bar_base + 8u * (2 * MAXS + 2 + b); };
     const uint32_t red_bar = bar_base + 8u * (2 * MAXS + 4);
+    const uint32_t stage_bar = bar_base + 8u * (2 * MAXS + 5);             // the four epilogue warps have parked their values
     uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
@@ -234,6 +289,7 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
             for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
             for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); }
             mbar_init(red_bar, 4);
+            mbar_init(stage_bar, 4);
             *abort_flag = 0u;
             *last_flag = 0u;
             fence_barrier_init();
@@ -321,6 +377,8 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
         uint32_t acc_ph = 0;
         int tile = first_tile, kb0 = first_kb, left = n_units, seg_idx = 0;
         bool ok = true;
+        float* stage = reinterpret_cast<float*>(smem_raw + (reduce_base - raw_addr));      // [MX][128] fp32: store staging
+        uint32_t stage_phase = 0;
         if (PAIR) {
             left = 0;                                          // the generic loop below is not used
             const int n = first_tile * R + nl;
@@ -350,12 +408,10 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     const float* peer = reinterpret_cast<const float*>(smem_raw + (reduce_base - raw_addr)) + nl;
 #pragma unroll
                     for (int m = 0; m < MX; ++m) acc[m] += peer[m * Cfg::LANES];       // rank 0 + rank 1
-                    if (row_ok) {
 #pragma unroll
-                        for (int m = 0; m < MX; ++m) {
-                            if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn));
-                        }
-                    }
+                    for (int m = 0; m < MX; ++m) acc[m] = apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn);
+                    // (each thread overwrites, in the same buffer, exactly the elements it has just read)
+                    skinny_store_band<OUT_BF16, MX>(p, stage, stage_bar, stage_phase, abort_flag, nl, epi_tid, lane, first_tile * R, R, row_ok, acc);
                 }
             }
         }
@@ -425,11 +481,15 @@ skinny_splitk_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_const
                     finalize = true;
                 }
             }
-            if (finalize && row_ok) {
+            if (finalize) {                // the same decision in all four epilogue warps
 #pragma unroll
-                for (int m = 0; m < MX; ++m) {
-                    if (m < p.M) skinny_store<OUT_BF16>(p, m, n, apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn));
-                }
+                for (int m = 0; m < MX; ++m) acc[m] = apply_act(p.act, FP8 ? fmaf(acc[m], p.acc_scale, bn) : acc[m] + bn);
+                if (!skinny_store_band<OUT_BF16, MX>(p, stage, stage_bar, stage_phase, abort_flag, nl, epi_tid, lane, tile * R, R, row_ok, acc)) { ok = false; break; }
+                // the next band parks its values in the same buffer: everybody has read this one first
+                __syncwarp();
+                if (lane == 0) mbar_arrive(stage_bar);
+                if (!mbar_wait(stage_bar, stage_phase, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 0xFu)) { ok = false; break; }
+                stage_phase ^= 1u;
             }
             ++tile;
             kb0 = 0;
