@@ -1161,17 +1161,18 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 
 // ---------------------------------------------------------------------------- block-scaled E4M3 (MXFP8)
 struct MxPlan { bool pair; int out_tile_n; int m_blocks, n_blocks, w_atoms, w_rows_per_block; size_t sfa_bytes, sfb_bytes; };
-// Large problems go to CTA pairs with 256 x 224 tiles (not SwiGLU, whose 112-column tile would not be a whole
-// number of epilogue chunks); everything else to single-CTA tiles of 128 x 128 (SwiGLU: 128 x 64).
+// Large problems go to CTA pairs with 256 x 224 tiles (SwiGLU: 256 x 96); everything else to single-CTA tiles of
+// 128 x 128 (SwiGLU: 128 x 64).
 MxPlan plan_mx(DeviceState* d, int epi, int64_t M, int64_t N, int64_t K) {
     MxPlan mp{};
     const size_t stages = static_cast<size_t>((K + 127) / 128);
-    mp.pair = epi != EPI_SWIGLU && d != nullptr && t_cta_pair >= 0 && gemm_pairs(d) > 0 && (t_cta_pair > 0 || (M >= 512 && N >= 224));
+    const int pair_tile_n = epi == EPI_SWIGLU ? 96 : 224;
+    mp.pair = d != nullptr && t_cta_pair >= 0 && gemm_pairs(d) > 0 && (t_cta_pair > 0 || (M >= 512 && N >= pair_tile_n));
     if (mp.pair) {
-        mp.out_tile_n = 224;
+        mp.out_tile_n = pair_tile_n;
         mp.m_blocks = 2 * static_cast<int>((M + 255) / 256);          // one 128-row block of X scales per CTA of a pair
-        mp.n_blocks = static_cast<int>((N + 223) / 224);
-        mp.w_atoms = 2; mp.w_rows_per_block = 224;
+        mp.n_blocks = static_cast<int>((N + pair_tile_n - 1) / pair_tile_n);
+        mp.w_atoms = 2; mp.w_rows_per_block = pair_tile_n;            // SwiGLU: 96 gate rows, then the same 96 up rows
     } else {
         mp.out_tile_n = epi == EPI_SWIGLU ? 64 : 128;
         mp.m_blocks = static_cast<int>((M + 127) / 128);
@@ -1259,7 +1260,7 @@ int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const
     p.act = act; p.bias = b; p.out = out; p.status = d->status;
     p.lse_partial = EPI == EPI_LSE ? reinterpret_cast<float2*>(sfb + mp.sfb_bytes) : nullptr;
     CUtensorMap tmA, tmB, tmB2;
-    const int w_box = mp.pair ? 112 : mp.out_tile_n;
+    const int w_box = mp.pair ? (EPI == EPI_SWIGLU ? 96 : 112) : mp.out_tile_n;
     if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, w_box)) ||
         (rc = encode_u8_2d(&tmB2, EPI == EPI_SWIGLU ? W28 : W8, N, K, w_box)))
         return rc;
@@ -1275,15 +1276,14 @@ int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const
         g_launches.fetch_add(2);
     }
     if (mp.pair) {
-        if constexpr (EPI != EPI_SWIGLU) {
-            CUtensorMap tmSFA, tmSFB;
-            if ((rc = encode_bytes_2d(&tmSFA, sfa, static_cast<int64_t>(p.k_blocks) * mp.m_blocks * 2, 2)) ||
-                (rc = encode_bytes_2d(&tmSFB, sfb, static_cast<int64_t>(p.k_blocks) * mp.n_blocks * 4, 4)))
-                return rc;
-            if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p)
-                                                               : launch_mx_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
-            else rc = launch_mx_pair<EPI_LSE, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
-        }
+        CUtensorMap tmSFA, tmSFB;
+        if ((rc = encode_bytes_2d(&tmSFA, sfa, static_cast<int64_t>(p.k_blocks) * mp.m_blocks * 2, 2)) ||
+            (rc = encode_bytes_2d(&tmSFB, sfb, static_cast<int64_t>(p.k_blocks) * mp.n_blocks * 4, 4)))
+            return rc;
+        if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx_pair<EPI_ACT, true>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p)
+                                                           : launch_mx_pair<EPI_ACT, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
+        else if (EPI == EPI_SWIGLU) rc = launch_mx_pair<EPI_SWIGLU, true>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
+        else rc = launch_mx_pair<EPI_LSE, false>(gemm_pairs(d), tmA, tmB, tmB2, tmSFA, tmSFB, p);
     } else if (EPI == EPI_ACT) rc = out_dtype == MTMC_OUT_BF16 ? launch_mx<EPI_ACT, true>(d, tmA, tmB, tmB2, sfa, sfb, p) : launch_mx<EPI_ACT, false>(d, tmA, tmB, tmB2, sfa, sfb, p);
     else if (EPI == EPI_SWIGLU) rc = launch_mx<EPI_SWIGLU, true>(d, tmA, tmB, tmB2, sfa, sfb, p);
     else rc = launch_mx<EPI_LSE, false>(d, tmA, tmB, tmB2, sfa, sfb, p);

@@ -1,7 +1,8 @@
 // Block-scaled E4M3 (MXFP8) on CTA pairs: the cta_group::2 form of gemm_mx.cuh for large problems.
 //
-// A pair owns a 256 x 224 output tile (256 x 112 for SwiGLU).  As in gemm_pair.cuh each CTA loads its own 128 rows
-// of X and its own half of the tile's W rows (112), the even CTA issues the MMAs for both
+// A pair owns a 256 x 224 output tile (SwiGLU: 256 x 96, from 96 gate and 96 up accumulator columns, so that the
+// tile is a whole number of 32-column epilogue chunks).  As in gemm_pair.cuh each CTA loads its own 128 rows
+// of X and its own half of the tile's W rows (112; SwiGLU: rank 0 the 96 gate rows, rank 1 the 96 up rows), the even CTA issues the MMAs for both
 // (tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale, M = 256, N = 224, K = 32), and each CTA keeps the
 // accumulator of its 128 rows in its own tensor memory, two buffers of 224 columns, so that a tile's epilogue
 // runs under the next tile's mainloop.  224 and not 256 columns: the scales need tensor memory too (two sets of
@@ -22,26 +23,26 @@ namespace mtmc {
 template <int EPI>
 struct MxPairCfg {
     static constexpr int BM = 256;                        // rows per pair tile (128 per CTA)
-    static constexpr int BN = 224;                        // accumulator columns (SwiGLU: 112 gate + 112 up)
+    static constexpr int BN = (EPI == EPI_SWIGLU) ? 192 : 224;   // accumulator columns (SwiGLU: 96 gate + 96 up)
     static constexpr int BK = 128;                        // E4M3 elements per ring stage: four MMAs of K = 32
     static constexpr int HALF_ROWS = BN / 2;              // W rows each CTA loads
     static constexpr int A_BYTES = 128 * BK;              // 16 KiB
-    static constexpr int B_BYTES = HALF_ROWS * BK;        // 14 KiB, in a 16 KiB slot
+    static constexpr int B_BYTES = HALF_ROWS * BK;        // 14 KiB (SwiGLU: 12 KiB), in a 16 KiB slot
     static constexpr int B_SLOT = 128 * BK;
     static constexpr int SFA_BYTES = 512;                 // scales of this CTA's 128 rows of X x 4 k-blocks
-    static constexpr int SFB_BYTES = 1024;                // scales of the tile's 224 (of 256) rows of W x 4 k-blocks
+    static constexpr int SFB_BYTES = 1024;                // scales of the tile's 224 or 192 (of 256) accumulator columns x 4 k-blocks
     static constexpr int SF_OFFSET = A_BYTES + B_SLOT;
     static constexpr int STAGE_BYTES = 34 * 1024;         // operands 32 KiB + scales 1.5 KiB, padded to keep stages 1024-byte aligned
     static constexpr int STAGES = 6;
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
-    static constexpr int SF_COL0 = 2 * BN;                // 448: then two sets of (4 + 8) scale columns
+    static constexpr int SF_COL0 = 448;                   // after two accumulator buffers: two sets of (4 + 8) scale columns
     static constexpr int TMEM_COLS = 512;
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int THREADS = 192;
     static_assert(SF_OFFSET + SFA_BYTES + SFB_BYTES <= STAGE_BYTES && SMEM_BYTES <= 227 * 1024, "a stage holds operands and scales; six stages fit");
     static_assert(SF_COL0 + 24 <= TMEM_COLS && EPI_HALVES == 1, "accumulators and scale columns fit tensor memory");
-    static_assert(EPI != EPI_SWIGLU, "a SwiGLU tile would have 112 output columns, not a whole number of 32-column epilogue chunks: it stays on gemm_mx.cuh");
+    static_assert(2 * BN <= SF_COL0 && OUT_TILE_N % 32 == 0 && HALF_ROWS % 8 == 0, "accumulator buffers below the scale columns; whole epilogue chunks; whole swizzle atoms");
 };
 
 __device__ __forceinline__ void tmem_cp_scales_pair(uint32_t taddr, uint64_t sdesc) {

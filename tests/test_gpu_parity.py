@@ -407,7 +407,7 @@ def test_fused_linear_mxfp8(M, N, K, act, odt):
     assert torch.equal(B.mtmc_fused_linear_mxfp8(Xd, SXd, Wd, SWd, bd, act, odt), out)
 
 
-@pytest.mark.parametrize("M,N,K", [(5, 8, 64), (100, 72, 160), (300, 392, 288), (600, 1000, 672)])
+@pytest.mark.parametrize("M,N,K", [(5, 8, 64), (100, 72, 160), (300, 392, 288), (600, 1000, 672), (1100, 520, 1056)])
 def test_swiglu_and_lse_mxfp8(M, N, K):
     mi = inputs.mx_linear_inputs(M, N, K, seed=7600 + M + N, spread=4)
     up = inputs.mx_linear_inputs(M, N, K, seed=7650 + M + N, spread=4)
