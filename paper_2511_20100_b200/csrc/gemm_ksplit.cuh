@@ -183,6 +183,8 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             if (warp == 2 && lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(ready_bar, lane));
             ok = mbar_wait_cluster(ready_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 8u);
         }
+        long long tx = tr.now();
+        if (tracer) tr.add(TR_XCHG_READY, tx - tb);
         if (ok) {
             // Everything this warp owes its peers goes out first (the TMEM load of the next chunk in flight while one
             // chunk is stored), then ONE fence orders all of it, then the peers are told: a fence per peer would
@@ -213,7 +215,9 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             fence_acq_rel_cluster();
             __syncwarp();
             if (lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(recv_bar, lane));
+            if (tracer) { const long long t1 = tr.now(); tr.add(TR_XCHG_SEND, t1 - tx); tx = t1; }
             ok = mbar_wait_cluster(recv_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 9u);
+            if (tracer) { const long long t1 = tr.now(); tr.add(TR_XCHG_RECV, t1 - tx); tx = t1; }
         }
         if (ok) {
             // sum of the KS partials of my columns, in rank order, back into TMEM
@@ -247,7 +251,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 tmem_st_32x32b_x32(t_addr + a * 32, r);
             }
             tmem_st_wait();
-            if (tracer) tr.add(TR_EPI_HANDOVER, tr.now() - tb);        // reduce-scatter through distributed shared memory
+            if (tracer) { tr.add(TR_XCHG_SUM, tr.now() - tx); tr.add(TR_EPI_HANDOVER, tr.now() - tb); }        // reduce-scatter through distributed shared memory
             const int row = mb * 128 + q * 32 + lane;
             epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, static_cast<int>(rank) * Cfg::OWN_OC,
                                          (static_cast<int>(rank) + 1) * Cfg::OWN_OC, Cfg::OUT_TILE_N, nb, static_cast<int>(rank), 0, vec_ok,

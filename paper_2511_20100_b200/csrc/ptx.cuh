@@ -397,6 +397,10 @@ enum {
     TR_EPI_ITEMS = 14,      // first epilogue warp: items
     TR_EPI_HANDOVER = 15,   // first epilogue warp: cycles inside stream-K / split-K hand-overs
     TR_END_NS = 16,         // teardown reached
+    TR_XCHG_READY = 17,     // cluster split-K, first epilogue warp: cycles until every peer's ring was idle
+    TR_XCHG_SEND = 18,      // ... cycles spent sending its parts to the peers (stores and fence)
+    TR_XCHG_RECV = 19,      // ... cycles until all peers' parts had arrived
+    TR_XCHG_SUM = 20,       // ... cycles adding the parts and writing the sum back to tensor memory
 };
 struct Trace {
 #ifdef MTMC_TRACE

@@ -26,7 +26,8 @@ from . import inputs  # noqa: E402
 
 WORDS = 32
 NAMES = ["start_ns", "setup_ns", "prod_first_ns", "prod_last_ns", "prod_stall", "mma_first_ns", "mma_last_ns", "mma_stall_data",
-         "mma_stall_acc", "mma_kblocks", "epi_first_ns", "epi_end_ns", "epi_stall", "epi_busy", "epi_items", "epi_handover", "end_ns"]
+         "mma_stall_acc", "mma_kblocks", "epi_first_ns", "epi_end_ns", "epi_stall", "epi_busy", "epi_items", "epi_handover", "end_ns",
+         "xchg_ready", "xchg_send", "xchg_recv", "xchg_sum"]
 
 
 def _problem(args):
@@ -109,6 +110,9 @@ def main():
     if has.any():
         print("  epilogue (first warp): %.1f items per CTA, busy %.0f cycles per item, waiting %.0f cycles per CTA, hand-overs %.0f cycles per CTA" % (
             items[has].mean(), (rec[has, 13] / items[has]).mean(), rec[has, 12].mean(), rec[has, 15].mean()))
+    if rec[:, 18].any():
+        print("  cluster split-K exchange (first warp), cycles per CTA: peers ready %.0f, send %.0f, wait for the peers' parts %.0f, sum %.0f" % (
+            rec[:, 17].mean(), rec[:, 18].mean(), rec[:, 19].mean(), rec[:, 20].mean()))
     if args.csv:
         with open(args.csv, "w") as f:
             f.write("cta," + ",".join(NAMES) + "\n")
