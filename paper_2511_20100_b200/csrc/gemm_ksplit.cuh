@@ -35,10 +35,19 @@ struct KSplitCfg {
     static constexpr int BLOCK_BYTES = 32 * 32 * 4;       // one chunk of one lane quadrant: 32 rows x 128 bytes
     static constexpr int RECV_BYTES = (KS - 1) * OWN_AC * 4 * BLOCK_BYTES;
     static_assert(RECV_BYTES <= STAGES * STAGE_BYTES, "the ring holds the peers' partials");
+    // Clusters of two and four send their parts as bulk copies from a staging area behind the receive area (the
+    // per-thread stores into a peer's shared memory run at about 16 bytes per cycle and CTA); a cluster of eight
+    // would need 2 x 112 KiB for that and keeps the stores.
+    static constexpr bool BULK = 2 * RECV_BYTES <= STAGES * STAGE_BYTES;
     static_assert(OWN_OC >= 1, "at least one output chunk per CTA");
     static constexpr int NUM_BARRIERS = 2 * STAGES + 3;   // ring, accumulator full, ready, received
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 4 * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
-    static constexpr int THREADS = 192;                   // producer, MMA issuer, four epilogue warps
+    // Epilogue warps: two per TMEM lane quadrant where the epilogue stores a tile (they share the exchange, the sums and
+    // the output chunks: the exchange is the exposed tail of a launch whose CTAs have one work item each); one per
+    // quadrant for the row reductions, whose partial per row has one writer.
+    static constexpr int EPI_W = (EPI == EPI_ACT || EPI == EPI_SWIGLU) ? 8 : 4;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_W * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
+    static constexpr int THREADS = 64 + 32 * EPI_W;       // producer, MMA issuer, epilogue warps
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory per CTA");
     static constexpr int TMEM_COLS = BN;                  // one accumulator: a CTA has exactly one work item
 };
 
@@ -47,7 +56,7 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t caddr, float a, fl
 }
 
 template <int EPI, bool OUT_BF16, int KS>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(64 + 32 * KSplitCfg<EPI, KS>::EPI_W, 1)
 gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
     using Cfg = KSplitCfg<EPI, KS>;
@@ -58,7 +67,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;
-    const uint32_t bar_base = epi_stage_base + 4 * EPI_STAGE_BYTES_PER_WARP;
+    const uint32_t bar_base = epi_stage_base + Cfg::EPI_W * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     const uint32_t accf_bar = bar_base + 8u * (2 * STAGES);
@@ -79,7 +88,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
         mbar_init(accf_bar, 1);
         mbar_init(ready_bar, KS - 1);             // one arrival per peer CTA
-        mbar_init(recv_bar, (KS - 1) * 4);        // one per epilogue warp of every peer
+        mbar_init(recv_bar, Cfg::BULK ? 1 : (KS - 1) * Cfg::EPI_W);   // bulk copies count bytes; else one arrival per epilogue warp of every peer
         *abort_flag = 0u;
         fence_barrier_init();
         fence_proxy_async_smem();
@@ -167,6 +176,8 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     } else {
         // ------------------------------------------------------------------ reduce-scatter + epilogue
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;            // which of the quadrant's (one or two) warps this is
+        constexpr int HALVES = Cfg::EPI_W / 4;
         const uint32_t lane_base = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t t_addr = tmem_base + lane_base;
         const bool vec_ok = OUT_BF16 ? (p.ldo % 8 == 0) : (p.ldo % 4 == 0);
@@ -179,6 +190,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         if (tracer) { tr.stamp(TR_EPI_FIRST_NS); tr.add(TR_EPI_ITEMS, 1); }
         if (ok) {
             tc_fence_after();
+            if (Cfg::BULK && warp == 2 && lane == 0) mbar_expect_tx(recv_bar, Cfg::RECV_BYTES);      // what the peers will copy in
             // my ring is idle (every MMA that read it has completed): the peers may write their partials into it
             if (warp == 2 && lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(ready_bar, lane));
             ok = mbar_wait_cluster(ready_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 8u);
@@ -190,11 +202,14 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             // chunk is stored), then ONE fence orders all of it, then the peers are told: a fence per peer would
             // cost a round trip through the cluster each.
             constexpr int SENDS = (KS - 1) * Cfg::OWN_AC;
+            // the quadrant's warps share the chunks: the first takes [0, ceil(SENDS / HALVES)), the second the rest
+            const int s_begin = HALVES == 2 && half ? (SENDS + 1) / 2 : 0;
+            const int s_end = HALVES == 2 && !half ? (SENDS + 1) / 2 : SENDS;
             auto chunk_of = [&](int idx) { return acc_chunk((static_cast<int>(rank) + 1 + idx / Cfg::OWN_AC) % KS, idx % Cfg::OWN_AC); };
             uint32_t r[32];
-            tmem_ld_32x32b_x32(t_addr + chunk_of(0) * 32, r);
+            if (s_begin < s_end) tmem_ld_32x32b_x32(t_addr + chunk_of(s_begin) * 32, r);
 #pragma unroll 1
-            for (int idx = 0; idx < SENDS; ++idx) {
+            for (int idx = s_begin; idx < s_end; ++idx) {
                 const int peer = (static_cast<int>(rank) + 1 + idx / Cfg::OWN_AC) % KS;
                 const int loc = idx % Cfg::OWN_AC;
                 const int sidx = static_cast<int>(rank) < peer ? static_cast<int>(rank) : static_cast<int>(rank) - 1;   // my place among the peer's senders
@@ -202,27 +217,47 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]);
-                if (idx + 1 < SENDS) tmem_ld_32x32b_x32(t_addr + chunk_of(idx + 1) * 32, r);
+                if (idx + 1 < s_end) tmem_ld_32x32b_x32(t_addr + chunk_of(idx + 1) * 32, r);
                 // the reader is the thread at the same place (quadrant, lane) of the peer, so the layout inside the 4 KiB
-                // block is private to the two: each store instruction of the warp writes 512 contiguous bytes, which
-                // the cluster network moves in a few large packets instead of 32 small ones
-                const uint32_t dst = cluster_map_shared(base, peer) +
-                                     static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 16);
+                // block is private to the two: each store instruction of the warp writes 512 contiguous bytes
+                const uint32_t slot = static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES);
+                if constexpr (Cfg::BULK) {
+                    // park the chunk in this CTA's staging area (behind the receive area), then one bulk copy moves it
+                    const uint32_t src = base + Cfg::RECV_BYTES + static_cast<uint32_t>((idx * 4 + q) * Cfg::BLOCK_BYTES);
 #pragma unroll
-                for (int g = 0; g < 8; ++g)
-                    st_shared_cluster_v4(dst + g * 512, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                    for (int g = 0; g < 8; ++g)
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(src + g * 512 + lane * 16), "f"(v[4 * g]), "f"(v[4 * g + 1]),
+                                     "f"(v[4 * g + 2]), "f"(v[4 * g + 3]) : "memory");
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) bulk_copy_to_peer(cluster_map_shared(base, peer) + slot, src, Cfg::BLOCK_BYTES, cluster_map_shared(recv_bar, peer));
+                } else {
+                    const uint32_t dst = cluster_map_shared(base, peer) + slot + lane * 16;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        st_shared_cluster_v4(dst + g * 512, v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
+                }
             }
-            fence_acq_rel_cluster();
-            __syncwarp();
-            if (lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(recv_bar, lane));
+            if constexpr (!Cfg::BULK) {
+                fence_acq_rel_cluster();
+                __syncwarp();
+                if (lane < KS && lane != static_cast<int>(rank)) mbar_arrive_remote(cluster_map_shared(recv_bar, lane));
+            }
             if (tracer) { const long long t1 = tr.now(); tr.add(TR_XCHG_SEND, t1 - tx); tx = t1; }
             ok = mbar_wait_cluster(recv_bar, 0u, abort_flag, p.status, STATUS_TIMEOUT_EPILOGUE | 9u);
             if (tracer) { const long long t1 = tr.now(); tr.add(TR_XCHG_RECV, t1 - tx); tx = t1; }
         }
-        if (ok) {
-            // sum of the KS partials of my columns, in rank order, back into TMEM
+        // The output chunks this warp finishes: its CTA's OWN_OC chunks, shared between the quadrant's warps.
+        const int j_begin = HALVES == 2 && half ? (Cfg::OWN_OC + 1) / 2 : 0;
+        const int j_end = HALVES == 2 && !half ? (Cfg::OWN_OC + 1) / 2 : Cfg::OWN_OC;
+        if (ok && j_begin < j_end) {
+            // sum of the KS partials of those columns (SwiGLU: of their gate and of their up columns), in rank order,
+            // back into TMEM
 #pragma unroll 1
-            for (int loc = 0; loc < Cfg::OWN_AC; ++loc) {
+            for (int part = 0; part < Cfg::OWN_AC / Cfg::OWN_OC; ++part) {
+#pragma unroll 1
+            for (int j = j_begin; j < j_end; ++j) {
+                const int loc = part * Cfg::OWN_OC + j;
                 const int a = acc_chunk(static_cast<int>(rank), loc);
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(t_addr + a * 32, r);
@@ -232,7 +267,7 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 for (int s = 0; s < KS; ++s) {
                     if (s == static_cast<int>(rank)) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) acc[j] = (s == 0) ? __uint_as_float(r[j]) : acc[j] + __uint_as_float(r[j]);
+                        for (int jj = 0; jj < 32; ++jj) acc[jj] = (s == 0) ? __uint_as_float(r[jj]) : acc[jj] + __uint_as_float(r[jj]);
                     } else {
                         const int sidx = s < static_cast<int>(rank) ? s : s - 1;
                         const uint32_t src = base + static_cast<uint32_t>(((sidx * Cfg::OWN_AC + loc) * 4 + q) * Cfg::BLOCK_BYTES + lane * 16);
@@ -247,14 +282,15 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     }
                 }
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(acc[j]);
+                for (int jj = 0; jj < 32; ++jj) r[jj] = __float_as_uint(acc[jj]);
                 tmem_st_32x32b_x32(t_addr + a * 32, r);
+            }
             }
             tmem_st_wait();
             if (tracer) { tr.add(TR_XCHG_SUM, tr.now() - tx); tr.add(TR_EPI_HANDOVER, tr.now() - tb); }        // reduce-scatter through distributed shared memory
             const int row = mb * 128 + q * 32 + lane;
-            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, static_cast<int>(rank) * Cfg::OWN_OC,
-                                         (static_cast<int>(rank) + 1) * Cfg::OWN_OC, Cfg::OUT_TILE_N, nb, static_cast<int>(rank), 0, vec_ok,
+            epilogue_item<EPI, OUT_BF16>(p, t_addr, row, nb * Cfg::OUT_TILE_N, static_cast<int>(rank) * Cfg::OWN_OC + j_begin,
+                                         static_cast<int>(rank) * Cfg::OWN_OC + j_end, Cfg::OUT_TILE_N, nb, static_cast<int>(rank), 0, vec_ok,
                                          smem_raw + (epi_stage_base - raw_addr) + (warp - 2) * EPI_STAGE_BYTES_PER_WARP, lane);
         }
         if (tracer) { tr.add(TR_EPI_BUSY, tr.now() - tb); tr.stamp(TR_EPI_END_NS); }
