@@ -1233,7 +1233,9 @@ int launch_mx_pair(int clusters, const CUtensorMap& tmA, const CUtensorMap& tmB,
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1 + pdl_attribute(attr + 1);
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmSFA, tmSFB, p));
+    GemmParams q = p;
+    q.trace = trace_for(cfg.gridDim.x);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, tmSFA, tmSFB, q));
     g_launches.fetch_add(1);
     note_kernel("gemm_mx_pair_kernel", EPI);
     return MTMC_OK;

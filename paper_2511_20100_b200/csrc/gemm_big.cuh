@@ -116,6 +116,8 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            long long t_stall = 0;
+            bool t_first = true;
             const uint32_t full0_base = cluster_map_shared(full_bar(0), 0);   // the even CTA's full barriers
             for (int t = pair_id; t < p.num_tiles && ok; t += num_pairs) {
                 int mb, nb;
@@ -129,8 +131,8 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int kb = 0; kb < p.k_blocks; ++kb, kx += p.bk_elems) {
                     const long long tw = tr.now();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 5u)) { ok = false; break; }
-                    tr.add(TR_PROD_STALL, tr.now() - tw);
-                    tr.stamp_once(TR_PROD_FIRST_NS);
+                    t_stall += tr.now() - tw;                 // trace totals live in registers and are written once, after the loop
+                    if (t_first) { tr.stamp(TR_PROD_FIRST_NS); t_first = false; }
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = full0_base + 8u * s;
                     tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
@@ -139,6 +141,7 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
+            tr.add(TR_PROD_STALL, t_stall);
             tr.stamp(TR_PROD_LAST_NS);
         }
         __syncwarp();
@@ -148,20 +151,22 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             int s = 0;
             uint32_t ph = 0, acc_ph = 0;
             bool ok = true;
+            long long t_data = 0, t_head = 0, t_max = 0, t_acc = 0, t_kb = 0;      // trace totals (dead code without -DMTMC_TRACE)
+            bool t_first = true;
             const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(256, Cfg::BN) : umma_idesc_bf16(256, Cfg::BN);
             for (int t = pair_id; t < p.num_tiles && ok; t += num_pairs) {
                 // the one accumulator set is free again once every epilogue warp of both CTAs has drained it
                 const long long ta = tr.now();
                 if (!mbar_wait_cluster(acce_bar, acc_ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 8u)) { ok = false; break; }
-                tr.add(TR_MMA_STALL_ACC, tr.now() - ta);
+                t_acc += tr.now() - ta;
                 acc_ph ^= 1u;
                 tc_fence_after();
                 for (int kb = 0; kb < p.k_blocks; ++kb) {
                     const long long tw = tr.now();
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 9u)) { ok = false; break; }
-                    tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
-                    tr.add(TR_MMA_KBLOCKS, 1);
-                    tr.stamp_once(TR_MMA_FIRST_NS);
+                    { const long long dw = tr.now() - tw; t_data += dw; t_max = dw > t_max ? dw : t_max; if (kb < STAGES) t_head += dw; }
+                    ++t_kb;
+                    if (t_first) { tr.stamp(TR_MMA_FIRST_NS); t_first = false; }
                     tc_fence_after();
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
                     const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
@@ -184,6 +189,8 @@ gemm_big_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
                 if (ok) umma_commit_pair(accf_bar, 3);           // both halves complete, in both CTAs
             }
+            tr.add(TR_MMA_STALL_DATA, t_data); tr.add(TR_MMA_STALL_HEAD, t_head); tr.max(TR_MMA_STALL_MAX, t_max);
+            tr.add(TR_MMA_STALL_ACC, t_acc); tr.add(TR_MMA_KBLOCKS, t_kb);
             tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();

@@ -1,8 +1,8 @@
 // The tiled tensor-core path for large problems: CTA pairs (thread-block clusters of two).
 //
 // A pair owns a 256 x 256 output tile (256 x 128 for SwiGLU).  Each CTA loads its own 128
-// rows of X and its own half of the W rows of the tile, so a ring stage is 32 KiB instead of
-// 48 KiB: six stages deep instead of four and a third less L2 -> shared-memory traffic per
+// rows of X and its own half of the W rows of the tile, so a k-block is 32 KiB instead of
+// 48 KiB (a ring of six k-blocks, handed over two at a time, instead of four) and a third less L2 -> shared-memory traffic per
 // FLOP.  The even CTA issues tcgen05.mma.cta_group::2 (M = 256) for both; each CTA keeps the
 // accumulator of its own 128 rows in its own TMEM and runs its own epilogue.
 //
@@ -35,8 +35,13 @@ struct PairCfg {
     static constexpr int BK = 64;
     static constexpr int A_BYTES = 128 * BK * 2;         // this CTA's X rows
     static constexpr int B_BYTES = 128 * BK * 2;         // this CTA's half of the W rows (at most)
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = 6;
+    // A ring stage carries two k-blocks.  The thread that issues the MMAs pays a fixed price per stage (the wait for
+    // the stage's data, the commit that frees it) on top of the MMAs themselves, and with one k-block per stage that
+    // thread, not the tensor pipe, set the pace: about 700 cycles per k-block against 512 of MMA.
+    static constexpr int KB_PER_STAGE = 2;
+    static constexpr int SUB_BYTES = A_BYTES + B_BYTES;  // one k-block: this CTA's X rows, then its W rows
+    static constexpr int STAGE_BYTES = KB_PER_STAGE * SUB_BYTES;
+    static constexpr int STAGES = 3;
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     static constexpr int TMEM_COLS = 2 * BN;
     static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
@@ -261,6 +266,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
+            long long t_stall = 0;
+            bool t_first = true;
             const uint32_t full0_base = cluster_map_shared(full_bar(0), 0);   // the even CTA's full barriers
             PairWalk walk(p, pair_id, num_pairs);
             PairWork w;
@@ -276,22 +283,28 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const CUtensorMap* mapB = (EPI == EPI_SWIGLU && rank == 1) ? (whole ? &tmB2 : &tmB2t) : (whole ? &tmB : &tmBt);
                 const uint32_t cta_bytes = Cfg::A_BYTES + static_cast<uint32_t>(b_rows) * Cfg::BK * 2;
                 int kx = w.kb0 * p.bk_elems;                             // K coordinate of the next k-block
-                for (int kb = w.kb0; kb < w.kb1; ++kb, kx += p.bk_elems) {
+                for (int kb = w.kb0; kb < w.kb1; kb += Cfg::KB_PER_STAGE, kx += Cfg::KB_PER_STAGE * p.bk_elems) {
+                    const bool two = kb + 1 < w.kb1;                     // an odd walk ends with half a stage
                     const long long tw = tr.now();
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 3u)) { ok = false; break; }
-                    tr.add(TR_PROD_STALL, tr.now() - tw);
-                    tr.stamp_once(TR_PROD_FIRST_NS);
+                    t_stall += tr.now() - tw;                 // trace totals live in registers and are written once, after the loop
+                    if (t_first) { tr.stamp(TR_PROD_FIRST_NS); t_first = false; }
                     // loads first, bookkeeping after: the time from "slot free" to "load issued" is on the ring's
                     // critical path (a transaction count may run ahead of its expect_tx within a phase)
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = full0_base + 8u * s;
-                    if (!MTMC_CHECK(a_dst + cta_bytes <= epi_stage_base && (kx & 7) == 0 && m0 >= 0 && n_row0 >= 0, p.status, 4u)) { ok = false; break; }
+                    if (!MTMC_CHECK(a_dst + Cfg::SUB_BYTES + cta_bytes <= epi_stage_base && (kx & 7) == 0 && m0 >= 0 && n_row0 >= 0, p.status, 4u)) { ok = false; break; }
                     tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
                     tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kx, n_row0);
-                    if (rank == 0) mbar_expect_tx(full_bar(s), 2u * cta_bytes);     // both CTAs' bytes
+                    if (two) {
+                        tma_load_2d_pair(a_dst + Cfg::SUB_BYTES, &tmA, full0, kx + p.bk_elems, m0);
+                        tma_load_2d_pair(a_dst + Cfg::SUB_BYTES + Cfg::A_BYTES, mapB, full0, kx + p.bk_elems, n_row0);
+                    }
+                    if (rank == 0) mbar_expect_tx(full_bar(s), (two ? 4u : 2u) * cta_bytes);     // both CTAs' bytes
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
+            tr.add(TR_PROD_STALL, t_stall);
             tr.stamp(TR_PROD_LAST_NS);
         }
         __syncwarp();
@@ -303,6 +316,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t acc_ph = 0;
             int it = 0;
             bool ok = true;
+            long long t_data = 0, t_head = 0, t_max = 0, t_acc = 0, t_kb = 0, t_issue = 0;      // trace totals (dead code without -DMTMC_TRACE)
+            bool t_first = true;
             PairWalk walk(p, pair_id, num_pairs);
             PairWork w;
             for (; ok && walk.next(w); ++it) {
@@ -312,35 +327,44 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(Cfg::BM, mma_n) : umma_idesc_bf16(Cfg::BM, mma_n);
                 const long long ta = tr.now();
                 if (!mbar_wait_cluster(acce_bar(buf), ((acc_ph >> buf) & 1u) ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA | 5u)) { ok = false; break; }
-                tr.add(TR_MMA_STALL_ACC, tr.now() - ta);
+                t_acc += tr.now() - ta;
                 acc_ph ^= 1u << buf;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * Cfg::BN);
-                for (int kb = w.kb0; kb < w.kb1; ++kb) {
+                for (int kb = w.kb0; kb < w.kb1; kb += Cfg::KB_PER_STAGE) {
+                    const int nsub = kb + 1 < w.kb1 ? 2 : 1;
                     const long long tw = tr.now();
                     if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 6u)) { ok = false; break; }
-                    tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
-                    tr.add(TR_MMA_KBLOCKS, 1);
-                    tr.stamp_once(TR_MMA_FIRST_NS);
+                    { const long long dw = tr.now() - tw; t_data += dw; t_max = dw > t_max ? dw : t_max; if (kb - w.kb0 < STAGES * Cfg::KB_PER_STAGE) t_head += dw; }
+                    t_kb += nsub;
+                    if (t_first) { tr.stamp(TR_MMA_FIRST_NS); t_first = false; }
                     tc_fence_after();
                     const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
-                    const uint64_t a_desc = umma_smem_desc_sw128(a_src);
-                    const uint64_t b_desc = umma_smem_desc_sw128(a_src + Cfg::A_BYTES);
-                    // four MMAs per 128-byte row either way: 4 x 16 bf16 or 4 x 32 E4M3, 32 bytes apart
-                    if (p.fp8) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_fp8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | k) != 0 ? 1u : 0u);
-                    } else {
+                    for (int j = 0; j < Cfg::KB_PER_STAGE; ++j) {
+                        if (j < nsub) {
+                            const uint64_t a_desc = umma_smem_desc_sw128(a_src + j * Cfg::SUB_BYTES);
+                            const uint64_t b_desc = umma_smem_desc_sw128(a_src + j * Cfg::SUB_BYTES + Cfg::A_BYTES);
+                            // four MMAs per 128-byte row either way: 4 x 16 bf16 or 4 x 32 E4M3, 32 bytes apart
+                            if (p.fp8) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | k) != 0 ? 1u : 0u);
+                                for (int k = 0; k < 4; ++k)
+                                    umma_fp8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | j | k) != 0 ? 1u : 0u);
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | j | k) != 0 ? 1u : 0u);
+                            }
+                        }
                     }
                     umma_commit_pair(empty_bar(s), 3);           // frees the stage in both CTAs
+                    t_issue += tr.now() - tw;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit_pair(accf_bar(buf), 3);      // accumulator complete, in both CTAs
             }
+            tr.add(TR_MMA_STALL_DATA, t_data); tr.add(TR_MMA_STALL_HEAD, t_head); tr.max(TR_MMA_STALL_MAX, t_max);
+            tr.add(TR_MMA_STALL_ACC, t_acc); tr.add(TR_MMA_KBLOCKS, t_kb); tr.add(TR_MMA_ISSUE, t_issue - t_data);
             tr.stamp(TR_MMA_LAST_NS);
         }
         __syncwarp();

@@ -408,22 +408,35 @@ enum {
     TR_XCHG_SEND = 18,      // ... cycles spent sending its parts to the peers (stores and fence)
     TR_XCHG_RECV = 19,      // ... cycles until all peers' parts had arrived
     TR_XCHG_SUM = 20,       // ... cycles adding the parts and writing the sum back to tensor memory
+    TR_START_CLK = 21,      // clock64 at TR_START_NS and at TR_END_NS: (end - start) cycles over (end - start) ns is the SM
+    TR_END_CLK = 22,        // clock the CTA ran at
+    TR_MMA_STALL_HEAD = 23, // the part of TR_MMA_STALL_DATA spent on the first ring-depth k-blocks of each work item
+    TR_MMA_STALL_MAX = 24,  // the longest single wait for data
+    TR_MMA_ISSUE = 25,      // cycles the issuing thread spent between a stage's data being there and its commit being issued
 };
 struct Trace {
 #ifdef MTMC_TRACE
     unsigned long long* rec;
     __device__ __forceinline__ explicit Trace(unsigned long long* base) : rec(base ? base + static_cast<size_t>(blockIdx.x) * TRACE_WORDS : nullptr) {}
     __device__ __forceinline__ void stamp(int i) const {
-        if (rec) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); rec[i] = t; }
+        if (rec) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            rec[i] = t;
+            if (i == TR_START_NS) rec[TR_START_CLK] = static_cast<unsigned long long>(clock64());
+            if (i == TR_END_NS) rec[TR_END_CLK] = static_cast<unsigned long long>(clock64());
+        }
     }
     __device__ __forceinline__ void stamp_once(int i) const { if (rec && rec[i] == 0ull) stamp(i); }
     __device__ __forceinline__ void add(int i, long long v) const { if (rec) rec[i] += static_cast<unsigned long long>(v); }
+    __device__ __forceinline__ void max(int i, long long v) const { if (rec && static_cast<unsigned long long>(v) > rec[i]) rec[i] = static_cast<unsigned long long>(v); }
     __device__ __forceinline__ long long now() const { return rec ? clock64() : 0ll; }
 #else
     __device__ __forceinline__ explicit Trace(unsigned long long*) {}
     __device__ __forceinline__ void stamp(int) const {}
     __device__ __forceinline__ void stamp_once(int) const {}
     __device__ __forceinline__ void add(int, long long) const {}
+    __device__ __forceinline__ void max(int, long long) const {}
     __device__ __forceinline__ long long now() const { return 0ll; }
 #endif
 };

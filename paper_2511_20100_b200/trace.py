@@ -27,7 +27,7 @@ from . import inputs  # noqa: E402
 WORDS = 32
 NAMES = ["start_ns", "setup_ns", "prod_first_ns", "prod_last_ns", "prod_stall", "mma_first_ns", "mma_last_ns", "mma_stall_data",
          "mma_stall_acc", "mma_kblocks", "epi_first_ns", "epi_end_ns", "epi_stall", "epi_busy", "epi_items", "epi_handover", "end_ns",
-         "xchg_ready", "xchg_send", "xchg_recv", "xchg_sum"]
+         "xchg_ready", "xchg_send", "xchg_recv", "xchg_sum", "start_clk", "end_clk", "mma_stall_head", "mma_stall_max", "mma_issue"]
 
 
 def _problem(args):
@@ -36,6 +36,14 @@ def _problem(args):
     else:
         M, N, K = (int(v) for v in args.what)
         c = dict(op="fused_linear", M=M, N=N, K=K, act="gelu_tanh", out_dtype="bf16", seed=1)
+    if c["op"] == "fused_linear_mxfp8":
+        mi = inputs.mx_linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+        d = [mi.X.cuda(), mi.SX.cuda(), mi.W.cuda(), mi.SW.cuda(), mi.b.cuda()]
+        return c, lambda: B.mtmc_fused_linear_mxfp8(d[0], d[1], d[2], d[3], d[4], c["act"], c["out_dtype"])
+    if c["op"] == "fused_linear_fp8":
+        fi = inputs.fp8_linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+        d = [fi.X.cuda(), fi.W.cuda(), fi.b.cuda()]
+        return c, lambda: B.mtmc_fused_linear_fp8(d[0], d[1], d[2], fi.scale_x, fi.scale_w, c["act"], c["out_dtype"])
     if c["op"] == "swiglu":
         si = inputs.swiglu_inputs(c["M"], c["N"], c["K"], c["seed"])
         d = [si.X.cuda(), si.Wg.cuda(), si.Wu.cuda()]
@@ -83,7 +91,7 @@ def main():
     rec = buf.cpu().view(-1, WORDS).numpy()
     rec = rec[rec[:, 0] != 0]
     if len(rec) == 0:
-        raise SystemExit("%s wrote no trace (only the CTA-pair and weight-streaming kernels are instrumented)" % kernel)
+        raise SystemExit("%s wrote no trace (the single-CTA tiled kernels are not instrumented)" % kernel)
     t0 = rec[:, 0].min()
     print("%s  M=%d N=%d K=%d  kernel %s  %d CTAs traced" % (" ".join(args.what), c["M"], c["N"], c["K"], kernel, len(rec)))
 
@@ -96,14 +104,21 @@ def main():
                        ("first accumulator ready", 10), ("last epilogue done", 11), ("teardown", 16)):
         lo, mean, hi = us(col)
         print("  %-26s min %9.2f  mean %9.2f  max %9.2f us" % (label, lo, mean, hi))
+    timed = (rec[:, 16] > rec[:, 0]) & (rec[:, 22] > rec[:, 21])
+    if timed.any():
+        mhz = (rec[timed, 22] - rec[timed, 21]).astype(float) / (rec[timed, 16] - rec[timed, 0]).astype(float) * 1e3
+        print("  SM clock over the CTAs' lifetimes: %.0f MHz (min %.0f, max %.0f)" % (mhz.mean(), mhz.min(), mhz.max()))
     issuers = rec[:, 9] > 0
     if issuers.any():
         kb = rec[issuers, 9].astype(float)
         span = (rec[issuers, 6] - rec[issuers, 5]).astype(float)      # ns from first MMA to last commit
         print("  MMA issuers: %d, k-blocks each %.1f (min %d, max %d); first MMA to last commit %.2f us mean = %.1f ns per k-block" % (
             int(issuers.sum()), kb.mean(), kb.min(), kb.max(), span.mean() / 1e3, (span / kb).mean()))
-        print("  MMA issuer waits, cycles per CTA: for data %.0f (%.0f per k-block), for a drained accumulator %.0f" % (
-            rec[issuers, 7].mean(), (rec[issuers, 7] / kb).mean(), rec[issuers, 8].mean()))
+        print("  MMA issuer waits, cycles per CTA: for data %.0f (%.0f per k-block; %.0f of it on the first ring-depth k-blocks of the work items; longest wait %.0f), "
+              "for a drained accumulator %.0f" % (rec[issuers, 7].mean(), (rec[issuers, 7] / kb).mean(), rec[issuers, 23].mean(), rec[issuers, 24].max(),
+                                                  rec[issuers, 8].mean()))
+    if issuers.any() and rec[issuers, 25].any():
+        print("  MMA issuer, from a stage's data being there to its commit issued: %.0f cycles per k-block" % (rec[issuers, 25] / kb).mean())
     print("  producer waits for a free stage: %.0f cycles per CTA" % rec[:, 4].mean())
     items = rec[:, 14].astype(float)
     has = items > 0
