@@ -529,7 +529,7 @@ void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
 bool use_pair(DeviceState* d, int64_t M, int64_t N) {
     if (t_cta_pair < 0 || t_tile_n == 128 || gemm_pairs(d) <= 0) return false;
     if (t_cta_pair > 0) return true;
-    return M >= 512 && N >= 256;
+    return M > 256 && N >= 256;        // from the second 128-row block of a second pair tile on (measured: 264 x 8192 x 8192 already 7 % ahead of 128-row tiles)
 }
 
 // Waves of 512 x 256 tiles against waves of 256 x 256 tiles, both counted in 256-row tile waves: the large tiles
@@ -543,34 +543,26 @@ bool big_waves_ok(int64_t M, int64_t N, int pairs, bool long_k) {
 }
 
 // The 512 x 256 pair tiles (gemm_big.cuh) against the 256 x 256 ones with overlapped epilogues (gemm_pair.cuh).
-// Measured on plain and GELU epilogues: per FLOP the large tiles are on a par at K = 4096 and 5-15 % ahead from
-// K = 8192 on (a quarter less operand traffic, and the exposed epilogue shrinks against the k-walk); their
-// tiles are twice as large, so with few waves they can lose more to the last, partial wave.  Hence: from 64
-// k-blocks on when their waves cost no more than the pair kernel's (a tenth more from 96 k-blocks on).  Tuning hook: cta_pair = 2 forces them, 1 forces the 256 x 256 pair tiles.
+// Since the pair kernel hands its ring over two k-blocks at a time its mainloop runs close to the tensor pipe's
+// pace as well, and its overlapped epilogue then decides: measured on GELU epilogues it is 4-5 % ahead at
+// K = 4096 (C2) and K = 14336, level at K = 8192 and 2 % behind at K = 16384; with E4M3 operands 5-15 % ahead up to
+// K = 14336; on the logsumexp epilogue 4 % ahead at K = 4096 (C4: 657 against 684 us).  So the large tiles are
+// chosen from 256 k-blocks on (K = 16384 in bf16), when their waves cost no more than a tenth above the pair
+// kernel's.  Tuning hook: cta_pair = 2 forces them, 1 forces the 256 x 256 pair tiles.
 bool use_big(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     const int pairs = gemm_pairs(d);
     if (pairs <= 0 || EPI_HALVES != 1 || t_tile_n != 0 || t_cta_pair < 0 || t_cta_pair == 1) return false;
     if (t_cta_pair == 2) return true;
     if (M < 512 || N < 256) return false;
     const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
-    if (k_blocks < 64) return false;
-    return big_waves_ok(M, N, pairs, k_blocks >= 96);
+    if (k_blocks < 256) return false;
+    return big_waves_ok(M, N, pairs, true);
 }
 
-// The same choice for the row reductions (logsumexp, row max, cross entropy).  Their epilogues store one partial
-// per row, so little is exposed when it is not overlapped: the large tiles are 4-5 % ahead at K = 4096 already
-// (C4: 680-714 us against 710-750 us).  From 32 k-blocks on, under the same wave rule.
+// The same choice for the row reductions (logsumexp, row max, cross entropy).
 // SwiGLU stays on the 256 x 256 tiles: its epilogue (two MUFU operations per element plus the stores) is too long
-// to expose (measured on C3: 2-3 % slower on the large tiles).
-bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
-    const int pairs = gemm_pairs(d);
-    if (pairs <= 0 || EPI_HALVES != 1 || t_tile_n != 0 || t_cta_pair < 0 || t_cta_pair == 1) return false;
-    if (t_cta_pair == 2) return true;
-    if (M < 512 || N < 256) return false;
-    const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
-    if (k_blocks < 32) return false;
-    return big_waves_ok(M, N, pairs, k_blocks >= 96);
-}
+// to expose.
+bool use_big_rowred(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) { return use_big(d, M, N, K, fp8); }
 
 // SwiGLU on the 512 x 256 tiles: only when the tuning hook forces them (cta_pair = 2); measured slower by default.
 bool use_big_swiglu(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
