@@ -526,10 +526,14 @@ int pick_ksplit(DeviceState* d, int64_t M, int64_t N, int64_t K, int out_tile_n,
 void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n, int ks, bool fp8);
 
 // Large problems go to CTA pairs (256-row tiles); small ones keep single-CTA 128-row tiles.
-bool use_pair(DeviceState* d, int64_t M, int64_t N) {
+bool use_pair(DeviceState* d, int64_t M, int64_t N, int64_t K = 1 << 20) {
     if (t_cta_pair < 0 || t_tile_n == 128 || gemm_pairs(d) <= 0) return false;
     if (t_cta_pair > 0) return true;
-    return M > 256 && N >= 256;        // from the second 128-row block of a second pair tile on (measured: 264 x 8192 x 8192 already 7 % ahead of 128-row tiles)
+    if (M * N * K < (1ll << 28)) return false;
+    // from a second 128-row block on: even with the pair tile's lower half mostly empty (M = 129) the pair kernel's
+    // mainloop makes up for it (129 ... 256 x 32000 x 4096: 62-70 us against 68-78 us on 128-row tiles)
+    // (tiny problems, a microsecond of work or less, keep the plain launch: 256-cube 8.1 us against 8.5-9.5 us as a cluster launch)
+    return M > 128 && N >= 256;
 }
 
 // Waves of 512 x 256 tiles against waves of 256 x 256 tiles, both counted in 256-row tile waves: the large tiles
@@ -927,7 +931,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     if (rc) return rc;
     const int ks = pick_ksplit(d, M, N, K, 256, fp8);
     const bool big = !ks && use_big_rowred(d, M, N, K, fp8);
-    const bool pair = !ks && !big && use_pair(d, M, N);
+    const bool pair = !ks && !big && use_pair(d, M, N, K);
     const int bn = (pair || ks || big) ? 256 : pick_tile_n(N);
     GemmParams p{};
     bool sk = false;
@@ -1009,7 +1013,7 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
         tr.stop();
         return rc;
     }
-    if (use_pair(d, M, N)) {
+    if (use_pair(d, M, N, K)) {
         GemmParams p{};
         const bool sk = plan_pair(d, p, M, N, K, 256, false);
         if ((rc = pair_scratch(d, p, sk))) return rc;
@@ -1083,7 +1087,7 @@ int swiglu_impl(const void* X, const void* Wg, const void* Wu, int64_t M, int64_
         tr.stop();
         return rc;
     }
-    if (use_pair(d, M, N)) {
+    if (use_pair(d, M, N, K)) {
         GemmParams p{};
         const bool sk = plan_pair(d, p, M, N, K, 128, fp8);
         if ((rc = pair_scratch(d, p, sk))) return rc;
@@ -1493,7 +1497,7 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
         tr.stop();
         return rc;
     }
-    const bool pair = use_pair(d, M, N);
+    const bool pair = use_pair(d, M, N, K);
     const int bn = pair ? 256 : pick_tile_n(N);
     GemmParams p{};
     if (pair) {
