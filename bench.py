@@ -291,6 +291,8 @@ def run_ours(args, rank, world, local_rank):
     B.load()
     # W, Wg, Wu are the weights of a layer: created once below and never written again, which is what this switch promises
     B.mtmc_set_static_weights(True)
+    if args.cta_pair:
+        B.mtmc_set_tuning(cta_pair=args.cta_pair)
     problems = [make_device_problem(n, device) for n in ORDER]
     peaks = measured_peaks()
 
@@ -585,6 +587,8 @@ def main():
     ap.add_argument("--full-cpu-baseline", action="store_true", help="time the oracle on all rows of every configuration (minutes)")
     ap.add_argument("--no-eager", action="store_true", help="skip the PyTorch-eager context timings")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-pointer end-to-end leg")
+    ap.add_argument("--cta-pair", type=int, default=0, help="tuning hook for every call (profiling aid): 1 forces the 256 x 256 pair tiles, "
+                    "2 the 512 x 256 pair tiles, -1 single-CTA tiles; 0 leaves the choice to the library")
     ap.add_argument("--configs", default=",".join(ORDER), help="comma-separated subset of C1..C5, or of the further operators X1.. (profiling aid)")
     args = ap.parse_args()
     ORDER = [c for c in args.configs.split(",") if c in inputs.CONFIGS or c in inputs.EXTRA_CONFIGS]

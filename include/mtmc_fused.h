@@ -329,19 +329,20 @@ float mtmc_last_kernel_ms(void);
  *   tile_n   : 128 or 256 forces single-CTA tiles with that accumulator width
  *   cta_pair : 1 forces the CTA-pair (cta_group::2) kernel with 256 x 256 tiles and overlapped
  *              epilogues, 2 the one with 512 x 256 tiles, < 0 forbids both;
- *              automatic = pairs when M >= 512 and N >= 256; the large tiles for the row
- *              reductions and for activation epilogues with a long K, never for SwiGLU
- *              (measured on a par at best) */
+ *              automatic = pairs when M > 128 and N >= 256 (and the problem is not tiny);
+ *              the large tiles from K = 16384 on (twice that for E4M3), never for SwiGLU */
 int mtmc_set_tuning(int split_k, int tile_n, int cta_pair);
 
 /* Device-side trace, for builds of the library compiled with -DMTMC_TRACE (the default build has none:
  * mtmc_trace_enabled() returns 0 and mtmc_set_trace() with a buffer fails with MTMC_ERR_INVALID_ARG).
  * dptr is a zero-filled device buffer of `bytes` bytes, 8-byte aligned, owned by the caller; (NULL, 0)
- * switches tracing off.  Thread-local.  While set, the CTA-pair kernels and the weight-streaming kernel
+ * switches tracing off.  Thread-local.  While set, the CTA-pair kernels (bf16 / E4M3 and MXFP8), the cluster
+ * split-K kernel and the weight-streaming kernel
  * write one record of 32 uint64 per CTA (launches of more CTAs than the buffer holds are not traced):
- * %globaltimer stamps of set-up, first / last load, first / last MMA, first / last epilogue, and cycle
+ * %globaltimer stamps of set-up, first / last load, first / last MMA, first / last epilogue, clock64 at both
+ * ends of the CTA's life, and cycle
  * totals of each role's waits (producer on a free stage, MMA issuer on data and on a drained accumulator,
- * epilogue on an accumulator, stream-K hand-overs); word indices are the TR_* constants of
+ * epilogue on an accumulator, stream-K hand-overs, the split-K exchange); word indices are the TR_* constants of
  * paper_2511_20100_b200/csrc/ptx.cuh, decoded by `python -m paper_2511_20100_b200.trace`.  Stall figures
  * quoted for this library come from there.  No counterpart in the paper. */
 int mtmc_trace_enabled(void);

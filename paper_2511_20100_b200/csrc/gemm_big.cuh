@@ -1,16 +1,16 @@
 // The tiled tensor-core path for large problems with a long K: CTA pairs on 512 x 256 tiles.
 //
 // gemm_pair.cuh gives each CTA 128 rows of a 256 x 256 pair tile and two accumulator buffers, so
-// that a tile's epilogue runs under the next tile's mainloop; its ring stage of 32 KiB feeds 512
-// clocks of MMA (64 B of shared-memory fill per clock and SM), and the mainloop is bound by the
-// shared-memory pipe at about 82 % tensor activity.  Here each CTA owns 256 rows: per 64-wide
+// that a tile's epilogue runs under the next tile's mainloop; a k-block of 32 KiB feeds 512
+// clocks of MMA (64 B of shared-memory fill per clock and SM).  Here each CTA owns 256 rows: per 64-wide
 // k-block it loads 256 rows of X (32 KiB) and its half of the tile's W rows (16 KiB) and issues the
 // MMAs of its two 128-row halves against the same W operand, so 48 KiB feed 1024 clocks of MMA
 // (48 B per clock): a quarter less fill per FLOP, from shared memory and from L2.  The price: the
 // two accumulators (2 x 256 columns) fill the tensor memory, so the epilogue cannot overlap the
 // next tile's mainloop; eight epilogue warps (two per TMEM lane quadrant, one per row half) keep
-// it short, and the producer refills the ring meanwhile.  It pays when the k-walk is long
-// against the epilogue.
+// it short, and the producer refills the ring meanwhile.  Eight MMAs per wait and commit keep the
+// issuing thread well ahead of the tensor pipe; it pays when the k-walk is long against the
+// exposed epilogue (measured: from K = 16384 on).
 //
 // Barriers as in gemm_pair.cuh: all TMA bytes of a stage are counted on the even CTA's `full`
 // barrier; tcgen05.commit with a cluster mask frees the stage in both CTAs and publishes the
