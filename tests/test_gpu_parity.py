@@ -224,19 +224,34 @@ def test_other_operators_on_strided_views(M, N, K, padx, padw, pado):
 
 
 def test_large_tile_pair_kernel_chosen_for_long_k():
-    """From 96 k-blocks on the 512 x 256 tiles are the default for M >= 512, N >= 256: bf16, residual and FP8 forms."""
+    """From 256 k-blocks on the 512 x 256 tiles are the default when their waves cost no more than the 256 x 256 pair
+    tiles' (1024 x 9472 x 16384: 74 large tiles, one wave).  That shape against the oracle on sampled points (every pair
+    tile, tile edges); a small one (15 tiles: cluster split-K by default) in full on each kernel family the hooks select."""
+    M, N, K = 1024, 9472, 16384
+    li = inputs.linear_inputs(M, N, K, seed=8899)
+    out = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), "silu", "bf16")
+    assert "gemm_big_kernel" in B.mtmc_last_kernel_name(), "ran %s" % B.mtmc_last_kernel_name()
+    B.mtmc_check_status()
+    rows, cols = inputs.sample_points(M, N, 3000, seed=7, tile_m=256, tile_n=256)
+    want = ref.fused_linear_points(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_SILU, rows, cols)
+    _assert_close(inputs.to_f64(out[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()]), want, TOL["bf16"], "1024 x 9472 x 16384 sampled")
+    assert bool(torch.isfinite(out.float()).all())
+    del out, li
+
     M, N, K = 600, 520, 6144
     li = inputs.linear_inputs(M, N, K, seed=8900)
     Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
     Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
-    out = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
-    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, ref.ACT_SILU), TOL["fp32"], "long K, default path")
-    B.mtmc_set_tuning(cta_pair=1)
-    try:
-        small_tiles = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
-    finally:
-        B.mtmc_set_tuning()
-    _assert_close(inputs.to_f64(small_tiles), ref.fused_linear(Xb, Wb, bf, ref.ACT_SILU), TOL["fp32"], "long K, 256-row tiles")
+    want = ref.fused_linear(Xb, Wb, bf, ref.ACT_SILU)
+    for tune, family in ((dict(), "gemm_ksplit_kernel"), (dict(cta_pair=1), "gemm_pair_kernel"), (dict(cta_pair=2), "gemm_big_kernel"),
+                         (dict(cta_pair=-1, split_k=1), "gemm_tiled_kernel")):
+        B.mtmc_set_tuning(**tune)
+        try:
+            out = B.mtmc_fused_linear(Xd, Wd, bd, "silu", "fp32")
+            assert family in B.mtmc_last_kernel_name(), "%r ran %s" % (tune, B.mtmc_last_kernel_name())
+        finally:
+            B.mtmc_set_tuning()
+        _assert_close(inputs.to_f64(out), want, TOL["fp32"], "long K, %s" % family)
     R = torch.randn(M, N, generator=torch.Generator().manual_seed(5)).bfloat16()
     res = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "none", "bf16")
     _assert_close(inputs.to_f64(res), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_NONE), TOL["bf16"],
@@ -246,6 +261,37 @@ def test_large_tile_pair_kernel_chosen_for_long_k():
     want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_GELU_TANH)
     _assert_close(inputs.to_f64(f8), want8, TOL["bf16"], "long K fp8")
     B.mtmc_check_status()
+
+
+@pytest.mark.parametrize("K", [40, 136, 264, 456, 520])
+def test_pair_kernel_odd_and_even_k_block_counts(K):
+    """The pair kernel hands its ring over two k-blocks at a time; a walk of 1, 3, 5 or 7 k-blocks ends with half a
+    stage (K = 40, 136, 264, 456; 520 is 9 k-blocks and wraps the three-stage ring).  All epilogues, bf16 and E4M3
+    operands, and tail pieces (300 x 520 leaves a partial wave that is cut into column pieces)."""
+    M, N = 300, 520
+    li = inputs.linear_inputs(M, N, K, seed=9100 + K)
+    si = inputs.swiglu_inputs(M, N, K, seed=9200 + K)
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=9300 + K)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    B.mtmc_set_tuning(cta_pair=1)
+    try:
+        out = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), "gelu_tanh", "fp32")
+        assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+        sw = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+        assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+        lse = B.mtmc_linear_lse(li.X.cuda(), li.W.cuda(), li.b.cuda())
+        f8 = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "relu", "fp32")
+        assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+    finally:
+        B.mtmc_set_tuning()
+    B.mtmc_check_status()
+    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, ref.ACT_GELU_TANH), TOL["fp32"], "pair, K = %d" % K)
+    _assert_close(inputs.to_f64(sw), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)), TOL["bf16"],
+                  "pair swiglu, K = %d" % K)
+    _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], "pair lse, K = %d" % K)
+    want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_RELU)
+    _assert_close(inputs.to_f64(f8), want8, TOL["fp32"], "pair fp8, K = %d" % (2 * K))
+
 
 @pytest.mark.parametrize("M,N,K", [(9, 520, 392), (16, 4096, 512), (129, 257, 72), (300, 520, 200), (600, 1000, 328)])
 @pytest.mark.parametrize("odt", ["fp32", "bf16"])
