@@ -70,7 +70,7 @@ struct DeviceState {
     cudaStream_t s_in = nullptr, s_out = nullptr;
     int max_pairs = -1;              // co-resident 2-CTA clusters of the skinny kernel (-1: not queried yet)
     int max_gemm_pairs = -1;         // the same for the CTA-pair tiled kernel
-    int max_ksplit[3] = {-1, -1, -1};   // co-resident clusters of two / four / eight CTAs of the cluster split-K kernel
+    int max_ksplit[6] = {-1, -1, -1, -1, -1, -1};   // co-resident clusters of two / four / eight CTAs of the cluster split-K kernel (256-, then 128-column tiles)
 };
 
 std::mutex g_mutex;
@@ -442,10 +442,10 @@ int gemm_pairs(DeviceState* d) {
     return d->max_gemm_pairs;
 }
 
-template <int EPI, bool OUT_BF16, int KS>
+template <int EPI, bool OUT_BF16, int KS, int BN = 256>
 int launch_ksplit_ks(int tiles, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
-    using Cfg = KSplitCfg<EPI, KS>;
-    auto kern = gemm_ksplit_kernel<EPI, OUT_BF16, KS>;
+    using Cfg = KSplitCfg<EPI, KS, BN>;
+    auto kern = gemm_ksplit_kernel<EPI, OUT_BF16, KS, BN>;
     if (int rc = ensure_smem_attr(kern, Cfg::SMEM_BYTES)) return rc;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(tiles * KS), 1, 1);
@@ -463,11 +463,16 @@ int launch_ksplit_ks(int tiles, const CUtensorMap& tmA, const CUtensorMap& tmB, 
     q.trace = trace_for(cfg.gridDim.x);
     CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmB2, q));
     g_launches.fetch_add(1);
-    note_kernel("gemm_ksplit_kernel", EPI, KS);
+    note_kernel(BN == 128 ? "gemm_ksplit_kernel (128-column tiles)" : "gemm_ksplit_kernel", EPI, KS);
     return MTMC_OK;
 }
+// ks: cluster size; negative: the same on 128-column tiles (activation epilogues only, clusters of two or four).
 template <int EPI, bool OUT_BF16>
 int launch_ksplit(int ks, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2, const GemmParams& p) {
+    if constexpr (EPI == EPI_ACT) {
+        if (ks == -4) return launch_ksplit_ks<EPI, OUT_BF16, 4, 128>(p.num_tiles, tmA, tmB, tmB2, p);
+        if (ks == -2) return launch_ksplit_ks<EPI, OUT_BF16, 2, 128>(p.num_tiles, tmA, tmB, tmB2, p);
+    }
     if constexpr (EPI != EPI_SWIGLU) {
         if (ks == 8) return launch_ksplit_ks<EPI, OUT_BF16, 8>(p.num_tiles, tmA, tmB, tmB2, p);
     }
@@ -476,12 +481,12 @@ int launch_ksplit(int ks, const CUtensorMap& tmA, const CUtensorMap& tmB, const 
 }
 
 // How many clusters of `ks` CTAs of the cluster split-K kernel the device holds at once (0: none).
-template <int KS>
+template <int KS, int BN = 256>
 int ksplit_clusters_ks(DeviceState* d) {
-    int& cached = d->max_ksplit[KS == 8 ? 2 : (KS == 4 ? 1 : 0)];
+    int& cached = d->max_ksplit[(BN == 128 ? 3 : 0) + (KS == 8 ? 2 : (KS == 4 ? 1 : 0))];
     if (cached < 0) {
-        using Cfg = KSplitCfg<EPI_ACT, KS>;
-        auto kern = gemm_ksplit_kernel<EPI_ACT, true, KS>;
+        using Cfg = KSplitCfg<EPI_ACT, KS, BN>;
+        auto kern = gemm_ksplit_kernel<EPI_ACT, true, KS, BN>;
         int n = 0;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(KS * d->sm_count), 1, 1);
@@ -519,6 +524,27 @@ int pick_ksplit(DeviceState* d, int64_t M, int64_t N, int64_t K, int out_tile_n,
     if (cap >= 4 && k_blocks >= 32 && tiles <= ksplit_clusters_ks<4>(d) && tiles * 4 <= d->sm_count) return 4;
     if (k_blocks >= 16 && tiles <= ksplit_clusters_ks<2>(d)) return 2;
     return 0;
+}
+
+// The same for activation epilogues, which also have 128-column tiles (clusters of two or four; returned as -2 / -4).
+// With as many CTAs at work the cluster is half as large and a CTA sends a third of the bytes through distributed
+// shared memory (48 KiB instead of 112 KiB in place of a cluster of eight), but half of its ring then holds X, so fewer
+// bytes of W are in flight per CTA and a long weight stream runs a tenth slower.  Measured (bias + GELU, 128 rows):
+// 4096 x 4096 14.2 us against 18.5 us, 8192 x 8192 32.1 us against 31.4 us.  So: in place of clusters of eight
+// always, in place of clusters of four when each CTA's walk is short (at most 64 k-blocks in all).
+int pick_ksplit_act(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
+    const int wide = pick_ksplit(d, M, N, K, 256, fp8);
+    if (wide == 0 || t_split_k == 2) return wide;             // (a cap of two is the hook for clusters of two on the wide tiles)
+    const int64_t wide_tiles = ((M + 127) / 128) * ((N + 255) / 256);
+    const int64_t tiles = ((M + 127) / 128) * ((N + 127) / 128);
+    const int64_t k_blocks = (K + (fp8 ? 127 : 63)) / (fp8 ? 128 : 64);
+    if (tiles > d->sm_count / 2) return wide;
+    int narrow = 0;
+    if (k_blocks >= 32 && tiles <= ksplit_clusters_ks<4, 128>(d) && tiles * 4 <= d->sm_count) narrow = 4;
+    else if (k_blocks >= 16 && tiles <= ksplit_clusters_ks<2, 128>(d)) narrow = 2;
+    if (narrow == 0 || tiles * narrow < wide_tiles * wide) return wide;
+    if (wide != 8 && k_blocks > 64) return wide;
+    return -narrow;
 }
 
 // The schedule of a cluster split-K launch: one whole tile per cluster; row-reduction partials are laid out as
@@ -990,12 +1016,13 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     if (rc) return rc;
     if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
 
-    if (const int ks = pick_ksplit(d, M, N, K, 256, false)) {
+    if (const int ks = pick_ksplit_act(d, M, N, K, false)) {
         GemmParams p{};
-        fill_ksplit(p, M, N, K, 256, ks, false);
+        const int bn = ks < 0 ? 128 : 256;
+        fill_ksplit(p, M, N, K, bn, ks < 0 ? -ks : ks, false);
         p.act = act; p.bias = b; p.residual = R; p.out = out; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB;
-        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, 256, ldw))) return rc;
+        if ((rc = encode_bf16_2d(&tmA, X, M, K, 128, ldx)) || (rc = encode_bf16_2d(&tmB, W, N, K, bn, ldw))) return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
         tr.stop();
@@ -1472,13 +1499,14 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     int rc = get_device(&d);
     if (rc) return rc;
     if (use_skinny(M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
-    if (const int ks = pick_ksplit(d, M, N, K, 256, true)) {
+    if (const int ks = pick_ksplit_act(d, M, N, K, true)) {
         GemmParams p{};
-        fill_ksplit(p, M, N, K, 256, ks, true);
+        const int bn = ks < 0 ? 128 : 256;
+        fill_ksplit(p, M, N, K, bn, ks < 0 ? -ks : ks, true);
         p.acc_scale = scale_x * scale_w;
         p.act = act; p.bias = b; p.residual = nullptr; p.out = out; p.lse_partial = nullptr; p.status = d->status;
         CUtensorMap tmA, tmB;
-        if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, 256))) return rc;
+        if ((rc = encode_u8_2d(&tmA, X8, M, K, 128)) || (rc = encode_u8_2d(&tmB, W8, N, K, bn))) return rc;
         TimedRegion tr(d);
         rc = out_dtype == MTMC_OUT_BF16 ? launch_ksplit<EPI_ACT, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI_ACT, false>(ks, tmA, tmB, tmB, p);
         tr.stop();

@@ -20,13 +20,20 @@
 
 namespace mtmc {
 
-template <int EPI, int KS>
+template <int EPI, int KS, int BN_ = 256>
 struct KSplitCfg {
     static_assert(KS == 2 || KS == 4 || KS == 8, "cluster of two, four or eight CTAs (eight: not for SwiGLU, whose tile has four output chunks)");
-    using Tile = TileCfg<EPI, 256>;
-    static constexpr int BN = 256;
-    static constexpr int STAGES = Tile::STAGES;
-    static constexpr int STAGE_BYTES = Tile::STAGE_BYTES;
+    static_assert(BN_ == 256 || (BN_ == 128 && KS <= 4 && EPI != EPI_SWIGLU), "128-column tiles: four accumulator chunks, clusters of two or four");
+    using Tile = TileCfg<EPI, BN_>;
+    static constexpr int BN = BN_;
+    // 128-column tiles: twice the tiles, so half the cluster size for the same number of CTAs and a third of the
+    // bytes to exchange (a CTA of a cluster of two sends 32 KiB where one of a cluster of four sends 96 KiB); each CTA
+    // then walks twice as many, half as heavy k-blocks, and its ring is handed over two k-blocks at a time so that the
+    // thread that issues the MMAs keeps ahead of the weight stream (three stages of 2 x 32 KiB).
+    static constexpr int KB_PER_STAGE = BN_ == 128 ? 2 : 1;
+    static constexpr int SUB_BYTES = Tile::STAGE_BYTES;   // one k-block: X rows, then W rows
+    static constexpr int STAGES = Tile::STAGES / KB_PER_STAGE;
+    static constexpr int STAGE_BYTES = KB_PER_STAGE * SUB_BYTES;
     static constexpr int OUT_TILE_N = Tile::OUT_TILE_N;
     static constexpr int AC = BN / 32;                    // 32-column chunks of the accumulator
     static constexpr int OC = OUT_TILE_N / 32;            // 32-column chunks of the output tile (SwiGLU: half of AC)
@@ -55,11 +62,11 @@ __device__ __forceinline__ void st_shared_cluster_v4(uint32_t caddr, float a, fl
     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(caddr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
 
-template <int EPI, bool OUT_BF16, int KS>
-__global__ void __launch_bounds__(64 + 32 * KSplitCfg<EPI, KS>::EPI_W, 1)
+template <int EPI, bool OUT_BF16, int KS, int BN = 256>
+__global__ void __launch_bounds__(64 + 32 * KSplitCfg<EPI, KS, BN>::EPI_W, 1)
 gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmB2, const GemmParams p) {
-    using Cfg = KSplitCfg<EPI, KS>;
+    using Cfg = KSplitCfg<EPI, KS, BN>;
     using Tile = typename Cfg::Tile;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -124,17 +131,20 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const int n0 = nb * Cfg::OUT_TILE_N;
             constexpr uint32_t b_rows_bytes = static_cast<uint32_t>(Cfg::OUT_TILE_N) * Tile::BK * 2;
             constexpr uint32_t tx = Tile::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes;
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int kb = kb0; kb < kb1; kb += Cfg::KB_PER_STAGE) {
+                const int nsub = (Cfg::KB_PER_STAGE == 2 && kb + 1 < kb1) ? 2 : 1;      // an odd walk ends with half a stage
                 const long long tw = tr.now();
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 7u)) break;
                 tr.add(TR_PROD_STALL, tr.now() - tw);
                 tr.stamp_once(TR_PROD_FIRST_NS);
-                const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
-                const uint32_t b_dst = a_dst + Tile::A_BYTES;
-                mbar_expect_tx(full_bar(s), tx);
-                tma_load_2d(a_dst, &tmA, full_bar(s), kb * p.bk_elems, m0);
-                tma_load_2d(b_dst, &tmB, full_bar(s), kb * p.bk_elems, n0);
-                if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), kb * p.bk_elems, n0);
+                mbar_expect_tx(full_bar(s), tx * nsub);
+                for (int j = 0; j < nsub; ++j) {
+                    const uint32_t a_dst = base + s * Cfg::STAGE_BYTES + j * Cfg::SUB_BYTES;
+                    const uint32_t b_dst = a_dst + Tile::A_BYTES;
+                    tma_load_2d(a_dst, &tmA, full_bar(s), (kb + j) * p.bk_elems, m0);
+                    tma_load_2d(b_dst, &tmB, full_bar(s), (kb + j) * p.bk_elems, n0);
+                    if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), (kb + j) * p.bk_elems, n0);
+                }
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
             tr.stamp(TR_PROD_LAST_NS);
@@ -147,24 +157,30 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             uint32_t ph = 0;
             bool ok = true;
             const uint32_t idesc = p.fp8 ? umma_idesc_e4m3(128, Cfg::BN) : umma_idesc_bf16(128, Cfg::BN);
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int kb = kb0; kb < kb1; kb += Cfg::KB_PER_STAGE) {
+                const int nsub = (Cfg::KB_PER_STAGE == 2 && kb + 1 < kb1) ? 2 : 1;
                 const long long tw = tr.now();
                 if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, STATUS_TIMEOUT_MMA | 7u)) { ok = false; break; }
                 tr.add(TR_MMA_STALL_DATA, tr.now() - tw);
-                tr.add(TR_MMA_KBLOCKS, 1);
+                tr.add(TR_MMA_KBLOCKS, nsub);
                 tr.stamp_once(TR_MMA_FIRST_NS);
                 tc_fence_after();
-                const uint32_t a_src = base + s * Cfg::STAGE_BYTES;
-                const uint64_t a_desc = umma_smem_desc_sw128(a_src);
-                const uint64_t b_desc = umma_smem_desc_sw128(a_src + Tile::A_BYTES);
-                if (p.fp8) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_fp8(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
-                } else {
+                for (int j = 0; j < Cfg::KB_PER_STAGE; ++j) {
+                    if (j < nsub) {
+                        const uint32_t a_src = base + s * Cfg::STAGE_BYTES + j * Cfg::SUB_BYTES;
+                        const uint64_t a_desc = umma_smem_desc_sw128(a_src);
+                        const uint64_t b_desc = umma_smem_desc_sw128(a_src + Tile::A_BYTES);
+                        if (p.fp8) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        umma_bf16(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < 4; ++k)
+                                umma_fp8(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | j | k) != 0 ? 1u : 0u);
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_bf16(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - kb0) | j | k) != 0 ? 1u : 0u);
+                        }
+                    }
                 }
                 umma_commit(empty_bar(s));
                 if (++s == STAGES) { s = 0; ph ^= 1u; }

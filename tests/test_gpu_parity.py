@@ -263,6 +263,34 @@ def test_large_tile_pair_kernel_chosen_for_long_k():
     B.mtmc_check_status()
 
 
+@pytest.mark.parametrize("M,N,K,want", [(100, 1000, 2304, "(128-column tiles)<EPI_ACT, 4>"), (200, 392, 1152, "(128-column tiles)<EPI_ACT, 2>"),
+                                        (128, 4096, 4096, "(128-column tiles)<EPI_ACT, 4>")])
+def test_cluster_split_k_on_128_column_tiles(M, N, K, want):
+    """Activation epilogues take the cluster split-K kernel on 128-column tiles when that halves the cluster: clusters of
+    four and of two, each CTA walking an odd number of k-blocks (9: the ring is handed over two at a time and ends with
+    half a stage), ragged N, fp32 and bf16 outputs, the residual form and E4M3 operands."""
+    li = inputs.linear_inputs(M, N, K, seed=9400 + M)
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    buf, out = _guarded((M, N), torch.float32)
+    B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32", out=out)
+    assert want in B.mtmc_last_kernel_name(), "ran %s" % B.mtmc_last_kernel_name()
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, ref.ACT_GELU_TANH), TOL["fp32"], "narrow split-K %dx%dx%d" % (M, N, K))
+    assert torch.equal(B.mtmc_fused_linear(Xd, Wd, bd, "gelu_tanh", "fp32"), out)          # bit-reproducible
+    R = torch.randn(M, N, generator=torch.Generator().manual_seed(M + N)).bfloat16()
+    res = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), "silu", "bf16")
+    assert want in B.mtmc_last_kernel_name()
+    _assert_close(inputs.to_f64(res), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), ref.ACT_SILU), TOL["bf16"], "narrow split-K residual")
+    fi = inputs.fp8_linear_inputs(M, N, 2 * K, seed=9500 + M)
+    f8 = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, "relu", "bf16")
+    assert want in B.mtmc_last_kernel_name(), "fp8 ran %s" % B.mtmc_last_kernel_name()
+    want8 = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, ref.ACT_RELU)
+    _assert_close(inputs.to_f64(f8), want8, TOL["bf16"], "narrow split-K fp8")
+    B.mtmc_check_status()
+
+
 @pytest.mark.parametrize("K", [40, 136, 264, 456, 520])
 def test_pair_kernel_odd_and_even_k_block_counts(K):
     """The pair kernel hands its ring over two k-blocks at a time; a walk of 1, 3, 5 or 7 k-blocks ends with half a
