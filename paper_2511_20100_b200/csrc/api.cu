@@ -759,7 +759,17 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t M, int64_t N, int64_t K,
     return s;
 }
 
-bool use_skinny(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 31) / 32 <= static_cast<int64_t>(TICKET_BYTES / 4); }
+// The weight-streaming kernel takes at most 64 rows of X.  From 17 rows on only while W is small enough for the pair
+// plan (one band per CTA pair: N <= 128 x pairs): on the ticket plan its time grows with the rows of X (wider MMAs and
+// partials through the workspace; 64 x 14336 x 4096: 40.7 us against 29.2 us on the tiled kernels, 64 x 11008 x 4096:
+// 35.6 against 25.8 us), while at 16 rows and below it is level or ahead.
+int skinny_pairs(DeviceState* d);
+bool use_skinny(DeviceState* d, int64_t M, int64_t N) {
+    if (M > SKINNY_MAX_M || (N + 31) / 32 > static_cast<int64_t>(TICKET_BYTES / 4)) return false;
+    if (M <= 16 || t_split_k > 0) return true;
+    const int pairs = skinny_pairs(d);
+    return pairs > 0 && N <= 128ll * pairs;
+}
 
 // One thread waits, with a one-millisecond limit, on an mbarrier that nothing ever arrives on:
 // the bounded wait gives up, records the status word and the kernel returns normally.
@@ -1014,7 +1024,7 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
+    if (use_skinny(d, M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
 
     if (const int ks = pick_ksplit_act(d, M, N, K, false)) {
         GemmParams p{};
@@ -1411,7 +1421,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     const size_t sk = pairs_possible ? streamk_bytes(gemm_pairs(d)) : 0;
     switch (op) {
         case MTMC_OP_FUSED_LINEAR: {
-            if (!use_skinny(M, N)) return sk;
+            if (!use_skinny(d, M, N)) return sk;
             // the larger of the bf16 and the E4M3 plan: mtmc_fused_linear_fp8 shares this op id
             SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
             SkinnyPlan s8 = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, 128);
@@ -1498,7 +1508,7 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
+    if (use_skinny(d, M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
     if (const int ks = pick_ksplit_act(d, M, N, K, true)) {
         GemmParams p{};
         const int bn = ks < 0 ? 128 : 256;
