@@ -531,7 +531,8 @@ int pick_ksplit(DeviceState* d, int64_t M, int64_t N, int64_t K, int out_tile_n,
 // shared memory (48 KiB instead of 112 KiB in place of a cluster of eight), but half of its ring then holds X, so fewer
 // bytes of W are in flight per CTA and a long weight stream runs a tenth slower.  Measured (bias + GELU, 128 rows):
 // 4096 x 4096 14.2 us against 18.5 us, 8192 x 8192 32.1 us against 31.4 us.  So: in place of clusters of eight
-// always, in place of clusters of four when each CTA's walk is short (at most 64 k-blocks in all).
+// always, in place of clusters of four when each CTA's walk is short (at most 64 k-blocks in all), and whenever they
+// put more CTAs to work.
 int pick_ksplit_act(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     const int wide = pick_ksplit(d, M, N, K, 256, fp8);
     if (wide == 0 || t_split_k == 2) return wide;             // (a cap of two is the hook for clusters of two on the wide tiles)
@@ -543,6 +544,7 @@ int pick_ksplit_act(DeviceState* d, int64_t M, int64_t N, int64_t K, bool fp8) {
     if (k_blocks >= 32 && tiles <= ksplit_clusters_ks<4, 128>(d) && tiles * 4 <= d->sm_count) narrow = 4;
     else if (k_blocks >= 16 && tiles <= ksplit_clusters_ks<2, 128>(d)) narrow = 2;
     if (narrow == 0 || tiles * narrow < wide_tiles * wide) return wide;
+    if (tiles * narrow > wide_tiles * wide) return -narrow;   // more CTAs streaming W (e.g. where no cluster of eight can be placed)
     if (wide != 8 && k_blocks > 64) return wide;
     return -narrow;
 }
@@ -636,6 +638,7 @@ void fill_ksplit(GemmParams& p, int64_t M, int64_t N, int64_t K, int out_tile_n,
     fill_tiling(p, M, N, K, out_tile_n, 1, false, 128, fp8);
     p.n_full = 0;
     p.tail_split = ks;
+    p.early_w = t_static_weights ? 1 : 0;
 }
 
 // Stream-K schedule of the pair kernel (see gemm_pair.cuh): the last full wave plus the remainder (everything, when
@@ -759,16 +762,20 @@ SkinnyPlan plan_skinny(int sm_count, int pairs, int64_t M, int64_t N, int64_t K,
     return s;
 }
 
-// The weight-streaming kernel takes at most 64 rows of X.  From 17 rows on only while W is small enough for the pair
-// plan (one band per CTA pair: N <= 128 x pairs): on the ticket plan its time grows with the rows of X (wider MMAs and
-// partials through the workspace; 64 x 14336 x 4096: 40.7 us against 29.2 us on the tiled kernels, 64 x 11008 x 4096:
-// 35.6 against 25.8 us), while at 16 rows and below it is level or ahead.
+// The weight-streaming kernel takes at most 64 rows of X.  skinny_possible: the shape fits it at all.  prefer_skinny: it is
+// the first choice -- when W has at least 64 rows per CTA pair (shorter bands leave its 128-lane MMAs mostly empty and its
+// CTAs bound by the k-blocks they issue, not by the bytes they stream: 16 x 4096 x 14336 34.7 us against 27.1 us on the
+// cluster split-K kernel, 64 x 1024 x 4096 30.8 against 10.9 us) and, from 17 rows of X on, only on its pair plan
+// (N <= 128 x pairs; on the ticket plan its time grows with the rows of X: 64 x 14336 x 4096 40.7 against 29.2 us).
+// Shapes it is not preferred for go to the cluster split-K kernel when that applies and come back here otherwise.
 int skinny_pairs(DeviceState* d);
-bool use_skinny(DeviceState* d, int64_t M, int64_t N) {
-    if (M > SKINNY_MAX_M || (N + 31) / 32 > static_cast<int64_t>(TICKET_BYTES / 4)) return false;
-    if (M <= 16 || t_split_k > 0) return true;
+bool skinny_possible(int64_t M, int64_t N) { return M <= SKINNY_MAX_M && (N + 31) / 32 <= static_cast<int64_t>(TICKET_BYTES / 4); }
+bool prefer_skinny(DeviceState* d, int64_t M, int64_t N) {
+    if (!skinny_possible(M, N)) return false;
+    if (t_split_k > 0) return true;
     const int pairs = skinny_pairs(d);
-    return pairs > 0 && N <= 128ll * pairs;
+    if (pairs <= 0) return M <= 16;
+    return N >= 64ll * pairs && (N <= 128ll * pairs || M <= 16);
 }
 
 // One thread waits, with a one-millisecond limit, on an mbarrier that nothing ever arrives on:
@@ -1024,7 +1031,7 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
     DeviceState* d = nullptr;
     rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(d, M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
+    if (prefer_skinny(d, M, N)) return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
 
     if (const int ks = pick_ksplit_act(d, M, N, K, false)) {
         GemmParams p{};
@@ -1038,6 +1045,8 @@ int fused_linear_impl(const void* X, const void* W, const float* b, const void* 
         tr.stop();
         return rc;
     }
+    if (skinny_possible(M, N) && t_tile_n == 0 && t_cta_pair <= 0)      // no cluster split-K for the shape (short K, too many tiles): stream the weights after all
+        return run_skinny(d, X, W, b, R, M, N, K, act, out_dtype, out, false, 1.0f, ldx, ldw, ldo);
     if (use_big(d, M, N, K, false)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512);
@@ -1421,7 +1430,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     const size_t sk = pairs_possible ? streamk_bytes(gemm_pairs(d)) : 0;
     switch (op) {
         case MTMC_OP_FUSED_LINEAR: {
-            if (!use_skinny(d, M, N)) return sk;
+            if (!skinny_possible(M, N)) return sk;
             // the larger of the bf16 and the E4M3 plan: mtmc_fused_linear_fp8 shares this op id
             SkinnyPlan s = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K);
             SkinnyPlan s8 = plan_skinny(d->sm_count, skinny_pairs(d), M, N, K, 128);
@@ -1508,7 +1517,7 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    if (use_skinny(d, M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
+    if (prefer_skinny(d, M, N)) return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
     if (const int ks = pick_ksplit_act(d, M, N, K, true)) {
         GemmParams p{};
         const int bn = ks < 0 ? 128 : 256;
@@ -1522,6 +1531,8 @@ int mtmc_fused_linear_fp8(const void* X8, const void* W8, const float* b, float 
         tr.stop();
         return rc;
     }
+    if (skinny_possible(M, N) && t_tile_n == 0 && t_cta_pair <= 0)
+        return run_skinny(d, X8, W8, b, nullptr, M, N, K, act, out_dtype, out, true, scale_x * scale_w);
     if (use_big(d, M, N, K, true)) {
         GemmParams p{};
         fill_tiling(p, M, N, K, 256, gemm_pairs(d), false, 512, true);

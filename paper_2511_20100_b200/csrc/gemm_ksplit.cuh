@@ -102,6 +102,27 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         tma_prefetch_desc(&tmA);
         tma_prefetch_desc(&tmB);
         if (EPI == EPI_SWIGLU) tma_prefetch_desc(&tmB2);
+        // Static weights: the W loads of the first ring go out now, before the cluster has met and before the wait on the
+        // preceding kernel -- they touch only this CTA's shared memory and barriers, which this thread has just initialised,
+        // and memory that nothing in flight writes.  The producer loop below adds the X loads of those stages.
+        if (p.early_w) {
+            int mb_e, nb_e;
+            tile_coords(p, tile, mb_e, nb_e);
+            const int kb0_e = static_cast<int>(static_cast<long long>(rank) * p.k_blocks / KS);
+            const int kb1_e = static_cast<int>(static_cast<long long>(rank + 1) * p.k_blocks / KS);
+            constexpr uint32_t b_rows_bytes_e = static_cast<uint32_t>(Cfg::OUT_TILE_N) * Tile::BK * 2;
+            constexpr uint32_t tx_e = Tile::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes_e;
+            int s = 0;
+            for (int kb = kb0_e; kb < kb1_e && s < STAGES; kb += Cfg::KB_PER_STAGE, ++s) {
+                const int nsub = (Cfg::KB_PER_STAGE == 2 && kb + 1 < kb1_e) ? 2 : 1;
+                mbar_expect_tx(full_bar(s), tx_e * nsub);
+                for (int j = 0; j < nsub; ++j) {
+                    const uint32_t b_dst = base + s * Cfg::STAGE_BYTES + j * Cfg::SUB_BYTES + Tile::A_BYTES;
+                    tma_load_2d(b_dst, &tmB, full_bar(s), (kb + j) * p.bk_elems, nb_e * Cfg::OUT_TILE_N);
+                    if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes_e, &tmB2, full_bar(s), (kb + j) * p.bk_elems, nb_e * Cfg::OUT_TILE_N);
+                }
+            }
+        }
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), Cfg::TMEM_COLS);
@@ -131,19 +152,24 @@ gemm_ksplit_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             const int n0 = nb * Cfg::OUT_TILE_N;
             constexpr uint32_t b_rows_bytes = static_cast<uint32_t>(Cfg::OUT_TILE_N) * Tile::BK * 2;
             constexpr uint32_t tx = Tile::A_BYTES + (EPI == EPI_SWIGLU ? 2u : 1u) * b_rows_bytes;
+            int begun = p.early_w ? STAGES : 0;          // stages whose bytes are announced and whose W loads are on their way
             for (int kb = kb0; kb < kb1; kb += Cfg::KB_PER_STAGE) {
                 const int nsub = (Cfg::KB_PER_STAGE == 2 && kb + 1 < kb1) ? 2 : 1;      // an odd walk ends with half a stage
+                const bool early = begun > 0;
+                if (early) --begun;
                 const long long tw = tr.now();
-                if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 7u)) break;
+                if (!early && !mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 7u)) break;
                 tr.add(TR_PROD_STALL, tr.now() - tw);
                 tr.stamp_once(TR_PROD_FIRST_NS);
-                mbar_expect_tx(full_bar(s), tx * nsub);
+                if (!early) mbar_expect_tx(full_bar(s), tx * nsub);
                 for (int j = 0; j < nsub; ++j) {
                     const uint32_t a_dst = base + s * Cfg::STAGE_BYTES + j * Cfg::SUB_BYTES;
                     const uint32_t b_dst = a_dst + Tile::A_BYTES;
                     tma_load_2d(a_dst, &tmA, full_bar(s), (kb + j) * p.bk_elems, m0);
-                    tma_load_2d(b_dst, &tmB, full_bar(s), (kb + j) * p.bk_elems, n0);
-                    if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), (kb + j) * p.bk_elems, n0);
+                    if (!early) {
+                        tma_load_2d(b_dst, &tmB, full_bar(s), (kb + j) * p.bk_elems, n0);
+                        if (EPI == EPI_SWIGLU) tma_load_2d(b_dst + b_rows_bytes, &tmB2, full_bar(s), (kb + j) * p.bk_elems, n0);
+                    }
                 }
                 if (++s == STAGES) { s = 0; ph ^= 1u; }
             }

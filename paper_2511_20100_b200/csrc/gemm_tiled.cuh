@@ -55,6 +55,8 @@ struct GemmParams {
                           // (max, index bits) for EPI_ROWMAX
     const long long* targets;   // [M] target column per row (EPI_XENT)
     float* target_logit;        // [M] logit at the target column, written by the one piece that holds it (EPI_XENT)
+    int early_w;          // 1: W is not written by any work still in flight (mtmc_set_static_weights), so the cluster split-K kernel
+                          // sends out its first ring of W loads before it waits for the preceding kernel (X, bias, outputs still wait)
     uint32_t* status;     // device status word
     unsigned long long* trace;   // per-CTA trace records (-DMTMC_TRACE builds, mtmc_set_trace), else null
     // Stream-K schedule of the CTA-pair kernel (gemm_pair.cuh): tiles [0, sk_first_tile) are dealt round-robin; the

@@ -1101,7 +1101,10 @@ def test_skinny_result_independent_of_split(split_k):
 
 
 def test_skinny_with_caller_workspace():
+    """The weight-streaming kernel's ticket plan (forced: a shape this small goes to the cluster split-K kernel by itself)
+    with partials and tickets in a caller's workspace; too small a workspace is refused before anything is launched."""
     li = inputs.linear_inputs(16, 512, 2048, seed=45)
+    B.mtmc_set_tuning(split_k=4)
     need = B.mtmc_workspace_bytes("fused_linear", 16, 512, 2048)
     assert need > 0
     ws = torch.full((need + 256,), 255, dtype=torch.uint8, device="cuda")   # dirty on purpose
@@ -1109,6 +1112,7 @@ def test_skinny_with_caller_workspace():
     B.mtmc_set_workspace(ws[off:off + need])
     try:
         out = B.mtmc_fused_linear(li.X.cuda(), li.W.cuda(), li.b.cuda(), "gelu_tanh", "bf16")
+        assert "ticket plan" in B.mtmc_last_kernel_name()
         B.mtmc_check_status()
         with pytest.raises(B.MtmcError) as e:
             B.mtmc_set_workspace(ws[off:off + 1024])
@@ -1116,6 +1120,7 @@ def test_skinny_with_caller_workspace():
         assert e.value.status == B.ERR_WORKSPACE
     finally:
         B.mtmc_set_workspace(None)
+        B.mtmc_set_tuning()
     want = ref.fused_linear(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), ref.ACT_GELU_TANH)
     _assert_close(inputs.to_f64(out), want, TOL["bf16"], "caller workspace")
 
