@@ -79,12 +79,13 @@ extern "C" {
  * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
  * the bias add and activation happen in fp32 on the fp32 accumulator, with no
  * intermediate rounding.)  X, W bf16; b fp32 or NULL; out fp32 or bf16 [M,N]
- * according to out_dtype.  Shapes with M <= 64 (decode batches) take the split-K
- * weight-streaming path (HBM-bound); problems of at most half a wave of 128 x 256
- * tiles with a long K a cluster split-K kernel (2, 4 or 8 CTAs per tile, reduction
- * through distributed shared memory); all others the tiled tensor-core kernels
- * (CTA pairs on 256 x 256 or 512 x 256 tiles for M >= 512 and N >= 256, single
- * CTAs otherwise).  Needs workspace only on the ticketed variant of the
+ * according to out_dtype.  Shapes with M <= 64 (decode batches) whose W has at
+ * least 64 rows per CTA pair take the split-K weight-streaming path (HBM-bound);
+ * problems of at most half a wave of 128 x 256 (or 128 x 128) tiles with a long K a
+ * cluster split-K kernel (2, 4 or 8 CTAs per tile, reduction through distributed
+ * shared memory); all others the tiled tensor-core kernels (CTA pairs on 256 x 256
+ * tiles from M > 128 and N >= 256 on, 512 x 256 tiles for very long K, single CTAs
+ * otherwise).  Needs workspace only on the ticketed variant of the
  * weight-streaming path (few rows of W, or a forced split; see mtmc_workspace_bytes). */
 int mtmc_fused_linear(const void* X, const void* W, const float* b,
                       int64_t M, int64_t N, int64_t K, int act, int out_dtype, void* out);

@@ -1426,7 +1426,7 @@ size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     // An upper bound over the kernels the library may pick for the shape under the current tuning: the stream-K
     // region of the pair kernel wherever CTA pairs are possible (whether or not this shape ends up on that schedule).
     const bool pairs_possible = gemm_pairs(d) > 0 && t_stream_k > 0 && t_cta_pair >= 0 && t_tile_n != 128 &&
-                                (t_cta_pair > 0 || (M >= 512 && N >= 256));
+                                (t_cta_pair > 0 || (M > 128 && N >= 256));
     const size_t sk = pairs_possible ? streamk_bytes(gemm_pairs(d)) : 0;
     switch (op) {
         case MTMC_OP_FUSED_LINEAR: {
