@@ -1002,10 +1002,11 @@ def test_stream_k_other_epilogues(M, N, K):
     _assert_close(inputs.to_f64(r["fp8"]), want8, TOL["bf16"], "stream-K fp8")
 
 
-def test_stream_k_with_caller_workspace():
-    """The accumulator parts and flag words in a caller's workspace of exactly mtmc_workspace_bytes, canaries around it."""
-    M, N, K = 2304, 2304, 328
-    li = inputs.linear_inputs(M, N, K, seed=8800)
+@pytest.mark.parametrize("M,N,K", [(2304, 2304, 328), (300, 2304, 2048)])
+def test_stream_k_with_caller_workspace(M, N, K):
+    """The accumulator parts and flag words in a caller's workspace of exactly mtmc_workspace_bytes, canaries around it
+    (also below 512 rows, where the pair kernel now starts)."""
+    li = inputs.linear_inputs(M, N, K, seed=8800 + M)
     Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
 
     def run():
