@@ -364,12 +364,13 @@ int mtmc_set_schedule(int stream_k);
 /* Static weights (thread-local, default 0 = off).  With enabled != 0 the caller promises, for
  * the calls that follow on this thread, that no work still in flight on the device writes
  * the W operand (the weights of a deployed model: written once, long before).  The
- * weight-streaming path (M <= 64) then issues its first ring of W loads before it waits
+ * weight-streaming path (M <= 64) and the cluster split-K kernel (decode and small
+ * prefill batches) then issue their first ring of W loads before they wait
  * for the preceding kernel on the stream to finish, so the start of the weight stream
  * overlaps that kernel's tail; X, the bias, the residual and every output still wait.
  * Results are the same bits as with the switch off.  If the promise is broken (W produced
  * by the kernel just before) the call may read stale weights.  The paper has no counterpart;
- * it follows its "pipeline" principle across a kernel boundary.  The tiled kernels ignore it. */
+ * it follows its "pipeline" principle across a kernel boundary.  The other tiled kernels ignore it. */
 int mtmc_set_static_weights(int enabled);
 
 /* Library version: major * 10000 + minor * 100 + patch. */
