@@ -1044,10 +1044,13 @@ def test_skinny_small(M, N, K, odt):
 
 
 @pytest.mark.parametrize("M,N,K,split_k", [(16, 8192, 8192, 0), (1, 4096, 1024, 0), (64, 9472, 136, 0), (5, 300, 2048, 0),
-                                           (16, 512, 1024, 4), (33, 2400, 1096, 0), (7, 128, 64, 0)])
+                                           (16, 512, 1024, 4), (33, 2400, 1096, 0), (7, 128, 64, 0),
+                                           (128, 4096, 4096, 0), (100, 8192, 4160, 0), (200, 1000, 1152, 0)])
 def test_skinny_static_weights_same_bits(M, N, K, split_k):
-    """With the static-weights promise the first ring of W loads goes out before the wait on the preceding kernel:
-    same bits as without it, launch after launch (each launch follows one of this library's own kernels)."""
+    """With the static-weights promise the first ring of W loads goes out before the wait on the preceding kernel, in the
+    weight-streaming kernel and in the cluster split-K kernel (the last three shapes and the short-band ones: 128- and
+    256-column tiles, an odd walk): same bits as without it, launch after launch (each launch follows one of this
+    library's own kernels)."""
     li = inputs.linear_inputs(M, N, K, seed=4100 + M + N)
     Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
     B.mtmc_set_tuning(split_k=split_k)
