@@ -2,7 +2,7 @@
 //
 // A pair owns a 256 x 256 output tile (256 x 128 for SwiGLU).  Each CTA loads its own 128
 // rows of X and its own half of the W rows of the tile, so a k-block is 32 KiB instead of
-// 48 KiB (a ring of six k-blocks, handed over two at a time, instead of four) and a third less L2 -> shared-memory traffic per
+// 48 KiB (a ring of six k-blocks, handed to the MMA issuer two at a time and back to the producer one by one, instead of four) and a third less L2 -> shared-memory traffic per
 // FLOP.  The even CTA issues tcgen05.mma.cta_group::2 (M = 256) for both; each CTA keeps the
 // accumulator of its own 128 rows in its own TMEM and runs its own epilogue.
 //
@@ -44,7 +44,7 @@ struct PairCfg {
     static constexpr int STAGES = 3;
     static constexpr int OUT_TILE_N = (EPI == EPI_SWIGLU) ? BN / 2 : BN;
     static constexpr int TMEM_COLS = 2 * BN;
-    static constexpr int NUM_BARRIERS = 2 * STAGES + 4;
+    static constexpr int NUM_BARRIERS = STAGES + KB_PER_STAGE * STAGES + 4;   // full per stage, empty per k-block, accumulators
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP + NUM_BARRIERS * 8 + 16 + 1024;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
 };
@@ -222,9 +222,11 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t epi_stage_base = base + STAGES * Cfg::STAGE_BYTES;        // warp-private store staging
     const uint32_t bar_base = epi_stage_base + EPI_WARPS * EPI_STAGE_BYTES_PER_WARP;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-    auto accf_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + b); };
-    auto acce_bar = [&](int b) { return bar_base + 8u * (2 * STAGES + 2 + b); };
+    // a stage's two k-blocks are handed to the MMA issuer together (one `full` barrier, two arrivals) but handed back
+    // one by one (an `empty` barrier each): the first is refilled while the second is still being multiplied
+    auto empty_bar = [&](int s, int j) { return bar_base + 8u * (STAGES + Cfg::KB_PER_STAGE * s + j); };
+    auto accf_bar = [&](int b) { return bar_base + 8u * ((1 + Cfg::KB_PER_STAGE) * STAGES + b); };
+    auto acce_bar = [&](int b) { return bar_base + 8u * ((1 + Cfg::KB_PER_STAGE) * STAGES + 2 + b); };
     uint8_t* ctrl = smem_raw + (bar_base - raw_addr) + 8 * Cfg::NUM_BARRIERS;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(ctrl + 4);
@@ -238,7 +240,10 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         tr.stamp(TR_START_NS);
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full_bar(s), Cfg::KB_PER_STAGE);           // one arrival (with its bytes) per k-block
+            for (int j = 0; j < Cfg::KB_PER_STAGE; ++j) mbar_init(empty_bar(s, j), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 2 * EPI_WARPS); }   // every epilogue warp of both CTAs
         *abort_flag = 0u;
         fence_barrier_init();
@@ -285,22 +290,26 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 int kx = w.kb0 * p.bk_elems;                             // K coordinate of the next k-block
                 for (int kb = w.kb0; kb < w.kb1; kb += Cfg::KB_PER_STAGE, kx += Cfg::KB_PER_STAGE * p.bk_elems) {
                     const bool two = kb + 1 < w.kb1;                     // an odd walk ends with half a stage
-                    const long long tw = tr.now();
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 3u)) { ok = false; break; }
-                    t_stall += tr.now() - tw;                 // trace totals live in registers and are written once, after the loop
-                    if (t_first) { tr.stamp(TR_PROD_FIRST_NS); t_first = false; }
-                    // loads first, bookkeeping after: the time from "slot free" to "load issued" is on the ring's
-                    // critical path (a transaction count may run ahead of its expect_tx within a phase)
-                    const uint32_t a_dst = base + s * Cfg::STAGE_BYTES;
                     const uint32_t full0 = full0_base + 8u * s;
-                    if (!MTMC_CHECK(a_dst + Cfg::SUB_BYTES + cta_bytes <= epi_stage_base && (kx & 7) == 0 && m0 >= 0 && n_row0 >= 0, p.status, 4u)) { ok = false; break; }
-                    tma_load_2d_pair(a_dst, &tmA, full0, kx, m0);
-                    tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kx, n_row0);
-                    if (two) {
-                        tma_load_2d_pair(a_dst + Cfg::SUB_BYTES, &tmA, full0, kx + p.bk_elems, m0);
-                        tma_load_2d_pair(a_dst + Cfg::SUB_BYTES + Cfg::A_BYTES, mapB, full0, kx + p.bk_elems, n_row0);
+#pragma unroll
+                    for (int j = 0; j < Cfg::KB_PER_STAGE; ++j) {
+                        const long long tw = tr.now();
+                        if (!mbar_wait(empty_bar(s, j), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_PRODUCER | 3u)) { ok = false; break; }
+                        t_stall += tr.now() - tw;                 // trace totals live in registers and are written once, after the loop
+                        if (t_first) { tr.stamp(TR_PROD_FIRST_NS); t_first = false; }
+                        if (j == 0 || two) {
+                            // loads first, bookkeeping after: the time from "slot free" to "load issued" is on the ring's
+                            // critical path (a transaction count may run ahead of its expect_tx within a phase)
+                            const uint32_t a_dst = base + s * Cfg::STAGE_BYTES + j * Cfg::SUB_BYTES;
+                            if (!MTMC_CHECK(a_dst + cta_bytes <= epi_stage_base && (kx & 7) == 0 && m0 >= 0 && n_row0 >= 0, p.status, 4u)) { ok = false; break; }
+                            tma_load_2d_pair(a_dst, &tmA, full0, kx + j * p.bk_elems, m0);
+                            tma_load_2d_pair(a_dst + Cfg::A_BYTES, mapB, full0, kx + j * p.bk_elems, n_row0);
+                            if (rank == 0) mbar_expect_tx(full_bar(s), 2u * cta_bytes);     // both CTAs' bytes of this k-block
+                        } else if (rank == 0) {
+                            mbar_arrive(full_bar(s));                                       // the missing half of an odd walk's last stage
+                        }
                     }
-                    if (rank == 0) mbar_expect_tx(full_bar(s), (two ? 4u : 2u) * cta_bytes);     // both CTAs' bytes
+                    if (!ok) break;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -356,8 +365,8 @@ gemm_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                     umma_bf16_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, ((kb - w.kb0) | j | k) != 0 ? 1u : 0u);
                             }
                         }
+                        umma_commit_pair(empty_bar(s, j), 3);    // frees this k-block's half of the stage in both CTAs (also the unused half of an odd walk's end)
                     }
-                    umma_commit_pair(empty_bar(s), 3);           // frees the stage in both CTAs
                     t_issue += tr.now() - tw;
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
