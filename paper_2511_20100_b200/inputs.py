@@ -44,6 +44,8 @@ EXTRA_CONFIGS = {
     # C2 and the 8192-cube with block-scaled E4M3 operands (MXFP8: one power-of-two scale per 32 elements of K)
     "X8": dict(op="fused_linear_mxfp8", M=4096, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=1),
     "X9": dict(op="fused_linear_mxfp8", M=8192, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=6),
+    # a decode batch against a 4096-wide layer: 32 tiles of 128 x 128, clusters of four CTAs per tile split along K
+    "X10": dict(op="fused_linear", M=128, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=8),
 }
 
 
