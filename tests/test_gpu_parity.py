@@ -1273,6 +1273,68 @@ def test_host_pointer_calls_without_waiting():
                   TOL["bf16"], "pipelined swiglu_host")
 
 
+def test_random_shapes_long_k_schedules_and_switches():
+    """Seeded sweep of 160 shapes with K up to 4480 (the cluster split-K kernels on 256- and 128-column tiles, odd and
+    even k-walks on the pair kernels' two-k-block ring), row counts on both sides of every kernel boundary, the
+    stream-K schedule and the static-weights switch on and off, bf16 and E4M3 operands, against the oracle."""
+    rng = np.random.default_rng(20251126)
+    tunings = [dict(), dict(), dict(cta_pair=1), dict(cta_pair=2), dict(cta_pair=-1), dict(split_k=1), dict(tile_n=128)]
+    seen = set()
+    for case in range(160):
+        M = int([rng.integers(1, 65), rng.integers(65, 300), rng.integers(257, 700), 128, 256, 512][case % 6])
+        N = 8 * int(rng.integers(1, 150))
+        K = 8 * int([rng.integers(1, 40), rng.integers(40, 560), 64, 128, 256, 264][int(rng.integers(0, 6))])
+        op = ["linear", "swiglu", "lse", "fp8", "linear", "residual", "rowmax"][int(rng.integers(0, 7))]
+        tune = tunings[int(rng.integers(0, len(tunings)))]
+        sk = int(rng.integers(0, 4) == 0)
+        static = bool(rng.integers(0, 2))
+        act = ["none", "relu", "gelu_tanh", "silu"][int(rng.integers(0, 4))]
+        odt = "bf16" if rng.integers(0, 2) else "fp32"
+        what = "case %d: %s %dx%dx%d %s %s %r stream-K %d static %d" % (case, op, M, N, K, act, odt, tune, sk, static)
+        B.mtmc_set_tuning(**tune)
+        B.mtmc_set_schedule(sk)
+        B.mtmc_set_static_weights(static)
+        try:
+            if op == "swiglu":
+                si = inputs.swiglu_inputs(M, N, K, seed=9800 + case)
+                got = B.mtmc_swiglu(si.X.cuda(), si.Wg.cuda(), si.Wu.cuda())
+                _assert_close(inputs.to_f64(got), ref.swiglu(inputs.bf16_bits(si.X), inputs.bf16_bits(si.Wg), inputs.bf16_bits(si.Wu)),
+                              TOL["bf16"], what)
+            elif op == "fp8":
+                K8 = (K + 15) // 16 * 16
+                fi = inputs.fp8_linear_inputs(M, N, K8, seed=9800 + case)
+                got = B.mtmc_fused_linear_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, act, odt)
+                want = ref.fused_linear_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b), fi.scale_x, fi.scale_w, B.ACT[act])
+                _assert_close(inputs.to_f64(got), want, TOL[odt], what)
+            else:
+                li = inputs.linear_inputs(M, N, K, seed=9800 + case)
+                Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+                Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+                if op == "linear":
+                    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+                    B.mtmc_fused_linear(Xd, Wd, bd, act, odt, out=out)
+                    B.mtmc_check_status()
+                    assert _canaries_intact(buf, M * N), what
+                    _assert_close(inputs.to_f64(out), ref.fused_linear(Xb, Wb, bf, B.ACT[act]), TOL[odt], what)
+                elif op == "residual":
+                    R = torch.randn(M, N, generator=torch.Generator().manual_seed(case)).bfloat16()
+                    got = B.mtmc_fused_linear_residual(Xd, Wd, bd, R.cuda(), act, "bf16")
+                    _assert_close(inputs.to_f64(got), ref.fused_linear_residual(Xb, Wb, bf, inputs.bf16_bits(R), B.ACT[act]), TOL["bf16"], what)
+                elif op == "lse":
+                    _assert_close(inputs.to_f64(B.mtmc_linear_lse(Xd, Wd, bd)), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], what)
+                else:
+                    mx, arg = B.mtmc_linear_rowmax(Xd, Wd, bd)
+                    _check_rowmax(li, mx, arg, what)
+            B.mtmc_check_status()
+            seen.add(B.mtmc_last_kernel_name().split("<")[0])
+        finally:
+            B.mtmc_set_tuning()
+            B.mtmc_set_schedule(0)
+            B.mtmc_set_static_weights(False)
+    for family in ("gemm_tiled_kernel", "gemm_pair_kernel", "gemm_big_kernel", "gemm_ksplit_kernel", "gemm_ksplit_kernel (128-column tiles)"):
+        assert family in seen, "the sweep never reached %s (ran %r)" % (family, sorted(seen))
+
+
 def test_random_shapes_all_operators_and_kernels():
     """Seeded sweep: 60 random shapes (ragged M, N, K; K a multiple of 8), each through a randomly chosen operator and
     kernel choice (automatic, 256 x 256 pairs, 512 x 256 pairs, single-CTA tiles of either width), against the oracle."""
