@@ -28,6 +28,8 @@
 //                   (the paper's own example of a fusion action joins a linear with a row max,
 //                   section "Training Process")
 //   cross entropy:  loss[m] = lse[m] - z[m][target[m]]   (softmax cross entropy of the logits row)
+//   row softmax  :  P[m][n] = exp(z[m][n] - max_n' z[m][n']) / sum_n' exp(z[m][n'] - max), the normalised
+//                   form of the same row reduction
 //
 // Layouts: X [M,K], W [N,K], out [M,N]; all dense row-major.  X/W arrive as bf16 bit
 // patterns (uint16_t: the upper half of an IEEE-754 binary32), b as binary32 and
@@ -37,7 +39,8 @@
 // Pins (see tests/test_oracle_pins.py): exact rational brute force on tiny
 // integer-valued problems, W = I, X = 0, K-split additivity, permutation and
 // scaling laws, closed-form activation and logsumexp values, act(z)-act(-z) = z,
-// lse(z+c) = lse(z)+c, softmax rows summing to one, and torch fp64 library
+// lse(z+c) = lse(z)+c, softmax rows summing to one, softmax of log-integers as exact
+// ratios, the two-class softmax as the logistic function, and torch fp64 library
 // routines.  No function here is "parity unpinned".
 #include <cmath>
 #include <cstdint>
@@ -330,6 +333,48 @@ int mtmc_ref_linear_lse_rows(const uint16_t* X, const uint16_t* W, const float* 
     }
     return 0;
 }
+
+// One row of logits -> its softmax by the definition with the maximum taken out first:
+// p[n] = exp(z[n] - max) / sum_n' exp(z[n'] - max), the sum in ascending n'.
+static void softmax_of_row(const double* z, int64_t N, double* p) {
+    double mx = z[0];
+    for (int64_t n = 1; n < N; ++n) mx = z[n] > mx ? z[n] : mx;
+    double s = 0.0;
+    for (int64_t n = 0; n < N; ++n) { p[n] = std::exp(z[n] - mx); s += p[n]; }
+    for (int64_t n = 0; n < N; ++n) p[n] /= s;
+}
+
+// P[m][n] = softmax over n of z[m][n] = X.W^T + b, all M rows.
+int mtmc_ref_linear_softmax(const uint16_t* X, const uint16_t* W, const float* b,
+                            int64_t M, int64_t N, int64_t K, double* P) {
+    if (!X || !W || !P || M <= 0 || N <= 0 || K <= 0) return 1;
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n) z[n] = preact(X, W, b, K, m, n);
+        softmax_of_row(z.data(), N, P + m * N);
+    });
+    return 0;
+}
+
+// The same for R listed rows only: P[r][·] belongs to row rows[r].
+int mtmc_ref_linear_softmax_rows(const uint16_t* X, const uint16_t* W, const float* b,
+                                 int64_t M, int64_t N, int64_t K,
+                                 const int64_t* rows, int64_t R, double* P) {
+    if (!X || !W || !P || !rows || M <= 0 || N <= 0 || K <= 0) return 1;
+    for (int64_t r = 0; r < R; ++r)
+        if (rows[r] < 0 || rows[r] >= M) return 1;
+    for (int64_t r = 0; r < R; ++r) {
+        std::vector<double> z(static_cast<size_t>(N));
+        double* zp = z.data();
+        int64_t m = rows[r];
+        parallel_for(N, [=](int64_t n) { zp[n] = preact(X, W, b, K, m, n); });
+        softmax_of_row(zp, N, P + r * N);
+    }
+    return 0;
+}
+
+// Softmax of a plain vector (for the closed-form pins).
+void mtmc_ref_softmax_vector(const double* z, int64_t N, double* p) { softmax_of_row(z, N, p); }
 
 // mx[m] = max_n z[m][n]; arg[m] = lowest column index attaining it.  arg may be null.
 int mtmc_ref_linear_rowmax(const uint16_t* X, const uint16_t* W, const float* b,

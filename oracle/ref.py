@@ -63,6 +63,10 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_linear_lse_rows.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
         L.mtmc_ref_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
         L.mtmc_ref_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
+        L.mtmc_ref_linear_softmax.argtypes = [vp, vp, vp, i64, i64, i64, vp]
+        L.mtmc_ref_linear_softmax_rows.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
+        L.mtmc_ref_softmax_vector.argtypes = [vp, i64, vp]
+        L.mtmc_ref_softmax_vector.restype = None
         L.mtmc_ref_lse_vector.argtypes = [vp, i64]
         L.mtmc_ref_lse_vector.restype = dbl
         L.mtmc_ref_compare.argtypes = [vp, vp, i64, dbl, dbl, vp]
@@ -360,6 +364,37 @@ def linear_cross_entropy_fp8(X, W, b, scale_x: float, scale_w: float, target):
                                                    target.ctypes.data, M, N, K, loss.ctypes.data, lse.ctypes.data),
            "mtmc_ref_linear_cross_entropy_fp8")
     return loss, lse
+
+
+def linear_softmax(X, W, b) -> np.ndarray:
+    """softmax over n of X.W^T + b, [M,N] float64."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    P = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_linear_softmax(X.ctypes.data, W.ctypes.data, bp, M, N, K, P.ctypes.data), "mtmc_ref_linear_softmax")
+    return P
+
+
+def linear_softmax_rows(X, W, b, rows) -> np.ndarray:
+    """The listed rows of linear_softmax, [len(rows), N] float64."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _bf16(X, (M, K)), _bf16(W, (N, K))
+    bk, bp = _bias(b, N)
+    rows = _idx(rows)
+    P = np.empty((rows.shape[0], N), dtype=np.float64)
+    _check(lib().mtmc_ref_linear_softmax_rows(X.ctypes.data, W.ctypes.data, bp, M, N, K,
+                                              rows.ctypes.data, rows.shape[0], P.ctypes.data), "mtmc_ref_linear_softmax_rows")
+    return P
+
+
+def softmax_vector(z) -> np.ndarray:
+    z = np.ascontiguousarray(np.asarray(z, dtype=np.float64))
+    p = np.empty_like(z)
+    lib().mtmc_ref_softmax_vector(z.ctypes.data, z.shape[0], p.ctypes.data)
+    return p
 
 
 def lse_vector(z) -> float:

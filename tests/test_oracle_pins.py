@@ -466,6 +466,60 @@ def test_linear_lse_end_to_end():
     np.testing.assert_array_equal(ref.linear_lse_rows(X, W, b, rows), lse[rows])
 
 
+def test_softmax_closed_forms_and_laws():
+    # logits ln(a_i) for integers a_i: p_i = a_i / sum(a) exactly in the rationals
+    a = [1, 2, 3, 10, 48]
+    p = ref.softmax_vector([math.log(v) for v in a])
+    for got, v in zip(p, a):
+        assert got == pytest.approx(float(Fraction(v, sum(a))), rel=4e-15)
+    # equal logits: 1/N; one logit: 1; far-apart and huge logits neither overflow nor lose the winner
+    np.testing.assert_allclose(ref.softmax_vector(np.full(37, -2.5)), np.full(37, 1.0 / 37), rtol=1e-15)
+    assert ref.softmax_vector([4.75])[0] == 1.0
+    np.testing.assert_array_equal(ref.softmax_vector([1000.0, 1000.0]), [0.5, 0.5])
+    np.testing.assert_array_equal(ref.softmax_vector([-1000.0, 0.0]), [0.0, 1.0])
+    # two classes: softmax([z, 0])[0] is the logistic function 1 / (1 + exp(-z))
+    for z in (-30.0, -2.25, 0.0, 0.5, 7.0, 40.0):
+        assert ref.softmax_vector([z, 0.0])[0] == pytest.approx(1.0 / (1.0 + math.exp(-z)), rel=4e-16, abs=0)
+    rng = np.random.default_rng(43)
+    z = rng.normal(size=200) * 3.0
+    p = ref.softmax_vector(z)
+    assert p.sum() == pytest.approx(1.0, abs=1e-14) and np.all(p > 0)
+    for c in (-700.0, -3.5, 12.25, 900.0):                                   # shift invariance
+        np.testing.assert_allclose(ref.softmax_vector(z + c), p, rtol=1e-12 * max(1.0, abs(c)))
+    perm = rng.permutation(200)                                              # permutation equivariance
+    np.testing.assert_allclose(ref.softmax_vector(z[perm]), p[perm], rtol=1e-13)
+    np.testing.assert_array_equal(np.argsort(p, kind="stable"), np.argsort(z, kind="stable"))   # monotone in the logits
+    i, j = 17, 133                                                           # ratios: p_i / p_j = exp(z_i - z_j)
+    assert p[i] / p[j] == pytest.approx(math.exp(z[i] - z[j]), rel=1e-13)
+    np.testing.assert_allclose(p, np.exp(z - ref.lse_vector(z)), rtol=1e-12)                  # the logsumexp form
+    np.testing.assert_allclose(p, torch.softmax(torch.from_numpy(z), 0).numpy(), rtol=1e-13)  # library routine
+
+
+def test_linear_softmax_end_to_end():
+    li = inputs.linear_inputs(5, 300, 48, seed=44)
+    X, W, b = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    P = ref.linear_softmax(X, W, b)
+    z = li.X.double() @ li.W.double().T + li.b.double()
+    np.testing.assert_allclose(P, torch.softmax(z, -1).numpy(), rtol=1e-12, atol=0)
+    np.testing.assert_allclose(P.sum(axis=1), np.ones(5), rtol=0, atol=1e-13)
+    # consistent with the other oracle routes to the same logits: exp(z - lse), and act = none pre-activations
+    lse = ref.linear_lse(X, W, b)
+    np.testing.assert_allclose(P, np.exp(ref.fused_linear(X, W, b, ref.ACT_NONE) - lse[:, None]), rtol=1e-12)
+    # the expected negative log-probability of a column is the cross entropy with that target
+    tgt = np.array([0, 299, 17, 150, 42])
+    loss, _ = ref.linear_cross_entropy(X, W, b, tgt)
+    np.testing.assert_allclose(-np.log(P[np.arange(5), tgt]), loss, rtol=0, atol=1e-12)
+    # zero weights: softmax(b) in every row; zero weights and no bias: 1/N; N = 1: all ones
+    W0 = np.zeros_like(W)
+    np.testing.assert_allclose(ref.linear_softmax(X, W0, b)[3], ref.softmax_vector(b.astype(np.float64)), rtol=1e-14)
+    np.testing.assert_array_equal(ref.linear_softmax(X, W0, None), np.full((5, 300), 1.0 / 300))
+    np.testing.assert_array_equal(ref.linear_softmax(X, W[:1].copy(), b[:1].copy()), np.ones((5, 1)))
+    # a transposed operand or a dropped bias would move the row maximum's place
+    assert np.array_equal(P.argmax(axis=1), z.numpy().argmax(axis=1))
+    rows = np.array([4, 0, 2])
+    np.testing.assert_array_equal(ref.linear_softmax_rows(X, W, b, rows), P[rows])
+
+
 def test_lse_expected_level_for_unit_variance_logits():
     # logits ~ N(0,1) + small bias over N columns: lse ~ ln N + 1/2 (lognormal mean)
     li = inputs.linear_inputs(4, 4000, 256, seed=43)
