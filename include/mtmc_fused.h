@@ -74,6 +74,7 @@ extern "C" {
 #define MTMC_OP_FUSED_LINEAR_MXFP8 5
 #define MTMC_OP_SWIGLU_MXFP8 6
 #define MTMC_OP_LINEAR_LSE_MXFP8 7
+#define MTMC_OP_LINEAR_SOFTMAX 8
 
 /* out[m][n] = act( sum_k X[m][k] W[n][k] + b[n] ).
  * (Fused GEMM + bias + activation: the Fusion principle applied to a linear layer;
@@ -203,6 +204,19 @@ int mtmc_linear_rowmax(const void* X, const void* W, const float* b,
  * row's (max, sum-exp).)  Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_CROSS_ENTROPY, M, N, K). */
 int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, const int64_t* targets,
                               int64_t M, int64_t N, int64_t K, float* loss_out, float* lse_out);
+
+/* Row softmax of the logits, written out as probabilities:
+ *   prob_out[m][n] = exp( z[m][n] - lse[m] ),  z[m][n] = sum_k X[m][k] W[n][k] + b[n],
+ * [M,N] dense row-major, fp32 or bf16 (out_dtype: MTMC_OUT_FP32 / MTMC_OUT_BF16), device, 16-byte
+ * aligned; lse_out (fp32 [M], device, may be NULL) also receives the row logsumexp.  (The
+ * normalised form of the same row reduction: the logits themselves are never written.  The GEMM's
+ * epilogue stores exp(z - max) with the maximum of the row's piece of the tile, which is at most 1
+ * whatever the logits' size, and leaves the piece's (max, sum-exp) in the workspace; after the
+ * merge one pass over prob_out multiplies every piece by exp(max - lse).  A bf16 result therefore
+ * carries two roundings of a value in [0, 1]: relative error up to 2^-8.)  N must be below
+ * 2^31 - 1024.  bf16 operands.  Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_SOFTMAX, M, N, K). */
+int mtmc_linear_softmax(const void* X, const void* W, const float* b,
+                        int64_t M, int64_t N, int64_t K, int out_dtype, void* prob_out, float* lse_out);
 
 /* Allocation-free variant of mtmc_linear_lse: same arguments, same result (same
  * kernels), but the (max, sum-exp) partials live in an 8 MiB array that is part of

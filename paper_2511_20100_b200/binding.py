@@ -22,11 +22,11 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_UNSUPPORTED_DEVICE, ERR_CUDA, ERR_DE
 ACT = {"none": 0, "relu": 1, "gelu_tanh": 2, "silu": 3}
 OUT_DTYPE = {"fp32": 0, "bf16": 1}
 OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "linear_cross_entropy": 4,
-      "fused_linear_mxfp8": 5, "swiglu_mxfp8": 6, "linear_lse_mxfp8": 7}
+      "fused_linear_mxfp8": 5, "swiglu_mxfp8": 6, "linear_lse_mxfp8": 7, "linear_softmax": 8}
 
 EXPORTS = [
     "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_fused_linear_fp8", "mtmc_swiglu", "mtmc_linear_lse",
-    "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy",
+    "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy", "mtmc_linear_softmax",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
@@ -81,6 +81,7 @@ def load() -> ctypes.CDLL:
         getattr(L, name).argtypes = [vp, vp, vp, i64, i64, i64, vp]
     L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
+    L.mtmc_linear_softmax.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp]
     L.mtmc_set_stream.argtypes = [vp]
     L.mtmc_set_workspace.argtypes = [vp, sz]
     L.mtmc_workspace_bytes.argtypes = [ci, i64, i64, i64]
@@ -371,6 +372,23 @@ def mtmc_linear_cross_entropy(X, W, b, targets, loss_out=None, lse_out=None, wan
                                             _dev(loss_out, torch.float32, (M,), "loss_out"),
                                             None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
     return (loss_out, lse_out) if want_lse else loss_out
+
+
+def mtmc_linear_softmax(X, W, b, out_dtype="fp32", prob_out=None, lse_out=None, want_lse=False):
+    """prob[m][n] = softmax over n of z = X @ W.T + b, [M,N] fp32 or bf16; the logits are never written."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if prob_out is None:
+        prob_out = torch.empty((M, N), dtype=odt, device=X.device)
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X.device)
+    _use_current_stream(X.device)
+    _check(load().mtmc_linear_softmax(_dev(X, torch.bfloat16, (M, K), "X"), _dev(W, torch.bfloat16, (N, K), "W"),
+                                      None if b is None else _dev(b, torch.float32, (N,), "b"), M, N, K, OUT_DTYPE[out_dtype],
+                                      _dev(prob_out, odt, (M, N), "prob_out"),
+                                      None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return (prob_out, lse_out) if want_lse else prob_out
 
 
 def mtmc_linear_rowmax_fp8(X8, W8, b, scale_x, scale_w, max_out=None, argmax_out=None, want_argmax=True):

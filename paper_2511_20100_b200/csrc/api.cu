@@ -104,7 +104,7 @@ thread_local char t_error[512] = "";
 thread_local char t_last_kernel[96] = "";     // main kernel of the last call of this thread (mtmc_last_kernel_name)
 
 void note_kernel(const char* family, int epi, int detail = 0) {
-    static const char* const epi_name[] = {"EPI_ACT", "EPI_SWIGLU", "EPI_LSE", "EPI_ROWMAX", "EPI_XENT"};
+    static const char* const epi_name[] = {"EPI_ACT", "EPI_SWIGLU", "EPI_LSE", "EPI_ROWMAX", "EPI_XENT", "EPI_SOFTMAX"};
     if (epi >= 0 && detail > 0) snprintf(t_last_kernel, sizeof t_last_kernel, "%s<%s, %d>", family, epi_name[epi], detail);
     else if (epi >= 0) snprintf(t_last_kernel, sizeof t_last_kernel, "%s<%s>", family, epi_name[epi]);
     else snprintf(t_last_kernel, sizeof t_last_kernel, "%s<MX=%d>", family, detail);
@@ -964,16 +964,20 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 // leaves one partial per (row, column piece) in the workspace, a merge kernel finishes the rows.
 //   EPI_LSE    : out_a = lse                     EPI_ROWMAX : out_a = max, out_i = argmax (may be null)
 //   EPI_XENT   : out_b = loss, out_a = lse (may be null); the target logits sit behind the partials
+//   EPI_SOFTMAX: prob = the [M,N] probabilities (fp32 / bf16, dense), out_a = lse (may be null: it then sits behind the
+//                partials); the tiled kernel leaves exp(z - max of the piece) in prob, a last kernel scales every piece
 template <int EPI>
 int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
-                      float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0) {
+                      float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0,
+                      void* prob = nullptr, int out_dtype = MTMC_OUT_FP32) {
     auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
     if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    const int ks = pick_ksplit(d, M, N, K, 256, fp8);
-    const bool big = !ks && use_big_rowred(d, M, N, K, fp8);
+    // the softmax epilogue runs on the pair kernel and the single-CTA tiles (whose pieces the scaling kernel knows)
+    const int ks = EPI == EPI_SOFTMAX ? 0 : pick_ksplit(d, M, N, K, 256, fp8);
+    const bool big = EPI != EPI_SOFTMAX && !ks && use_big_rowred(d, M, N, K, fp8);
     const bool pair = !ks && !big && use_pair(d, M, N, K);
     const int bn = (pair || ks || big) ? 256 : pick_tile_n(N);
     GemmParams p{};
@@ -984,13 +988,13 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     else fill_tiling(p, M, N, K, bn, d->sm_count, true, 128, fp8);
     p.acc_scale = acc_scale;
     const size_t partial_bytes = lse_partial_bytes(p);         // what the chosen plan writes and the merge reads
-    const size_t extra = EPI == EPI_XENT ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
+    const size_t extra = (EPI == EPI_XENT || EPI == EPI_SOFTMAX) ? round256(static_cast<size_t>(M) * sizeof(float)) : 0;
     const int sk_clusters = sk ? gemm_pairs(d) : 0;
     void* ws = nullptr;
     rc = get_workspace(d, partial_bytes + extra + (sk ? streamk_bytes(sk_clusters) : 0), &ws);
     if (rc) return rc;
     if (sk && (rc = attach_streamk(d, p, sk_clusters, ws, partial_bytes + extra))) return rc;
-    p.act = ACT_NONE; p.bias = b; p.out = nullptr; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
+    p.act = ACT_NONE; p.bias = b; p.out = prob; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
     p.targets = reinterpret_cast<const long long*>(targets);
     p.target_logit = EPI == EPI_XENT ? reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes) : nullptr;
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
@@ -1000,14 +1004,47 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
         (rc = encode(&tmBt, W, N, K, (pair || big) ? p.tail_width / 2 : p.tail_width, ldw)))
         return rc;
     TimedRegion tr(d);
-    if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
-    else if (big) rc = launch_big<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, p);
-    else if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
-    else rc = bn == 256 ? launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
-                        : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    if constexpr (EPI == EPI_SOFTMAX) {
+        const bool bf = out_dtype == MTMC_OUT_BF16;
+        if (pair) rc = bf ? launch_pair<EPI, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
+                          : launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+        else if (bn == 256) rc = bf ? launch_tiled<EPI, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                                    : launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+        else rc = bf ? launch_tiled<EPI, 128, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                     : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    } else {
+        if (ks) rc = launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
+        else if (big) rc = launch_big<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, p);
+        else if (pair) rc = launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
+        else rc = bn == 256 ? launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p)
+                            : launch_tiled<EPI, 128, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
+    }
     tr.stop();
     if (rc) return rc;
     const unsigned blocks = static_cast<unsigned>((M + 7) / 8);
+    if constexpr (EPI == EPI_SOFTMAX) {
+        float* lse = out_a ? out_a : reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes);
+        lse_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
+                                                       p.n_full, p.tail_split, lse, nullptr, nullptr);
+        CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(1);
+        // one warp per row and span of columns: enough warps to fill the device a few times over, spans of whole tiles
+        const int out_tile_n = (pair || bn == 256) ? 256 : 128;
+        int64_t spans = std::max<int64_t>(1, (static_cast<int64_t>(d->sm_count) * 64 + M - 1) / M);
+        const int64_t max_spans = (N + 1023) / 1024;
+        if (spans > max_spans) spans = max_spans;
+        const int span = static_cast<int>(((N + spans - 1) / spans + 1023) / 1024 * 1024);
+        const dim3 grid(blocks, static_cast<unsigned>((N + span - 1) / span), 1);
+        if (out_dtype == MTMC_OUT_BF16)
+            softmax_scale_kernel<true><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
+                                                                   p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, span);
+        else
+            softmax_scale_kernel<false><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
+                                                                    p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, span);
+        CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(1);
+        return MTMC_OK;
+    }
     if (EPI == EPI_ROWMAX)
         rowmax_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
                                                           p.n_full, p.tail_split, out_a, out_i);
@@ -1413,8 +1450,8 @@ const char* mtmc_last_kernel_name(void) { return t_last_kernel; }
 
 size_t mtmc_workspace_bytes(int op, int64_t M, int64_t N, int64_t K) {
     if (M <= 0 || N <= 0 || K <= 0) return static_cast<size_t>(-1);
-    if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_LSE_MXFP8) return static_cast<size_t>(-1);
-    if (op >= MTMC_OP_FUSED_LINEAR_MXFP8) {      // the re-arranged scales (+ the logsumexp partials of 128-column tiles, the most pieces)
+    if (op < MTMC_OP_FUSED_LINEAR || op > MTMC_OP_LINEAR_SOFTMAX) return static_cast<size_t>(-1);
+    if (op >= MTMC_OP_FUSED_LINEAR_MXFP8 && op <= MTMC_OP_LINEAR_LSE_MXFP8) {      // the re-arranged scales (+ the logsumexp partials of 128-column tiles, the most pieces)
         DeviceState* dm = nullptr;
         if (get_device(&dm) != MTMC_OK) return static_cast<size_t>(-1);
         const MxPlan mp = plan_mx(dm, op == MTMC_OP_SWIGLU_MXFP8 ? EPI_SWIGLU : (op == MTMC_OP_LINEAR_LSE_MXFP8 ? EPI_LSE : EPI_ACT), M, N, K);
@@ -1681,6 +1718,16 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
     if (!targets) return fail(MTMC_ERR_INVALID_ARG, "null pointer argument");
     if (reinterpret_cast<uintptr_t>(targets) & 7u) return fail(MTMC_ERR_INVALID_ARG, "targets must be 8-byte aligned");
     return run_row_reduction<EPI_XENT>(X, W, b, targets, M, N, K, lse_out, loss_out, nullptr);
+}
+
+int mtmc_linear_softmax(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int out_dtype,
+                        void* prob_out, float* lse_out) {
+    int rc = check_common(X, W, prob_out, M, N, K);
+    if (rc) return rc;
+    if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
+    if (N >= (1ll << 31) - 1024) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "N = %lld: N must be below 2^31 - 1024", (long long)N);
+    if (lse_out && (reinterpret_cast<uintptr_t>(lse_out) & 3u)) return fail(MTMC_ERR_INVALID_ARG, "lse_out must be 4-byte aligned");
+    return run_row_reduction<EPI_SOFTMAX>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr, false, 1.0f, 0, 0, prob_out, out_dtype);
 }
 
 int mtmc_linear_rowmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,

@@ -15,7 +15,7 @@
 
 namespace mtmc {
 
-enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2, EPI_ROWMAX = 3, EPI_XENT = 4 };
+enum { EPI_ACT = 0, EPI_SWIGLU = 1, EPI_LSE = 2, EPI_ROWMAX = 3, EPI_XENT = 4, EPI_SOFTMAX = 5 };
 enum { ACT_NONE = 0, ACT_RELU = 1, ACT_GELU_TANH = 2, ACT_SILU = 3 };
 
 // Epilogue warps per CTA: EPI_HALVES per TMEM lane quadrant, each draining its share of an item's
@@ -335,6 +335,7 @@ __device__ __forceinline__ void tile_bias_chunk(const GemmParams& p, const float
 //   EPI_LSE    : online (max, sum-exp) in base-2 units, one partial per (row, column piece)
 //   EPI_XENT   : the same, and the logit at the row's target column is set aside
 //   EPI_ROWMAX : running (max, lowest column attaining it), one partial per (row, column piece)
+//   EPI_SOFTMAX: the (max, sum-exp) partial of EPI_LSE, and exp(z - max of the piece) stored to out for every column
 template <int EPI, bool OUT_BF16>
 __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_addr, int row, int n_tile0, int c_begin,
                                               int c_end, int width, int nb, int sub, int half, bool vec_ok, uint8_t* stage,
@@ -438,6 +439,56 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
         }
         if (row < p.M && MTMC_CHECK((nb * p.tail_split + sub) * EPI_HALVES + half < p.n_tiles * p.tail_split * EPI_HALVES, p.status, 2u))
             p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] = make_float2(mx, __int_as_float(arg));
+    } else if (EPI == EPI_SOFTMAX) {
+        // Two passes over the piece's accumulator columns, which stay in tensor memory meanwhile: first the row's
+        // maximum over the piece, then e = 2^(t - max) for every column, stored as the still unnormalised output and
+        // summed.  The (max, sum) partial goes the way of EPI_LSE; softmax_scale_kernel multiplies the piece by
+        // exp(max - lse) once the row's lse is known.
+        constexpr float LOG2E = 1.4426950408889634f;
+        const float zscale = LOG2E * p.acc_scale;
+        const int live = min(c_end, (p.N - n_tile0 + 31) / 32);
+        float mx = -INFINITY, sum = 0.0f;
+        uint32_t r[32];
+        if (c_begin < live) tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
+#pragma unroll 1
+        for (int c = c_begin; c < live; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            float bv[32];
+            tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
+            tmem_ld_wait();
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float t = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);
+                m4[j & 3] = fmaxf(m4[j & 3], (n0 + j < p.N) ? t : -INFINITY);     // columns past N are zero-filled weight rows
+            }
+            if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
+            mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+        }
+        if (c_begin < live) tmem_ld_32x32b_x32(t_addr + c_begin * 32, r);
+#pragma unroll 1
+        for (int c = c_begin; c < live; ++c) {
+            const int n0 = n_tile0 + c * 32;
+            float bv[32], y[32];
+            tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
+            tmem_ld_wait();
+            float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const float t = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);       // the same bits as in the first pass
+                y[j] = (n0 + j < p.N) ? ex2_approx(t - mx) : 0.0f;
+                s4[j & 3] += y[j];
+            }
+            if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
+            sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);
+            if (!MTMC_CHECK(n0 >= 0 && n0 < p.N && p.ldo >= p.N, p.status, 5u)) continue;
+            if (vec_ok && n0 + 32 <= p.N) store_chunk_coalesced<OUT_BF16>(stage, p.out, row - lane, n0, p.M, p.ldo, y, lane);
+            else if (row < p.M) store_row_chunk<OUT_BF16>(p.out, row, n0, p.N, p.ldo, y, false);
+        }
+        // a piece that lies wholly past N (only possible in the last column tile) stays neutral
+        if (row < p.M && MTMC_CHECK((nb * p.tail_split + sub) * EPI_HALVES + half < p.n_tiles * p.tail_split * EPI_HALVES, p.status, 2u))
+            p.lse_partial[static_cast<size_t>((nb * p.tail_split + sub) * EPI_HALVES + half) * p.M + row] =
+                make_float2(mx * 0.6931471805599453f, sum);
     } else {
         // Online (max, sum-exp) over this tile's columns, in base-2 units: t = z * log2(e).
         constexpr float LOG2E = 1.4426950408889634f;
@@ -739,6 +790,82 @@ __global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, i
     if (lane == 0) {
         max_out[row] = mx;
         if (argmax_out) argmax_out[row] = arg;
+    }
+}
+
+// Turns the unnormalised exponentials that EPI_SOFTMAX left in out into probabilities: every element is multiplied
+// by exp(max of its piece - lse of its row), the piece being the (column tile, tail piece, share of the piece) whose
+// epilogue thread wrote it.  One warp per row and span of columns, 16 bytes per lane and step where the pitch allows.
+template <bool OUT_BF16>
+__global__ void softmax_scale_kernel(void* __restrict__ out, int ldo, const float2* __restrict__ partial,
+                                     const float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
+                                     int group_m, int n_full, int tail_split, int out_tile_n, int span) {
+    pdl_launch_dependents();
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    const int mb = row / rows_per_tile;
+    const float l = __ldcg(lse + row);
+    const int c_first = blockIdx.y * span, c_last = min(N, c_first + span);
+    // the factor of the piece that holds column col
+    auto factor = [&](int col) -> float {
+        const int nb = col / out_tile_n;
+        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+        const int width = out_tile_n / pieces;
+        const int in_tile = col - nb * out_tile_n;
+        const int sub = in_tile / width;
+        const int chunk = (in_tile - sub * width) >> 5, chunks = width >> 5;
+        const int half = (EPI_HALVES == 2 && chunk >= (chunks + 1) / 2) ? 1 : 0;
+        const float2 v = __ldcg(partial + static_cast<size_t>((nb * tail_split + sub) * EPI_HALVES + half) * M + row);
+        return __expf(v.x - l);
+    };
+    constexpr int PER = OUT_BF16 ? 8 : 4;                    // elements per 16 bytes
+    const size_t elem = OUT_BF16 ? 2 : 4;
+    uint8_t* base = reinterpret_cast<uint8_t*>(out) + static_cast<size_t>(row) * ldo * elem;
+    const bool vec = (ldo % PER == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0);
+    if (vec) {
+        constexpr int UNROLL = 4;
+        const int n_vec = c_last == N ? (N / PER) * PER : c_last;       // span and c_first are multiples of 32
+        for (int c0 = c_first + lane * PER; c0 < n_vec; c0 += 32 * PER * UNROLL) {
+            uint4 q[UNROLL];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int c = c0 + u * 32 * PER;
+                if (c < n_vec) q[u] = *reinterpret_cast<const uint4*>(base + c * elem);
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int c = c0 + u * 32 * PER;
+                if (c >= n_vec) continue;
+                const float f = factor(c);                   // 16 bytes lie inside one 32-column chunk
+                uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    if (OUT_BF16) w[h] = pack_bf16x2(__uint_as_float(w[h] << 16) * f, __uint_as_float(w[h] & 0xffff0000u) * f);
+                    else w[h] = __float_as_uint(__uint_as_float(w[h]) * f);
+                }
+                *reinterpret_cast<uint4*>(base + c * elem) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        }
+        for (int c = n_vec + lane; c < c_last; c += 32) {                  // the last N mod PER columns
+            const float f = factor(c);
+            if (OUT_BF16) {
+                __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(base) + c;
+                *e = __float2bfloat16_rn(__bfloat162float(*e) * f);
+            } else {
+                reinterpret_cast<float*>(base)[c] *= f;
+            }
+        }
+    } else {
+        for (int c = c_first + lane; c < c_last; c += 32) {
+            const float f = factor(c);
+            if (OUT_BF16) {
+                __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(base) + c;
+                *e = __float2bfloat16_rn(__bfloat162float(*e) * f);
+            } else {
+                reinterpret_cast<float*>(base)[c] *= f;
+            }
+        }
     }
 }
 

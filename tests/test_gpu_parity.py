@@ -798,6 +798,126 @@ def test_rowmax_and_cross_entropy_at_lm_head_size_on_sampled_rows():
     assert bool((loss >= lse - mx - 2e-3).all())
 
 
+# ------------------------------------------------------------------ row softmax written out as probabilities
+# Probabilities are compared relative to their own size (a row of N of them averages 1/N, far below any absolute
+# tolerance that suits activations): logit error (bf16 products, fp32 sums) and the hardware exp2 give a few 1e-4;
+# a bf16 result adds two roundings of a value in [0, 1], 2^-8 together.  The absolute term only covers results that
+# fp32 flushes to zero (below 2^-126).
+SOFTMAX_TOL = {"fp32": (1e-30, 2e-3), "bf16": (1e-30, 1e-2)}
+
+
+def _check_softmax(li, prob, lse, odt, what):
+    Xb, Wb, bf = inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b)
+    want = ref.linear_softmax(Xb, Wb, bf)
+    _assert_close(inputs.to_f64(prob), want, SOFTMAX_TOL[odt], what)
+    if lse is not None:
+        _assert_close(inputs.to_f64(lse), ref.linear_lse(Xb, Wb, bf), TOL["fp32"], what + ": lse")
+    sums = prob.double().sum(dim=1).cpu().numpy()
+    np.testing.assert_allclose(sums, np.ones_like(sums), rtol=0, atol=4e-3 if odt == "bf16" else 1e-4, err_msg=what + ": row sums")
+
+
+@pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 8, 64), (200, 1000, 256), (129, 257, 72), (64, 3000, 128), (260, 512, 320),
+                                   (300, 2304, 2048), (130, 4100, 512), (700, 1300, 328)])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_linear_softmax_small(M, N, K, odt):
+    """Single-CTA tiles and pair tiles, whole and split wave tails, N a multiple of 32, of 8, of 4 and odd."""
+    li = inputs.linear_inputs(M, N, K, seed=5400 + M + N, bias=(M % 2 == 0))
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    bufl, lse = _guarded((M,), torch.float32)
+    B.mtmc_linear_softmax(li.X.cuda(), li.W.cuda(), None if li.b is None else li.b.cuda(), odt, prob_out=out, lse_out=lse)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N) and _canaries_intact(bufl, M)
+    _check_softmax(li, out, lse, odt, "softmax %dx%dx%d %s" % (M, N, K, odt))
+    again = B.mtmc_linear_softmax(li.X.cuda(), li.W.cuda(), None if li.b is None else li.b.cuda(), odt)   # lse in the workspace
+    B.mtmc_check_status()
+    assert torch.equal(again, out), "run-to-run bits"
+
+
+SOFTMAX_FAMILIES = [("single-CTA tiles", dict(cta_pair=-1), 0, (300, 1000, 328)), ("128-column tiles", dict(tile_n=128), 0, (300, 1000, 328)),
+                    ("256 x 256 pair tiles", dict(cta_pair=1), -1, (600, 1000, 328)), ("pair tiles, stream-K", dict(cta_pair=1), 1, (600, 2304, 328))]
+
+
+@pytest.mark.parametrize("family,tune,sk,shape", SOFTMAX_FAMILIES, ids=[f[0] for f in SOFTMAX_FAMILIES])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_linear_softmax_edge_cases(family, tune, sk, shape, odt):
+    """On every kernel that carries the epilogue: equal logits (W = 0: softmax(b), without bias 1/N), one dominant logit
+    (a weight row scaled by 64: one probability near 1, the rest tiny but right), and shifts of +-500 in the bias,
+    which leave the probabilities alone although exp of the logits themselves overflows or vanishes in fp32."""
+    M, N, K = shape
+    li = inputs.linear_inputs(M, N, K, seed=9800 + M)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    W0 = torch.zeros_like(li.W)
+    Wdom = li.W.clone()
+    Wdom[N // 3] = (Wdom[N // 3].float() * 64.0).bfloat16()
+    B.mtmc_set_tuning(**tune)
+    B.mtmc_set_schedule(sk)
+    try:
+        plain = B.mtmc_linear_softmax(Xd, Wd, bd, odt)
+        want_kernel = "gemm_pair_kernel" if "pair" in family else "gemm_tiled_kernel"
+        assert want_kernel in B.mtmc_last_kernel_name(), "%s: ran %s" % (family, B.mtmc_last_kernel_name())
+        zero_b = B.mtmc_linear_softmax(Xd, W0.cuda(), bd, odt)
+        zero_nob = B.mtmc_linear_softmax(Xd, W0.cuda(), None, odt)
+        dom = B.mtmc_linear_softmax(Xd, Wdom.cuda(), bd, odt)
+        up = B.mtmc_linear_softmax(Xd, Wd, (li.b + 500.0).cuda(), odt)
+        down = B.mtmc_linear_softmax(Xd, Wd, (li.b - 500.0).cuda(), odt)
+        B.mtmc_check_status()
+    finally:
+        B.mtmc_set_schedule(0)
+        B.mtmc_set_tuning()
+    tol = SOFTMAX_TOL[odt]
+    _check_softmax(li, plain, None, odt, family)
+    _check_softmax(inputs.LinearInputs(li.X, W0, li.b), zero_b, None, odt, family + ": W = 0")
+    _assert_close(inputs.to_f64(zero_nob), np.full((M, N), 1.0 / N), tol, family + ": W = 0, no bias = 1/N")
+    _check_softmax(inputs.LinearInputs(li.X, Wdom, li.b), dom, None, odt, family + ": dominant logit")
+    _check_softmax(inputs.LinearInputs(li.X, li.W, li.b + 500.0), up, None, odt, family + ": bias + 500")
+    _check_softmax(inputs.LinearInputs(li.X, li.W, li.b - 500.0), down, None, odt, family + ": bias - 500")
+
+
+def test_linear_softmax_with_caller_workspace_and_bad_arguments():
+    M, N, K = 300, 2304, 2048
+    li = inputs.linear_inputs(M, N, K, seed=5500)
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    for sk in (1, -1):
+        B.mtmc_set_schedule(sk)
+        try:
+            need = B.mtmc_workspace_bytes("linear_softmax", M, N, K)      # under the schedule that the call will run with
+            assert need >= B.mtmc_workspace_bytes("linear_lse", M, N, K) > 0
+            guard = torch.full((need + 8192,), 0x5A, dtype=torch.uint8, device="cuda")
+            off = (-guard.data_ptr()) % 256 + 3840
+            B.mtmc_set_workspace(guard[off:off + need])
+            prob = B.mtmc_linear_softmax(Xd, Wd, bd, "bf16")
+            B.mtmc_check_status()
+        finally:
+            B.mtmc_set_schedule(0)
+            B.mtmc_set_workspace(None)
+        assert bool((guard[:off] == 0x5A).all()) and bool((guard[off + need:] == 0x5A).all())
+        _check_softmax(li, prob, None, "bf16", "softmax, caller workspace, schedule %d" % sk)
+    L = B.load()
+    assert L.mtmc_linear_softmax(Xd.data_ptr(), Wd.data_ptr(), None, M, N, K, 7, prob.data_ptr(), None) == B.ERR_INVALID_ARG
+    assert L.mtmc_linear_softmax(Xd.data_ptr(), Wd.data_ptr(), None, M, N, K, 0, None, None) == B.ERR_INVALID_ARG
+    assert L.mtmc_linear_softmax(Xd.data_ptr(), Wd.data_ptr(), None, M, N, K + 4, 0, prob.data_ptr(), None) == B.ERR_UNSUPPORTED_SHAPE
+    B.mtmc_check_status()
+
+
+def test_linear_softmax_at_lm_head_size_on_sampled_rows():
+    c = inputs.CONFIGS["C4"]
+    li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
+    Xd, Wd, bd = li.X.cuda(), li.W.cuda(), li.b.cuda()
+    prob, lse = B.mtmc_linear_softmax(Xd, Wd, bd, "bf16", want_lse=True)
+    assert "gemm_pair_kernel" in B.mtmc_last_kernel_name()
+    lse_alone = B.mtmc_linear_lse(Xd, Wd, bd)
+    B.mtmc_check_status()
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, c["M"] - 1], np.random.default_rng(6).integers(0, c["M"], size=4)]))
+    want = ref.linear_softmax_rows(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b), rows)
+    idx = torch.from_numpy(rows).cuda()
+    _assert_close(inputs.to_f64(prob[idx]), want, SOFTMAX_TOL["bf16"], "C4 softmax sampled rows")
+    # properties at full size: every row sums to one, no probability above one or below zero, lse as the reduction alone
+    sums = prob.float().sum(dim=1)
+    assert bool(((sums - 1.0).abs() <= 4e-3).all()), "row sums %.5f .. %.5f" % (float(sums.min()), float(sums.max()))
+    assert bool((prob >= 0).all()) and bool((prob <= 1).all())
+    assert torch.allclose(lse, lse_alone, rtol=0, atol=1e-4)
+
+
 # ------------------------------------------------------------------ cluster split-K (few tiles, long K)
 # Problems of at most half a wave of 128 x 256 tiles: a cluster of 2, 4 or 8 CTAs per tile, reduce-scatter through
 # distributed shared memory.  Ragged in every dimension, k-blocks that do not divide evenly among the CTAs,
