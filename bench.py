@@ -61,6 +61,8 @@ def algorithmic_bytes(c) -> float:
         extra = {"linear_lse": 0.0, "linear_rowmax": 4.0 * M, "linear_cross_entropy": 8.0 * M}[c["op"]]
         return 2.0 * (M * K + N * K) + 4.0 * N + 4.0 * M + extra
     out_b = 2.0 if c["out_dtype"] == "bf16" else 4.0
+    if c["op"] == "linear_softmax":         # the probabilities are written, read back and written again by the finishing pass
+        return 2.0 * (M * K + N * K) + 4.0 * N + 3.0 * out_b * M * N
     res = out_b * M * N if c["op"] == "fused_linear_residual" else 0.0
     return 2.0 * (M * K + N * K) + 4.0 * N + out_b * M * N + res
 
@@ -180,6 +182,8 @@ def call_device(B, pr):
         B.mtmc_linear_rowmax(d[0], d[1], d[2], max_out=pr["out"], want_argmax=False)
     elif c["op"] == "linear_cross_entropy":
         B.mtmc_linear_cross_entropy(d[0], d[1], d[2], d[3], loss_out=pr["out"])
+    elif c["op"] == "linear_softmax":
+        B.mtmc_linear_softmax(d[0], d[1], d[2], c["out_dtype"], prob_out=pr["out"])
     elif c["op"] == "fused_linear_residual":
         B.mtmc_fused_linear_residual(d[0], d[1], d[2], d[3], c["act"], c["out_dtype"], out=pr["out"])
     elif c["op"] == "fused_linear_fp8":
@@ -215,6 +219,8 @@ def eager_call(pr, dev):
     if c["op"] == "linear_cross_entropy":
         return torch.nn.functional.cross_entropy((dev[0] @ dev[1].T).float() + dev[2], dev[3], reduction="none")
     z = (dev[0] @ dev[1].T).float() + dev[2]
+    if c["op"] == "linear_softmax":
+        return torch.softmax(z, dim=-1).to(torch.bfloat16)
     if c["op"] == "fused_linear_residual":
         return (z + dev[3].float()).to(torch.bfloat16)
     z = torch.relu(z) if c["act"] == "relu" else torch.nn.functional.gelu(z, approximate="tanh")

@@ -1028,19 +1028,16 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
                                                        p.n_full, p.tail_split, lse, nullptr, nullptr);
         CUDA_TRY(cudaGetLastError());
         g_launches.fetch_add(1);
-        // one warp per row and span of columns: enough warps to fill the device a few times over, spans of whole tiles
+        // one warp per row and span of eight column tiles: many short blocks, so that the last wave costs little
         const int out_tile_n = (pair || bn == 256) ? 256 : 128;
-        int64_t spans = std::max<int64_t>(1, (static_cast<int64_t>(d->sm_count) * 64 + M - 1) / M);
-        const int64_t max_spans = (N + 1023) / 1024;
-        if (spans > max_spans) spans = max_spans;
-        const int span = static_cast<int>(((N + spans - 1) / spans + 1023) / 1024 * 1024);
-        const dim3 grid(blocks, static_cast<unsigned>((N + span - 1) / span), 1);
+        const int tiles_per_span = std::max(8, (p.n_tiles + 65534) / 65535);      // grid.y stays within its limit
+        const dim3 grid(blocks, static_cast<unsigned>((p.n_tiles + tiles_per_span - 1) / tiles_per_span), 1);
         if (out_dtype == MTMC_OUT_BF16)
-            softmax_scale_kernel<true><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
-                                                                   p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, span);
+            softmax_finish_kernel<true><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
+                                                                    p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
         else
-            softmax_scale_kernel<false><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
-                                                                    p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, span);
+            softmax_finish_kernel<false><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
+                                                                     p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
         CUDA_TRY(cudaGetLastError());
         g_launches.fetch_add(1);
         return MTMC_OK;

@@ -793,78 +793,89 @@ __global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, i
     }
 }
 
-// Turns the unnormalised exponentials that EPI_SOFTMAX left in out into probabilities: every element is multiplied
-// by exp(max of its piece - lse of its row), the piece being the (column tile, tail piece, share of the piece) whose
-// epilogue thread wrote it.  One warp per row and span of columns, 16 bytes per lane and step where the pitch allows.
+// Finishes EPI_SOFTMAX once lse_merge_kernel has left the rows' lse: turns the unnormalised exponentials in out into
+// probabilities -- every element is multiplied by exp(max of its piece - lse of its row), the piece being the
+// (column tile, tail piece, share of the piece) whose epilogue thread wrote it.  One warp per row and span of column
+// tiles; 16 bytes per lane and step where the pitch allows, four tiles' loads in flight.
 template <bool OUT_BF16>
-__global__ void softmax_scale_kernel(void* __restrict__ out, int ldo, const float2* __restrict__ partial,
-                                     const float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
-                                     int group_m, int n_full, int tail_split, int out_tile_n, int span) {
+__global__ void softmax_finish_kernel(void* __restrict__ out, int ldo, const float2* __restrict__ partial,
+                                      const float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
+                                      int group_m, int n_full, int tail_split, int out_tile_n, int tiles_per_span) {
     pdl_launch_dependents();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
     const int mb = row / rows_per_tile;
     const float l = __ldcg(lse + row);
-    const int c_first = blockIdx.y * span, c_last = min(N, c_first + span);
-    // the factor of the piece that holds column col
-    auto factor = [&](int col) -> float {
-        const int nb = col / out_tile_n;
-        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
-        const int width = out_tile_n / pieces;
-        const int in_tile = col - nb * out_tile_n;
-        const int sub = in_tile / width;
-        const int chunk = (in_tile - sub * width) >> 5, chunks = width >> 5;
-        const int half = (EPI_HALVES == 2 && chunk >= (chunks + 1) / 2) ? 1 : 0;
-        const float2 v = __ldcg(partial + static_cast<size_t>((nb * tail_split + sub) * EPI_HALVES + half) * M + row);
-        return __expf(v.x - l);
-    };
+
     constexpr int PER = OUT_BF16 ? 8 : 4;                    // elements per 16 bytes
+    constexpr int UNROLL = 4;                                // tiles in flight
+    constexpr int UPL = OUT_BF16 ? 1 : 2;                    // 16-byte units of a 256-column tile per lane
     const size_t elem = OUT_BF16 ? 2 : 4;
     uint8_t* base = reinterpret_cast<uint8_t*>(out) + static_cast<size_t>(row) * ldo * elem;
     const bool vec = (ldo % PER == 0) && ((reinterpret_cast<uintptr_t>(out) & 15u) == 0);
-    if (vec) {
-        constexpr int UNROLL = 4;
-        const int n_vec = c_last == N ? (N / PER) * PER : c_last;       // span and c_first are multiples of 32
-        for (int c0 = c_first + lane * PER; c0 < n_vec; c0 += 32 * PER * UNROLL) {
-            uint4 q[UNROLL];
+    const int nb_first = blockIdx.y * tiles_per_span, nb_last = min(n_tiles, nb_first + tiles_per_span);
+    const int n_vec = vec ? (N / PER) * PER : 0;             // columns below n_vec travel as whole 16-byte units
+    // the partial of the piece of tile nb that holds the tile's column in_tile
+    auto piece_of = [&](int nb, int pieces, int in_tile) -> const float2* {
+        const int width = out_tile_n / pieces;
+        const int sub = in_tile / width;
+        const int chunk = (in_tile - sub * width) >> 5, chunks = width >> 5;
+        const int half = (EPI_HALVES == 2 && chunk >= (chunks + 1) / 2) ? 1 : 0;
+        return partial + static_cast<size_t>((nb * tail_split + sub) * EPI_HALVES + half) * M + row;
+    };
+    const int units = out_tile_n / PER;                      // 16-byte units per tile: 16, 32 or 64
+    for (int nb0 = nb_first; nb0 < nb_last; nb0 += UNROLL) {
+        uint4 q[UNROLL][UPL];
+        float pm[UNROLL][UPL];                               // the pieces' maxima, fetched while the data is on its way
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const int c = c0 + u * 32 * PER;
-                if (c < n_vec) q[u] = *reinterpret_cast<const uint4*>(base + c * elem);
+        for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+            for (int k = 0; k < UPL; ++k) {
+                const int unit = lane + 32 * k, col = (nb0 + u) * out_tile_n + unit * PER;
+                if (nb0 + u < nb_last && unit < units && col < n_vec) q[u][k] = __ldcs(reinterpret_cast<const uint4*>(base + col * elem));
             }
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const int c = c0 + u * 32 * PER;
-                if (c >= n_vec) continue;
-                const float f = factor(c);                   // 16 bytes lie inside one 32-column chunk
-                uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+        for (int u = 0; u < UNROLL; ++u) {
+            const int nb = nb0 + u;
+            if (nb >= nb_last) break;
+            const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+#pragma unroll
+            for (int k = 0; k < UPL; ++k) {
+                const int unit = lane + 32 * k;
+                if (unit < units && nb * out_tile_n + unit * PER < n_vec) pm[u][k] = __ldcg(piece_of(nb, pieces, unit * PER)).x;   // 16 bytes lie inside one 32-column chunk
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int nb = nb0 + u;
+            if (nb >= nb_last) break;
+#pragma unroll
+            for (int k = 0; k < UPL; ++k) {
+                const int unit = lane + 32 * k, col = nb * out_tile_n + unit * PER;
+                if (unit >= units || col >= n_vec) continue;
+                const float f = __expf(pm[u][k] - l);
+                uint32_t w[4] = {q[u][k].x, q[u][k].y, q[u][k].z, q[u][k].w};
 #pragma unroll
                 for (int h = 0; h < 4; ++h) {
                     if (OUT_BF16) w[h] = pack_bf16x2(__uint_as_float(w[h] << 16) * f, __uint_as_float(w[h] & 0xffff0000u) * f);
                     else w[h] = __float_as_uint(__uint_as_float(w[h]) * f);
                 }
-                *reinterpret_cast<uint4*>(base + c * elem) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(base + col * elem) = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
-        for (int c = n_vec + lane; c < c_last; c += 32) {                  // the last N mod PER columns
-            const float f = factor(c);
-            if (OUT_BF16) {
-                __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(base) + c;
-                *e = __float2bfloat16_rn(__bfloat162float(*e) * f);
-            } else {
-                reinterpret_cast<float*>(base)[c] *= f;
-            }
-        }
-    } else {
-        for (int c = c_first + lane; c < c_last; c += 32) {
-            const float f = factor(c);
-            if (OUT_BF16) {
-                __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(base) + c;
-                *e = __float2bfloat16_rn(__bfloat162float(*e) * f);
-            } else {
-                reinterpret_cast<float*>(base)[c] *= f;
-            }
+    }
+    // what does not travel as 16-byte units: the last N mod PER columns, or every column of an unaligned output
+    const int c_first = max(n_vec, nb_first * out_tile_n), c_last = min(N, nb_last * out_tile_n);
+    for (int c = c_first + lane; c < c_last; c += 32) {
+        const int nb = c / out_tile_n;
+        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+        const float f = __expf(__ldcg(piece_of(nb, pieces, c - nb * out_tile_n)).x - l);
+        if (OUT_BF16) {
+            __nv_bfloat16* e = reinterpret_cast<__nv_bfloat16*>(base) + c;
+            *e = __float2bfloat16_rn(__bfloat162float(*e) * f);
+        } else {
+            reinterpret_cast<float*>(base)[c] *= f;
         }
     }
 }
