@@ -29,7 +29,7 @@
 //                   section "Training Process")
 //   cross entropy:  loss[m] = lse[m] - z[m][target[m]]   (softmax cross entropy of the logits row)
 //   row softmax  :  P[m][n] = exp(z[m][n] - max_n' z[m][n']) / sum_n' exp(z[m][n'] - max), the normalised
-//                   form of the same row reduction
+//                   form of the same row reduction (also with E4M3 operands and per-tensor scales)
 //
 // Layouts: X [M,K], W [N,K], out [M,N]; all dense row-major.  X/W arrive as bf16 bit
 // patterns (uint16_t: the upper half of an IEEE-754 binary32), b as binary32 and
@@ -414,6 +414,19 @@ static double preact_fp8(const uint8_t* X, const uint8_t* W, const float* b, dou
     double acc = 0.0;
     for (int64_t k = 0; k < K; ++k) acc += e4m3_to_double(X[m * K + k]) * e4m3_to_double(W[n * K + k]);
     return scale * acc + (b ? static_cast<double>(b[n]) : 0.0);
+}
+
+// Row softmax of the E4M3 layer's logits: P[m][n] = softmax over n of sx*sw * Xq.Wq^T + b.
+int mtmc_ref_linear_softmax_fp8(const uint8_t* X, const uint8_t* W, const float* b, float scale_x, float scale_w,
+                                int64_t M, int64_t N, int64_t K, double* P) {
+    if (!X || !W || !P || M <= 0 || N <= 0 || K <= 0) return 1;
+    const double scale = static_cast<double>(scale_x) * static_cast<double>(scale_w);
+    parallel_for(M, [=](int64_t m) {
+        std::vector<double> z(static_cast<size_t>(N));
+        for (int64_t n = 0; n < N; ++n) z[n] = preact_fp8(X, W, b, scale, K, m, n);
+        softmax_of_row(z.data(), N, P + m * N);
+    });
+    return 0;
 }
 
 // Row maximum and the lowest column attaining it, E4M3 operands.

@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.mtmc_ref_linear_softmax.argtypes = [vp, vp, vp, i64, i64, i64, vp]
         L.mtmc_ref_linear_softmax_rows.argtypes = [vp, vp, vp, i64, i64, i64, vp, i64, vp]
         L.mtmc_ref_softmax_vector.argtypes = [vp, i64, vp]
+        L.mtmc_ref_linear_softmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, vp]
         L.mtmc_ref_softmax_vector.restype = None
         L.mtmc_ref_lse_vector.argtypes = [vp, i64]
         L.mtmc_ref_lse_vector.restype = dbl
@@ -387,6 +388,18 @@ def linear_softmax_rows(X, W, b, rows) -> np.ndarray:
     P = np.empty((rows.shape[0], N), dtype=np.float64)
     _check(lib().mtmc_ref_linear_softmax_rows(X.ctypes.data, W.ctypes.data, bp, M, N, K,
                                               rows.ctypes.data, rows.shape[0], P.ctypes.data), "mtmc_ref_linear_softmax_rows")
+    return P
+
+
+def linear_softmax_fp8(X, W, b, scale_x: float, scale_w: float) -> np.ndarray:
+    """softmax over n of scale_x*scale_w * Xq.Wq^T + b with E4M3 bit patterns (uint8), [M,N] float64."""
+    M, K = X.shape
+    N = W.shape[0]
+    X, W = _fp8(X, (M, K)), _fp8(W, (N, K))
+    bk, bp = _bias(b, N)
+    P = np.empty((M, N), dtype=np.float64)
+    _check(lib().mtmc_ref_linear_softmax_fp8(X.ctypes.data, W.ctypes.data, bp, float(scale_x), float(scale_w), M, N, K,
+                                             P.ctypes.data), "mtmc_ref_linear_softmax_fp8")
     return P
 
 

@@ -271,6 +271,26 @@ def test_fp8_rowmax_and_cross_entropy_pins():
     assert np.array_equal(floss, gloss)
 
 
+def test_fp8_softmax_pins():
+    fi = inputs.fp8_linear_inputs(6, 41, 48, seed=75)
+    X8, W8, b = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    P = ref.linear_softmax_fp8(X8, W8, b, fi.scale_x, fi.scale_w)
+    z = ref.fused_linear_fp8(X8, W8, b, fi.scale_x, fi.scale_w, ref.ACT_NONE)          # the pinned FP8 logits
+    np.testing.assert_allclose(P, torch.softmax(torch.from_numpy(z), dim=-1).numpy(), rtol=1e-13, atol=0)
+    assert np.array_equal(P, np.stack([ref.softmax_vector(row) for row in z]))         # the pinned row routine on them
+    lse = ref.linear_lse_fp8(X8, W8, b, fi.scale_x, fi.scale_w)
+    np.testing.assert_allclose(P, np.exp(z - lse[:, None]), rtol=1e-12)
+    np.testing.assert_allclose(P.sum(axis=1), np.ones(6), rtol=0, atol=1e-13)
+    # doubling one scale and halving the other changes nothing; doubling one doubles the logits' spread
+    assert np.array_equal(ref.linear_softmax_fp8(X8, W8, b, 2.0 * fi.scale_x, 0.5 * fi.scale_w), P)
+    P2 = ref.linear_softmax_fp8(X8, W8, None, 2.0 * fi.scale_x, fi.scale_w)
+    z0 = ref.fused_linear_fp8(X8, W8, None, fi.scale_x, fi.scale_w, ref.ACT_NONE)
+    np.testing.assert_allclose(P2, torch.softmax(torch.from_numpy(2.0 * z0), dim=-1).numpy(), rtol=1e-12)
+    # with power-of-two scales folded into bf16 copies of the operands: the bf16 function, bit for bit
+    folded = ref.linear_softmax(_as_bf16_bits(fi.X, 2.0 ** -4), _as_bf16_bits(fi.W, 2.0 ** -8), b)
+    assert np.array_equal(ref.linear_softmax_fp8(X8, W8, b, 2.0 ** -4, 2.0 ** -8), folded)
+
+
 # ---------------------------------------------------------------- activations
 def _closed_forms():
     rows = []
