@@ -217,6 +217,13 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
  * 2^31 - 1024.  bf16 operands.  Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_SOFTMAX, M, N, K). */
 int mtmc_linear_softmax(const void* X, const void* W, const float* b,
                         int64_t M, int64_t N, int64_t K, int out_dtype, void* prob_out, float* lse_out);
+/* The same on row-major views (X, W rows ldx, ldw elements apart: >= K, multiples of 8; prob_out rows ldo >= N
+ * elements apart, any value, e.g. the probabilities written into a wider buffer), and with E4M3 operands and
+ * per-tensor scales (as mtmc_linear_lse_fp8: K % 16 == 0, z = scale_x * scale_w * sum_k X8 W8 + b).  Same kernels. */
+int mtmc_linear_softmax_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b,
+                                int64_t M, int64_t N, int64_t K, int out_dtype, void* prob_out, int64_t ldo, float* lse_out);
+int mtmc_linear_softmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w,
+                            int64_t M, int64_t N, int64_t K, int out_dtype, void* prob_out, float* lse_out);
 
 /* Allocation-free variant of mtmc_linear_lse: same arguments, same result (same
  * kernels), but the (max, sum-exp) partials live in an 8 MiB array that is part of

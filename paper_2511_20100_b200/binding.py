@@ -27,6 +27,7 @@ OP = {"fused_linear": 0, "swiglu": 1, "linear_lse": 2, "linear_rowmax": 3, "line
 EXPORTS = [
     "mtmc_fused_linear", "mtmc_fused_linear_residual", "mtmc_fused_linear_fp8", "mtmc_swiglu", "mtmc_linear_lse",
     "mtmc_linear_lse_noalloc", "mtmc_linear_rowmax", "mtmc_linear_cross_entropy", "mtmc_linear_softmax",
+    "mtmc_linear_softmax_strided", "mtmc_linear_softmax_fp8",
     "mtmc_fused_linear_host", "mtmc_swiglu_host", "mtmc_linear_lse_host",
     "mtmc_fused_linear_host_async", "mtmc_swiglu_host_async", "mtmc_linear_lse_host_async", "mtmc_host_sync",
     "mtmc_set_stream", "mtmc_set_workspace", "mtmc_workspace_bytes", "mtmc_check_status",
@@ -82,6 +83,8 @@ def load() -> ctypes.CDLL:
     L.mtmc_linear_rowmax.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_linear_cross_entropy.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp]
     L.mtmc_linear_softmax.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp]
+    L.mtmc_linear_softmax_strided.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, ci, vp, i64, vp]
+    L.mtmc_linear_softmax_fp8.argtypes = [vp, vp, vp, ctypes.c_float, ctypes.c_float, i64, i64, i64, ci, vp, vp]
     L.mtmc_set_stream.argtypes = [vp]
     L.mtmc_set_workspace.argtypes = [vp, sz]
     L.mtmc_workspace_bytes.argtypes = [ci, i64, i64, i64]
@@ -388,6 +391,40 @@ def mtmc_linear_softmax(X, W, b, out_dtype="fp32", prob_out=None, lse_out=None, 
                                       None if b is None else _dev(b, torch.float32, (N,), "b"), M, N, K, OUT_DTYPE[out_dtype],
                                       _dev(prob_out, odt, (M, N), "prob_out"),
                                       None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
+    return (prob_out, lse_out) if want_lse else prob_out
+
+
+def mtmc_linear_softmax_strided(X, W, b, out_dtype="fp32", prob_out=None):
+    """mtmc_linear_softmax with X, W and prob_out as row-major views (column slices of wider matrices)."""
+    M, K = X.shape
+    N = W.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if prob_out is None:
+        prob_out = torch.empty((M, N), dtype=odt, device=X.device)
+    _use_current_stream(X.device)
+    (xp, ldx), (wp, ldw), (op, ldo) = (_view2d(X, torch.bfloat16, (M, K), "X"), _view2d(W, torch.bfloat16, (N, K), "W"),
+                                       _view2d(prob_out, odt, (M, N), "prob_out"))
+    _check(load().mtmc_linear_softmax_strided(xp, ldx, wp, ldw, None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                              M, N, K, OUT_DTYPE[out_dtype], op, ldo, None))
+    return prob_out
+
+
+def mtmc_linear_softmax_fp8(X8, W8, b, scale_x, scale_w, out_dtype="fp32", prob_out=None, lse_out=None, want_lse=False):
+    """mtmc_linear_softmax with float8_e4m3fn operands and per-tensor scales."""
+    M, K = X8.shape
+    N = W8.shape[0]
+    odt = torch.bfloat16 if out_dtype == "bf16" else torch.float32
+    if prob_out is None:
+        prob_out = torch.empty((M, N), dtype=odt, device=X8.device)
+    if lse_out is None and want_lse:
+        lse_out = torch.empty((M,), dtype=torch.float32, device=X8.device)
+    _use_current_stream(X8.device)
+    f8 = torch.float8_e4m3fn
+    _check(load().mtmc_linear_softmax_fp8(_dev(X8, f8, (M, K), "X8"), _dev(W8, f8, (N, K), "W8"),
+                                          None if b is None else _dev(b, torch.float32, (N,), "b"),
+                                          float(scale_x), float(scale_w), M, N, K, OUT_DTYPE[out_dtype],
+                                          _dev(prob_out, odt, (M, N), "prob_out"),
+                                          None if lse_out is None else _dev(lse_out, torch.float32, (M,), "lse_out")))
     return (prob_out, lse_out) if want_lse else prob_out
 
 

@@ -969,7 +969,7 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 template <int EPI>
 int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
                       float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0,
-                      void* prob = nullptr, int out_dtype = MTMC_OUT_FP32) {
+                      void* prob = nullptr, int out_dtype = MTMC_OUT_FP32, int64_t ldo = 0) {
     auto encode = fp8 ? encode_u8_2d : encode_bf16_2d;
     if (b && !aligned16(b)) return fail(MTMC_ERR_INVALID_ARG, "bias must be 16-byte aligned");
     DeviceState* d = nullptr;
@@ -994,7 +994,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     rc = get_workspace(d, partial_bytes + extra + (sk ? streamk_bytes(sk_clusters) : 0), &ws);
     if (rc) return rc;
     if (sk && (rc = attach_streamk(d, p, sk_clusters, ws, partial_bytes + extra))) return rc;
-    p.act = ACT_NONE; p.bias = b; p.out = prob; p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
+    p.act = ACT_NONE; p.bias = b; p.out = prob; if (ldo > 0) p.ldo = static_cast<int>(ldo); p.lse_partial = static_cast<float2*>(ws); p.status = d->status;
     p.targets = reinterpret_cast<const long long*>(targets);
     p.target_logit = EPI == EPI_XENT ? reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes) : nullptr;
     // a target outside [0, N) matches no column: its row's loss comes out as NaN instead of a stale value
@@ -1717,14 +1717,37 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
     return run_row_reduction<EPI_XENT>(X, W, b, targets, M, N, K, lse_out, loss_out, nullptr);
 }
 
-int mtmc_linear_softmax(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int out_dtype,
-                        void* prob_out, float* lse_out) {
-    int rc = check_common(X, W, prob_out, M, N, K);
-    if (rc) return rc;
+namespace {
+int check_softmax(int64_t N, int out_dtype, const float* lse_out) {
     if (out_dtype != MTMC_OUT_FP32 && out_dtype != MTMC_OUT_BF16) return fail(MTMC_ERR_INVALID_ARG, "unknown output type id %d", out_dtype);
     if (N >= (1ll << 31) - 1024) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "N = %lld: N must be below 2^31 - 1024", (long long)N);
     if (lse_out && (reinterpret_cast<uintptr_t>(lse_out) & 3u)) return fail(MTMC_ERR_INVALID_ARG, "lse_out must be 4-byte aligned");
+    return MTMC_OK;
+}
+}  // namespace
+
+int mtmc_linear_softmax(const void* X, const void* W, const float* b, int64_t M, int64_t N, int64_t K, int out_dtype,
+                        void* prob_out, float* lse_out) {
+    int rc = check_common(X, W, prob_out, M, N, K);
+    if (rc || (rc = check_softmax(N, out_dtype, lse_out))) return rc;
     return run_row_reduction<EPI_SOFTMAX>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr, false, 1.0f, 0, 0, prob_out, out_dtype);
+}
+
+int mtmc_linear_softmax_strided(const void* X, int64_t ldx, const void* W, int64_t ldw, const float* b, int64_t M, int64_t N, int64_t K,
+                                int out_dtype, void* prob_out, int64_t ldo, float* lse_out) {
+    int rc = check_common(X, W, prob_out, M, N, K);
+    if (rc || (rc = check_row_pitches(ldx, ldw, K)) || (rc = check_softmax(N, out_dtype, lse_out))) return rc;
+    if (ldo < N) return fail(MTMC_ERR_INVALID_ARG, "row pitches must cover the rows (ldo >= N)");
+    if (ldo >= (1ll << 31)) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "row pitches must be below 2^31");
+    return run_row_reduction<EPI_SOFTMAX>(X, W, b, nullptr, M, N, K, lse_out, nullptr, nullptr, false, 1.0f, ldx, ldw, prob_out, out_dtype, ldo);
+}
+
+int mtmc_linear_softmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,
+                            int64_t K, int out_dtype, void* prob_out, float* lse_out) {
+    if (K % 16 != 0) return fail(MTMC_ERR_UNSUPPORTED_SHAPE, "K = %lld: K must be a multiple of 16 for E4M3 operands", (long long)K);
+    int rc = check_common(X8, W8, prob_out, M, N, K);
+    if (rc || (rc = check_softmax(N, out_dtype, lse_out))) return rc;
+    return run_row_reduction<EPI_SOFTMAX>(X8, W8, b, nullptr, M, N, K, lse_out, nullptr, nullptr, true, scale_x * scale_w, 0, 0, prob_out, out_dtype);
 }
 
 int mtmc_linear_rowmax_fp8(const void* X8, const void* W8, const float* b, float scale_x, float scale_w, int64_t M, int64_t N,

@@ -899,6 +899,41 @@ def test_linear_softmax_with_caller_workspace_and_bad_arguments():
     B.mtmc_check_status()
 
 
+@pytest.mark.parametrize("M,N,K,padx,padw,pado", [(100, 72, 136, 8, 24, 3), (300, 520, 328, 16, 8, 8), (300, 2304, 2048, 64, 64, 1024),
+                                                  (1100, 1300, 1024, 8, 16, 4)])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_linear_softmax_on_strided_views(M, N, K, padx, padw, pado, odt):
+    """X, W and the probabilities as column slices of wider matrices (single-CTA and pair kernels; pitches that allow
+    16-byte accesses and pitches that do not): the dense call's bits, the neighbours untouched."""
+    li = inputs.linear_inputs(M, N, K, seed=9070 + M + N)
+    tdt = torch.bfloat16 if odt == "bf16" else torch.float32
+    Xw = torch.full((M, K + padx), 3.0, dtype=torch.bfloat16, device="cuda")
+    Ww = torch.full((N, K + padw), -2.0, dtype=torch.bfloat16, device="cuda")
+    Ow = torch.full((M, N + pado), 7.0, dtype=tdt, device="cuda")
+    offx, offw, offo = (8 if padx >= 16 else 0), (8 if padw >= 16 else 0), (8 if pado >= 16 else 0)
+    Xv, Wv, Ov = Xw[:, offx:offx + K], Ww[:, offw:offw + K], Ow[:, offo:offo + N]
+    Xv.copy_(li.X.cuda()); Wv.copy_(li.W.cuda())
+    B.mtmc_linear_softmax_strided(Xv, Wv, li.b.cuda(), odt, prob_out=Ov)
+    B.mtmc_check_status()
+    _check_softmax(li, Ov.contiguous(), None, odt, "strided softmax %dx%dx%d %s" % (M, N, K, odt))
+    assert bool((Ow[:, :offo] == 7.0).all()) and bool((Ow[:, offo + N:] == 7.0).all())
+    assert torch.equal(B.mtmc_linear_softmax(li.X.cuda(), li.W.cuda(), li.b.cuda(), odt), Ov.contiguous())
+
+
+@pytest.mark.parametrize("M,N,K", [(5, 8, 64), (200, 1000, 256), (129, 257, 80), (600, 3000, 128), (1024, 4096, 512)])
+@pytest.mark.parametrize("odt", ["fp32", "bf16"])
+def test_linear_softmax_fp8(M, N, K, odt):
+    fi = inputs.fp8_linear_inputs(M, N, K, seed=7500 + M + N)
+    buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
+    _, lse = B.mtmc_linear_softmax_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda(), fi.scale_x, fi.scale_w, odt, prob_out=out, want_lse=True)
+    B.mtmc_check_status()
+    assert _canaries_intact(buf, M * N)
+    X8, W8, bf = inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b)
+    _assert_close(inputs.to_f64(out), ref.linear_softmax_fp8(X8, W8, bf, fi.scale_x, fi.scale_w), SOFTMAX_TOL[odt],
+                  "softmax fp8 %dx%dx%d %s" % (M, N, K, odt))
+    _assert_close(inputs.to_f64(lse), ref.linear_lse_fp8(X8, W8, bf, fi.scale_x, fi.scale_w), TOL["fp32"], "lse of softmax fp8")
+
+
 def test_linear_softmax_at_lm_head_size_on_sampled_rows():
     c = inputs.CONFIGS["C4"]
     li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
