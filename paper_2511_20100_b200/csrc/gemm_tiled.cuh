@@ -457,10 +457,18 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            const bool ragged = n0 + 32 > p.N;               // columns past N are zero-filled weight rows: masked out
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float t = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);
-                m4[j & 3] = fmaxf(m4[j & 3], (n0 + j < p.N) ? t : -INFINITY);     // columns past N are zero-filled weight rows
+            for (int j = 0; j < 32; j += 2) {                // packed fp32 pairs: half the issue slots of the FP part
+                float b0, b1, t0, t1;
+                mul_f32x2(b0, b1, bv[j], bv[j + 1], LOG2E, LOG2E);
+                fma_f32x2(t0, t1, __uint_as_float(r[j]), __uint_as_float(r[j + 1]), zscale, zscale, b0, b1);
+                if (ragged) {
+                    if (n0 + j >= p.N) t0 = -INFINITY;
+                    if (n0 + j + 1 >= p.N) t1 = -INFINITY;
+                }
+                m4[j & 3] = fmaxf(m4[j & 3], t0);
+                m4[(j + 1) & 3] = fmaxf(m4[(j + 1) & 3], t1);
             }
             if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
             mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
@@ -473,11 +481,20 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
             tile_bias_chunk(p, bias_tile, n_tile0, n0, bv);
             tmem_ld_wait();
             float s4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            const bool ragged = n0 + 32 > p.N;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-                const float t = fmaf(__uint_as_float(r[j]), zscale, bv[j] * LOG2E);       // the same bits as in the first pass
-                y[j] = (n0 + j < p.N) ? ex2_approx(t - mx) : 0.0f;
-                s4[j & 3] += y[j];
+            for (int j = 0; j < 32; j += 2) {
+                float b0, b1, t0, t1, d0, d1;
+                mul_f32x2(b0, b1, bv[j], bv[j + 1], LOG2E, LOG2E);
+                fma_f32x2(t0, t1, __uint_as_float(r[j]), __uint_as_float(r[j + 1]), zscale, zscale, b0, b1);   // the same bits as in the first pass
+                add_f32x2(d0, d1, t0, t1, -mx, -mx);
+                y[j] = ex2_approx(d0);
+                y[j + 1] = ex2_approx(d1);
+                if (ragged) {
+                    if (n0 + j >= p.N) y[j] = 0.0f;
+                    if (n0 + j + 1 >= p.N) y[j + 1] = 0.0f;
+                }
+                add_f32x2(s4[j & 3], s4[(j + 1) & 3], s4[j & 3], s4[(j + 1) & 3], y[j], y[j + 1]);
             }
             if (c + 1 < live) tmem_ld_32x32b_x32(t_addr + (c + 1) * 32, r);
             sum += (s4[0] + s4[1]) + (s4[2] + s4[3]);

@@ -56,6 +56,11 @@ def _problem(args):
         return c, lambda: B.mtmc_linear_lse(d[0], d[1], d[2])
     if c["op"] == "linear_rowmax":
         return c, lambda: B.mtmc_linear_rowmax(d[0], d[1], d[2])
+    if c["op"] == "linear_cross_entropy":
+        tgt = inputs.targets(c["M"], c["N"], c["seed"]).cuda()
+        return c, lambda: B.mtmc_linear_cross_entropy(d[0], d[1], d[2], tgt)
+    if c["op"] == "linear_softmax":
+        return c, lambda: B.mtmc_linear_softmax(d[0], d[1], d[2], c["out_dtype"])
     if c["op"] == "fused_linear_residual":
         R = inputs.residual(c["M"], c["N"], c["seed"]).cuda()
         return c, lambda: B.mtmc_fused_linear_residual(d[0], d[1], d[2], R, c["act"], c["out_dtype"])
