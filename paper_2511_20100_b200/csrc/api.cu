@@ -341,6 +341,23 @@ int pdl_attribute(cudaLaunchAttribute* attr) {
     return 1;
 }
 
+// A small follow-up kernel (merge, scaling pass) as a programmatic dependent of the kernel before it: its blocks are
+// placed while that kernel still runs and proceed, from their griddepcontrol.wait, the moment it has completed.
+template <class Kern, class... Args>
+int launch_follow_up(Kern kern, dim3 grid, unsigned threads, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = t_stream;
+    cudaLaunchAttribute attr[1];
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_attribute(attr);
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, args...));
+    g_launches.fetch_add(1);
+    return MTMC_OK;
+}
+
 template <int EPI, int BN, bool OUT_BF16>
 int launch_tiled(DeviceState* d, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmB2,
                  const CUtensorMap& tmBt, const CUtensorMap& tmB2t, GemmParams p) {
@@ -1024,33 +1041,23 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     const unsigned blocks = static_cast<unsigned>((M + 7) / 8);
     if constexpr (EPI == EPI_SOFTMAX) {
         float* lse = out_a ? out_a : reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes);
-        lse_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
-                                                       p.n_full, p.tail_split, lse, nullptr, nullptr);
-        CUDA_TRY(cudaGetLastError());
-        g_launches.fetch_add(1);
+        if ((rc = launch_follow_up(lse_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+                                   p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse, static_cast<const float*>(nullptr),
+                                   static_cast<float*>(nullptr))))
+            return rc;
         // one warp per row and span of eight column tiles: many short blocks, so that the last wave costs little
         const int out_tile_n = (pair || bn == 256) ? 256 : 128;
         const int tiles_per_span = std::max(8, (p.n_tiles + 65534) / 65535);      // grid.y stays within its limit
         const dim3 grid(blocks, static_cast<unsigned>((p.n_tiles + tiles_per_span - 1) / tiles_per_span), 1);
-        if (out_dtype == MTMC_OUT_BF16)
-            softmax_finish_kernel<true><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
-                                                                    p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
-        else
-            softmax_finish_kernel<false><<<grid, 256, 0, t_stream>>>(prob, p.ldo, p.lse_partial, lse, p.M, p.N, p.rows_per_tile, p.m_tiles,
-                                                                     p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
-        CUDA_TRY(cudaGetLastError());
-        g_launches.fetch_add(1);
-        return MTMC_OK;
+        auto finish = out_dtype == MTMC_OUT_BF16 ? softmax_finish_kernel<true> : softmax_finish_kernel<false>;
+        return launch_follow_up(finish, grid, 256u, prob, p.ldo, static_cast<const float2*>(p.lse_partial), static_cast<const float*>(lse),
+                                p.M, p.N, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
     }
     if (EPI == EPI_ROWMAX)
-        rowmax_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
-                                                          p.n_full, p.tail_split, out_a, out_i);
-    else
-        lse_merge_kernel<<<blocks, 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
-                                                       p.n_full, p.tail_split, out_a, p.target_logit, out_b);
-    CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return MTMC_OK;
+        return launch_follow_up(rowmax_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+                                p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_a, out_i);
+    return launch_follow_up(lse_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+                            p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_a, static_cast<const float*>(p.target_logit), out_b);
 }
 
 // out = act(X.W^T + b) (+ R): picks the weight-streaming path for decode batches, CTA pairs for

@@ -754,6 +754,7 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
                                  int group_m, int n_full, int tail_split, float* __restrict__ lse,
                                  const float* __restrict__ target_logit, float* __restrict__ loss) {
     pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
+    pdl_wait();                  // launched as a programmatic dependent: the tiled kernel's partials are complete from here on
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -784,6 +785,7 @@ __global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, i
                                     int group_m, int n_full, int tail_split, float* __restrict__ max_out,
                                     int* __restrict__ argmax_out) {
     pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
+    pdl_wait();                  // launched as a programmatic dependent: the tiled kernel's partials are complete from here on
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -819,6 +821,7 @@ __global__ void softmax_finish_kernel(void* __restrict__ out, int ldo, const flo
                                       const float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
                                       int group_m, int n_full, int tail_split, int out_tile_n, int tiles_per_span) {
     pdl_launch_dependents();
+    pdl_wait();                  // launched as a programmatic dependent of the merge kernel
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
