@@ -934,6 +934,44 @@ def test_linear_softmax_fp8(M, N, K, odt):
     _assert_close(inputs.to_f64(lse), ref.linear_lse_fp8(X8, W8, bf, fi.scale_x, fi.scale_w), TOL["fp32"], "lse of softmax fp8")
 
 
+def test_linear_softmax_random_shapes_kernels_and_schedules():
+    """Seeded sweep: 60 shapes (M to 900, N to 6000, K to 2560) over output types, bias or none, logits spread by a
+    bias forty times as wide, the kernel choices of the tuning hook, the stream-K schedule and E4M3 operands."""
+    rng = np.random.default_rng(20261)
+    for it in range(60):
+        M, N = int(rng.integers(1, 900)), int(rng.integers(1, 6000))
+        K = int(rng.integers(1, 160)) * 8 if rng.random() < 0.7 else int(rng.integers(1, 40)) * 64
+        odt = "bf16" if rng.random() < 0.5 else "fp32"
+        bias = rng.random() < 0.7
+        r = rng.random()
+        tune = dict(cta_pair=1) if r < 0.2 else dict(cta_pair=-1) if r < 0.35 else dict(tile_n=128) if r < 0.45 else {}
+        sk = int(rng.choice([0, 1, -1]))
+        fp8 = rng.random() < 0.25
+        what = "case %d: %dx%dx%d %s bias=%s %r stream_k=%d fp8=%s" % (it, M, N, K, odt, bias, tune, sk, fp8)
+        B.mtmc_set_tuning(**tune)
+        B.mtmc_set_schedule(sk)
+        try:
+            if fp8:
+                K = max(16, K // 16 * 16)
+                fi = inputs.fp8_linear_inputs(M, N, K, seed=it)
+                out = B.mtmc_linear_softmax_fp8(fi.X.cuda(), fi.W.cuda(), fi.b.cuda() if bias else None, fi.scale_x, fi.scale_w, odt)
+                want = ref.linear_softmax_fp8(inputs.fp8_bits(fi.X), inputs.fp8_bits(fi.W), inputs.f32(fi.b) if bias else None,
+                                              fi.scale_x, fi.scale_w)
+            else:
+                li = inputs.linear_inputs(M, N, K, seed=it, bias=bias)
+                if bias and rng.random() < 0.3:
+                    li.b = li.b * 40.0
+                out = B.mtmc_linear_softmax(li.X.cuda(), li.W.cuda(), None if li.b is None else li.b.cuda(), odt)
+                want = ref.linear_softmax(inputs.bf16_bits(li.X), inputs.bf16_bits(li.W), inputs.f32(li.b))
+            B.mtmc_check_status()
+        finally:
+            B.mtmc_set_schedule(0)
+            B.mtmc_set_tuning()
+        _assert_close(inputs.to_f64(out), want, SOFTMAX_TOL[odt], what)
+        sums = out.double().sum(dim=1)
+        assert bool(((sums - 1.0).abs() <= (4e-3 if odt == "bf16" else 1e-4)).all()), what + ": row sums"
+
+
 def test_linear_softmax_at_lm_head_size_on_sampled_rows():
     c = inputs.CONFIGS["C4"]
     li = inputs.linear_inputs(c["M"], c["N"], c["K"], c["seed"])
