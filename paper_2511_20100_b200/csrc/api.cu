@@ -1038,10 +1038,12 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     }
     tr.stop();
     if (rc) return rc;
-    const unsigned blocks = static_cast<unsigned>((M + 7) / 8);
+    const unsigned blocks = static_cast<unsigned>((M + 7) / 8);      // eight rows per block of the finishing pass
+    const dim3 merge_grid(static_cast<unsigned>((M + 31) / 32), 1, 1);
+    const unsigned merge_threads = 32u * MERGE_WARPS;
     if constexpr (EPI == EPI_SOFTMAX) {
         float* lse = out_a ? out_a : reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes);
-        if ((rc = launch_follow_up(lse_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+        if ((rc = launch_follow_up(lse_merge_rows_kernel, merge_grid, merge_threads, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
                                    p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse, static_cast<const float*>(nullptr),
                                    static_cast<float*>(nullptr))))
             return rc;
@@ -1054,9 +1056,9 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
                                 p.M, p.N, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
     }
     if (EPI == EPI_ROWMAX)
-        return launch_follow_up(rowmax_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+        return launch_follow_up(rowmax_merge_rows_kernel, merge_grid, merge_threads, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
                                 p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_a, out_i);
-    return launch_follow_up(lse_merge_kernel, dim3(blocks, 1, 1), 256u, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
+    return launch_follow_up(lse_merge_rows_kernel, merge_grid, merge_threads, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
                             p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_a, static_cast<const float*>(p.target_logit), out_b);
 }
 
@@ -1375,10 +1377,9 @@ int run_mx(const void* X8, const void* SX, const void* W8, const void* SW, const
     tr.stop();
     if (rc) return rc;
     if (EPI == EPI_LSE) {
-        lse_merge_kernel<<<static_cast<unsigned>((M + 7) / 8), 256, 0, t_stream>>>(p.lse_partial, p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m,
-                                                                                  p.n_full, p.tail_split, lse_out, nullptr, nullptr);
-        CUDA_TRY(cudaGetLastError());
-        g_launches.fetch_add(1);
+        return launch_follow_up(lse_merge_rows_kernel, dim3(static_cast<unsigned>((M + 31) / 32), 1, 1), 32u * MERGE_WARPS,
+                                static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full,
+                                p.tail_split, lse_out, static_cast<const float*>(nullptr), static_cast<float*>(nullptr));
     }
     return MTMC_OK;
 }

@@ -749,7 +749,8 @@ __device__ __forceinline__ void lse_combine(float& m, float& s, float om, float 
 // lse[row] = max + ln(sum).  One warp per row; lanes stride over the column tiles and
 // combine with shuffles.  Every piece left EPI_HALVES partials; a whole tile is one piece, a tile
 // of the split wave tail is tail_split pieces.  With target_logit / loss given it also writes the
-// softmax cross entropy loss[row] = lse[row] - logit[row][target[row]].
+// softmax cross entropy loss[row] = lse[row] - logit[row][target[row]].  (The warp-per-row form: the allocation-free entry
+// point launches it with the block size it chose; everything else uses lse_merge_rows_kernel below.)
 __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
                                  int group_m, int n_full, int tail_split, float* __restrict__ lse,
                                  const float* __restrict__ target_logit, float* __restrict__ loss) {
@@ -780,33 +781,110 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
     }
 }
 
-// Merges the (max, column) partials of each row: the largest value, ties to the lowest column.
-__global__ void rowmax_merge_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles,
-                                    int group_m, int n_full, int tail_split, float* __restrict__ max_out,
-                                    int* __restrict__ argmax_out) {
+// The logsumexp merge with the roles of lanes and warps exchanged, and the row-maximum merge (the largest value, ties
+// to the lowest column) in the same form: a block owns 32 consecutive rows, lane = row,
+// and its warps share out the column tiles (warp w takes tiles w, w + warps, ...).  partial[piece][row] is then read
+// as whole 256-byte lines (the warp-per-row form fetches a 32-byte sector for every 8 bytes it uses), four tiles'
+// loads are in flight per thread, and warp 0 adds the warps' results in warp order through shared memory, so the
+// result does not depend on timing.  Launched with 32 * MERGE_WARPS threads per block and ceil(M / 32) blocks.
+constexpr int MERGE_WARPS = 16;
+
+__global__ void __launch_bounds__(32 * MERGE_WARPS)
+lse_merge_rows_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles, int group_m,
+                      int n_full, int tail_split, float* __restrict__ lse, const float* __restrict__ target_logit,
+                      float* __restrict__ loss) {
     pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
     pdl_wait();                  // launched as a programmatic dependent: the tiled kernel's partials are complete from here on
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= M) return;
-    const int mb = row / rows_per_tile;
-    float mx = -INFINITY;
-    int arg = 0x7fffffff;
-    for (int nb = lane; nb < n_tiles; nb += 32) {
-        const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
-        for (int sl = 0; sl < EPI_HALVES * pieces; ++sl) {
-            const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
-            const int a = __float_as_int(v.y);
-            if (v.x > mx || (v.x == mx && a < arg)) { mx = v.x; arg = a; }
+    __shared__ float2 part[MERGE_WARPS][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int row = blockIdx.x * 32 + lane;
+    float mx = -INFINITY, sum = 0.0f;
+    if (row < M) {
+        const int mb = row / rows_per_tile;
+        for (int nb0 = w; nb0 < n_tiles; nb0 += 4 * MERGE_WARPS) {
+            float2 v[4];
+            int more[4];                                      // further partials of the tile (pieces of the wave tail, shares of a piece)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int nb = nb0 + u * MERGE_WARPS;
+                v[u] = make_float2(-INFINITY, 0.0f);
+                more[u] = 0;
+                if (nb < n_tiles) {
+                    const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+                    more[u] = EPI_HALVES * pieces - 1;
+                    v[u] = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES) * M + row);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                lse_combine(mx, sum, v[u].x, v[u].y);         // (-inf, 0) past the last tile: neutral
+                const int nb = nb0 + u * MERGE_WARPS;
+                for (int sl = 1; sl <= more[u]; ++sl) {       // ascending columns
+                    const float2 x = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
+                    lse_combine(mx, sum, x.x, x.y);
+                }
+            }
         }
     }
+    part[w][lane] = make_float2(mx, sum);
+    __syncthreads();
+    if (w == 0 && row < M) {
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-        const float om = __shfl_xor_sync(0xffffffffu, mx, off);
-        const int oa = __shfl_xor_sync(0xffffffffu, arg, off);
-        if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+        for (int k = 1; k < MERGE_WARPS; ++k) lse_combine(mx, sum, part[k][lane].x, part[k][lane].y);
+        const float l = mx + __logf(sum);
+        if (lse) lse[row] = l;
+        if (loss) loss[row] = l - __ldcg(target_logit + row);
     }
-    if (lane == 0) {
+}
+
+__global__ void __launch_bounds__(32 * MERGE_WARPS)
+rowmax_merge_rows_kernel(const float2* __restrict__ partial, int M, int rows_per_tile, int m_tiles, int n_tiles, int group_m,
+                         int n_full, int tail_split, float* __restrict__ max_out, int* __restrict__ argmax_out) {
+    pdl_launch_dependents();
+    pdl_wait();
+    __shared__ float2 part[MERGE_WARPS][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int row = blockIdx.x * 32 + lane;
+    float mx = -INFINITY;
+    int arg = 0x7fffffff;
+    if (row < M) {
+        const int mb = row / rows_per_tile;
+        for (int nb0 = w; nb0 < n_tiles; nb0 += 4 * MERGE_WARPS) {
+            float2 v[4];
+            int more[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int nb = nb0 + u * MERGE_WARPS;
+                v[u] = make_float2(-INFINITY, __int_as_float(0x7fffffff));
+                more[u] = 0;
+                if (nb < n_tiles) {
+                    const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+                    more[u] = EPI_HALVES * pieces - 1;
+                    v[u] = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES) * M + row);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                int a = __float_as_int(v[u].y);
+                if (v[u].x > mx || (v[u].x == mx && a < arg)) { mx = v[u].x; arg = a; }
+                const int nb = nb0 + u * MERGE_WARPS;
+                for (int sl = 1; sl <= more[u]; ++sl) {
+                    const float2 x = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
+                    a = __float_as_int(x.y);
+                    if (x.x > mx || (x.x == mx && a < arg)) { mx = x.x; arg = a; }
+                }
+            }
+        }
+    }
+    part[w][lane] = make_float2(mx, __int_as_float(arg));
+    __syncthreads();
+    if (w == 0 && row < M) {
+#pragma unroll
+        for (int k = 1; k < MERGE_WARPS; ++k) {
+            const float om = part[k][lane].x;
+            const int oa = __float_as_int(part[k][lane].y);
+            if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+        }
         max_out[row] = mx;
         if (argmax_out) argmax_out[row] = arg;
     }
