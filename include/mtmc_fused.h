@@ -212,7 +212,8 @@ int mtmc_linear_cross_entropy(const void* X, const void* W, const float* b, cons
  * normalised form of the same row reduction: the logits themselves are never written.  The GEMM's
  * epilogue stores exp(z - max) with the maximum of the row's piece of the tile, which is at most 1
  * whatever the logits' size, and leaves the piece's (max, sum-exp) in the workspace; after the
- * merge one pass over prob_out multiplies every piece by exp(max - lse).  A bf16 result therefore
+ * merge (a launch of its own, or the first step of the last pass when a row has few pieces) one
+ * pass over prob_out multiplies every piece by exp(max - lse).  A bf16 result therefore
  * carries two roundings of a value in [0, 1]: relative error up to 2^-8.)  N must be below
  * 2^31 - 1024.  bf16 operands.  Needs mtmc_workspace_bytes(MTMC_OP_LINEAR_SOFTMAX, M, N, K). */
 int mtmc_linear_softmax(const void* X, const void* W, const float* b,

@@ -992,8 +992,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    // the softmax epilogue runs on the pair kernel and the single-CTA tiles (whose pieces the scaling kernel knows)
-    const int ks = EPI == EPI_SOFTMAX ? 0 : pick_ksplit(d, M, N, K, 256, fp8);
+    // the softmax epilogue runs on the kernels whose pieces the scaling kernel knows: all but the 512 x 256 tiles
+    const int ks = pick_ksplit(d, M, N, K, 256, fp8);
     const bool big = EPI != EPI_SOFTMAX && !ks && use_big_rowred(d, M, N, K, fp8);
     const bool pair = !ks && !big && use_pair(d, M, N, K);
     const int bn = (pair || ks || big) ? 256 : pick_tile_n(N);
@@ -1023,7 +1023,8 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     TimedRegion tr(d);
     if constexpr (EPI == EPI_SOFTMAX) {
         const bool bf = out_dtype == MTMC_OUT_BF16;
-        if (pair) rc = bf ? launch_pair<EPI, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
+        if (ks) rc = bf ? launch_ksplit<EPI, true>(ks, tmA, tmB, tmB, p) : launch_ksplit<EPI, false>(ks, tmA, tmB, tmB, p);
+        else if (pair) rc = bf ? launch_pair<EPI, true>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p)
                           : launch_pair<EPI, false>(gemm_pairs(d), tmA, tmB, tmB, tmBt, tmBt, p);
         else if (bn == 256) rc = bf ? launch_tiled<EPI, 256, true>(d, tmA, tmB, tmB, tmBt, tmBt, p)
                                     : launch_tiled<EPI, 256, false>(d, tmA, tmB, tmB, tmBt, tmBt, p);
@@ -1042,18 +1043,24 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     const dim3 merge_grid(static_cast<unsigned>((M + 31) / 32), 1, 1);
     const unsigned merge_threads = 32u * MERGE_WARPS;
     if constexpr (EPI == EPI_SOFTMAX) {
+        // one warp per row and span of eight column tiles: many short blocks, so that the last wave costs little
+        const int out_tile_n = (pair || ks || bn == 256) ? 256 : 128;
+        const int tiles_per_span = std::max(8, (p.n_tiles + 65534) / 65535);      // grid.y stays within its limit
+        const dim3 grid(blocks, static_cast<unsigned>((p.n_tiles + tiles_per_span - 1) / tiles_per_span), 1);
+        const bool bf = out_dtype == MTMC_OUT_BF16;
+        if (p.n_tiles * p.tail_split <= 256) {      // few pieces per row: every warp of the finishing kernel merges them itself
+            auto finish = bf ? softmax_finish_kernel<true, true> : softmax_finish_kernel<false, true>;
+            return launch_follow_up(finish, grid, 256u, prob, p.ldo, static_cast<const float2*>(p.lse_partial), out_a, p.M, p.N,
+                                    p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
+        }
         float* lse = out_a ? out_a : reinterpret_cast<float*>(static_cast<char*>(ws) + partial_bytes);
         if ((rc = launch_follow_up(lse_merge_rows_kernel, merge_grid, merge_threads, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,
                                    p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, lse, static_cast<const float*>(nullptr),
                                    static_cast<float*>(nullptr))))
             return rc;
-        // one warp per row and span of eight column tiles: many short blocks, so that the last wave costs little
-        const int out_tile_n = (pair || bn == 256) ? 256 : 128;
-        const int tiles_per_span = std::max(8, (p.n_tiles + 65534) / 65535);      // grid.y stays within its limit
-        const dim3 grid(blocks, static_cast<unsigned>((p.n_tiles + tiles_per_span - 1) / tiles_per_span), 1);
-        auto finish = out_dtype == MTMC_OUT_BF16 ? softmax_finish_kernel<true> : softmax_finish_kernel<false>;
-        return launch_follow_up(finish, grid, 256u, prob, p.ldo, static_cast<const float2*>(p.lse_partial), static_cast<const float*>(lse),
-                                p.M, p.N, p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
+        auto finish = bf ? softmax_finish_kernel<true, false> : softmax_finish_kernel<false, false>;
+        return launch_follow_up(finish, grid, 256u, prob, p.ldo, static_cast<const float2*>(p.lse_partial), lse, p.M, p.N,
+                                p.rows_per_tile, p.m_tiles, p.n_tiles, p.group_m, p.n_full, p.tail_split, out_tile_n, tiles_per_span);
     }
     if (EPI == EPI_ROWMAX)
         return launch_follow_up(rowmax_merge_rows_kernel, merge_grid, merge_threads, static_cast<const float2*>(p.lse_partial), p.M, p.rows_per_tile,

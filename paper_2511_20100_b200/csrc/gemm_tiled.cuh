@@ -890,21 +890,43 @@ rowmax_merge_rows_kernel(const float2* __restrict__ partial, int M, int rows_per
     }
 }
 
-// Finishes EPI_SOFTMAX once lse_merge_kernel has left the rows' lse: turns the unnormalised exponentials in out into
-// probabilities -- every element is multiplied by exp(max of its piece - lse of its row), the piece being the
-// (column tile, tail piece, share of the piece) whose epilogue thread wrote it.  One warp per row and span of column
-// tiles; 16 bytes per lane and step where the pitch allows, four tiles' loads in flight.
-template <bool OUT_BF16>
+// Finishes EPI_SOFTMAX: turns the unnormalised exponentials in out into probabilities -- every element is multiplied
+// by exp(max of its piece - lse of its row), the piece being the (column tile, tail piece, share of the piece) whose
+// epilogue thread wrote it.  One warp per row and span of column tiles; 16 bytes per lane and step where the pitch
+// allows, four tiles' loads in flight.  MERGE = false: lse_merge_rows_kernel has left the rows' lse in `lse`.
+// MERGE = true (rows of few pieces): every warp merges its row's (max, sum-exp) partials itself first, lanes striding
+// the column tiles, and the first span's warp writes the lse if the caller wants it -- one launch less.
+template <bool OUT_BF16, bool MERGE>
 __global__ void softmax_finish_kernel(void* __restrict__ out, int ldo, const float2* __restrict__ partial,
-                                      const float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
+                                      float* __restrict__ lse, int M, int N, int rows_per_tile, int m_tiles, int n_tiles,
                                       int group_m, int n_full, int tail_split, int out_tile_n, int tiles_per_span) {
     pdl_launch_dependents();
-    pdl_wait();                  // launched as a programmatic dependent of the merge kernel
+    pdl_wait();                  // launched as a programmatic dependent of the kernel that wrote the partials / the lse
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
     const int mb = row / rows_per_tile;
-    const float l = __ldcg(lse + row);
+    float l;
+    if (MERGE) {
+        float mx = -INFINITY, sum = 0.0f;
+        for (int nb = lane; nb < n_tiles; nb += 32) {
+            const int pieces = tile_index(group_m, m_tiles, n_tiles, mb, nb) < n_full ? 1 : tail_split;
+            for (int sl = 0; sl < EPI_HALVES * pieces; ++sl) {    // ascending columns
+                const float2 v = __ldcg(partial + static_cast<size_t>(nb * tail_split * EPI_HALVES + sl) * M + row);
+                lse_combine(mx, sum, v.x, v.y);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, mx, off);
+            const float os = __shfl_xor_sync(0xffffffffu, sum, off);
+            lse_combine(mx, sum, om, os);
+        }
+        l = __shfl_sync(0xffffffffu, mx + __logf(sum), 0);
+        if (blockIdx.y == 0 && lane == 0 && lse) lse[row] = l;
+    } else {
+        l = __ldcg(lse + row);
+    }
 
     constexpr int PER = OUT_BF16 ? 8 : 4;                    // elements per 16 bytes
     constexpr int UNROLL = 4;                                // tiles in flight

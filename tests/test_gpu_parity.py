@@ -817,10 +817,12 @@ def _check_softmax(li, prob, lse, odt, what):
 
 
 @pytest.mark.parametrize("M,N,K", [(1, 1, 8), (5, 8, 64), (200, 1000, 256), (129, 257, 72), (64, 3000, 128), (260, 512, 320),
-                                   (300, 2304, 2048), (130, 4100, 512), (700, 1300, 328)])
+                                   (300, 2304, 2048), (130, 4100, 512), (700, 1300, 328),
+                                   (128, 300, 4096), (200, 1100, 4096), (64, 2048, 2048), (16, 520, 1024)])
 @pytest.mark.parametrize("odt", ["fp32", "bf16"])
 def test_linear_softmax_small(M, N, K, odt):
-    """Single-CTA tiles and pair tiles, whole and split wave tails, N a multiple of 32, of 8, of 4 and odd."""
+    """Single-CTA tiles, pair tiles and cluster split-K (clusters of two, four and eight, also with pieces that lie
+    wholly past N), whole and split wave tails, N a multiple of 32, of 8, of 4 and odd."""
     li = inputs.linear_inputs(M, N, K, seed=5400 + M + N, bias=(M % 2 == 0))
     buf, out = _guarded((M, N), torch.bfloat16 if odt == "bf16" else torch.float32)
     bufl, lse = _guarded((M,), torch.float32)
@@ -834,7 +836,8 @@ def test_linear_softmax_small(M, N, K, odt):
 
 
 SOFTMAX_FAMILIES = [("single-CTA tiles", dict(cta_pair=-1), 0, (300, 1000, 328)), ("128-column tiles", dict(tile_n=128), 0, (300, 1000, 328)),
-                    ("256 x 256 pair tiles", dict(cta_pair=1), -1, (600, 1000, 328)), ("pair tiles, stream-K", dict(cta_pair=1), 1, (600, 2304, 328))]
+                    ("256 x 256 pair tiles", dict(cta_pair=1), -1, (600, 1000, 328)), ("pair tiles, stream-K", dict(cta_pair=1), 1, (600, 2304, 328)),
+                    ("cluster split-K", dict(), 0, (128, 1024, 4096))]
 
 
 @pytest.mark.parametrize("family,tune,sk,shape", SOFTMAX_FAMILIES, ids=[f[0] for f in SOFTMAX_FAMILIES])
@@ -853,7 +856,7 @@ def test_linear_softmax_edge_cases(family, tune, sk, shape, odt):
     B.mtmc_set_schedule(sk)
     try:
         plain = B.mtmc_linear_softmax(Xd, Wd, bd, odt)
-        want_kernel = "gemm_pair_kernel" if "pair" in family else "gemm_tiled_kernel"
+        want_kernel = "gemm_pair_kernel" if "pair" in family else "gemm_ksplit_kernel" if "split-K" in family else "gemm_tiled_kernel"
         assert want_kernel in B.mtmc_last_kernel_name(), "%s: ran %s" % (family, B.mtmc_last_kernel_name())
         zero_b = B.mtmc_linear_softmax(Xd, W0.cuda(), bd, odt)
         zero_nob = B.mtmc_linear_softmax(Xd, W0.cuda(), None, odt)
