@@ -486,6 +486,18 @@ def test_linear_lse_end_to_end():
     np.testing.assert_array_equal(ref.linear_lse_rows(X, W, b, rows), lse[rows])
 
 
+def test_softmax_golden_values():
+    """40-digit values of exp(z_i - lse(z)) for five logit vectors (moderate, spread over 40 units, offset by 1000)."""
+    seen = 0
+    for kind, arg, val in _closed_forms():
+        if kind == "softmax":
+            logits, idx = arg.split("|")
+            p = ref.softmax_vector([float(t) for t in logits.split(",")])
+            assert p[int(idx)] == pytest.approx(val, rel=2e-13), arg      # exp(-20) near 1e-9: fp64 keeps 13 digits of it
+            seen += 1
+    assert seen == 19
+
+
 def test_softmax_closed_forms_and_laws():
     # logits ln(a_i) for integers a_i: p_i = a_i / sum(a) exactly in the rationals
     a = [1, 2, 3, 10, 48]
