@@ -798,6 +798,27 @@ def test_rowmax_and_cross_entropy_at_lm_head_size_on_sampled_rows():
     assert bool((loss >= lse - mx - 2e-3).all())
 
 
+def test_decode_and_prefill_sweep_at_full_size():
+    """M = 64 ... 512 rows against one 8192 x 8192 weight matrix (bias + GELU-tanh, bf16), every output against the
+    oracle, and the kernel family that each batch size lands on: weight streaming up to 64 rows, cluster split-K
+    up to 256, CTA pairs from there."""
+    N = K = 8192
+    li = inputs.linear_inputs(512, N, K, seed=8100)
+    Wd, bd = li.W.cuda(), li.b.cuda()
+    Wb, bf = inputs.bf16_bits(li.W), inputs.f32(li.b)
+    for M, family in ((64, "skinny_splitk_kernel"), (65, "gemm_ksplit_kernel"), (96, "gemm_ksplit_kernel"), (128, "gemm_ksplit_kernel"),
+                      (192, "gemm_ksplit_kernel"), (256, "gemm_ksplit_kernel"), (384, "gemm_pair_kernel"), (512, "gemm_pair_kernel")):
+        X = li.X[:M].contiguous()
+        buf, out = _guarded((M, N), torch.bfloat16)
+        B.mtmc_fused_linear(X.cuda(), Wd, bd, "gelu_tanh", "bf16", out=out)
+        ran = B.mtmc_last_kernel_name()
+        B.mtmc_check_status()
+        assert family in ran, "M = %d: ran %s" % (M, ran)
+        assert _canaries_intact(buf, M * N)
+        want = ref.fused_linear(inputs.bf16_bits(X), Wb, bf, ref.ACT_GELU_TANH)
+        _assert_close(inputs.to_f64(out), want, TOL["bf16"], "%d x 8192 x 8192 on %s" % (M, ran))
+
+
 # ------------------------------------------------------------------ row softmax written out as probabilities
 # Probabilities are compared relative to their own size (a row of N of them averages 1/N, far below any absolute
 # tolerance that suits activations): logit error (bf16 products, fp32 sums) and the hardware exp2 give a few 1e-4;
