@@ -46,6 +46,9 @@ EXTRA_CONFIGS = {
     "X9": dict(op="fused_linear_mxfp8", M=8192, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=6),
     # a decode batch against a 4096-wide layer: 32 tiles of 128 x 128, clusters of four CTAs per tile split along K
     "X10": dict(op="fused_linear", M=128, N=4096, K=4096, act="gelu_tanh", out_dtype="bf16", seed=8),
+    # X7's 8192-wide layer against 256 rows (clusters of two CTAs per tile) and 512 rows (64 pair tiles on 74 pairs)
+    "X12": dict(op="fused_linear", M=256, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=9),
+    "X13": dict(op="fused_linear", M=512, N=8192, K=8192, act="gelu_tanh", out_dtype="bf16", seed=10),
     # C4's logits as probabilities: the row softmax written out in bf16 (the logits themselves never are)
     "X11": dict(op="linear_softmax", M=4096, N=32000, K=4096, out_dtype="bf16", seed=3),
 }
