@@ -442,7 +442,7 @@ __device__ __forceinline__ void epilogue_item(const GemmParams& p, uint32_t t_ad
     } else if (EPI == EPI_SOFTMAX) {
         // Two passes over the piece's accumulator columns, which stay in tensor memory meanwhile: first the row's
         // maximum over the piece, then e = 2^(t - max) for every column, stored as the still unnormalised output and
-        // summed.  The (max, sum) partial goes the way of EPI_LSE; softmax_scale_kernel multiplies the piece by
+        // summed.  The (max, sum) partial goes the way of EPI_LSE; softmax_finish_kernel multiplies the piece by
         // exp(max - lse) once the row's lse is known.
         constexpr float LOG2E = 1.4426950408889634f;
         const float zscale = LOG2E * p.acc_scale;
@@ -755,7 +755,6 @@ __global__ void lse_merge_kernel(const float2* __restrict__ partial, int M, int 
                                  int group_m, int n_full, int tail_split, float* __restrict__ lse,
                                  const float* __restrict__ target_logit, float* __restrict__ loss) {
     pdl_launch_dependents();     // the next kernel of this library may set up (and prefetch static weights) beside this one
-    pdl_wait();                  // launched as a programmatic dependent: the tiled kernel's partials are complete from here on
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
