@@ -981,8 +981,9 @@ int linear_lse_host_impl(const void* X, const void* W, const float* b, int64_t M
 // leaves one partial per (row, column piece) in the workspace, a merge kernel finishes the rows.
 //   EPI_LSE    : out_a = lse                     EPI_ROWMAX : out_a = max, out_i = argmax (may be null)
 //   EPI_XENT   : out_b = loss, out_a = lse (may be null); the target logits sit behind the partials
-//   EPI_SOFTMAX: prob = the [M,N] probabilities (fp32 / bf16, dense), out_a = lse (may be null: it then sits behind the
-//                partials); the tiled kernel leaves exp(z - max of the piece) in prob, a last kernel scales every piece
+//   EPI_SOFTMAX: prob = the [M,N] probabilities (fp32 / bf16, rows ldo elements apart), out_a = lse (may be null: a merge
+//                launch then leaves it behind the partials); the tiled kernel leaves exp(z - max of the piece) in prob,
+//                the finishing kernel scales every piece (and merges the partials itself when a row has few of them)
 template <int EPI>
 int run_row_reduction(const void* X, const void* W, const float* b, const int64_t* targets, int64_t M, int64_t N, int64_t K,
                       float* out_a, float* out_b, int32_t* out_i, bool fp8 = false, float acc_scale = 1.0f, int64_t ldx = 0, int64_t ldw = 0,
@@ -992,7 +993,7 @@ int run_row_reduction(const void* X, const void* W, const float* b, const int64_
     DeviceState* d = nullptr;
     int rc = get_device(&d);
     if (rc) return rc;
-    // the softmax epilogue runs on the kernels whose pieces the scaling kernel knows: all but the 512 x 256 tiles
+    // the softmax epilogue runs on the kernels whose pieces the finishing kernel knows: all but the 512 x 256 tiles
     const int ks = pick_ksplit(d, M, N, K, 256, fp8);
     const bool big = EPI != EPI_SOFTMAX && !ks && use_big_rowred(d, M, N, K, fp8);
     const bool pair = !ks && !big && use_pair(d, M, N, K);
